@@ -1,0 +1,174 @@
+/*
+ * sketchssm.h -- C ABI of the SketchSSM decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * SketchSSM keeps the full recurrent state S (K x V, fp32) of a linear-attention
+ * layer exact, but lets the decode steps between two state updates read only a
+ * compact sketch U = S^T Omega (V x r) of it.  One window of L tokens is
+ * (Algorithm 1, inference part):
+ *     L-1 times  sketchssm_decode_step   : append token, o = U C q~ + o_buffer
+ *     once       sketchssm_state_update  : append token, replay the L buffered
+ *                                          tokens into S, o = S^T q, U = S^T Omega
+ * sketchssm_full_read_decode is the exact decode that reads all of S every step
+ * (the buffered-replay baseline of Eq. 4); it is kept as the in-library baseline.
+ *
+ * Recurrences (Section 3.1, Eq. 1-4), per (batch b, head h):
+ *   S_t = M_t S_{t-1} + beta_t k_t v_t^T,  M_t = (I - beta_t k_t k_t^T) D_t  (GDN, KDA)
+ *                                          M_t = D_t                         (Mamba-2)
+ *   D_t = a_t I (Mamba-2), alpha_t I (GDN), Diag(g_t) (KDA)
+ *   o_t = S_0^T q~_t + sum_{s<=t} a_s v_s,  q~_t = M_{1:t}^T q_t,
+ *   a_s = beta_s <M_{s+1:t} k_s, q_t>.
+ *
+ * General rules
+ *   - Every pointer in sketchssm_buffers and every tensor argument of the three
+ *     hot-path calls is a DEVICE pointer on the configured device, owned by the
+ *     caller, 16-byte aligned, densely packed in the layouts below.  The library
+ *     allocates no device memory and keeps no copy of any tensor.
+ *   - The hot-path calls only enqueue work on `stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and return; they never synchronise.
+ *   - Return value: SKETCHSSM_OK (0) or a negative sketchssm_status.  Nothing
+ *     throws, aborts or traps.  Kernels bound every wait; a wait that runs out
+ *     records a code in the caller's status word (see sketchssm_buffers.status).
+ *   - The window phase is the caller's: `n_before` (tokens already buffered) is
+ *     the same for the whole batch.
+ *
+ * Layouts (B = batch, H = heads, K = dk, V = dv, r = rank, L = buf_len; "io" is
+ * float or bfloat16 as configured):
+ *   state  S      [B][H][K][V]  fp32
+ *   sketch U      [B][H][r][V]  fp32   (U^T of the paper's V x r matrix: row g is S^T omega_g)
+ *   omega  Omega  [H][K][r]     fp32   (fixed offline, shared by the batch)
+ *   coef   C      [H][r][K]     fp32   (fixed offline coefficient map, Eq. 10)
+ *   ring          [B][H] blocks of sketchssm_sizes.ring_head_bytes, each
+ *                   k     [L][K] io
+ *                   v     [L][V] io
+ *                   beta  [L]    fp32
+ *                   decay [L]    fp32 (Mamba-2 a_t, GDN alpha_t)  or  [L][K] io (KDA g_t)
+ *   token inputs  q,k [B][H][K] io;  v [B][H][V] io;  beta [B][H] fp32;
+ *                 decay [B][H] fp32 (Mamba-2, GDN) or [B][H][K] io (KDA)
+ *   output        o [B][H][V] fp32 or bfloat16 (config.out_dtype)
+ */
+#ifndef SKETCHSSM_H_
+#define SKETCHSSM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum sketchssm_kind { SKETCHSSM_MAMBA2 = 0, SKETCHSSM_GDN = 1, SKETCHSSM_KDA = 2 };
+enum sketchssm_dtype { SKETCHSSM_F32 = 0, SKETCHSSM_BF16 = 1 };
+
+typedef enum sketchssm_status {
+    SKETCHSSM_OK = 0,
+    SKETCHSSM_INVALID_ARG = -1,       /* null pointer, misaligned pointer, n out of range, bad flag mix */
+    SKETCHSSM_UNSUPPORTED_SHAPE = -2, /* shape outside the compiled set (see sketchssm_create) */
+    SKETCHSSM_NOT_BOUND = -3,         /* hot-path call before sketchssm_bind */
+    SKETCHSSM_CUDA_ERROR = -4,        /* a CUDA runtime call failed (launch, attribute, device) */
+    SKETCHSSM_DEVICE_TIMEOUT = -5     /* read back from the status word: a bounded device wait ran out */
+} sketchssm_status;
+
+/* flags of sketchssm_state_update */
+#define SKETCHSSM_NO_SKETCH 0x1u      /* do not write U (the flush kernel without the sketch) */
+/* flags of sketchssm_decode_step / sketchssm_full_read_decode */
+#define SKETCHSSM_NO_APPEND 0x1u      /* use the token for this step's output but do not store it in the ring */
+
+typedef struct sketchssm_config {
+    int32_t kind;       /* sketchssm_kind */
+    int32_t batch;      /* B >= 1 */
+    int32_t heads;      /* H >= 1 */
+    int32_t dk;         /* K: 64 or 128 */
+    int32_t dv;         /* V: 64 or 128 */
+    int32_t rank;       /* r: 1..64 */
+    int32_t buf_len;    /* L: 4..64, multiple of 4 */
+    int32_t io_dtype;   /* sketchssm_dtype of q, k, v, KDA g and of the ring's k, v, g */
+    int32_t out_dtype;  /* sketchssm_dtype of o */
+    int32_t device;     /* CUDA device ordinal */
+} sketchssm_config;
+
+typedef struct sketchssm_sizes {
+    size_t state_bytes, sketch_bytes, ring_bytes, omega_bytes, coef_bytes;
+    size_t status_bytes;     /* size of the status word block (16) */
+    size_t ring_head_bytes;  /* stride of one (b, h) ring block */
+    size_t ring_v_offset, ring_beta_offset, ring_decay_offset; /* byte offsets inside a ring block (k is at 0) */
+    size_t alignment;        /* required alignment of every pointer (16) */
+} sketchssm_sizes;
+
+typedef struct sketchssm_buffers {
+    void* state;   /* S      */
+    void* sketch;  /* U      */
+    void* ring;    /* ring   */
+    void* omega;   /* Omega  */
+    void* coef;    /* C      */
+    void* status;  /* int32[4], zero-initialised by the caller: [0] first device fault code
+                      (0 = none), [1] which wait, [2..3] reserved.  Kernels only ever write
+                      non-zero codes; sketchssm_read_status reads it back. */
+} sketchssm_buffers;
+
+typedef struct sketchssm_ctx sketchssm_ctx; /* host-only metadata; owns no device memory */
+
+/* Validate the configuration and create a context.  Host-only (no CUDA call).
+ * Supported: dk in {64,128}, dv in {64,128}, 1 <= rank <= 64, buf_len in 4..64 and a
+ * multiple of 4, any kind / dtype combination.  Returns INVALID_ARG / UNSUPPORTED_SHAPE. */
+int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out);
+int sketchssm_destroy(sketchssm_ctx* ctx);
+
+/* Byte sizes and ring sub-offsets for this configuration.  Host-only. */
+int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out);
+
+/* Record the caller's device buffers (all six required, 16-byte aligned).  The context
+ * stores the pointers only; the caller keeps ownership and must keep them alive. */
+int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* bufs);
+
+/* Flush step of Algorithm 1: (optionally) append the current token, replay every buffered
+ * token into S exactly (Eq. 3), then o = S^T q from the updated state and U = S^T Omega
+ * (Eq. 7) while the updated tile is still on chip, so S is read once and written once.
+ *   n_before : tokens already in the ring, 0..L (0..L-1 when a token is given).
+ *   k, v, beta, decay : the current token, all given or all NULL.  When given it is
+ *              replayed last (it need not be stored: the ring is empty afterwards).
+ *   q, out   : both given or both NULL; out = S_new^T q (exact output of the flush step).
+ *   flags    : SKETCHSSM_NO_SKETCH leaves U untouched.
+ * With n_before = 0 and no token, S is left untouched and only U (and out) are produced:
+ * this builds the initial sketch from a prefilled state.
+ * After the call the caller's ring count is 0. */
+int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
+                           const void* v, const void* beta, const void* decay, void* out,
+                           uint32_t flags, void* stream);
+
+/* Non-flush decode step of Algorithm 1: store the token in ring slot n_before, form q~_t and
+ * the buffer weights from the n_before+1 buffered tokens (Eq. 4), c_t = C q~_t, and write
+ * o = U c_t + sum_s a_s v_s.  S is not touched.  n_before in 0..L-1; all pointers required.
+ * After the call the caller's ring count is n_before + 1 (unless SKETCHSSM_NO_APPEND). */
+int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
+                          const void* v, const void* beta, const void* decay, void* out,
+                          uint32_t flags, void* stream);
+
+/* Exact decode step that reads the whole state: o = S_0^T q~_t + sum_s a_s v_s (Eq. 4).
+ * Same arguments and ring behaviour as sketchssm_decode_step; U and C are not read. */
+int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
+                               const void* v, const void* beta, const void* decay, void* out,
+                               uint32_t flags, void* stream);
+
+/* Copy the status word back (synchronises `stream`).  Returns SKETCHSSM_OK if no kernel
+ * recorded a fault, SKETCHSSM_DEVICE_TIMEOUT otherwise; `detail`, if not NULL, receives the
+ * four status ints. */
+int sketchssm_read_status(sketchssm_ctx* ctx, int32_t detail[4], void* stream);
+
+/* Text of the CUDA runtime error behind the most recent SKETCHSSM_CUDA_ERROR of this context. */
+const char* sketchssm_last_cuda_error(const sketchssm_ctx* ctx);
+
+/* Number of kernels the last hot-path call on this context launched (host counter). */
+int sketchssm_last_launch_count(const sketchssm_ctx* ctx);
+
+/* Optional launch tuning, host-only.  Keys: "decode_batches_per_cta" (batch entries one CTA of
+ * the decode kernels serves for its head; 0 = library default), "decode_stages" (1 or 2 shared-memory
+ * stages per warp; 0 = library default).  Results never depend on these. */
+int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value);
+
+const char* sketchssm_status_string(int status);
+const char* sketchssm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKETCHSSM_H_ */

@@ -1,0 +1,231 @@
+// C ABI of the SketchSSM decode hot path: argument checking and kernel dispatch.
+#include <new>
+
+#include "internal.cuh"
+
+using namespace sketchssm;
+
+struct sketchssm_ctx : public Ctx {
+    int tune_batches_per_cta;
+    int tune_stages;
+};
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+RingLayout ring_layout(const sketchssm_config& c, int io) {
+    RingLayout r;
+    r.v_off = (size_t)c.buf_len * c.dk * io;
+    r.beta_off = r.v_off + (size_t)c.buf_len * c.dv * io;
+    r.decay_off = r.beta_off + (size_t)c.buf_len * 4;
+    const size_t decay_bytes = c.kind == SKETCHSSM_KDA ? (size_t)c.buf_len * c.dk * io : (size_t)c.buf_len * 4;
+    r.head_bytes = r.decay_off + decay_bytes;
+    return r;
+}
+
+int check_token_ptrs(const void* q, const void* k, const void* v, const void* beta, const void* decay, const void* out) {
+    const void* ps[6] = {q, k, v, beta, decay, out};
+    for (const void* p : ps) {
+        if (p == nullptr || !aligned16(p)) return SKETCHSSM_INVALID_ARG;
+    }
+    return SKETCHSSM_OK;
+}
+
+Params base_params(const sketchssm_ctx* ctx) {
+    Params p{};
+    p.state = static_cast<float*>(ctx->bufs.state);
+    p.sketch = static_cast<float*>(ctx->bufs.sketch);
+    p.ring = static_cast<unsigned char*>(ctx->bufs.ring);
+    p.omega = static_cast<const float*>(ctx->bufs.omega);
+    p.coef = static_cast<const float*>(ctx->bufs.coef);
+    p.status = static_cast<int*>(ctx->bufs.status);
+    p.rl = ctx->ring;
+    p.B = ctx->cfg.batch; p.H = ctx->cfg.heads; p.R = ctx->cfg.rank; p.L = ctx->cfg.buf_len;
+    p.dk = ctx->cfg.dk; p.dv = ctx->cfg.dv;
+    p.out_bf16 = ctx->cfg.out_dtype == SKETCHSSM_BF16;
+    p.batches_per_cta = ctx->tune_batches_per_cta;
+    p.stages = ctx->tune_stages;
+    return p;
+}
+
+int set_device(const sketchssm_ctx* ctx) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+    if (cur != ctx->cfg.device && cudaSetDevice(ctx->cfg.device) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+    return SKETCHSSM_OK;
+}
+
+int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q, const void* k, const void* v,
+                  const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    ctx->last_launches = 0;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    if (n_before < 0 || n_before > ctx->cfg.buf_len - 1) return SKETCHSSM_INVALID_ARG;
+    if (flags & ~SKETCHSSM_NO_APPEND) return SKETCHSSM_INVALID_ARG;
+    int rc = check_token_ptrs(q, k, v, beta, decay, out);
+    if (rc != SKETCHSSM_OK) return rc;
+    rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    Params p = base_params(ctx);
+    p.q = q; p.k = k; p.v = v; p.beta = static_cast<const float*>(beta); p.decay = decay; p.out = out;
+    p.n_before = n_before;
+    p.has_token = 1;
+    p.append = (flags & SKETCHSSM_NO_APPEND) ? 0 : 1;
+    p.full_read = full_read;
+    return launch_decode(ctx, p, static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+
+extern "C" {
+
+int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
+    if (cfg == nullptr || out == nullptr) return SKETCHSSM_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->kind < SKETCHSSM_MAMBA2 || cfg->kind > SKETCHSSM_KDA) return SKETCHSSM_INVALID_ARG;
+    if (cfg->io_dtype != SKETCHSSM_F32 && cfg->io_dtype != SKETCHSSM_BF16) return SKETCHSSM_INVALID_ARG;
+    if (cfg->out_dtype != SKETCHSSM_F32 && cfg->out_dtype != SKETCHSSM_BF16) return SKETCHSSM_INVALID_ARG;
+    if (cfg->batch < 1 || cfg->heads < 1 || cfg->device < 0) return SKETCHSSM_INVALID_ARG;
+    if (cfg->rank < 1 || cfg->buf_len < 1) return SKETCHSSM_INVALID_ARG;
+    if ((cfg->dk != 64 && cfg->dk != 128) || (cfg->dv != 64 && cfg->dv != 128)) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (cfg->rank > kMaxRank) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (cfg->buf_len < 4 || cfg->buf_len > kMaxBufLen || (cfg->buf_len & 3)) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if ((size_t)cfg->batch * cfg->heads > (size_t)1 << 24) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    sketchssm_ctx* c = new (std::nothrow) sketchssm_ctx();
+    if (c == nullptr) return SKETCHSSM_INVALID_ARG;
+    c->cfg = *cfg;
+    c->io_size = cfg->io_dtype == SKETCHSSM_BF16 ? 2 : 4;
+    c->ring = ring_layout(*cfg, c->io_size);
+    c->bound = false;
+    c->bufs = sketchssm_buffers{};
+    c->last_launches = 0;
+    c->last_cuda_error = cudaSuccess;
+    c->tune_batches_per_cta = 0;
+    c->tune_stages = 0;
+    *out = c;
+    return SKETCHSSM_OK;
+}
+
+int sketchssm_destroy(sketchssm_ctx* ctx) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    delete ctx;
+    return SKETCHSSM_OK;
+}
+
+int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
+    if (ctx == nullptr || out == nullptr) return SKETCHSSM_INVALID_ARG;
+    const sketchssm_config& c = ctx->cfg;
+    const size_t bh = (size_t)c.batch * c.heads;
+    out->state_bytes = bh * c.dk * c.dv * 4;
+    out->sketch_bytes = bh * c.rank * c.dv * 4;
+    out->ring_bytes = bh * ctx->ring.head_bytes;
+    out->omega_bytes = (size_t)c.heads * c.dk * c.rank * 4;
+    out->coef_bytes = (size_t)c.heads * c.rank * c.dk * 4;
+    out->status_bytes = kStatusInts * sizeof(int32_t);
+    out->ring_head_bytes = ctx->ring.head_bytes;
+    out->ring_v_offset = ctx->ring.v_off;
+    out->ring_beta_offset = ctx->ring.beta_off;
+    out->ring_decay_offset = ctx->ring.decay_off;
+    out->alignment = 16;
+    return SKETCHSSM_OK;
+}
+
+int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* b) {
+    if (ctx == nullptr || b == nullptr) return SKETCHSSM_INVALID_ARG;
+    const void* ps[6] = {b->state, b->sketch, b->ring, b->omega, b->coef, b->status};
+    for (const void* p : ps) {
+        if (p == nullptr || !aligned16(p)) return SKETCHSSM_INVALID_ARG;
+    }
+    ctx->bufs = *b;
+    ctx->bound = true;
+    return SKETCHSSM_OK;
+}
+
+int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
+                           const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    ctx->last_launches = 0;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    if (flags & ~SKETCHSSM_NO_SKETCH) return SKETCHSSM_INVALID_ARG;
+    const int n_tok = (k != nullptr) + (v != nullptr) + (beta != nullptr) + (decay != nullptr);
+    if (n_tok != 0 && n_tok != 4) return SKETCHSSM_INVALID_ARG;
+    const bool has_token = n_tok == 4;
+    if ((q == nullptr) != (out == nullptr)) return SKETCHSSM_INVALID_ARG;
+    if (n_before < 0 || n_before + (has_token ? 1 : 0) > ctx->cfg.buf_len) return SKETCHSSM_INVALID_ARG;
+    const void* ps[6] = {q, k, v, beta, decay, out};
+    for (const void* p : ps) {
+        if (p != nullptr && !aligned16(p)) return SKETCHSSM_INVALID_ARG;
+    }
+    const bool sketch = !(flags & SKETCHSSM_NO_SKETCH);
+    const int n_tot = n_before + (has_token ? 1 : 0);
+    if (n_tot == 0 && !sketch && out == nullptr) return SKETCHSSM_OK;  // nothing to do
+    int rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    Params p = base_params(ctx);
+    p.q = q; p.k = k; p.v = v; p.beta = static_cast<const float*>(beta); p.decay = decay; p.out = out;
+    p.n_before = n_before;
+    p.has_token = has_token ? 1 : 0;
+    p.write_sketch = sketch ? 1 : 0;
+    p.write_state = n_tot > 0 ? 1 : 0;
+    return launch_update(ctx, p, static_cast<cudaStream_t>(stream));
+}
+
+int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
+                          const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    return decode_common(ctx, 0, n_before, q, k, v, beta, decay, out, flags, stream);
+}
+
+int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
+                               const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    return decode_common(ctx, 1, n_before, q, k, v, beta, decay, out, flags, stream);
+}
+
+int sketchssm_read_status(sketchssm_ctx* ctx, int32_t detail[4], void* stream) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    int rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    int32_t host[kStatusInts] = {0, 0, 0, 0};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(host, ctx->bufs.status, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+    if (detail != nullptr) {
+        for (int i = 0; i < kStatusInts; ++i) detail[i] = host[i];
+    }
+    return host[0] == 0 ? SKETCHSSM_OK : SKETCHSSM_DEVICE_TIMEOUT;
+}
+
+const char* sketchssm_last_cuda_error(const sketchssm_ctx* ctx) {
+    return ctx == nullptr ? "no context" : cudaGetErrorString(ctx->last_cuda_error);
+}
+
+int sketchssm_last_launch_count(const sketchssm_ctx* ctx) { return ctx == nullptr ? 0 : ctx->last_launches; }
+
+int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value) {
+    if (ctx == nullptr || key == nullptr) return SKETCHSSM_INVALID_ARG;
+    auto eq = [](const char* a, const char* b) {
+        while (*a && *b && *a == *b) { ++a; ++b; }
+        return *a == *b;
+    };
+    if (eq(key, "decode_batches_per_cta")) { ctx->tune_batches_per_cta = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_stages")) { ctx->tune_stages = value; return SKETCHSSM_OK; }
+    return SKETCHSSM_INVALID_ARG;
+}
+
+const char* sketchssm_status_string(int status) {
+    switch (status) {
+        case SKETCHSSM_OK: return "ok";
+        case SKETCHSSM_INVALID_ARG: return "invalid argument";
+        case SKETCHSSM_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case SKETCHSSM_NOT_BOUND: return "buffers not bound";
+        case SKETCHSSM_CUDA_ERROR: return "CUDA runtime error";
+        case SKETCHSSM_DEVICE_TIMEOUT: return "bounded device wait ran out";
+    }
+    return "unknown status";
+}
+
+const char* sketchssm_version(void) { return "sketchssm-b200 0.1"; }
+
+}  // extern "C"

@@ -1,0 +1,197 @@
+// Internal declarations shared by the SketchSSM CUDA translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sketchssm.h"
+
+namespace sketchssm {
+
+constexpr int kMaxBufLen = 64;
+constexpr int kMaxRank = 64;
+constexpr int kStatusInts = 4;
+// device fault codes written to the status word
+constexpr int kFaultDecodeWait = 1;
+constexpr int kFaultFullReadWait = 2;
+constexpr int kFaultUpdateWait = 3;
+
+struct RingLayout {
+    size_t head_bytes, v_off, beta_off, decay_off;
+};
+
+struct Ctx {
+    sketchssm_config cfg;
+    sketchssm_buffers bufs;
+    RingLayout ring;
+    bool bound;
+    int io_size;
+    int sm_count;       // filled lazily on first launch
+    int max_smem_optin; // ditto
+    int last_launches;
+    cudaError_t last_cuda_error;  // of the most recent failing runtime call
+};
+
+// Arguments common to the three kernels.
+struct Params {
+    // token inputs
+    const void* q;
+    const void* k;
+    const void* v;
+    const float* beta;
+    const void* decay;
+    void* out;
+    // caller buffers
+    float* state;
+    float* sketch;
+    unsigned char* ring;
+    const float* omega;
+    const float* coef;
+    int* status;
+    RingLayout rl;
+    int B, H, R, L;
+    int dk, dv;
+    int n_before;    // tokens already in the ring
+    int has_token;   // current token given
+    int append;      // store the token in the ring
+    int out_bf16;
+    int write_sketch;
+    int write_state;
+    int full_read;   // decode: read S instead of U, C
+    int batches_per_cta;
+    int stages;
+};
+
+int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// Bounded wait: returns false if the barrier phase did not complete within the iteration limit.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit = (1u << 22)) {
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    return false;
+}
+
+// 1-D bulk asynchronous copy global -> shared of this CTA (no multicast), completion on an mbarrier.
+// src, dst 16-byte aligned; bytes a positive multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void record_fault(int* status, int code, int where) {
+    if (status != nullptr) {
+        if (atomicCAS(status, 0, code) == 0) status[1] = where;
+    }
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Load N consecutive io elements (float or bf16) starting at element index `idx` as floats.
+template <int N>
+__device__ __forceinline__ void load_io(const float* base, int idx, float (&dst)[N]) {
+    if constexpr (N == 4) {
+        float4 t = *reinterpret_cast<const float4*>(base + idx);
+        dst[0] = t.x; dst[1] = t.y; dst[2] = t.z; dst[3] = t.w;
+    } else if constexpr (N == 2) {
+        float2 t = *reinterpret_cast<const float2*>(base + idx);
+        dst[0] = t.x; dst[1] = t.y;
+    } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) dst[i] = base[idx + i];
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void load_io(const __nv_bfloat16* base, int idx, float (&dst)[N]) {
+    if constexpr (N == 4) {
+        uint2 t = *reinterpret_cast<const uint2*>(base + idx);
+        __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&t.x);
+        __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&t.y);
+        float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+        dst[0] = fa.x; dst[1] = fa.y; dst[2] = fb.x; dst[3] = fb.y;
+    } else if constexpr (N == 2) {
+        __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(base + idx);
+        float2 fa = __bfloat1622float2(a);
+        dst[0] = fa.x; dst[1] = fa.y;
+    } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) dst[i] = __bfloat162float(base[idx + i]);
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void store_io(float* base, int idx, const float (&src)[N]) {
+    if constexpr (N == 4) {
+        *reinterpret_cast<float4*>(base + idx) = make_float4(src[0], src[1], src[2], src[3]);
+    } else if constexpr (N == 2) {
+        *reinterpret_cast<float2*>(base + idx) = make_float2(src[0], src[1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) base[idx + i] = src[i];
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void store_io(__nv_bfloat16* base, int idx, const float (&src)[N]) {
+    if constexpr (N == 4) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(src[0], src[1]);
+        __nv_bfloat162 b = __floats2bfloat162_rn(src[2], src[3]);
+        uint2 t;
+        t.x = *reinterpret_cast<uint32_t*>(&a);
+        t.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(base + idx) = t;
+    } else if constexpr (N == 2) {
+        *reinterpret_cast<__nv_bfloat162*>(base + idx) = __floats2bfloat162_rn(src[0], src[1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < N; ++i) base[idx + i] = __float2bfloat16_rn(src[i]);
+    }
+}
+
+#endif  // __CUDACC__
+
+}  // namespace sketchssm

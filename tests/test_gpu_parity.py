@@ -1,0 +1,282 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle, element by element.
+
+Norm: per decode step, max |o_gpu - o_oracle| over max |o_oracle| across all compared (b, h, v);
+the same for the final state S and sketch U.  Bars: 1e-5 for float32 I/O, 2e-3 for bfloat16 I/O
+(float32 state and accumulation in both cases).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sketchssm_oracle as orc
+from paper_2609_33051_b200 import synth
+from tests import harness
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-3}
+# the kernels accumulate in float32 on the same input bits, so the observed error sits far below the
+# bf16 bar; a regression guard at this level catches wrong-but-small mistakes the bar would hide
+FP32_GUARD = 5e-5
+
+
+def _device():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return torch.device("cuda", 0)
+
+
+def make_layer(w, layer=0, out="f32"):
+    from paper_2609_33051_b200.binding import SketchSSM
+    dev = _device()
+    Om, C = harness.basis_for(w, layer)
+    m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out=out, device=0)
+    S0 = synth.initial_state(w, layer)
+    m.state.copy_(torch.from_numpy(S0))
+    m.omega.copy_(torch.from_numpy(Om))
+    m.coef.copy_(torch.from_numpy(C))
+    return m, S0, Om, C, dev
+
+
+def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32"):
+    """Algorithm 1 on GPU and oracle; returns the worst per-step relative error and the final-state errors."""
+    m, S0, Om, C, dev = make_layer(w, out=out)
+    for key, val in (tune or {}).items():
+        m.tune(key, val)
+    bs, hs = harness.select_heads(w, max_heads)
+    m.state_update(0)                                   # initial sketch from the prefilled state
+    S = S0[bs, hs].astype(np.float64)
+    Om_s, C_s = Om[hs].astype(np.float64), C[hs].astype(np.float64)
+    U = orc.sketch_of(S, Om_s)
+    errs = {"u0": harness.rel_err(m.sketch.cpu().numpy()[bs, hs].transpose(0, 2, 1), U)}
+    worst = 0.0
+    ring = []
+    o_dev = m.new_output()
+    L = w.buf_len
+    for t in range(steps):
+        x = synth.step_inputs(w, 0, t)
+        tt = harness.token_tensors(w, x, dev)
+        n = t % L
+        ring.append(harness.oracle_token(x, bs, hs))
+        q = x["q"][bs, hs].astype(np.float64)
+        if n < L - 1:
+            if mode == "sketch":
+                m.decode_step(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
+                ref = orc.decode_step(w.kind, U, C_s, ring, q)
+            else:
+                m.full_read_decode(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
+                ref = orc.full_read_decode(w.kind, S, ring, q)
+        else:
+            m.state_update(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
+            S, U, ref = orc.state_update(w.kind, S, ring, Om_s, q)
+            ring = []
+        assert m.last_launch_count() == 1
+        got = o_dev.float().cpu().numpy()[bs, hs]
+        assert np.all(np.isfinite(got))
+        worst = max(worst, harness.rel_err(got, ref))
+    m.check_status()
+    errs["out"] = worst
+    errs["S"] = harness.rel_err(m.state.cpu().numpy()[bs, hs], S)
+    errs["U"] = harness.rel_err(m.sketch.cpu().numpy()[bs, hs].transpose(0, 2, 1), U)
+    return errs
+
+
+def check(errs, io, guard=FP32_GUARD):
+    for key, e in errs.items():
+        assert e <= TOL[io], (key, e, errs)
+        assert e <= guard, (key, e, errs)
+
+
+# ---------------------------------------------------------------------------------------------
+# config 1 in full, and reduced-batch versions of configs 2-4 (all heads compared)
+# ---------------------------------------------------------------------------------------------
+
+def test_config1_gdn_tiny_full_run():
+    w = synth.CONFIGS["c1_gdn_tiny"]
+    errs = run_schedule(w, w.steps, max_heads=10**9)
+    check(errs, "f32", guard=1e-5)
+
+
+@pytest.mark.parametrize("name,batch,steps", [("c2_mamba2", 6, 40), ("c3_gdn", 5, 40), ("c4_kda", 3, 70)])
+def test_configs_2_to_4_reduced_batch(name, batch, steps):
+    w = synth.CONFIGS[name].replace(batch=batch, heads=4)
+    check(run_schedule(w, steps, max_heads=10**9), w.io)
+
+
+@pytest.mark.parametrize("name", ["c2_mamba2", "c3_gdn", "c4_kda"])
+def test_full_read_decode_reduced_batch(name):
+    w = synth.CONFIGS[name].replace(batch=5, heads=3)
+    check(run_schedule(w, w.buf_len + 5, max_heads=10**9, mode="full_read"), w.io)
+
+
+# ---------------------------------------------------------------------------------------------
+# shapes, ranks, window lengths, launch tunings
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind", synth.KINDS)
+@pytest.mark.parametrize("dk,dv", [(64, 64), (64, 128), (128, 64), (128, 128)])
+@pytest.mark.parametrize("io", ["f32", "bf16"])
+def test_shapes_and_dtypes(kind, dk, dv, io):
+    w = synth.Workload("t", kind, 3, 2, dk, dv, 8, 8, 20, io, 4242, basis="qr")
+    check(run_schedule(w, 20, max_heads=10**9), io, guard=1e-5 if io == "f32" else FP32_GUARD)
+    check(run_schedule(w, 11, max_heads=10**9, mode="full_read"), io, guard=1e-5 if io == "f32" else FP32_GUARD)
+
+
+@pytest.mark.parametrize("kind", synth.KINDS)
+@pytest.mark.parametrize("rank,buf_len", [(1, 4), (5, 12), (32, 64), (64, 8)])
+def test_ranks_and_window_lengths(kind, rank, buf_len):
+    w = synth.Workload("t", kind, 2, 3, 128, 64, rank, buf_len, 0, "bf16", 99, basis="qr")
+    check(run_schedule(w, buf_len + 3, max_heads=10**9), "bf16")
+
+
+@pytest.mark.parametrize("kind", synth.KINDS)
+@pytest.mark.parametrize("tune", [{"decode_stages": 1, "decode_batches_per_cta": 1},
+                                  {"decode_stages": 2, "decode_batches_per_cta": 64},
+                                  {"decode_stages": 2, "decode_batches_per_cta": 7}])
+def test_launch_tunings_and_ragged_batches(kind, tune):
+    w = synth.Workload("t", kind, 37, 3, 128, 128, 16, 16, 0, "bf16", 7, basis="qr")
+    check(run_schedule(w, 20, max_heads=10**9, tune=tune), "bf16")
+    check(run_schedule(w, 18, max_heads=10**9, mode="full_read", tune=tune), "bf16")
+
+
+def test_bf16_output_mode():
+    w = synth.Workload("t", "gdn", 4, 2, 128, 128, 16, 8, 0, "bf16", 5, basis="qr")
+    errs = run_schedule(w, 12, max_heads=10**9, out="bf16")
+    # a bf16-stored output carries its own rounding of 2^-8 relative on top of the arithmetic error
+    assert errs["out"] <= 2e-3 + 2.0 ** -8, errs
+    assert errs["S"] <= FP32_GUARD and errs["U"] <= FP32_GUARD
+
+
+# ---------------------------------------------------------------------------------------------
+# special cases the method has
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind", synth.KINDS)
+def test_identity_basis_gives_exact_read(kind):
+    """r = K, Omega = I, C = I: the sketch path equals the full-read path and the recurrence itself."""
+    from paper_2609_33051_b200.binding import SketchSSM
+    dev = _device()
+    w = synth.Workload("t", kind, 3, 2, 64, 64, 64, 8, 0, "f32", 31)
+    m = SketchSSM(kind, w.batch, w.heads, 64, 64, 64, 8, io="f32", device=0)
+    S0 = synth.initial_state(w)
+    eye = np.broadcast_to(np.eye(64, dtype=np.float32), (w.heads, 64, 64)).copy()
+    m.state.copy_(torch.from_numpy(S0)); m.omega.copy_(torch.from_numpy(eye)); m.coef.copy_(torch.from_numpy(eye))
+    m.state_update(0)
+    np.testing.assert_allclose(m.sketch.cpu().numpy(), S0, rtol=0, atol=1e-7)   # U[g, v] = S[g, v]
+    S = S0.astype(np.float64)
+    o1, o2 = m.new_output(), m.new_output()
+    for t in range(7):
+        x = synth.step_inputs(w, 0, t)
+        tt = harness.token_tensors(w, x, dev)
+        m.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o1, flags=1)   # NO_APPEND
+        m.full_read_decode(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o2)
+        S = orc.transition(kind, S, x["k"], x["v"], x["beta"], x["decay"])
+        ref = orc.exact_read(S, x["q"])
+        assert harness.rel_err(o1.cpu().numpy(), ref) <= 1e-5
+        assert harness.rel_err(o2.cpu().numpy(), ref) <= 1e-5
+    m.check_status()
+
+
+@pytest.mark.parametrize("kind", synth.KINDS)
+def test_replay_equals_single_token_updates_and_flags(kind):
+    """Replaying L buffered tokens equals L updates of one token; NO_SKETCH leaves U alone;
+    a replay without a current token (n_before = L) works; the ring holds what was appended."""
+    from paper_2609_33051_b200.binding import SketchSSM, NO_SKETCH
+    dev = _device()
+    w = synth.Workload("t", kind, 4, 3, 128, 64, 8, 8, 0, "bf16", 17, basis="qr")
+    ma, S0, Om, C, _ = make_layer(w)
+    mb, *_ = make_layer(w)
+    ma.state_update(0); mb.state_update(0)
+    o = ma.new_output()
+    toks = [harness.token_tensors(w, synth.step_inputs(w, 0, t), dev) for t in range(w.buf_len)]
+    for t, tt in enumerate(toks):                      # a: buffer all L tokens (decode steps), replay at once
+        ma.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o) if t < w.buf_len - 1 else None
+    # ring contents are exactly what was appended
+    rk, rv, rb, rd = ma.ring_views()
+    for t in range(w.buf_len - 1):
+        assert torch.equal(rk[:, :, t], toks[t]["k"]) and torch.equal(rv[:, :, t], toks[t]["v"])
+        assert torch.equal(rb[:, :, t], toks[t]["beta"]) and torch.equal(rd[:, :, t], toks[t]["decay"])
+    last = toks[-1]
+    sketch_before = ma.sketch.clone()
+    ma.state_update(w.buf_len - 1, last["q"], last["k"], last["v"], last["beta"], last["decay"], o, flags=NO_SKETCH)
+    assert torch.equal(ma.sketch, sketch_before)
+    ma.state_update(0)                                  # now refresh the sketch from the updated state
+    ob = mb.new_output()
+    for tt in toks:                                     # b: one-token updates ("standard" execution)
+        mb.state_update(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], ob)
+    assert harness.rel_err(ma.state.cpu().numpy(), mb.state.cpu().numpy().astype(np.float64)) <= 2e-5
+    assert harness.rel_err(ma.sketch.cpu().numpy(), mb.sketch.cpu().numpy().astype(np.float64)) <= 2e-5
+    assert harness.rel_err(o.cpu().numpy(), ob.cpu().numpy().astype(np.float64)) <= 2e-5
+    # c: replay a full ring without a current token
+    mc, *_ = make_layer(w)
+    mc.state_update(0)
+    w2 = w.replace(buf_len=8)
+    for t, tt in enumerate(toks[:-1]):
+        mc.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+    # append the last one by a decode step with n_before = L-1, then replay with n_before = L and no token
+    mc.decode_step(w.buf_len - 1, last["q"], last["k"], last["v"], last["beta"], last["decay"], o)
+    mc.state_update(w.buf_len)
+    assert harness.rel_err(mc.state.cpu().numpy(), mb.state.cpu().numpy().astype(np.float64)) <= 2e-5
+    for m in (ma, mb, mc):
+        m.check_status()
+
+
+@pytest.mark.parametrize("kind", synth.KINDS)
+def test_empty_buffer_output_is_U_C_q(kind):
+    """A token with beta = 0 and unit decay contributes nothing: o = U C q_t."""
+    dev = _device()
+    w = synth.Workload("t", kind, 3, 2, 128, 128, 16, 8, 0, "f32", 23, basis="qr")
+    m, S0, Om, C, _ = make_layer(w)
+    m.state_update(0)
+    x = synth.step_inputs(w, 0, 0)
+    x["beta"] = np.zeros_like(x["beta"]); x["decay"] = np.ones_like(x["decay"])
+    tt = harness.token_tensors(w, x, dev)
+    o = m.new_output()
+    m.decode_step(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+    U = orc.sketch_of(S0.astype(np.float64), Om.astype(np.float64)[None])
+    ref = np.einsum("bhvg,bhg->bhv", U, np.einsum("hgk,bhk->bhg", C.astype(np.float64), x["q"].astype(np.float64)))
+    assert harness.rel_err(o.cpu().numpy(), ref) <= 1e-5
+    m.check_status()
+
+
+def test_checkpoint_resume_mid_window():
+    """(S, ring, n) is the whole recurrent truth: restoring them and rebuilding U continues identically."""
+    dev = _device()
+    w = synth.Workload("t", "kda", 3, 2, 128, 128, 16, 8, 0, "bf16", 29, basis="qr")
+    ma, *_ = make_layer(w)
+    ma.state_update(0)
+    oa, ob = ma.new_output(), ma.new_output()
+    toks = [harness.token_tensors(w, synth.step_inputs(w, 0, t), dev) for t in range(8)]
+    for t in range(3):
+        tt = toks[t]
+        ma.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], oa)
+    mb, *_ = make_layer(w)
+    mb.state.copy_(ma.state); mb.ring.copy_(ma.ring)
+    mb.state_update(0)                                   # rebuild U from the restored state
+    for t in range(3, 8):
+        tt = toks[t]
+        for m, o in ((ma, oa), (mb, ob)):
+            if t < 7:
+                m.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+            else:
+                m.state_update(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+        assert torch.equal(oa, ob)
+    assert torch.equal(ma.state, mb.state) and torch.equal(ma.sketch, mb.sketch)
+
+
+def test_repeat_runs_are_bitwise_identical():
+    w = synth.CONFIGS["c3_gdn"].replace(batch=9, heads=2)
+    outs = []
+    for _ in range(2):
+        m, *_ = make_layer(w)
+        dev = _device()
+        m.state_update(0)
+        o = m.new_output()
+        for t in range(16):
+            tt = harness.token_tensors(w, synth.step_inputs(w, 0, t), dev)
+            if t < 15:
+                m.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+            else:
+                m.state_update(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+        outs.append((o.clone(), m.state.clone(), m.sketch.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
