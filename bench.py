@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the SketchSSM decode hot path on B200.
+
+One *step* is one window of Algorithm 1 over a stack of layers: for every layer, L-1 non-flush decode
+steps (sketchssm_decode_step) and one flush (sketchssm_state_update with the sketch refresh), over the
+whole batch of the workload.  The metric is decode tokens/s per layer:  B * L * n_layers / step time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With --impl reference the CPU oracle is timed on a bounded sample of the
+same workload instead.  Under torchrun (N > 1) every rank runs the same per-GPU workload (weak scaling,
+no data-path collective: heads are independent); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_33051_b200 import synth, traffic  # noqa: E402
+
+METRIC = "decode tokens/s per layer"
+UNIT = "tokens/s/layer"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (None until a capture of that kernel/workload exists)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    def __init__(self, device_index: int, period_s: float = 0.01):
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for name, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+# ---------------------------------------------------------------------------------------------
+# workload construction
+# ---------------------------------------------------------------------------------------------
+def fitted_basis(w: synth.Workload):
+    """Omega [H,K,r], C [H,r,K] float32 from the workload's calibration queries (E_0 = I)."""
+    from paper_2609_33051_b200 import calibrate
+    if w.basis == "qr":
+        Om = synth.qr_basis(w)
+        return Om, np.ascontiguousarray(np.swapaxes(Om, 1, 2))
+    Om = np.empty((w.heads, w.dk, w.rank), np.float32)
+    C = np.empty((w.heads, w.rank, w.dk), np.float32)
+    for h in range(w.heads):
+        O, Cm = calibrate.fit_head(torch.from_numpy(synth.calibration_queries(w, 0, h)), w.rank)
+        Om[h], C[h] = O.numpy().astype(np.float32), Cm.numpy().astype(np.float32)
+    return Om, C
+
+
+class Stack:
+    """n_layers independent layers of one workload on one GPU, with one window of device-resident inputs each."""
+
+    def __init__(self, w: synth.Workload, n_layers: int, device: int):
+        from paper_2609_33051_b200.binding import SketchSSM
+        self.w, self.n_layers, self.device = w, n_layers, device
+        dev = torch.device("cuda", device)
+        Om, C = fitted_basis(w)
+        S0 = torch.from_numpy(synth.initial_state(w, 0)).to(dev)
+        dec_io = w.io if w.kind == "kda" else "f32"
+        window = []
+        for t in range(w.buf_len):
+            x = synth.step_inputs(w, 0, t)
+            window.append(dict(q=synth.to_torch(x["q"], w.io, dev), k=synth.to_torch(x["k"], w.io, dev),
+                               v=synth.to_torch(x["v"], w.io, dev), beta=synth.to_torch(x["beta"], "f32", dev),
+                               decay=synth.to_torch(x["decay"], dec_io, dev)))
+        self.host_window = None
+        self.layers, self.inputs, self.outs = [], [], []
+        for _ in range(n_layers):
+            m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out="f32", device=device)
+            m.state.copy_(S0)
+            m.omega.copy_(torch.from_numpy(Om))
+            m.coef.copy_(torch.from_numpy(C))
+            m.state_update(0)
+            self.layers.append(m)
+            # every layer gets its own copy of the window so that no input is served from L2 across layers
+            self.inputs.append([{k: v.clone() for k, v in tok.items()} for tok in window])
+            self.outs.append(m.new_output())
+        self.window0 = window
+        torch.cuda.synchronize(dev)
+
+    def device_bytes(self) -> int:
+        m = self.layers[0]
+        per = m.state.numel() * 4 + m.sketch.numel() * 4 + m.ring.numel()
+        per += sum(v.numel() * v.element_size() for tok in self.inputs[0] for v in tok.values())
+        return per * self.n_layers
+
+    def run_window(self, mode: str = "sketch", events=None):
+        """One step: L tokens through every layer.  mode: "sketch" (decode_step + state_update) or
+        "full_read" (full_read_decode + state_update without the sketch write).  `events`, if given, receives
+        (kind, n_before, start_event, end_event) per launch."""
+        from paper_2609_33051_b200.binding import NO_SKETCH
+        L = self.w.buf_len
+        launches = 0
+        for t in range(L):
+            for li, m in enumerate(self.layers):
+                tok, o = self.inputs[li][t], self.outs[li]
+                if events is not None:
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                if t < L - 1:
+                    if mode == "sketch":
+                        m.decode_step(t, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], o)
+                    else:
+                        m.full_read_decode(t, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], o)
+                else:
+                    m.state_update(t, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], o,
+                                   flags=0 if mode == "sketch" else NO_SKETCH)
+                launches += m.last_launch_count()
+                if events is not None:
+                    e1.record()
+                    events.append(("decode" if t < L - 1 else "update", t, e0, e1))
+        return launches
+
+    # -- end-to-end: host buffers, copies inside the timed region ---------------------------------
+    def setup_host(self):
+        m = self.layers[0]
+        self.host_window = []
+        for tok in self.window0:
+            hb = m.new_token_buffers(pinned_host=True)
+            for k in ("q", "k", "v", "beta", "decay"):
+                hb[k].copy_(tok[k])
+            self.host_window.append(hb)
+        self.staging = [m.new_token_buffers(pinned_host=False) for _ in range(2)]
+
+    def run_window_host(self):
+        from paper_2609_33051_b200 import binding
+        L = self.w.buf_len
+        h2d = d2h = 0
+        i = 0
+        for t in range(L):
+            hb = self.host_window[t]
+            for m in self.layers:
+                op = binding.OP_DECODE if t < L - 1 else binding.OP_UPDATE
+                m.step_host(op, t, hb, self.staging[i & 1])
+                i += 1
+                h2d += sum(hb[k].numel() * hb[k].element_size() for k in ("q", "k", "v", "beta", "decay"))
+                d2h += hb["out"].numel() * hb["out"].element_size()
+        return h2d, d2h
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------------------------
+def oracle_window(w: synth.Workload, sample_heads: int, reps: int = 1):
+    """Time the oracle, as it stands, on one window of `sample_heads` heads of the workload.
+    Returns (seconds per window, head-steps per window, threads used)."""
+    from oracle import sketchssm_oracle as orc
+    total = w.batch * w.heads
+    idx = np.sort(np.random.default_rng(1).choice(total, size=min(sample_heads, total), replace=False))
+    bs, hs = idx // w.heads, idx % w.heads
+    Om, C = fitted_basis(w.replace(heads=w.heads))
+    Om_s, C_s = Om[hs].astype(np.float64), C[hs].astype(np.float64)
+    S = synth.initial_state(w.replace(batch=min(w.batch, 8)), 0)
+    bsel = bs % S.shape[0]
+    S0 = S[bsel, hs].astype(np.float64)
+    toks, qs = [], []
+    for t in range(w.buf_len):
+        x = synth.step_inputs(w, 0, t)
+        toks.append(tuple(x[n][bs, hs].astype(np.float64) for n in ("k", "v", "beta", "decay")))
+        qs.append(x["q"][bs, hs].astype(np.float64))
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        orc.run_schedule(w.kind, S0, Om_s, C_s, toks, qs, w.buf_len)
+        times.append(time.perf_counter() - t0)
+    return times, len(bs) * w.buf_len, 1
+
+
+# ---------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_mamba2")
+    ap.add_argument("--layers", type=int, default=8, help="layer copies in the stack (distinct memory)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch")
+    ap.add_argument("--buf-len", type=int, default=0)
+    ap.add_argument("--rank", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-launch-events", action="store_true", help="do not bracket every launch with events")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-full-read", action="store_true")
+    ap.add_argument("--tune", default="", help="comma list key=value passed to sketchssm_tune")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    w = synth.CONFIGS[args.workload]
+    if args.batch or args.buf_len or args.rank:
+        w = w.replace(batch=args.batch or w.batch, buf_len=args.buf_len or w.buf_len, rank=args.rank or w.rank)
+    cfg = {"workload": f"{w.name}: {w.kind} B{w.batch} H{w.heads} K{w.dk} V{w.dv} r{w.rank} L{w.buf_len} "
+                       f"{w.io} I/O, fp32 state/sketch", "layers": args.layers,
+           "schedule": "per layer and window: L-1 decode_step + 1 state_update(+sketch)"}
+
+    # ----------------------------------------------------------------------------------------
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        sample = 64
+        times, head_steps, cores = oracle_window(w, sample, reps=args.warmup + args.steps)
+        timed = times[args.warmup:]
+        sec = sum(timed) / len(timed)
+        value = head_steps / sec / w.heads
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                 "sample": f"{sample} (batch, head) pairs x one window of {w.buf_len} tokens per step; "
+                                           f"rate scaled to a layer of {w.heads} heads"},
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    # ----------------------------------------------------------------------------------------
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    from paper_2609_33051_b200 import build as _build
+    if not os.path.exists(_build.LIB_PATH):
+        _build.build()
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    stack = Stack(w, args.layers, local_rank)
+    for kv in filter(None, args.tune.split(",")):
+        k, v = kv.split("=")
+        for m in stack.layers:
+            m.tune(k, int(v))
+    L, B, H = w.buf_len, w.batch, w.heads
+    tokens_per_step = B * L * args.layers
+    cfg.update({"device_bytes": stack.device_bytes(), "l2": "inputs larger than L2: every layer has its own state, "
+                "sketch, ring and token tensors; %.1f GB touched between re-uses" % (stack.device_bytes() / 1e9),
+                "per_kernel_timing": "second timed pass of the same launches with CUDA events around every launch "
+                                     "(bracketing costs a few % of step time, so the headline pass has none)"})
+
+    def timed_region(fn, steps, warmup, sampler=None):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        if sampler is not None:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        out = None
+        for _ in range(steps):
+            out = fn()
+        e1.record()
+        barrier()
+        clocks = sampler.stop() if sampler is not None else None
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / steps, out, clocks
+
+    # ---- device-resident timing (the headline value): no events between launches ----
+    launches_per_step = [0]
+
+    def step():
+        launches_per_step[0] = stack.run_window("sketch", None)
+
+    ms_step, _, clocks = timed_region(step, args.steps, args.warmup, ClockSampler(local_rank))
+    for m in stack.layers:
+        m.check_status()
+    value = world * tokens_per_step / (ms_step * 1e-3)
+
+    # ---- the same region again with every launch bracketed by events: per-kernel durations ----
+    events = None if args.no_launch_events else []
+    ms_step_instrumented = None
+    if events is not None:
+        ms_step_instrumented, _, _ = timed_region(lambda: stack.run_window("sketch", events),
+                                                  max(3, args.steps // 2), 1)
+
+    # ---- per-kernel durations and roofline of the dominant kernel ----
+    peak, peak_kind = measured_peaks()
+    kern = {}
+    if events:
+        agg = {"decode": [0.0, 0, 0], "update": [0.0, 0, 0]}            # ms, launches, bytes
+        for kind, t, a, b in events:
+            agg[kind][0] += a.elapsed_time(b)
+            agg[kind][1] += 1
+            agg[kind][2] += (traffic.decode_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io) if kind == "decode"
+                             else traffic.update_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io))
+        for kind, (ms, n, by) in agg.items():
+            if n:
+                kern[kind] = {"launches": n, "avg_us": 1e3 * ms / n, "share": ms / (agg["decode"][0] + agg["update"][0]),
+                              "algorithmic_bytes_per_launch": by / n, "achieved_gbs": by / (ms * 1e-3) / 1e9}
+    dominant = max(kern, key=lambda k: kern[k]["share"]) if kern else None
+    roofline = None
+    if dominant:
+        kname = "decode_kernel" if dominant == "decode" else "update_kernel"
+        roofline = {"bound": "hbm", "kernel": kname, "achieved": kern[dominant]["achieved_gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": kern[dominant]["achieved_gbs"] / peak, "peak_source": peak_kind,
+                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((kname, w.name)),
+                    "frac_of_8TBs_nominal": kern[dominant]["achieved_gbs"] / 8000.0}
+
+    # ---- in-library full-read baseline (buffered replay that reads all of S every step) ----
+    full = None
+    if not args.skip_full_read:
+        ms_full, _, _ = timed_region(lambda: stack.run_window("full_read", None), max(3, args.steps // 4), 3)
+        full = {"value": world * tokens_per_step / (ms_full * 1e-3), "unit": UNIT, "ms_per_step": ms_full,
+                "what": "sketchssm_full_read_decode x (L-1) + sketchssm_state_update(NO_SKETCH) per layer and window",
+                "sketch_speedup": ms_full / ms_step}
+        stack.run_window("sketch", None)     # leave a fresh sketch behind
+
+    # ---- end to end through the C ABI with host buffers ----
+    e2e = None
+    if not args.skip_e2e:
+        stack.setup_host()
+        bytes_io = [0, 0]
+
+        def host_step():
+            bytes_io[0], bytes_io[1] = stack.run_window_host()
+
+        ms_e2e, _, _ = timed_region(host_step, args.e2e_steps, 3)
+        e2e = {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io[0],
+               "d2h_bytes_per_step": bytes_io[1], "ms_per_step": ms_e2e, "steps": args.e2e_steps,
+               "what": "sketchssm_step_host per layer-step: pinned host q,k,v,beta,decay -> device, kernel, o -> host"}
+    for m in stack.layers:
+        m.check_status()
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu_baseline:
+        probe, head_steps, cores = oracle_window(w, 512, reps=1)
+        sample = int(min(w.batch * w.heads, max(512, 512 * 12.0 / max(probe[0], 1e-3))))
+        times, head_steps, cores = oracle_window(w, sample, reps=1)
+        cpu = {"value": head_steps / times[0] / H, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "seconds": times[0],
+               "sample": f"{sample} (batch, head) pairs x one window of {L} tokens (L-1 decode steps + 1 state "
+                         f"update), fp64 NumPy; rate scaled to a layer of {H} heads"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
+                "e2e": e2e, "gpu_launches": launches_per_step[0] * args.steps, "roofline": roofline,
+                "kernels": kern, "ms_per_step_with_launch_events": ms_step_instrumented, "full_read_baseline": full, "cpu_baseline": cpu,
+                "per_gpu_heads": B * H}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -149,6 +149,24 @@ int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, 
                                const void* v, const void* beta, const void* decay, void* out,
                                uint32_t flags, void* stream);
 
+/* Device staging for one step's token tensors, caller-owned, same shapes/dtypes as the token
+ * arguments of the hot-path calls (q,k [B][H][K] io; v [B][H][V] io; beta [B][H] fp32; decay;
+ * out [B][H][V]).  Used only by sketchssm_step_host. */
+typedef struct sketchssm_staging {
+    void *q, *k, *v, *beta, *decay, *out;
+} sketchssm_staging;
+
+enum sketchssm_op { SKETCHSSM_OP_DECODE = 0, SKETCHSSM_OP_FULL_READ = 1, SKETCHSSM_OP_UPDATE = 2 };
+
+/* One step of Algorithm 1 with HOST token tensors: enqueue on `stream` the host->device copies of
+ * q, k, v, beta, decay into `staging`, the chosen hot-path call (decode step, full-read decode, or
+ * state update with the token and the exact output), and the device->host copy of the output into
+ * `host_out`.  Host buffers should be page-locked for the copies to be asynchronous; they must stay
+ * valid until the stream has passed this step.  Same n_before / flags rules as the underlying call. */
+int sketchssm_step_host(sketchssm_ctx* ctx, int op, int n_before, const void* host_q, const void* host_k,
+                        const void* host_v, const void* host_beta, const void* host_decay, void* host_out,
+                        const sketchssm_staging* staging, uint32_t flags, void* stream);
+
 /* Copy the status word back (synchronises `stream`).  Returns SKETCHSSM_OK if no kernel
  * recorded a fault, SKETCHSSM_DEVICE_TIMEOUT otherwise; `detail`, if not NULL, receives the
  * four status ints. */

@@ -25,8 +25,9 @@ EXPORTED = (
     "sketchssm_create", "sketchssm_destroy", "sketchssm_query_sizes", "sketchssm_bind",
     "sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode",
     "sketchssm_read_status", "sketchssm_last_launch_count", "sketchssm_tune",
-    "sketchssm_status_string", "sketchssm_version", "sketchssm_last_cuda_error",
+    "sketchssm_status_string", "sketchssm_version", "sketchssm_last_cuda_error", "sketchssm_step_host",
 )
+OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 
 
 class Config(ctypes.Structure):
@@ -42,6 +43,10 @@ class Sizes(ctypes.Structure):
 
 class Buffers(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status")]
+
+
+class Staging(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("q", "k", "v", "beta", "decay", "out")]
 
 
 class SketchSSMError(RuntimeError):
@@ -70,6 +75,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sketchssm_bind.argtypes = [vp, ctypes.POINTER(Buffers)]
     for name in ("sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode"):
         getattr(lib, name).argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u32, vp]
+    lib.sketchssm_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.POINTER(Staging), u32, vp]
     lib.sketchssm_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32 * 4), vp]
     lib.sketchssm_last_launch_count.argtypes = [vp]
     lib.sketchssm_tune.argtypes = [vp, ctypes.c_char_p, i32]
@@ -190,6 +196,27 @@ class SketchSSM:
                                                  _ptr(decay), _ptr(out), flags, self._stream(stream))
         self._check("sketchssm_full_read_decode", rc)
         return out
+
+    def new_token_buffers(self, pinned_host: bool = False):
+        """Empty q, k, v, beta, decay, out tensors of the C ABI's shapes: on the device, or page-locked host."""
+        iod = TORCH_DTYPE[self.io]
+        kw = dict(device="cpu", pin_memory=True) if pinned_host else dict(device=self.device)
+        dec = (torch.empty(self.B, self.H, self.K, dtype=iod, **kw) if self.kind == "kda"
+               else torch.empty(self.B, self.H, dtype=torch.float32, **kw))
+        return dict(q=torch.empty(self.B, self.H, self.K, dtype=iod, **kw),
+                    k=torch.empty(self.B, self.H, self.K, dtype=iod, **kw),
+                    v=torch.empty(self.B, self.H, self.V, dtype=iod, **kw),
+                    beta=torch.empty(self.B, self.H, dtype=torch.float32, **kw), decay=dec,
+                    out=torch.empty(self.B, self.H, self.V, dtype=TORCH_DTYPE[self.out], **kw))
+
+    def step_host(self, op: int, n_before: int, host: dict, staging: dict, flags: int = 0, stream=None):
+        """sketchssm_step_host: host token tensors in, host output out, copies and kernel on one stream."""
+        st = Staging(*[staging[n].data_ptr() for n in ("q", "k", "v", "beta", "decay", "out")])
+        rc = self.lib.sketchssm_step_host(self._ctx, op, n_before, _ptr(host["q"]), _ptr(host["k"]), _ptr(host["v"]),
+                                          _ptr(host["beta"]), _ptr(host["decay"]), _ptr(host["out"]),
+                                          ctypes.byref(st), flags, self._stream(stream))
+        self._check("sketchssm_step_host", rc)
+        return host["out"]
 
     def read_status(self, stream=None):
         detail = (ctypes.c_int32 * 4)()

@@ -181,6 +181,41 @@ int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, 
     return decode_common(ctx, 1, n_before, q, k, v, beta, decay, out, flags, stream);
 }
 
+int sketchssm_step_host(sketchssm_ctx* ctx, int op, int n_before, const void* hq, const void* hk, const void* hv,
+                        const void* hbeta, const void* hdecay, void* hout, const sketchssm_staging* st,
+                        uint32_t flags, void* stream) {
+    if (ctx == nullptr || st == nullptr) return SKETCHSSM_INVALID_ARG;
+    if (op < SKETCHSSM_OP_DECODE || op > SKETCHSSM_OP_UPDATE) return SKETCHSSM_INVALID_ARG;
+    if (hq == nullptr || hk == nullptr || hv == nullptr || hbeta == nullptr || hdecay == nullptr || hout == nullptr)
+        return SKETCHSSM_INVALID_ARG;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    int rc = check_token_ptrs(st->q, st->k, st->v, st->beta, st->decay, st->out);
+    if (rc != SKETCHSSM_OK) return rc;
+    rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    const sketchssm_config& c = ctx->cfg;
+    const size_t bh = (size_t)c.batch * c.heads;
+    const size_t qk_bytes = bh * c.dk * ctx->io_size, v_bytes = bh * c.dv * ctx->io_size;
+    const size_t dec_bytes = c.kind == SKETCHSSM_KDA ? qk_bytes : bh * 4;
+    const size_t out_bytes = bh * c.dv * (c.out_dtype == SKETCHSSM_BF16 ? 2 : 4);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(st->q, hq, qk_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(st->k, hk, qk_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(st->v, hv, v_bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(st->beta, hbeta, bh * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(st->decay, hdecay, dec_bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) { ctx->last_cuda_error = e; return SKETCHSSM_CUDA_ERROR; }
+    if (op == SKETCHSSM_OP_UPDATE)
+        rc = sketchssm_state_update(ctx, n_before, st->q, st->k, st->v, st->beta, st->decay, st->out, flags, stream);
+    else
+        rc = decode_common(ctx, op == SKETCHSSM_OP_FULL_READ, n_before, st->q, st->k, st->v, st->beta, st->decay,
+                           st->out, flags, stream);
+    if (rc != SKETCHSSM_OK) return rc;
+    e = cudaMemcpyAsync(hout, st->out, out_bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) { ctx->last_cuda_error = e; return SKETCHSSM_CUDA_ERROR; }
+    return SKETCHSSM_OK;
+}
+
 int sketchssm_read_status(sketchssm_ctx* ctx, int32_t detail[4], void* stream) {
     if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
     if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
