@@ -89,6 +89,7 @@ typedef struct sketchssm_config {
 typedef struct sketchssm_sizes {
     size_t state_bytes, sketch_bytes, ring_bytes, omega_bytes, coef_bytes;
     size_t status_bytes;     /* size of the status word block (16) */
+    size_t work_bytes;       /* per-head weight hand-off between the two decode kernels: B*H*(K+L) floats */
     size_t ring_head_bytes;  /* stride of one (b, h) ring block */
     size_t ring_v_offset, ring_beta_offset, ring_decay_offset; /* byte offsets inside a ring block (k is at 0) */
     size_t alignment;        /* required alignment of every pointer (16) */
@@ -103,6 +104,9 @@ typedef struct sketchssm_buffers {
     void* status;  /* int32[4], zero-initialised by the caller: [0] first device fault code
                       (0 = none), [1] which wait, [2..3] reserved.  Kernels only ever write
                       non-zero codes; sketchssm_read_status reads it back. */
+    void* work;    /* work_bytes of scratch for the decode calls (contents are transient: written and
+                      consumed inside one call; calls that overlap on the GPU need separate contexts
+                      with separate work buffers) */
 } sketchssm_buffers;
 
 typedef struct sketchssm_ctx sketchssm_ctx; /* host-only metadata; owns no device memory */
@@ -116,7 +120,7 @@ int sketchssm_destroy(sketchssm_ctx* ctx);
 /* Byte sizes and ring sub-offsets for this configuration.  Host-only. */
 int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out);
 
-/* Record the caller's device buffers (all six required, 16-byte aligned).  The context
+/* Record the caller's device buffers (all seven required, 16-byte aligned).  The context
  * stores the pointers only; the caller keeps ownership and must keep them alive. */
 int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* bufs);
 
@@ -144,7 +148,9 @@ int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const
                           uint32_t flags, void* stream);
 
 /* Exact decode step that reads the whole state: o = S_0^T q~_t + sum_s a_s v_s (Eq. 4).
- * Same arguments and ring behaviour as sketchssm_decode_step; U and C are not read. */
+ * Same arguments and ring behaviour as sketchssm_decode_step; U and C are not read.
+ * Both decode calls run as two kernels: the first forms the buffer weights a_s and the coefficients
+ * (c_t, or q~_t for the full read) into `work`, the second forms the weighted sum of rows. */
 int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
                                const void* v, const void* beta, const void* decay, void* out,
                                uint32_t flags, void* stream);
@@ -180,7 +186,10 @@ int sketchssm_last_launch_count(const sketchssm_ctx* ctx);
 
 /* Optional launch tuning, host-only.  Keys: "decode_batches_per_cta" (batch entries one CTA of
  * the decode kernels serves for its head; 0 = library default), "decode_stages" (1 or 2 shared-memory
- * stages per warp; 0 = library default).  Results never depend on these. */
+ * stages per lane group; 0 = library default), "decode_warps_per_cta", "decode_max_warps_per_sm",
+ * "decode_lanes_per_head", "decode_l2_prefetch", "decode_impl" (0 = two kernels, the default; 1 = one fused
+ * kernel with a warp per head; 2 = one fused kernel with 8 or 16 lanes per head).  Results depend on these
+ * only through floating-point summation order. */
 int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value);
 
 const char* sketchssm_status_string(int status);

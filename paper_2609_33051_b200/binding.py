@@ -38,11 +38,11 @@ class Config(ctypes.Structure):
 class Sizes(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("state_bytes", "sketch_bytes", "ring_bytes", "omega_bytes", "coef_bytes", "status_bytes",
-                 "ring_head_bytes", "ring_v_offset", "ring_beta_offset", "ring_decay_offset", "alignment")]
+                 "work_bytes", "ring_head_bytes", "ring_v_offset", "ring_beta_offset", "ring_decay_offset", "alignment")]
 
 
 class Buffers(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status", "work")]
 
 
 class Staging(ctypes.Structure):
@@ -115,7 +115,7 @@ class SketchSSM:
         self._check("sketchssm_create", self.lib.sketchssm_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.sizes = Sizes()
         self._check("sketchssm_query_sizes", self.lib.sketchssm_query_sizes(self._ctx, ctypes.byref(self.sizes)))
-        self.state = self.sketch = self.ring = self.omega = self.coef = self.status = None
+        self.state = self.sketch = self.ring = self.omega = self.coef = self.status = self.work = None
         if allocate:
             self.allocate()
 
@@ -128,6 +128,7 @@ class SketchSSM:
         self.omega = torch.zeros(self.H, self.K, self.R, dtype=torch.float32, device=d)
         self.coef = torch.zeros(self.H, self.R, self.K, dtype=torch.float32, device=d)
         self.status = torch.zeros(4, dtype=torch.int32, device=d)
+        self.work = torch.zeros(self.sizes.work_bytes // 4, dtype=torch.float32, device=d)
         self.bind()
 
     def bind(self):
@@ -135,7 +136,7 @@ class SketchSSM:
         assert self.sketch.numel() * 4 == self.sizes.sketch_bytes
         assert self.ring.numel() == self.sizes.ring_bytes
         b = Buffers(self.state.data_ptr(), self.sketch.data_ptr(), self.ring.data_ptr(),
-                    self.omega.data_ptr(), self.coef.data_ptr(), self.status.data_ptr())
+                    self.omega.data_ptr(), self.coef.data_ptr(), self.status.data_ptr(), self.work.data_ptr())
         self._check("sketchssm_bind", self.lib.sketchssm_bind(self._ctx, ctypes.byref(b)))
 
     def close(self):

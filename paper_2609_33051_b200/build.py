@@ -10,8 +10,14 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsketchssm.so")
-SOURCES = ["api.cu", "decode.cu", "update.cu"]
-HEADERS = [os.path.join(CSRC, "internal.cuh"), os.path.join(ROOT, "include", "sketchssm.h")]
+# (source, object suffix, extra defines); the lane-group decode kernel is compiled once per (recurrence kind, I/O type)
+UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []),
+         *[("decode_fused.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
+           for k in range(3) for io in range(2)],
+         *[("decode_split.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
+           for k in range(3) for io in range(2)]]
+HEADERS = [os.path.join(CSRC, "internal.cuh"), os.path.join(CSRC, "lanegroup.cuh"),
+           os.path.join(ROOT, "include", "sketchssm.h")]
 
 
 def _nvcc() -> str:
@@ -38,12 +44,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         flags += ["-Xptxas", "-v"]
     procs, objs = [], []
-    for src in SOURCES:
+    for src, suffix, defs in UNITS:
         sp = os.path.join(CSRC, src)
-        obj = os.path.join(objdir, src.replace(".cu", ".o"))
+        obj = os.path.join(objdir, src.replace(".cu", suffix + ".o"))
         objs.append(obj)
         if force or _stale(obj, [sp] + HEADERS):
-            procs.append((src, subprocess.Popen([nvcc, *flags, "-c", sp, "-o", obj],
+            procs.append((src + suffix, subprocess.Popen([nvcc, *flags, *defs, "-c", sp, "-o", obj],
                                                 stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     for src, pr in procs:
         out, _ = pr.communicate()

@@ -8,6 +8,11 @@ using namespace sketchssm;
 struct sketchssm_ctx : public Ctx {
     int tune_batches_per_cta;
     int tune_stages;
+    int tune_warps_per_cta;
+    int tune_lanes_per_head;
+    int tune_decode_impl;   // 0: two kernels (weights + output rows), 1: warp-per-head kernel, 2: fused lane-group kernel
+    int tune_max_warps;
+    int tune_l2_prefetch;   // lane-group kernel: 1 (default) / 0
 };
 
 namespace {
@@ -40,12 +45,18 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.omega = static_cast<const float*>(ctx->bufs.omega);
     p.coef = static_cast<const float*>(ctx->bufs.coef);
     p.status = static_cast<int*>(ctx->bufs.status);
+    p.work = static_cast<float*>(ctx->bufs.work);
+    p.wstride = ctx->cfg.dk + ctx->cfg.buf_len;
     p.rl = ctx->ring;
     p.B = ctx->cfg.batch; p.H = ctx->cfg.heads; p.R = ctx->cfg.rank; p.L = ctx->cfg.buf_len;
     p.dk = ctx->cfg.dk; p.dv = ctx->cfg.dv;
     p.out_bf16 = ctx->cfg.out_dtype == SKETCHSSM_BF16;
     p.batches_per_cta = ctx->tune_batches_per_cta;
     p.stages = ctx->tune_stages;
+    p.warps_per_cta = ctx->tune_warps_per_cta;
+    p.lanes_per_head = ctx->tune_lanes_per_head;
+    p.l2_prefetch = ctx->tune_l2_prefetch;
+    p.max_warps_per_sm = ctx->tune_max_warps;
     return p;
 }
 
@@ -73,7 +84,27 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     p.has_token = 1;
     p.append = (flags & SKETCHSSM_NO_APPEND) ? 0 : 1;
     p.full_read = full_read;
-    return launch_decode(ctx, p, static_cast<cudaStream_t>(stream));
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
+    if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
+    if (ctx->tune_decode_impl == 2) {
+        switch (ctx->cfg.kind) {
+            case SKETCHSSM_MAMBA2:
+                return bf ? launch_decode_group_mamba2_bf16(ctx, p, cs) : launch_decode_group_mamba2_f32(ctx, p, cs);
+            case SKETCHSSM_GDN:
+                return bf ? launch_decode_group_gdn_bf16(ctx, p, cs) : launch_decode_group_gdn_f32(ctx, p, cs);
+            default:
+                return bf ? launch_decode_group_kda_bf16(ctx, p, cs) : launch_decode_group_kda_f32(ctx, p, cs);
+        }
+    }
+    switch (ctx->cfg.kind) {
+        case SKETCHSSM_MAMBA2:
+            return bf ? launch_decode_split_mamba2_bf16(ctx, p, cs) : launch_decode_split_mamba2_f32(ctx, p, cs);
+        case SKETCHSSM_GDN:
+            return bf ? launch_decode_split_gdn_bf16(ctx, p, cs) : launch_decode_split_gdn_f32(ctx, p, cs);
+        default:
+            return bf ? launch_decode_split_kda_bf16(ctx, p, cs) : launch_decode_split_kda_f32(ctx, p, cs);
+    }
 }
 
 }  // namespace
@@ -103,6 +134,11 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     c->last_cuda_error = cudaSuccess;
     c->tune_batches_per_cta = 0;
     c->tune_stages = 0;
+    c->tune_warps_per_cta = 0;
+    c->tune_lanes_per_head = 0;
+    c->tune_decode_impl = 1;
+    c->tune_l2_prefetch = 1;
+    c->tune_max_warps = 0;
     *out = c;
     return SKETCHSSM_OK;
 }
@@ -123,6 +159,7 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
     out->omega_bytes = (size_t)c.heads * c.dk * c.rank * 4;
     out->coef_bytes = (size_t)c.heads * c.rank * c.dk * 4;
     out->status_bytes = kStatusInts * sizeof(int32_t);
+    out->work_bytes = bh * (size_t)(c.dk + c.buf_len) * 4;
     out->ring_head_bytes = ctx->ring.head_bytes;
     out->ring_v_offset = ctx->ring.v_off;
     out->ring_beta_offset = ctx->ring.beta_off;
@@ -133,7 +170,7 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
 
 int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* b) {
     if (ctx == nullptr || b == nullptr) return SKETCHSSM_INVALID_ARG;
-    const void* ps[6] = {b->state, b->sketch, b->ring, b->omega, b->coef, b->status};
+    const void* ps[7] = {b->state, b->sketch, b->ring, b->omega, b->coef, b->status, b->work};
     for (const void* p : ps) {
         if (p == nullptr || !aligned16(p)) return SKETCHSSM_INVALID_ARG;
     }
@@ -246,6 +283,11 @@ int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value) {
     };
     if (eq(key, "decode_batches_per_cta")) { ctx->tune_batches_per_cta = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_stages")) { ctx->tune_stages = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_warps_per_cta")) { ctx->tune_warps_per_cta = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_lanes_per_head")) { ctx->tune_lanes_per_head = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_l2_prefetch")) { ctx->tune_l2_prefetch = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_max_warps_per_sm")) { ctx->tune_max_warps = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_impl")) { ctx->tune_decode_impl = value; return SKETCHSSM_OK; }
     return SKETCHSSM_INVALID_ARG;
 }
 

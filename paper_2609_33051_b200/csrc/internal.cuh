@@ -49,6 +49,8 @@ struct Params {
     const float* omega;
     const float* coef;
     int* status;
+    float* work;        // [B][H][wstride]: per-head weights handed from the decode weights kernel to the output kernel
+    int wstride;        // dk + buf_len floats: [0, dk) coefficients c (or q~), [dk + s] buffer weight a_s
     RingLayout rl;
     int B, H, R, L;
     int dk, dv;
@@ -61,9 +63,27 @@ struct Params {
     int full_read;   // decode: read S instead of U, C
     int batches_per_cta;
     int stages;
+    int warps_per_cta;   // decode: 0 = library default
+    int lanes_per_head;  // decode (group kernel): 8 or 16; 0 = library default
+    int l2_prefetch;     // decode (group kernel): request the following item's operands into L2
+    int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
 };
 
-int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head
+// 8 or 16 lanes per head, one entry per recurrence kind
+// decode as two kernels (weights, then output rows), one entry per (kind, I/O type)
+int launch_decode_split_mamba2_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_split_mamba2_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_split_gdn_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_split_gdn_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_split_kda_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_split_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_group_mamba2_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_group_mamba2_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_group_gdn_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_group_gdn_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_group_kda_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_decode_group_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------

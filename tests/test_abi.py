@@ -77,6 +77,7 @@ def test_sizes_and_ring_layout(lib, kind, io, K, V, L, expect_head):
     assert s.ring_beta_offset == s.ring_v_offset + L * V * esz
     assert s.ring_decay_offset == s.ring_beta_offset + L * 4
     assert s.alignment == 16 and s.status_bytes == 16
+    assert s.work_bytes == 15 * (K + L) * 4
     for off in (s.ring_head_bytes, s.ring_v_offset, s.ring_beta_offset, s.ring_decay_offset):
         assert off % 16 == 0
     lib.sketchssm_destroy(ctx)
@@ -88,11 +89,11 @@ def test_calls_are_rejected_before_bind_and_on_bad_arguments(lib):
     assert lib.sketchssm_decode_step(ctx, 0, dummy, dummy, dummy, dummy, dummy, dummy, 0, None) == -3
     assert lib.sketchssm_state_update(ctx, 0, None, None, None, None, None, None, 0, None) == -3
     assert lib.sketchssm_read_status(ctx, None, None) == -3
-    bufs = binding.Buffers(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0)
+    bufs = binding.Buffers(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0, 0x7000)
     assert lib.sketchssm_bind(ctx, ctypes.byref(bufs)) == -1            # null status
-    bufs = binding.Buffers(0x1000, 0x2000, 0x3008, 0x4000, 0x5000, 0x6000)
+    bufs = binding.Buffers(0x1000, 0x2000, 0x3008, 0x4000, 0x5000, 0x6000, 0x7000)
     assert lib.sketchssm_bind(ctx, ctypes.byref(bufs)) == -1            # misaligned ring
-    bufs = binding.Buffers(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000)
+    bufs = binding.Buffers(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000)
     assert lib.sketchssm_bind(ctx, ctypes.byref(bufs)) == 0
     # argument checks happen on the host before any CUDA call
     assert lib.sketchssm_decode_step(ctx, 16, dummy, dummy, dummy, dummy, dummy, dummy, 0, None) == -1   # n_before > L-1

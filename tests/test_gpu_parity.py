@@ -69,7 +69,7 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32"):
             m.state_update(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
             S, U, ref = orc.state_update(w.kind, S, ring, Om_s, q)
             ring = []
-        assert m.last_launch_count() == 1
+        assert m.last_launch_count() in (1, 2)   # the two-kernel decode launches twice
         got = o_dev.float().cpu().numpy()[bs, hs]
         assert np.all(np.isfinite(got))
         worst = max(worst, harness.rel_err(got, ref))
@@ -129,9 +129,13 @@ def test_ranks_and_window_lengths(kind, rank, buf_len):
 
 
 @pytest.mark.parametrize("kind", synth.KINDS)
-@pytest.mark.parametrize("tune", [{"decode_stages": 1, "decode_batches_per_cta": 1},
-                                  {"decode_stages": 2, "decode_batches_per_cta": 64},
-                                  {"decode_stages": 2, "decode_batches_per_cta": 7}])
+@pytest.mark.parametrize("tune", [{"decode_impl": 1, "decode_stages": 1, "decode_batches_per_cta": 1},
+                                  {"decode_impl": 1, "decode_stages": 2, "decode_batches_per_cta": 7},
+                                  {"decode_impl": 2, "decode_stages": 1, "decode_warps_per_cta": 1},
+                                  {"decode_impl": 2, "decode_stages": 2, "decode_warps_per_cta": 3},
+                                  {"decode_impl": 2, "decode_l2_prefetch": 0},
+                                  {"decode_impl": 0, "decode_stages": 2, "decode_warps_per_cta": 2},
+                                  {"decode_impl": 0, "decode_stages": 1, "decode_max_warps_per_sm": 4}])
 def test_launch_tunings_and_ragged_batches(kind, tune):
     w = synth.Workload("t", kind, 37, 3, 128, 128, 16, 16, 0, "bf16", 7, basis="qr")
     check(run_schedule(w, 20, max_heads=10**9, tune=tune), "bf16")
