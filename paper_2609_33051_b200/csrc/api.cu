@@ -12,6 +12,7 @@ struct sketchssm_ctx : public Ctx {
     int tune_lanes_per_head;
     int tune_decode_impl;   // 0: two kernels (weights + output rows), 1: warp-per-head kernel, 2: fused lane-group kernel
     int tune_max_warps;
+    int tune_update_impl;
     int tune_l2_prefetch;   // lane-group kernel: 1 (default) / 0
 };
 
@@ -57,6 +58,7 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.lanes_per_head = ctx->tune_lanes_per_head;
     p.l2_prefetch = ctx->tune_l2_prefetch;
     p.max_warps_per_sm = ctx->tune_max_warps;
+    p.update_impl = ctx->tune_update_impl;
     return p;
 }
 
@@ -139,6 +141,7 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     c->tune_decode_impl = 1;
     c->tune_l2_prefetch = 1;
     c->tune_max_warps = 0;
+    c->tune_update_impl = 0;
     *out = c;
     return SKETCHSSM_OK;
 }
@@ -205,6 +208,10 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     p.has_token = has_token ? 1 : 0;
     p.write_sketch = sketch ? 1 : 0;
     p.write_state = n_tot > 0 ? 1 : 0;
+    if (p.update_impl == 0) {
+        rc = launch_update_tc(ctx, p, static_cast<cudaStream_t>(stream));
+        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+    }
     return launch_update(ctx, p, static_cast<cudaStream_t>(stream));
 }
 
@@ -287,6 +294,7 @@ int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value) {
     if (eq(key, "decode_lanes_per_head")) { ctx->tune_lanes_per_head = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_l2_prefetch")) { ctx->tune_l2_prefetch = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_max_warps_per_sm")) { ctx->tune_max_warps = value; return SKETCHSSM_OK; }
+    if (eq(key, "update_impl")) { ctx->tune_update_impl = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_impl")) { ctx->tune_decode_impl = value; return SKETCHSSM_OK; }
     return SKETCHSSM_INVALID_ARG;
 }

@@ -246,10 +246,10 @@ __global__ void __launch_bounds__(256) decode_fused_kernel(const Params p) {
                     part[i] = acc;
                 }
                 group_reduce_transpose<LPH, NB>(part, j);
-                if (NB >= LPH || (j % (LPH / NB)) == 0) {
+                if (NB >= LPH || (j % (LPH > NB ? LPH / NB : 1)) == 0) {
 #pragma unroll
                     for (int i = 0; i < PPL; ++i) {
-                        const int idx = NB >= LPH ? PPL * j + i : j / (LPH / NB);
+                        const int idx = NB >= LPH ? PPL * j + i : j / (LPH > NB ? LPH / NB : 1);
                         if (s0 + idx < n) sA[s0 + idx] = part[i];
                     }
                 }
@@ -311,8 +311,8 @@ __global__ void __launch_bounds__(256) decode_fused_kernel(const Params p) {
             if (RP >= LPH) {
 #pragma unroll
                 for (int i = 0; i < CPL; ++i) sW[CPL * j + i] = part[i];
-            } else if ((j % (LPH / RP)) == 0) {
-                sW[j / (LPH / RP)] = part[0];
+            } else if ((j % (LPH > RP ? LPH / RP : 1)) == 0) {
+                sW[j / (LPH > RP ? LPH / RP : 1)] = part[0];
             }
         } else {
             store_row<EK, LPH>(sW, j, x);

@@ -236,10 +236,10 @@ __global__ void __launch_bounds__(256) decode_weights_kernel(const Params p) {
                     part[i] = acc;
                 }
                 group_reduce_transpose<LPH, NB>(part, j);
-                if (NB >= LPH || (j % (LPH / NB)) == 0) {
+                if (NB >= LPH || (j % (LPH > NB ? LPH / NB : 1)) == 0) {
 #pragma unroll
                     for (int i = 0; i < PPL; ++i) {
-                        const int idx = NB >= LPH ? PPL * j + i : j / (LPH / NB);
+                        const int idx = NB >= LPH ? PPL * j + i : j / (LPH > NB ? LPH / NB : 1);
                         if (s0 + idx < n) sA[s0 + idx] = part[i];
                     }
                 }
@@ -303,8 +303,8 @@ __global__ void __launch_bounds__(256) decode_weights_kernel(const Params p) {
 #pragma unroll
                     for (int i = 0; i < CPL; ++i)
                         if (CPL * j + i < R) wk[CPL * j + i] = part[i];
-                } else if ((j % (LPH / RP)) == 0 && j / (LPH / RP) < R) {
-                    wk[j / (LPH / RP)] = part[0];
+                } else if ((j % (LPH > RP ? LPH / RP : 1)) == 0 && j / (LPH > RP ? LPH / RP : 1) < R) {
+                    wk[j / (LPH > RP ? LPH / RP : 1)] = part[0];
                 }
             }
         } else if (active) {

@@ -67,6 +67,7 @@ struct Params {
     int lanes_per_head;  // decode (group kernel): 8 or 16; 0 = library default
     int l2_prefetch;     // decode (group kernel): request the following item's operands into L2
     int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
+    int update_impl;      // 0: tensor cores where supported, 1: CUDA cores only
 };
 
 int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head
@@ -84,7 +85,8 @@ int launch_decode_group_gdn_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_group_gdn_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_group_kda_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_group_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);
+int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);       // CUDA cores, every configuration
+int launch_update_tc(Ctx* ctx, const Params& p, cudaStream_t stream);    // tcgen05 tensor cores; UNSUPPORTED_SHAPE outside its domain
 
 // ---------------------------------------------------------------------------------------------
 // device helpers

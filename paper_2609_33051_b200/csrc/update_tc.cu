@@ -1,0 +1,447 @@
+// State-update (flush) kernel on the 5th-generation tensor cores (tcgen05 + TMEM), sm_100a.
+//
+// Mamba-2 transition (M_t = D_t = a_t I): the replay of n buffered tokens is the closed form of Eq. 3
+//     S_new = d S_0 + sum_s (beta_s prod_{j>s} a_j) k_s v_s^T,   d = prod_j a_j,
+// a rank-n update, and the sketch rows and the exact output are one more contraction over the state rows,
+//     U[g, :] = S_new^T omega_g  (Eq. 7),   o = S_new^T q.
+// Both contractions run as tcgen05.mma with fp32 accumulators in tensor memory; the fp32 state itself only
+// ever passes through registers once (read S_0, fused multiply-add with the accumulator, write S_new), so S is
+// streamed from HBM exactly once per update.
+//
+// Tile: 128 TMEM lanes = the value columns j of one head (V = 128) or of two heads of the same head index
+// (V = 64, block-diagonal operand); TMEM columns = the state rows i (K = 128).  Thread t owns lane t.
+//   MMA 1 (kind::f16, bf16 x bf16 -> fp32):  T[t, i] = sum_s w_s v_s[j(t)] k_s[i]
+//       A = w_s v_s split into bf16 hi + lo (w_s is fp32), B = the raw bf16 keys: exact products, fp32 sums
+//   epilogue: S_new[i, j] = d S_0[i, j] + T[t, i]  (coalesced global loads/stores, one element per thread and row),
+//       S_new split into bf16 hi + lo and written to shared memory as the A operand of MMA 2, 32 rows at a time
+//   MMA 2: UT[t, g] = sum_i S_new[i, j(t)] W[i, g],  W = [Omega | q] split hi + lo; three products
+//       (hi*hi + lo*hi + hi*lo) keep ~16 mantissa bits, accumulated in fp32
+// Operands use the no-swizzle canonical shared-memory layouts (8 x 16-byte core matrices).
+#include "internal.cuh"
+
+namespace sketchssm {
+
+namespace {
+
+constexpr int kTcThreads = 128;
+constexpr int kK = 128;              // state rows handled by this kernel
+constexpr int kTokBlock = 16;        // tokens per head and MMA-1 block
+constexpr int kChunk = 32;           // state rows per epilogue chunk
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    // shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets in 16-byte units
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32]) {
+    uint32_t u[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
+          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]),
+          "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]),
+          "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16]) {
+    uint32_t u[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
+          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(u[i]);
+}
+
+// bf16 hi + lo split of a float: x ~= hi + lo with ~16 mantissa bits
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
+    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+}
+
+struct TcSmem {
+    uint32_t a1_hi, a1_lo, b1, a2, b2_hi, b2_lo, w, bars, tmem_slot, total;
+};
+
+__host__ __device__ inline TcSmem make_tc_smem(int NH, int NP) {
+    TcSmem s;
+    const uint32_t kd1 = (uint32_t)(kTokBlock * NH);
+    uint32_t off = 0;
+    s.a1_hi = off; off += 128u * kd1 * 2u;
+    s.a1_lo = off; off += 128u * kd1 * 2u;
+    s.b1 = off; off += 128u * kd1 * 2u;
+    s.a2 = off; off += 2u * 2u * 128u * kChunk * 2u;     // two chunk buffers, each hi + lo
+    s.b2_hi = off; off += (uint32_t)NP * kK * 2u;
+    s.b2_lo = off; off += (uint32_t)NP * kK * 2u;
+    s.w = off; off += 2u * 208u * 4u;                    // per head: w_s (64), total decay (16), beta_s (64), a_s (64)
+    s.bars = off; off += 64u;
+    s.tmem_slot = off; off += 64u;
+    s.total = off;
+    return s;
+}
+
+}  // namespace
+
+// V = 128: one head per tile; V = 64: two heads (same head index, consecutive batch entries) per tile.
+template <int V>
+__global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Params p) {
+    constexpr int K = kK;
+    constexpr int NH = 128 / V;
+    constexpr int KD1 = kTokBlock * NH;                 // contraction length of one MMA-1 block
+    extern __shared__ __align__(1024) unsigned char smem[];
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int R = p.R, H = p.H, B = p.B;
+    const int NP = (R + NH + 15) & ~15;                   // sketch ranks + one query column per head, padded
+    const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);
+    const TcSmem sm = make_tc_smem(NH, NP);
+    __nv_bfloat16* sA1hi = reinterpret_cast<__nv_bfloat16*>(smem + sm.a1_hi);
+    __nv_bfloat16* sA1lo = reinterpret_cast<__nv_bfloat16*>(smem + sm.a1_lo);
+    __nv_bfloat16* sB1 = reinterpret_cast<__nv_bfloat16*>(smem + sm.b1);
+    unsigned char* sA2 = smem + sm.a2;
+    __nv_bfloat16* sB2hi = reinterpret_cast<__nv_bfloat16*>(smem + sm.b2_hi);
+    __nv_bfloat16* sB2lo = reinterpret_cast<__nv_bfloat16*>(smem + sm.b2_lo);
+    float* sW = reinterpret_cast<float*>(smem + sm.w);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);     // [0] MMA 1, [1..2] MMA 2 chunk buffers, [3] MMA 2 all
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.tmem_slot);
+
+    const uint32_t tmem_cols = NP <= 32 ? 128u : 256u;
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 4; ++i) mbar_init(&bars[i], 1);
+        mbar_fence_init();
+    }
+    // the off-diagonal blocks of the block-diagonal A operand (and unused token rows) stay zero for the whole kernel
+    for (int i = tid; i < (int)(3u * 128u * KD1 * 2u / 16u); i += kTcThreads)
+        reinterpret_cast<uint4*>(smem + sm.a1_hi)[i] = make_uint4(0, 0, 0, 0);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_t = tmem_base;                          // T: 128 columns
+    const uint32_t tmem_u = tmem_base + (NP <= 32 ? 0u : 128u); // UT: NP columns (re-uses consumed T columns if it fits)
+    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+
+    // instruction descriptors: bf16 x bf16 -> fp32
+    const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+    const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)NP >> 3) << 17) | ((128u >> 4) << 24);
+
+    // canonical no-swizzle layouts (byte offsets)
+    //   MN-major (MMA 1): elem(mn, k) at (k%8)*16 + (mn%8)*2 + (mn/8)*128 + (k/8)*2048
+    //   K-major  (MMA 2): elem(mn, k) at (mn%8)*16 + (mn/8)*128 + (k/8)*LBO + (k%8)*2,  LBO = 16*MN
+    constexpr uint32_t LBO1 = 2048, SBO = 128;
+    constexpr uint32_t LBO2A = 2048;
+    const uint32_t LBO2B = (uint32_t)NP * 16u;
+
+    const int tiles_per_h = B / NH;
+    const long long n_tiles = (long long)H * tiles_per_h;
+    const int tile0 = (int)(n_tiles * blockIdx.x / gridDim.x);
+    const int tile1 = (int)(n_tiles * (blockIdx.x + 1) / gridDim.x);
+
+    const int my_head = tid / V;          // which head of the tile this thread's lane belongs to
+    const int j = tid % V;
+    int cur_h = -1;
+    uint32_t ph0 = 0, ph1[2] = {0, 0}, ph3 = 0;   // mbarrier phases
+    bool dead = false;
+
+    for (int tile = tile0; tile < tile1 && !dead; ++tile) {
+        const int h = tile / tiles_per_h;
+        const int b0 = (tile - h * tiles_per_h) * NH;
+        const size_t bh = (size_t)(b0 + my_head) * H + h;
+
+        // ---- W = [Omega | q ...] hi/lo, K-major; Omega part once per head index ----
+        if (h != cur_h) {
+            const float* og = p.omega + (size_t)h * K * R;
+            for (int idx = tid; idx < K * NP; idx += kTcThreads) {
+                const int i = idx / NP, g = idx % NP;
+                __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi;
+                if (g < R && p.write_sketch) split_bf16(og[(size_t)i * R + g], hi, lo);
+                const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO2B + (i & 7) * 2) >> 1;
+                sB2hi[o2] = hi;
+                sB2lo[o2] = lo;
+            }
+            cur_h = h;
+        }
+        if (p.q != nullptr) {       // query columns R .. R+NH-1 (bf16-exact: lo = 0)
+            for (int idx = tid; idx < K * NH; idx += kTcThreads) {
+                const int i = idx % K, hd = idx / K, g = R + hd;
+                const size_t bq = (size_t)(b0 + hd) * H + h;
+                const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO2B + (i & 7) * 2) >> 1;
+                sB2hi[o2] = reinterpret_cast<const __nv_bfloat16*>(p.q)[bq * K + i];
+            }
+        }
+
+        // ---- token weights w_s = beta_s prod_{j>s} a_j and the total decay ----
+        // gates are fetched in parallel, then one thread per head runs the short serial scan from shared memory
+        for (int idx = tid; idx < NH * 64; idx += kTcThreads) {
+            const int hd = idx >> 6, s = idx & 63;
+            if (s < n_tot) {
+                const size_t bw = (size_t)(b0 + hd) * H + h;
+                const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
+                sW[hd * 208 + 80 + s] = s < n_ring ? reinterpret_cast<const float*>(rh + p.rl.beta_off)[s] : p.beta[bw];
+                sW[hd * 208 + 144 + s] = s < n_ring ? reinterpret_cast<const float*>(rh + p.rl.decay_off)[s]
+                                                    : reinterpret_cast<const float*>(p.decay)[bw];
+            }
+        }
+        __syncthreads();
+        if (tid < NH) {
+            float suf = 1.f;
+            for (int s = n_tot - 1; s >= 0; --s) {
+                sW[tid * 208 + s] = sW[tid * 208 + 80 + s] * suf;
+                suf *= sW[tid * 208 + 144 + s];
+            }
+            sW[tid * 208 + 64] = suf;
+        }
+        // prefetch the first chunk of S_0 while the operands are being prepared
+        const float* Sg = p.state + bh * (size_t)K * V + j;
+        float s0[kChunk];
+#pragma unroll
+        for (int ii = 0; ii < kChunk; ++ii) s0[ii] = Sg[(size_t)ii * V];
+        __syncthreads();
+
+        // ---- MMA 1 over blocks of kTokBlock tokens per head ----
+        const int n_blocks = (n_tot + kTokBlock - 1) / kTokBlock;
+        for (int blk = 0; blk < n_blocks; ++blk) {
+            if (blk > 0) {      // the previous block's MMAs must have read the operand buffers
+                if (!mbar_wait_bounded(&bars[0], ph0)) { record_fault(p.status, kFaultUpdateWait, 1); dead = true; }
+                ph0 ^= 1;
+                tc_fence_after();
+            }
+            // B operand: keys, MN-major (mn = state row i, k = token slot)
+            for (int idx = tid; idx < KD1 * (K / 8); idx += kTcThreads) {
+                const int sp = idx / (K / 8), a = idx % (K / 8);        // operand row (token), 8-element vector index
+                const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
+                const size_t bk = (size_t)(b0 + hd) * H + h;
+                uint4 val = make_uint4(0, 0, 0, 0);
+                if (s < n_ring) {
+                    val = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + ((size_t)s * K + a * 8) * 2);
+                } else if (s < n_tot) {
+                    val = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.k) + bk * K + a * 8);
+                }
+                *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(sB1) + (sp & 7) * 16 + a * SBO + (sp >> 3) * LBO1) = val;
+            }
+            // A operand: w_s v_s hi/lo, MN-major (mn = lane t = head*V + j, k = token slot), block diagonal over heads
+            for (int idx = tid; idx < KD1 * (V / 8); idx += kTcThreads) {
+                const int sp = idx / (V / 8), a = idx % (V / 8);
+                const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
+                const size_t bk = (size_t)(b0 + hd) * H + h;
+                uint4 vraw = make_uint4(0, 0, 0, 0);
+                float w = 0.f;
+                if (s < n_ring) {
+                    vraw = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + p.rl.v_off + ((size_t)s * V + a * 8) * 2);
+                    w = sW[hd * 208 + s];
+                } else if (s < n_tot) {
+                    vraw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.v) + bk * V + a * 8);
+                    w = sW[hd * 208 + s];
+                }
+                const uint32_t vin[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
+                uint32_t ohi[4], olo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float f0 = w * __uint_as_float(vin[e] << 16), f1 = w * __uint_as_float(vin[e] & 0xffff0000u);
+                    __nv_bfloat16 h0, l0, h1, l1;
+                    split_bf16(f0, h0, l0);
+                    split_bf16(f1, h1, l1);
+                    ohi[e] = pack_bf16(h0, h1);
+                    olo[e] = pack_bf16(l0, l1);
+                }
+                const uint32_t off = (sp & 7) * 16 + (hd * (V / 8) + a) * SBO + (sp >> 3) * LBO1;
+                *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(sA1hi) + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(sA1lo) + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+            }
+            proxy_fence();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < KD1 / 16; ++ks) {
+                    const uint64_t bd = make_desc(smem_u32(sB1) + ks * 2 * LBO1, LBO1, SBO);
+                    tc_mma_bf16(tmem_t, make_desc(smem_u32(sA1hi) + ks * 2 * LBO1, LBO1, SBO), bd, idesc1, (blk | ks) ? 1u : 0u);
+                    tc_mma_bf16(tmem_t, make_desc(smem_u32(sA1lo) + ks * 2 * LBO1, LBO1, SBO), bd, idesc1, 1u);
+                }
+                tc_commit(&bars[0]);
+            }
+        }
+        if (n_blocks > 0) {
+            if (!mbar_wait_bounded(&bars[0], ph0)) { record_fault(p.status, kFaultUpdateWait, 2); dead = true; }
+            ph0 ^= 1;
+            tc_fence_after();
+        }
+        dead = __syncthreads_or(dead ? 1 : 0) != 0;
+        if (dead) break;
+
+        // ---- epilogue: S_new = d S_0 + T, written back; S_new hi/lo -> A operand of MMA 2, 32 rows at a time ----
+        const float dtot = n_tot > 0 ? sW[my_head * 208 + 64] : 1.f;
+        float* So = p.state + bh * (size_t)K * V + j;
+        for (int c = 0; c < K / kChunk; ++c) {
+            float s0n[kChunk];
+            if (c + 1 < K / kChunk) {
+#pragma unroll
+                for (int ii = 0; ii < kChunk; ++ii) s0n[ii] = Sg[(size_t)((c + 1) * kChunk + ii) * V];
+            }
+            float t[kChunk];
+            if (n_blocks > 0) {
+                tmem_ld32(tmem_t + lane_sel + (uint32_t)(c * kChunk), t);
+            } else {
+#pragma unroll
+                for (int ii = 0; ii < kChunk; ++ii) t[ii] = 0.f;
+            }
+            if (c >= 2) {       // chunk buffer c&1 was read by the MMAs of chunk c-2
+                if (!mbar_wait_bounded(&bars[1 + (c & 1)], ph1[c & 1])) { record_fault(p.status, kFaultUpdateWait, 3); dead = true; }
+                ph1[c & 1] ^= 1;
+            }
+            unsigned char* a2hi = sA2 + (size_t)(c & 1) * (2u * 128u * kChunk * 2u);
+            unsigned char* a2lo = a2hi + 128u * kChunk * 2u;
+#pragma unroll
+            for (int v8 = 0; v8 < kChunk / 8; ++v8) {
+                uint32_t ohi[4], olo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i0 = v8 * 8 + 2 * e;
+                    const float x0 = fmaf(dtot, s0[i0], t[i0]), x1 = fmaf(dtot, s0[i0 + 1], t[i0 + 1]);
+                    if (p.write_state) {
+                        So[(size_t)(c * kChunk + i0) * V] = x0;
+                        So[(size_t)(c * kChunk + i0 + 1) * V] = x1;
+                    }
+                    __nv_bfloat16 h0, l0, h1, l1;
+                    split_bf16(x0, h0, l0);
+                    split_bf16(x1, h1, l1);
+                    ohi[e] = pack_bf16(h0, h1);
+                    olo[e] = pack_bf16(l0, l1);
+                }
+                const uint32_t off = (tid & 7) * 16 + (tid >> 3) * SBO + v8 * LBO2A;
+                *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                *reinterpret_cast<uint4*>(a2lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+            }
+            proxy_fence();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kChunk / 16; ++ks) {
+                    const uint32_t kb = (uint32_t)(c * (kChunk / 8) + ks * 2) * LBO2B;      // W rows of this K-step
+                    const uint64_t ahi = make_desc(smem_u32(a2hi) + ks * 2 * LBO2A, LBO2A, SBO);
+                    const uint64_t alo = make_desc(smem_u32(a2lo) + ks * 2 * LBO2A, LBO2A, SBO);
+                    const uint64_t bhi = make_desc(smem_u32(sB2hi) + kb, LBO2B, SBO);
+                    const uint64_t blo = make_desc(smem_u32(sB2lo) + kb, LBO2B, SBO);
+                    tc_mma_bf16(tmem_u, ahi, bhi, idesc2, (c | ks) ? 1u : 0u);
+                    tc_mma_bf16(tmem_u, alo, bhi, idesc2, 1u);
+                    tc_mma_bf16(tmem_u, ahi, blo, idesc2, 1u);
+                }
+                tc_commit(c + 1 < K / kChunk ? &bars[1 + (c & 1)] : &bars[3]);
+            }
+            if (c + 1 < K / kChunk) {
+#pragma unroll
+                for (int ii = 0; ii < kChunk; ++ii) s0[ii] = s0n[ii];
+            }
+        }
+        // drain: chunk 2's commit (buffer 0) is still pending on its barrier; the final commit covers everything
+        if (!mbar_wait_bounded(&bars[1], ph1[0])) { record_fault(p.status, kFaultUpdateWait, 4); dead = true; }
+        ph1[0] ^= 1;
+        if (!mbar_wait_bounded(&bars[3], ph3)) { record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
+        ph3 ^= 1;
+        tc_fence_after();
+
+        // ---- UT rows -> sketch and exact output ----
+        for (int g0 = 0; g0 < NP; g0 += 16) {
+            float u[16];
+            tmem_ld16(tmem_u + lane_sel + (uint32_t)g0, u);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const int g = g0 + e;
+                if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u[e];
+                if (g == R + my_head && p.out != nullptr) {
+                    if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u[e]);
+                    else reinterpret_cast<float*>(p.out)[bh * V + j] = u[e];
+                }
+            }
+        }
+        tc_fence_before();
+        dead = __syncthreads_or(dead ? 1 : 0) != 0;   // T / UT are free again; also publishes any fault
+        tc_fence_after();
+    }
+
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// Returns SKETCHSSM_UNSUPPORTED_SHAPE when the configuration is outside this kernel's domain (the caller then
+// uses the CUDA-core kernel).
+int launch_update_tc(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+    const sketchssm_config& c = ctx->cfg;
+    if (c.kind != SKETCHSSM_MAMBA2 || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int NH = 128 / c.dv;
+    if (c.batch % NH != 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int NP = (c.rank + NH + 15) & ~15;
+    if (NP > 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    Params p = p_in;
+    if (ctx->sm_count == 0) {
+        int dev = 0, sms = 0;
+        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return SKETCHSSM_CUDA_ERROR;
+        ctx->sm_count = sms;
+    }
+    const TcSmem sm = make_tc_smem(NH, NP);
+    const int tmem_cols = NP <= 32 ? 128 : 256;
+    int ctas = (int)((228u * 1024u) / (sm.total + 1024u));
+    if (ctas > 512 / tmem_cols) ctas = 512 / tmem_cols;     // tensor memory: 512 columns per SM
+    if (ctas > 4) ctas = 4;
+    if (p.max_warps_per_sm > 0 && ctas > p.max_warps_per_sm / 4) ctas = p.max_warps_per_sm / 4 > 0 ? p.max_warps_per_sm / 4 : 1;
+    const long long n_tiles = (long long)c.batch * c.heads / NH;
+    long long grid = (long long)ctx->sm_count * ctas;
+    if (grid > n_tiles) grid = n_tiles;
+    auto kern = c.dv == 128 ? update_tc_mamba2_kernel<128> : update_tc_mamba2_kernel<64>;
+    if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)sm.total)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    kern<<<dim3((unsigned)grid), kTcThreads, sm.total, stream>>>(p);
+    if ((ctx->last_cuda_error = cudaGetLastError()) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+    ctx->last_launches = 1;
+    return SKETCHSSM_OK;
+}
+
+}  // namespace sketchssm
