@@ -89,6 +89,15 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
     lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
+// two floats -> packed bf16x2 hi and packed bf16x2 lo (element 0 in the low half)
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+    hi = *reinterpret_cast<uint32_t*>(&h);
+    const float r0 = x0 - __uint_as_float(hi << 16), r1 = x1 - __uint_as_float(hi & 0xffff0000u);
+    __nv_bfloat162 l = __floats2bfloat162_rn(r0, r1);
+    lo = *reinterpret_cast<uint32_t*>(&l);
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
     return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
@@ -101,10 +110,14 @@ __host__ __device__ inline TcSmem make_tc_smem(int NH, int NP) {
     TcSmem s;
     const uint32_t kd1 = (uint32_t)(kTokBlock * NH);
     uint32_t off = 0;
-    s.a1_hi = off; off += 128u * kd1 * 2u;
-    s.a1_lo = off; off += 128u * kd1 * 2u;
-    s.b1 = off; off += 128u * kd1 * 2u;
-    s.a2 = off; off += 2u * 2u * 128u * kChunk * 2u;     // two chunk buffers, each hi + lo
+    // the MMA-1 operands are dead once MMA 1 has completed, before the epilogue writes the MMA-2 chunk buffers:
+    // both live in the same region
+    s.a1_hi = off;
+    s.a1_lo = off + 128u * kd1 * 2u;
+    s.b1 = off + 2u * 128u * kd1 * 2u;
+    s.a2 = off;
+    const uint32_t mma1_bytes = 3u * 128u * kd1 * 2u, mma2_bytes = 2u * 2u * 128u * kChunk * 2u;   // two chunk buffers, hi + lo
+    off += mma1_bytes > mma2_bytes ? mma1_bytes : mma2_bytes;
     s.b2_hi = off; off += (uint32_t)NP * kK * 2u;
     s.b2_lo = off; off += (uint32_t)NP * kK * 2u;
     s.w = off; off += 2u * 208u * 4u;                    // per head: w_s (64), total decay (16), beta_s (64), a_s (64)
@@ -150,9 +163,6 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
         for (int i = 0; i < 4; ++i) mbar_init(&bars[i], 1);
         mbar_fence_init();
     }
-    // the off-diagonal blocks of the block-diagonal A operand (and unused token rows) stay zero for the whole kernel
-    for (int i = tid; i < (int)(3u * 128u * KD1 * 2u / 16u); i += kTcThreads)
-        reinterpret_cast<uint4*>(smem + sm.a1_hi)[i] = make_uint4(0, 0, 0, 0);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -246,9 +256,11 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                 ph0 ^= 1;
                 tc_fence_after();
             }
+            // Operand rows are written 16 bytes per thread; consecutive threads walk the 8 token rows of a core matrix
+            // first and then the next 8-element vector, so that a warp writes 512 contiguous bytes (no bank conflicts).
             // B operand: keys, MN-major (mn = state row i, k = token slot)
             for (int idx = tid; idx < KD1 * (K / 8); idx += kTcThreads) {
-                const int sp = idx / (K / 8), a = idx % (K / 8);        // operand row (token), 8-element vector index
+                const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
                 const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
                 const size_t bk = (size_t)(b0 + hd) * H + h;
                 uint4 val = make_uint4(0, 0, 0, 0);
@@ -259,32 +271,32 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                 }
                 *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(sB1) + (sp & 7) * 16 + a * SBO + (sp >> 3) * LBO1) = val;
             }
-            // A operand: w_s v_s hi/lo, MN-major (mn = lane t = head*V + j, k = token slot), block diagonal over heads
-            for (int idx = tid; idx < KD1 * (V / 8); idx += kTcThreads) {
-                const int sp = idx / (V / 8), a = idx % (V / 8);
+            // A operand: w_s v_s hi/lo, MN-major (mn = lane t = head*V + j, k = token slot), block diagonal over heads:
+            // lanes of head hd see only the token rows of head hd, the other block is zero
+            for (int idx = tid; idx < KD1 * 16; idx += kTcThreads) {
+                const int a128 = (idx >> 3) & 15, sp = (idx & 7) + 8 * (idx >> 7);     // a128: vector index over all 128 lanes
                 const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
+                const int hd_lane = a128 / (V / 8), a = a128 % (V / 8);
                 const size_t bk = (size_t)(b0 + hd) * H + h;
                 uint4 vraw = make_uint4(0, 0, 0, 0);
                 float w = 0.f;
-                if (s < n_ring) {
-                    vraw = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + p.rl.v_off + ((size_t)s * V + a * 8) * 2);
-                    w = sW[hd * 208 + s];
-                } else if (s < n_tot) {
-                    vraw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.v) + bk * V + a * 8);
-                    w = sW[hd * 208 + s];
+                if (hd_lane == hd) {
+                    if (s < n_ring) {
+                        vraw = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + p.rl.v_off + ((size_t)s * V + a * 8) * 2);
+                        w = sW[hd * 208 + s];
+                    } else if (s < n_tot) {
+                        vraw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.v) + bk * V + a * 8);
+                        w = sW[hd * 208 + s];
+                    }
                 }
                 const uint32_t vin[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
                 uint32_t ohi[4], olo[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const float f0 = w * __uint_as_float(vin[e] << 16), f1 = w * __uint_as_float(vin[e] & 0xffff0000u);
-                    __nv_bfloat16 h0, l0, h1, l1;
-                    split_bf16(f0, h0, l0);
-                    split_bf16(f1, h1, l1);
-                    ohi[e] = pack_bf16(h0, h1);
-                    olo[e] = pack_bf16(l0, l1);
+                    split_bf16x2(f0, f1, ohi[e], olo[e]);
                 }
-                const uint32_t off = (sp & 7) * 16 + (hd * (V / 8) + a) * SBO + (sp >> 3) * LBO1;
+                const uint32_t off = (sp & 7) * 16 + a128 * SBO + (sp >> 3) * LBO1;
                 *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(sA1hi) + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
                 *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(sA1lo) + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
             }
@@ -343,11 +355,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                         So[(size_t)(c * kChunk + i0) * V] = x0;
                         So[(size_t)(c * kChunk + i0 + 1) * V] = x1;
                     }
-                    __nv_bfloat16 h0, l0, h1, l1;
-                    split_bf16(x0, h0, l0);
-                    split_bf16(x1, h1, l1);
-                    ohi[e] = pack_bf16(h0, h1);
-                    olo[e] = pack_bf16(l0, l1);
+                    split_bf16x2(x0, x1, ohi[e], olo[e]);
                 }
                 const uint32_t off = (tid & 7) * 16 + (tid >> 3) * SBO + v8 * LBO2A;
                 *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
