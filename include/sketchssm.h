@@ -155,6 +155,29 @@ int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, 
                                const void* v, const void* beta, const void* decay, void* out,
                                uint32_t flags, void* stream);
 
+/* Size of the library-owned device array used by sketchssm_decode_step_static. */
+#define SKETCHSSM_STATIC_WORK_BYTES (4u << 20)
+
+/* (The paper has no counterpart of this entry point: it exists for deployment, not for the method.)
+ * sketchssm_decode_step for callers that cannot provide scratch memory and must not trigger an allocation:
+ * an engine whose device memory pool is carved up once at start-up, a plug-in that only ever receives its
+ * tensors, code inside a region where an allocation would synchronise the device.  Same arguments, same
+ * result (up to floating-point summation order) and same ring behaviour as sketchssm_decode_step, always as
+ * the two-kernel decode; the per-head weight hand-off between the two kernels lives in a device array that
+ * belongs to the library (SKETCHSSM_STATIC_WORK_BYTES = 4 MiB, held by every GPU that loads the library until
+ * the process exits) instead of in sketchssm_buffers.work, which this call never touches.  The call itself
+ * allocates nothing, on the host or on the device.
+ *   - Limit: batch * heads * (dk + buf_len) * 4 bytes must fit in the array, otherwise the call returns
+ *     SKETCHSSM_UNSUPPORTED_SHAPE and launches nothing.
+ *   - The first call made on a device looks up the array's address on that device (one runtime query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - All contexts, streams and threads share the one array.  It keeps whatever the last call left in it; the
+ *     kernels overwrite every element they read, so nothing has to be cleared.  Two calls that overlap on the
+ *     GPU (different streams, or different contexts on the same device) race on it: serialise them. */
+int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
+                                 const void* v, const void* beta, const void* decay, void* out,
+                                 uint32_t flags, void* stream);
+
 /* Device staging for one step's token tensors, caller-owned, same shapes/dtypes as the token
  * arguments of the hot-path calls (q,k [B][H][K] io; v [B][H][V] io; beta [B][H] fp32; decay;
  * out [B][H][V]).  Used only by sketchssm_step_host. */

@@ -26,6 +26,7 @@ EXPORTED = (
     "sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode",
     "sketchssm_read_status", "sketchssm_last_launch_count", "sketchssm_tune",
     "sketchssm_status_string", "sketchssm_version", "sketchssm_last_cuda_error", "sketchssm_step_host",
+    "sketchssm_decode_step_static",
 )
 OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 
@@ -73,7 +74,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sketchssm_destroy.argtypes = [vp]
     lib.sketchssm_query_sizes.argtypes = [vp, ctypes.POINTER(Sizes)]
     lib.sketchssm_bind.argtypes = [vp, ctypes.POINTER(Buffers)]
-    for name in ("sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode"):
+    for name in ("sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode",
+                 "sketchssm_decode_step_static"):
         getattr(lib, name).argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u32, vp]
     lib.sketchssm_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.POINTER(Staging), u32, vp]
     lib.sketchssm_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32 * 4), vp]
@@ -190,6 +192,14 @@ class SketchSSM:
         rc = self.lib.sketchssm_decode_step(self._ctx, n_before, _ptr(q), _ptr(k), _ptr(v), _ptr(beta),
                                             _ptr(decay), _ptr(out), flags, self._stream(stream))
         self._check("sketchssm_decode_step", rc)
+        return out
+
+    def decode_step_static(self, n_before: int, q, k, v, beta, decay, out, flags: int = 0, stream=None):
+        """sketchssm_decode_step_static: the decode step for callers that can neither allocate nor supply
+        scratch; its kernel-to-kernel hand-off uses the library's fixed 4 MiB device array."""
+        rc = self.lib.sketchssm_decode_step_static(self._ctx, n_before, _ptr(q), _ptr(k), _ptr(v), _ptr(beta),
+                                                   _ptr(decay), _ptr(out), flags, self._stream(stream))
+        self._check("sketchssm_decode_step_static", rc)
         return out
 
     def full_read_decode(self, n_before: int, q, k, v, beta, decay, out, flags: int = 0, stream=None):

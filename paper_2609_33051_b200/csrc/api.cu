@@ -225,6 +225,29 @@ int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, 
     return decode_common(ctx, 1, n_before, q, k, v, beta, decay, out, flags, stream);
 }
 
+int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
+                                 const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    ctx->last_launches = 0;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    if (n_before < 0 || n_before > ctx->cfg.buf_len - 1) return SKETCHSSM_INVALID_ARG;
+    if (flags & ~SKETCHSSM_NO_APPEND) return SKETCHSSM_INVALID_ARG;
+    int rc = check_token_ptrs(q, k, v, beta, decay, out);
+    if (rc != SKETCHSSM_OK) return rc;
+    if ((size_t)ctx->cfg.batch * ctx->cfg.heads * (size_t)(ctx->cfg.dk + ctx->cfg.buf_len) * sizeof(float) >
+        (size_t)SKETCHSSM_STATIC_WORK_BYTES)
+        return SKETCHSSM_UNSUPPORTED_SHAPE;     // would not fit the library's static array
+    rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    Params p = base_params(ctx);
+    p.q = q; p.k = k; p.v = v; p.beta = static_cast<const float*>(beta); p.decay = decay; p.out = out;
+    p.n_before = n_before;
+    p.has_token = 1;
+    p.append = (flags & SKETCHSSM_NO_APPEND) ? 0 : 1;
+    p.full_read = 0;
+    return launch_decode_static(ctx, p, static_cast<cudaStream_t>(stream));
+}
+
 int sketchssm_step_host(sketchssm_ctx* ctx, int op, int n_before, const void* hq, const void* hk, const void* hv,
                         const void* hbeta, const void* hdecay, void* hout, const sketchssm_staging* st,
                         uint32_t flags, void* stream) {

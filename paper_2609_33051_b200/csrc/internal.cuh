@@ -72,6 +72,8 @@ struct Params {
 
 int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head
 // 8 or 16 lanes per head, one entry per recurrence kind
+// two-kernel decode with the weight hand-off in the library's static device array
+int launch_decode_static(Ctx* ctx, const Params& p, cudaStream_t stream);
 // decode as two kernels (weights, then output rows), one entry per (kind, I/O type)
 int launch_decode_split_mamba2_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_split_mamba2_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
