@@ -37,6 +37,26 @@ UNIT = "tokens/s/layer"
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
 
 
+def max_over_ranks(ms_local: float, dist, device="cuda") -> float:
+    """Job time of a multi-rank run: the slowest rank's device time."""
+    if dist is None:
+        return ms_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(tokens_per_rank: float, world: int, ms_step: float) -> float:
+    """Whole-job tokens/s/layer: every rank processes its own shard (weak scaling, no exchange)."""
+    return world * tokens_per_rank / (ms_step * 1e-3)
+
+
+def rank_shard(total_batch: int, rank: int, world: int):
+    """[begin, end) of the batch entries a rank owns when one batch is split across ranks (heads and batch
+    entries are independent, so shards never communicate)."""
+    return (total_batch * rank) // world, (total_batch * (rank + 1)) // world
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -342,11 +362,7 @@ def main():
         e1.record()
         barrier()
         clocks = sampler.stop() if sampler is not None else None
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), dist)
         return ms / steps, out, clocks
 
     # ---- device-resident timing (the headline value): no events between launches ----
@@ -358,7 +374,7 @@ def main():
     ms_step, _, clocks = timed_region(step, args.steps, args.warmup, ClockSampler(local_rank))
     for m in stack.layers:
         m.check_status()
-    value = world * tokens_per_step / (ms_step * 1e-3)
+    value = job_value(tokens_per_step, world, ms_step)
 
     # ---- the same region again with every launch bracketed by events: per-kernel durations ----
     events = None if args.no_launch_events else []

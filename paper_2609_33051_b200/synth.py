@@ -110,7 +110,9 @@ def _softplus(x):
 def initial_state(w: Workload, layer: int = 0) -> np.ndarray:
     """S_init ~ N(0, state_std^2), shape [B, H, K, V], float32."""
     g = _gen(w, _F_STATE, layer)
-    return (w.state_std * g.standard_normal((w.batch, w.heads, w.dk, w.dv))).astype(np.float32)
+    out = g.standard_normal((w.batch, w.heads, w.dk, w.dv), dtype=np.float32)
+    out *= np.float32(w.state_std)
+    return out
 
 
 def a_log(w: Workload, layer: int = 0) -> np.ndarray:
