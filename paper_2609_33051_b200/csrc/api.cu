@@ -13,6 +13,7 @@ struct sketchssm_ctx : public Ctx {
     int tune_decode_impl;   // 0: two kernels (weights + output rows), 1: warp-per-head kernel, 2: fused lane-group kernel
     int tune_max_warps;
     int tune_update_impl;
+    int tune_decode_mma;
     int tune_l2_prefetch;   // lane-group kernel: 1 (default) / 0
 };
 
@@ -59,6 +60,7 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.l2_prefetch = ctx->tune_l2_prefetch;
     p.max_warps_per_sm = ctx->tune_max_warps;
     p.update_impl = ctx->tune_update_impl;
+    p.decode_mma = ctx->tune_decode_mma;
     return p;
 }
 
@@ -88,7 +90,13 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     p.full_read = full_read;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
-    if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
+    if (ctx->tune_decode_impl == 1) {
+        if (p.decode_mma) {
+            const int rc = launch_decode_mma(ctx, p, cs);
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        }
+        return launch_decode(ctx, p, cs);
+    }
     if (ctx->tune_decode_impl == 2) {
         switch (ctx->cfg.kind) {
             case SKETCHSSM_MAMBA2:
@@ -142,6 +150,7 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     c->tune_l2_prefetch = 1;
     c->tune_max_warps = 0;
     c->tune_update_impl = 0;
+    c->tune_decode_mma = 0;
     *out = c;
     return SKETCHSSM_OK;
 }
@@ -317,6 +326,7 @@ int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value) {
     if (eq(key, "decode_lanes_per_head")) { ctx->tune_lanes_per_head = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_l2_prefetch")) { ctx->tune_l2_prefetch = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_max_warps_per_sm")) { ctx->tune_max_warps = value; return SKETCHSSM_OK; }
+    if (eq(key, "decode_mma")) { ctx->tune_decode_mma = value; return SKETCHSSM_OK; }
     if (eq(key, "update_impl")) { ctx->tune_update_impl = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_impl")) { ctx->tune_decode_impl = value; return SKETCHSSM_OK; }
     return SKETCHSSM_INVALID_ARG;

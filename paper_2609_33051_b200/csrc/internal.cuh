@@ -68,9 +68,11 @@ struct Params {
     int l2_prefetch;     // decode (group kernel): request the following item's operands into L2
     int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
     int update_impl;      // 0: tensor cores where supported, 1: CUDA cores only
+    int decode_mma;       // warp-per-head decode: 1 = tensor-core dot products where supported
 };
 
 int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head
+int launch_decode_mma(Ctx* ctx, const Params& p, cudaStream_t stream);    // Mamba-2 with tensor-core dot products; UNSUPPORTED_SHAPE outside its domain
 // 8 or 16 lanes per head, one entry per recurrence kind
 // two-kernel decode with the weight hand-off in the library's static device array
 int launch_decode_static(Ctx* ctx, const Params& p, cudaStream_t stream);
@@ -113,6 +115,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
                  : "memory");
 }
 
+// One potentially blocking poll of the barrier phase.  (An explicit suspend-time hint was measured: waiting warps
+// then woke only when the hint ran out, which cost the kernels with few warps up to 2x, so none is given.)
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t done;
     asm volatile(

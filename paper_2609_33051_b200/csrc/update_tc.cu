@@ -98,10 +98,6 @@ __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, u
     lo = *reinterpret_cast<uint32_t*>(&l);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
-    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
-}
-
 struct TcSmem {
     uint32_t a1_hi, a1_lo, b1, a2, b2_hi, b2_lo, w, bars, tmem_slot, total;
 };

@@ -135,11 +135,20 @@ def test_ranks_and_window_lengths(kind, rank, buf_len):
                                   {"decode_impl": 2, "decode_stages": 2, "decode_warps_per_cta": 3},
                                   {"decode_impl": 2, "decode_l2_prefetch": 0},
                                   {"decode_impl": 0, "decode_stages": 2, "decode_warps_per_cta": 2},
-                                  {"decode_impl": 0, "decode_stages": 1, "decode_max_warps_per_sm": 4}])
+                                  {"decode_impl": 0, "decode_stages": 1, "decode_max_warps_per_sm": 4},
+                                  {"decode_impl": 1, "decode_mma": 1}, {"update_impl": 1}])
 def test_launch_tunings_and_ragged_batches(kind, tune):
     w = synth.Workload("t", kind, 37, 3, 128, 128, 16, 16, 0, "bf16", 7, basis="qr")
     check(run_schedule(w, 20, max_heads=10**9, tune=tune), "bf16")
     check(run_schedule(w, 18, max_heads=10**9, mode="full_read", tune=tune), "bf16")
+
+
+@pytest.mark.parametrize("dv,rank,buf_len", [(64, 16, 16), (128, 40, 48), (64, 5, 64)])
+def test_mamba2_tensor_core_variants(dv, rank, buf_len):
+    """Mamba-2 decode with mma.sync dot products, and the tcgen05 update against the CUDA-core update."""
+    w = synth.Workload("t", "mamba2", 6, 3, 128, dv, rank, buf_len, 0, "bf16", 77, basis="qr")
+    check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"decode_mma": 1}), "bf16")
+    check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"update_impl": 1}), "bf16")
 
 
 def test_bf16_output_mode():
