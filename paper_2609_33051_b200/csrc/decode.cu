@@ -1,27 +1,36 @@
-// Decode-step kernels of the SketchSSM hot path (sm_100a).
+// Decode-step kernel, one warp per (batch, head) (sm_100a): the default for decode_step and full_read_decode.
 //
-// One warp owns one (batch, head) at a time.  Its per-head operands -- the sketch U and the
-// buffered keys / values / gates of the ring -- are brought from HBM into a private shared-memory
-// stage by 1-D bulk asynchronous copies (TMA, no multicast) that complete on an mbarrier, so the
-// copies of the next head overlap the arithmetic of the current one and no register is spent on
-// data in flight.  The per-head coefficient map C is shared by the whole batch: a CTA serves one
-// head index h for a chunk of batch entries and stages C in shared memory once.
+// CTAs are persistent: each walks a contiguous range of (head index, batch) items, so a single wave of CTAs
+// covers the launch, the coefficient map C of at most two head indices is staged in shared memory once per CTA,
+// and no per-CTA start-up cost is paid more than once per SM slot.  A warp owns one head at a time.  All of the
+// head's operands -- the sketch U, the buffered keys / values / gates of the ring and the current token's
+// q, k, v rows -- arrive in the warp's private shared-memory stage by 1-D bulk asynchronous copies (TMA, no
+// multicast) completing on the warp's mbarrier; the copies of the warp's next head are issued as soon as the
+// current one is done, and the token's scalar gates are fetched one head ahead, so no global-memory latency sits
+// on the per-head critical path except the stage itself.
 //
 // Arithmetic per head (Algorithm 1, non-flush step; Eq. 4):
-//   x <- q_t;  for s = t .. 1:  a_s = beta_s <k_s, x>;  x <- D_s (x - a_s k_s)   [Mamba-2: x <- a_s-decay * x]
+//   x <- q_t;  for s = t .. 1:  a_s = beta_s <k_s, x>;  x <- D_s (x - a_s k_s)   [Mamba-2: a_s = beta_s (prod_{j>s} a_j) <k_s, q_t>]
 //   sketch mode:    o = sum_g (C x)_g U[g,:] + sum_s a_s v_s
 //   full-read mode: o = S_0^T x            + sum_s a_s v_s
+// Sets of independent dot products (C x, and all of Mamba-2's <k_s, q_t>) are reduced eight at a time with a
+// transposing butterfly (9 shuffles per 8 sums instead of 40); the delta-rule chain keeps one 5-step reduction
+// per buffered token.
 #include "internal.cuh"
+#include "lanegroup.cuh"
 
 namespace sketchssm {
 
+namespace {
+
 struct StageLayout {
-    uint32_t u_off, u_bytes;      // sketch U (sketch mode only)
-    uint32_t k_off, k_bytes;      // n buffered keys
-    uint32_t v_off, v_bytes;      // n buffered values
+    uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
+    uint32_t k_off, k_bytes;        // n buffered keys
+    uint32_t v_off, v_bytes;        // n buffered values
     uint32_t gate_off, gate_bytes;  // beta[L] (+ decay[L] for scalar kinds)
-    uint32_t g_off, g_bytes;      // KDA: n per-channel decays
-    uint32_t total;               // stage stride, multiple of 128
+    uint32_t g_off, g_bytes;        // KDA: n per-channel decays
+    uint32_t tq_off, tk_off, tv_off, tg_off, tqk_bytes, tv_bytes, tg_bytes;   // the current token's rows
+    uint32_t total;                 // stage stride, multiple of 128
 };
 
 __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K, int V, int R, int L, int n,
@@ -35,161 +44,138 @@ __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K
     s.gate_bytes = n > 0 ? (uint32_t)((kind == SKETCHSSM_KDA ? 1 : 2) * L * 4) : 0u;
     off += s.gate_bytes;
     s.g_off = off; s.g_bytes = kind == SKETCHSSM_KDA ? (uint32_t)(n * K * io) : 0u; off += s.g_bytes;
+    s.tqk_bytes = (uint32_t)(K * io); s.tv_bytes = (uint32_t)(V * io);
+    s.tg_bytes = kind == SKETCHSSM_KDA ? (uint32_t)(K * io) : 0u;
+    s.tq_off = off; off += s.tqk_bytes;
+    s.tk_off = off; off += s.tqk_bytes;
+    s.tv_off = off; off += s.tv_bytes;
+    s.tg_off = off; off += s.tg_bytes;
     s.total = (off + 127u) & ~127u;
     return s;
 }
 
 struct DecodeSmem {
-    uint32_t coef_bytes, bar_off, x_off, stage_off, total;
+    uint32_t coef_slot_bytes, bar_off, scratch_off, scratch_stride, stage_off, total;
 };
 
 __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps, int stages, int full_read,
                                                        uint32_t stage_bytes) {
     DecodeSmem d;
-    d.coef_bytes = full_read ? 0u : (uint32_t)(R * K * 4);
-    d.bar_off = d.coef_bytes;
+    const int RP = (R + 7) & ~7;                       // coefficient rows padded to the reduction width
+    d.coef_slot_bytes = full_read ? 0u : (uint32_t)(RP * K * 4);
+    d.bar_off = 2u * d.coef_slot_bytes;
     uint32_t off = d.bar_off + (((uint32_t)(nwarps * stages * 8) + 127u) & ~127u);
-    d.x_off = off;
-    off += full_read ? (uint32_t)(nwarps * K * 4) : 0u;
+    d.scratch_stride = (uint32_t)((K + 80) * 4);       // per warp: q~ (full read) or c (K floats), then 64+ dot products
+    d.scratch_off = off; off += (uint32_t)nwarps * d.scratch_stride;
     d.stage_off = off;
     d.total = off + (uint32_t)(nwarps * stages) * stage_bytes;
     return d;
 }
 
+}  // namespace
+
 template <int KIND, typename IO, int K, int V>
 __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
     constexpr int EV = V / 32;
+    constexpr int NB = 8;                               // dot products per transposing reduction
     extern __shared__ __align__(128) unsigned char smem[];
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
-    const int R = p.R, L = p.L, H = p.H, n = p.n_before;
+    const int R = p.R, L = p.L, H = p.H, B = p.B, n = p.n_before;
+    const int RP = (R + 7) & ~7;
     const int stages = p.stages;
-
-    const int chunks = (p.B + p.batches_per_cta - 1) / p.batches_per_cta;
-    const int h = blockIdx.x / chunks;
-    const int b0 = (blockIdx.x % chunks) * p.batches_per_cta;
-    const int b1 = min(p.B, b0 + p.batches_per_cta);
 
     const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n, p.full_read);
     const DecodeSmem ds = make_decode_smem(K, R, nwarps, stages, p.full_read, sl.total);
-    float* sC = reinterpret_cast<float*>(smem);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * stages;
-    float* sX = reinterpret_cast<float*>(smem + ds.x_off) + warp * K;
+    float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
+    float* sP = sX + K;                                                                               // dot products
     unsigned char* my_stage = smem + ds.stage_off + (size_t)warp * stages * sl.total;
+
+    // contiguous range of items for this CTA; item = h * B + b
+    const long long total = (long long)H * B;
+    const int item0 = (int)(total * blockIdx.x / gridDim.x);
+    const int item1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    const int h_first = item0 / B;
+    const int h_last = item1 > item0 ? (item1 - 1) / B : h_first;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < nwarps * stages; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + ds.bar_off) + i, 1);
         mbar_fence_init();
     }
-    if (!p.full_read) {
-        const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)h * R * K);
-        float4* dst = reinterpret_cast<float4*>(sC);
-        for (int i = threadIdx.x; i < R * K / 4; i += blockDim.x) dst[i] = src[i];
-    }
     __syncthreads();
 
-    const uint32_t tx_bytes = sl.u_bytes + sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes;
-    const bool has_copies = tx_bytes > 0;
+    const uint32_t tx_bytes = sl.u_bytes + sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes + 2u * sl.tqk_bytes +
+                              sl.tv_bytes + sl.tg_bytes;
 
-    auto issue = [&](int b, int st) {
-        // lane 0 only
+    auto issue = [&](int item, int st) {   // lane 0 only
         uint64_t* bar = &bars[st];
         unsigned char* sb = my_stage + (size_t)st * sl.total;
+        const int h = item / B, b = item - h * B;
         const size_t bh = (size_t)b * H + h;
         const unsigned char* rh = p.ring + bh * p.rl.head_bytes;
         mbar_expect_tx(bar, tx_bytes);
-        if (sl.u_bytes) bulk_g2s(sb + sl.u_off, p.sketch + bh * (size_t)R * V, sl.u_bytes, bar);
+        bulk_g2s(sb + sl.tq_off, reinterpret_cast<const IO*>(p.q) + bh * K, sl.tqk_bytes, bar);
+        bulk_g2s(sb + sl.tk_off, reinterpret_cast<const IO*>(p.k) + bh * K, sl.tqk_bytes, bar);
+        bulk_g2s(sb + sl.tv_off, reinterpret_cast<const IO*>(p.v) + bh * V, sl.tv_bytes, bar);
+        if (sl.tg_bytes) bulk_g2s(sb + sl.tg_off, reinterpret_cast<const IO*>(p.decay) + bh * K, sl.tg_bytes, bar);
         if (sl.k_bytes) {
             bulk_g2s(sb + sl.k_off, rh, sl.k_bytes, bar);
-            bulk_g2s(sb + sl.v_off, rh + p.rl.v_off, sl.v_bytes, bar);
             bulk_g2s(sb + sl.gate_off, rh + p.rl.beta_off, sl.gate_bytes, bar);
             if (sl.g_bytes) bulk_g2s(sb + sl.g_off, rh + p.rl.decay_off, sl.g_bytes, bar);
+            bulk_g2s(sb + sl.v_off, rh + p.rl.v_off, sl.v_bytes, bar);
         }
+        if (sl.u_bytes) bulk_g2s(sb + sl.u_off, p.sketch + bh * (size_t)R * V, sl.u_bytes, bar);
     };
 
-    const int first_b = b0 + warp;
-    const int count = first_b < b1 ? (b1 - first_b + nwarps - 1) / nwarps : 0;
+    const int n_items = item1 - item0;
+    const int count = warp < n_items ? (n_items - warp + nwarps - 1) / nwarps : 0;
+    auto item_of = [&](int it) { return item0 + warp + it * nwarps; };
+
+    if (count > 0 && lane == 0) issue(item_of(0), 0);
+
+    // coefficient maps of the (at most two) head indices of this range, rows padded with zeros
+    if (!p.full_read && item1 > item0) {
+        const int nslots = h_last > h_first ? 2 : 1;
+        for (int s = 0; s < nslots; ++s) {
+            const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
+            float4* dst = reinterpret_cast<float4*>(smem + (size_t)s * ds.coef_slot_bytes);
+            for (int i = threadIdx.x; i < RP * K / 4; i += blockDim.x)
+                dst[i] = i < R * K / 4 ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+    __syncthreads();
+
+    // the token's scalar gates travel in registers, fetched one head ahead
+    auto scalar_gates = [&](int item, float& bt, float& dsc) {
+        const int h = item / B, b = item - h * B;
+        const size_t bh = (size_t)b * H + h;
+        bt = p.beta[bh];
+        dsc = 1.f;
+        if constexpr (KIND != SKETCHSSM_KDA) dsc = reinterpret_cast<const float*>(p.decay)[bh];
+    };
+    float bt_next = 0.f, dsc_next = 1.f;
+    if (count > 0) scalar_gates(item_of(0), bt_next, dsc_next);
     bool dead = false;
 
-    if (has_copies && count > 0 && lane == 0) issue(first_b, 0);
-
     for (int it = 0; it < count; ++it) {
-        const int b = first_b + it * nwarps;
+        const int item = item_of(it);
         const int st = stages == 2 ? (it & 1) : 0;
         const uint32_t parity = stages == 2 ? ((it >> 1) & 1) : (it & 1);
-        if (stages == 2 && has_copies && it + 1 < count && lane == 0) issue(b + nwarps, st ^ 1);
+        if (stages == 2 && it + 1 < count && lane == 0) issue(item_of(it + 1), st ^ 1);
 
+        const int h = item / B, b = item - h * B;
         const size_t bh = (size_t)b * H + h;
-        const IO* qg = reinterpret_cast<const IO*>(p.q) + bh * K;
-        const IO* kg = reinterpret_cast<const IO*>(p.k) + bh * K;
-        const IO* vg = reinterpret_cast<const IO*>(p.v) + bh * V;
+        const float bt = bt_next, dsc = dsc_next;
+        if (it + 1 < count) scalar_gates(item_of(it + 1), bt_next, dsc_next);
 
-        float q0[EK], x[EK], kk[EK], gg[EK], vv[EV], o[EV];
-        load_io<EK>(qg, lane * EK, q0);
-        load_io<EK>(kg, lane * EK, kk);
-        load_io<EV>(vg, lane * EV, vv);
-        float bt = p.beta[bh];
-        float dsc = 1.f;
-        if constexpr (KIND == SKETCHSSM_KDA) {
-            load_io<EK>(reinterpret_cast<const IO*>(p.decay) + bh * K, lane * EK, gg);
-        } else {
-            dsc = reinterpret_cast<const float*>(p.decay)[bh];
-        }
-#pragma unroll
-        for (int e = 0; e < EK; ++e) x[e] = q0[e];
-#pragma unroll
-        for (int e = 0; e < EV; ++e) o[e] = 0.f;
-
-        if (p.append) {
-            unsigned char* rh = p.ring + bh * p.rl.head_bytes;
-            store_io<EK>(reinterpret_cast<IO*>(rh) + (size_t)n * K, lane * EK, kk);
-            store_io<EV>(reinterpret_cast<IO*>(rh + p.rl.v_off) + (size_t)n * V, lane * EV, vv);
-            if constexpr (KIND == SKETCHSSM_KDA) {
-                store_io<EK>(reinterpret_cast<IO*>(rh + p.rl.decay_off) + (size_t)n * K, lane * EK, gg);
-                if (lane == 0) reinterpret_cast<float*>(rh + p.rl.beta_off)[n] = bt;
-            } else {
-                if (lane == 0) {
-                    reinterpret_cast<float*>(rh + p.rl.beta_off)[n] = bt;
-                    reinterpret_cast<float*>(rh + p.rl.decay_off)[n] = dsc;
-                }
-            }
-        }
-
-        // One step of the backward sweep (M_s^T applied to the running vector) for the token held in
-        // (kk, vv, bt, dsc / gg).  Mamba-2 has no erase, so its running vector is dsuf * q_t.
-        float dsuf = 1.f;
-        auto sweep = [&]() {
-            float part = 0.f;
-#pragma unroll
-            for (int e = 0; e < EK; ++e) part = fmaf(kk[e], x[e], part);
-            const float dot = warp_sum(part);
-            float a;
-            if constexpr (KIND == SKETCHSSM_MAMBA2) {
-                a = bt * dsuf * dot;
-                dsuf *= dsc;
-            } else if constexpr (KIND == SKETCHSSM_GDN) {
-                a = bt * dot;
-#pragma unroll
-                for (int e = 0; e < EK; ++e) x[e] = dsc * fmaf(-a, kk[e], x[e]);
-            } else {
-                a = bt * dot;
-#pragma unroll
-                for (int e = 0; e < EK; ++e) x[e] = gg[e] * fmaf(-a, kk[e], x[e]);
-            }
-#pragma unroll
-            for (int e = 0; e < EV; ++e) o[e] = fmaf(a, vv[e], o[e]);
-        };
-        sweep();  // the current token, s = t
-
-        if (has_copies) {
-            if (!mbar_wait_bounded(&bars[st], parity)) {
-                record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
-                dead = true;
-                break;
-            }
+        if (!mbar_wait_bounded(&bars[st], parity)) {
+            record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
+            dead = true;
+            break;
         }
         const unsigned char* sb = my_stage + (size_t)st * sl.total;
         const IO* sK = reinterpret_cast<const IO*>(sb + sl.k_off);
@@ -198,37 +184,129 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
         const float* sDec = sBeta + L;
         const IO* sG = reinterpret_cast<const IO*>(sb + sl.g_off);
 
-        for (int s = n - 1; s >= 0; --s) {
-            load_io<EK>(sK, s * K + lane * EK, kk);
-            load_io<EV>(sV, s * V + lane * EV, vv);
-            bt = sBeta[s];
+        float q0[EK], x[EK], kk[EK], gg[EK], vv[EV], o[EV];
+        load_io<EK>(reinterpret_cast<const IO*>(sb + sl.tq_off), lane * EK, q0);
+        load_io<EK>(reinterpret_cast<const IO*>(sb + sl.tk_off), lane * EK, kk);
+        load_io<EV>(reinterpret_cast<const IO*>(sb + sl.tv_off), lane * EV, vv);
+        if constexpr (KIND == SKETCHSSM_KDA) load_io<EK>(reinterpret_cast<const IO*>(sb + sl.tg_off), lane * EK, gg);
+
+        if (p.append) {
+            unsigned char* rh = p.ring + bh * p.rl.head_bytes;
+            store_io<EK>(reinterpret_cast<IO*>(rh) + (size_t)n * K, lane * EK, kk);
+            store_io<EV>(reinterpret_cast<IO*>(rh + p.rl.v_off) + (size_t)n * V, lane * EV, vv);
             if constexpr (KIND == SKETCHSSM_KDA) {
-                load_io<EK>(sG, s * K + lane * EK, gg);
-            } else {
-                dsc = sDec[s];
+                store_io<EK>(reinterpret_cast<IO*>(rh + p.rl.decay_off) + (size_t)n * K, lane * EK, gg);
+                if (lane == 0) reinterpret_cast<float*>(rh + p.rl.beta_off)[n] = bt;
+            } else if (lane == 0) {
+                reinterpret_cast<float*>(rh + p.rl.beta_off)[n] = bt;
+                reinterpret_cast<float*>(rh + p.rl.decay_off)[n] = dsc;
             }
-            sweep();
         }
+
+        // ---- current token, s = t ----
+        float dsuf = 1.f;
+        {
+            float part = 0.f;
+#pragma unroll
+            for (int e = 0; e < EK; ++e) part = fmaf(kk[e], q0[e], part);
+            const float a = bt * warp_sum(part);
+#pragma unroll
+            for (int e = 0; e < EV; ++e) o[e] = a * vv[e];
+            if constexpr (KIND == SKETCHSSM_MAMBA2) {
+                dsuf = dsc;
+            } else if constexpr (KIND == SKETCHSSM_GDN) {
+#pragma unroll
+                for (int e = 0; e < EK; ++e) x[e] = dsc * fmaf(-a, kk[e], q0[e]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < EK; ++e) x[e] = gg[e] * fmaf(-a, kk[e], q0[e]);
+            }
+        }
+
+        // ---- buffered tokens ----
         if constexpr (KIND == SKETCHSSM_MAMBA2) {
+            // independent dot products <k_s, q_t>, eight per transposing reduction; lane l ends up with slot s0 + l/4
+            for (int s0 = 0; s0 < n; s0 += NB) {
+                float part[NB];
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
+                    float kr[EK];
+                    load_io<EK>(sK, min(s0 + i, n - 1) * K + lane * EK, kr);
+                    float acc = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EK; ++e) acc = fmaf(kr[e], q0[e], acc);
+                    part[i] = acc;
+                }
+                group_reduce_transpose<32, NB>(part, lane);
+                if ((lane & 3) == 0) sP[s0 + (lane >> 2)] = part[0];
+            }
+            __syncwarp();
+#pragma unroll 4
+            for (int s = n - 1; s >= 0; --s) {
+                const float a = sBeta[s] * dsuf * sP[s];
+                dsuf *= sDec[s];
+                float vr[EV];
+                load_io<EV>(sV, s * V + lane * EV, vr);
+#pragma unroll
+                for (int e = 0; e < EV; ++e) o[e] = fmaf(a, vr[e], o[e]);
+            }
 #pragma unroll
             for (int e = 0; e < EK; ++e) x[e] = dsuf * q0[e];
+        } else {
+#pragma unroll 2
+            for (int s = n - 1; s >= 0; --s) {
+                float kr[EK], vr[EV];
+                load_io<EK>(sK, s * K + lane * EK, kr);
+                load_io<EV>(sV, s * V + lane * EV, vr);
+                float part = 0.f;
+#pragma unroll
+                for (int e = 0; e < EK; ++e) part = fmaf(kr[e], x[e], part);
+                const float a = sBeta[s] * warp_sum(part);
+                if constexpr (KIND == SKETCHSSM_GDN) {
+                    const float d = sDec[s];
+#pragma unroll
+                    for (int e = 0; e < EK; ++e) x[e] = d * fmaf(-a, kr[e], x[e]);
+                } else {
+                    float gr[EK];
+                    load_io<EK>(sG, s * K + lane * EK, gr);
+#pragma unroll
+                    for (int e = 0; e < EK; ++e) x[e] = gr[e] * fmaf(-a, kr[e], x[e]);
+                }
+#pragma unroll
+                for (int e = 0; e < EV; ++e) o[e] = fmaf(a, vr[e], o[e]);
+            }
         }
 
         if (!p.full_read) {
+            // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
+            const float* sC = reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
+            __syncwarp();
+            for (int g0 = 0; g0 < RP; g0 += NB) {
+                float part[NB];
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
+                    float cw[EK];
+                    load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
+                    float acc = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EK; ++e) acc = fmaf(cw[e], x[e], acc);
+                    part[i] = acc;
+                }
+                group_reduce_transpose<32, NB>(part, lane);
+                if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
+            }
+            __syncwarp();
             const float* sU = reinterpret_cast<const float*>(sb + sl.u_off);
 #pragma unroll 4
             for (int g = 0; g < R; ++g) {
-                float cw[EK], uu[EV];
-                load_io<EK>(sC, g * K + lane * EK, cw);
+                const float cg = sX[g];
+                float uu[EV];
                 load_io<EV>(sU, g * V + lane * EV, uu);
-                float part = 0.f;
-#pragma unroll
-                for (int e = 0; e < EK; ++e) part = fmaf(cw[e], x[e], part);
-                const float cg = warp_sum(part);
 #pragma unroll
                 for (int e = 0; e < EV; ++e) o[e] = fmaf(cg, uu[e], o[e]);
             }
         } else {
+            __syncwarp();
             store_io<EK>(sX, lane * EK, x);
             __syncwarp();
             const float* Sg = p.state + bh * (size_t)K * V + lane * EV;
@@ -244,7 +322,6 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
                     for (int e = 0; e < EV; ++e) o[e] = fmaf(rows[r][e], xi, o[e]);
                 }
             }
-            __syncwarp();
         }
 
         if (p.out_bf16) {
@@ -253,12 +330,11 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
             store_io<EV>(reinterpret_cast<float*>(p.out) + bh * V, lane * EV, o);
         }
 
-        __syncwarp();  // every lane is done reading this stage before it is refilled
-        if (stages == 1 && has_copies && it + 1 < count && lane == 0) issue(b + nwarps, 0);
+        __syncwarp();  // every lane is done with this stage and the scratch before either is reused
+        if (stages == 1 && it + 1 < count && lane == 0) issue(item_of(it + 1), 0);
     }
 
-    if (dead && stages == 2 && has_copies) {
-        // give the other stage's copies a bounded chance to land before the CTA retires
+    if (dead && stages == 2) {   // bounded grace period for the other stage's copies before the CTA retires
         mbar_wait_bounded(&bars[0], 0, 1u << 16);
         mbar_wait_bounded(&bars[1], 0, 1u << 16);
     }
@@ -268,48 +344,42 @@ template <int KIND, typename IO, int K, int V>
 static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     const int io = (int)sizeof(IO);
     const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read);
-    const size_t smem_budget = 227u * 1024u;
-    // choose warps per CTA and stage count: as many resident warps per SM as shared memory allows
-    int best_nw = 1, best_stages = 1, best_warps = 0;
-    const int stage_opts[2] = {1, 2};
-    for (int si = 0; si < 2; ++si) {
-        for (int nw = 8; nw >= 1; --nw) {
-            const DecodeSmem d = make_decode_smem(K, p.R, nw, stage_opts[si], p.full_read, sl.total);
-            if (d.total > smem_budget) continue;
-            int ctas = (int)(smem_budget / (d.total + 1024u));
-            if (ctas < 1) ctas = 1;
-            if (ctas * nw > 48) ctas = 48 / nw;   // 48 warps is plenty; keeps register pressure irrelevant
-            if (ctas > 32) ctas = 32;
-            const int warps = ctas * nw;
-            // prefer more resident warps; at equal warps prefer a single stage with more CTAs
-            if (warps > best_warps) { best_warps = warps; best_nw = nw; best_stages = stage_opts[si]; }
-        }
+    const uint32_t smem_budget = 227u * 1024u;
+    if (ctx->sm_count == 0) {
+        int dev = 0, sms = 0;
+        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return SKETCHSSM_CUDA_ERROR;
+        ctx->sm_count = sms;
     }
-    if (p.stages == 1 || p.stages == 2) {
-        // explicit request: re-pick the warp count for that stage count
-        best_warps = 0;
-        for (int nw = 8; nw >= 1; --nw) {
-            const DecodeSmem d = make_decode_smem(K, p.R, nw, p.stages, p.full_read, sl.total);
-            if (d.total > smem_budget) continue;
-            int ctas = (int)(smem_budget / (d.total + 1024u));
-            if (ctas < 1) ctas = 1;
-            if (ctas * nw > 48) ctas = 48 / nw;
-            const int warps = ctas * nw;
-            if (warps > best_warps) { best_warps = warps; best_nw = nw; }
-        }
-        best_stages = p.stages;
+    // warps per CTA / stages / CTAs per SM: as many resident warps per SM as shared memory allows (capped),
+    // preferring a single stage (more heads in flight per byte of shared memory) and fewer, larger CTAs
+    const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
+    const int want_st = (p.stages == 1 || p.stages == 2) ? p.stages : 1;
+    int best_nw = 0, best_ctas = 1, best_warps = 0;
+    for (int nw = 8; nw >= 1; --nw) {
+        if (p.warps_per_cta && nw != p.warps_per_cta) continue;
+        const DecodeSmem d = make_decode_smem(K, p.R, nw, want_st, p.full_read, sl.total);
+        if (d.total > smem_budget) continue;
+        int ctas = (int)((228u * 1024u) / (d.total + 1024u));
+        if (ctas * nw > cap) ctas = cap / nw;
+        if (ctas < 1) continue;
+        if (ctas * nw > best_warps) { best_warps = ctas * nw; best_nw = nw; best_ctas = ctas; }
     }
-    if (best_warps == 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    p.stages = best_stages;
-    if (p.batches_per_cta <= 0) p.batches_per_cta = best_nw * 2;
-    const DecodeSmem d = make_decode_smem(K, p.R, best_nw, best_stages, p.full_read, sl.total);
+    if (best_nw == 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    p.stages = want_st;
+    const DecodeSmem d = make_decode_smem(K, p.R, best_nw, want_st, p.full_read, sl.total);
     auto kern = decode_kernel<KIND, IO, K, V>;
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)d.total)) != cudaSuccess)
         return SKETCHSSM_CUDA_ERROR;
-    const int chunks = (p.B + p.batches_per_cta - 1) / p.batches_per_cta;
-    const dim3 grid((unsigned)(p.H * chunks));
-    kern<<<grid, best_nw * 32, d.total, stream>>>(p);
+    long long grid = (long long)ctx->sm_count * best_ctas;
+    const long long total = (long long)p.B * p.H;
+    if (p.batches_per_cta > 0) grid = (total + p.batches_per_cta - 1) / p.batches_per_cta;   // explicit items per CTA
+    if (grid > (total + best_nw - 1) / best_nw) grid = (total + best_nw - 1) / best_nw;      // at least one head per warp
+    if (grid < p.H) grid = p.H;                                  // a CTA's range then spans at most two head indices
+    if (grid > total) grid = total;
+    kern<<<dim3((unsigned)grid), best_nw * 32, d.total, stream>>>(p);
     if ((ctx->last_cuda_error = cudaGetLastError()) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
     ctx->last_launches = 1;
     return SKETCHSSM_OK;
