@@ -32,9 +32,19 @@ from paper_2609_33051_b200 import synth, traffic  # noqa: E402
 
 METRIC = "decode tokens/s per layer"
 UNIT = "tokens/s/layer"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (None until a capture of that kernel/workload exists)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/:
+# (kernel, workload) -> (captured bytes, algorithmic bytes of the captured launches).  Traffic grows in proportion
+# to the algorithmic bytes (ring fill), so the bench line scales the captured figure to its own average launch.
+NCU_TRAFFIC_CAPTURES = {
+    ("decode_kernel", "c2_mamba2"): (117.74e6, 0.5 * (traffic.decode_bytes("mamba2", 256, 64, 128, 64, 16, 4, "bf16")
+                                                      + traffic.decode_bytes("mamba2", 256, 64, 128, 64, 16, 5, "bf16"))),
+    ("update_kernel", "c2_mamba2"): (1199.06e6, float(traffic.update_bytes("mamba2", 256, 64, 128, 64, 16, 15, "bf16"))),
+}
+
+
+def ncu_traffic(kernel: str, workload: str, algorithmic_bytes_per_launch: float):
+    cap = NCU_TRAFFIC_CAPTURES.get((kernel, workload))
+    return None if cap is None else cap[0] * algorithmic_bytes_per_launch / cap[1]
 
 
 def max_over_ranks(ms_local: float, dist, device="cuda") -> float:
@@ -403,7 +413,8 @@ def main():
         kname = "decode_kernel" if dominant == "decode" else "update_kernel"
         roofline = {"bound": "hbm", "kernel": kname, "achieved": kern[dominant]["achieved_gbs"], "peak": peak,
                     "unit": "GB/s", "frac": kern[dominant]["achieved_gbs"] / peak, "peak_source": peak_kind,
-                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get((kname, w.name)),
+                    "traffic": ncu_traffic(kname, w.name, kern[dominant]["algorithmic_bytes_per_launch"]),
+                    "algorithmic_bytes_per_launch": kern[dominant]["algorithmic_bytes_per_launch"],
                     "frac_of_8TBs_nominal": kern[dominant]["achieved_gbs"] / 8000.0}
 
     # ---- in-library full-read baseline (buffered replay that reads all of S every step) ----
