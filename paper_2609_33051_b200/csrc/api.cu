@@ -14,6 +14,7 @@ struct sketchssm_ctx : public Ctx {
     int tune_max_warps;
     int tune_update_impl;
     int tune_decode_mma;
+    int tune_pdl;
     int tune_l2_prefetch;   // lane-group kernel: 1 (default) / 0
 };
 
@@ -61,6 +62,7 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.max_warps_per_sm = ctx->tune_max_warps;
     p.update_impl = ctx->tune_update_impl;
     p.decode_mma = ctx->tune_decode_mma;
+    p.pdl = ctx->tune_pdl;
     return p;
 }
 
@@ -151,6 +153,7 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     c->tune_max_warps = 0;
     c->tune_update_impl = 0;
     c->tune_decode_mma = 0;
+    c->tune_pdl = 1;
     *out = c;
     return SKETCHSSM_OK;
 }
@@ -326,6 +329,7 @@ int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value) {
     if (eq(key, "decode_lanes_per_head")) { ctx->tune_lanes_per_head = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_l2_prefetch")) { ctx->tune_l2_prefetch = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_max_warps_per_sm")) { ctx->tune_max_warps = value; return SKETCHSSM_OK; }
+    if (eq(key, "pdl")) { ctx->tune_pdl = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_mma")) { ctx->tune_decode_mma = value; return SKETCHSSM_OK; }
     if (eq(key, "update_impl")) { ctx->tune_update_impl = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_impl")) { ctx->tune_decode_impl = value; return SKETCHSSM_OK; }

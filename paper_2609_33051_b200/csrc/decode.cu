@@ -106,7 +106,20 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
         for (int i = 0; i < nwarps * stages; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + ds.bar_off) + i, 1);
         mbar_fence_init();
     }
+    // coefficient maps of the (at most two) head indices of this range, rows padded with zeros.  C is a constant of
+    // the layer (never written by these kernels), so it may be staged before the predecessor in the stream is done.
+    if (!p.full_read && item1 > item0) {
+        const int nslots = h_last > h_first ? 2 : 1;
+        for (int s = 0; s < nslots; ++s) {
+            const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
+            float4* dst = reinterpret_cast<float4*>(smem + (size_t)s * ds.coef_slot_bytes);
+            for (int i = threadIdx.x; i < RP * K / 4; i += blockDim.x)
+                dst[i] = i < R * K / 4 ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
     __syncthreads();
+    grid_dep_wait();                 // from here on the ring, the sketch and the token tensors are read
+    grid_dep_launch_dependents();
 
     const uint32_t tx_bytes = sl.u_bytes + sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes + 2u * sl.tqk_bytes +
                               sl.tv_bytes + sl.tg_bytes;
@@ -136,18 +149,6 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
     auto item_of = [&](int it) { return item0 + warp + it * nwarps; };
 
     if (count > 0 && lane == 0) issue(item_of(0), 0);
-
-    // coefficient maps of the (at most two) head indices of this range, rows padded with zeros
-    if (!p.full_read && item1 > item0) {
-        const int nslots = h_last > h_first ? 2 : 1;
-        for (int s = 0; s < nslots; ++s) {
-            const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
-            float4* dst = reinterpret_cast<float4*>(smem + (size_t)s * ds.coef_slot_bytes);
-            for (int i = threadIdx.x; i < RP * K / 4; i += blockDim.x)
-                dst[i] = i < R * K / 4 ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    }
-    __syncthreads();
 
     // the token's scalar gates travel in registers, fetched one head ahead
     auto scalar_gates = [&](int item, float& bt, float& dsc) {
@@ -379,8 +380,8 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     if (grid > (total + best_nw - 1) / best_nw) grid = (total + best_nw - 1) / best_nw;      // at least one head per warp
     if (grid < p.H) grid = p.H;                                  // a CTA's range then spans at most two head indices
     if (grid > total) grid = total;
-    kern<<<dim3((unsigned)grid), best_nw * 32, d.total, stream>>>(p);
-    if ((ctx->last_cuda_error = cudaGetLastError()) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+    if ((ctx->last_cuda_error = launch_kernel(kern, dim3((unsigned)grid), dim3(best_nw * 32), d.total, stream, p, p.pdl != 0)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
     ctx->last_launches = 1;
     return SKETCHSSM_OK;
 }

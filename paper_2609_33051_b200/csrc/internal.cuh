@@ -69,6 +69,7 @@ struct Params {
     int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
     int update_impl;      // 0: tensor cores where supported, 1: CUDA cores only
     int decode_mma;       // warp-per-head decode: 1 = tensor-core dot products where supported
+    int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
 };
 
 int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head
@@ -96,6 +97,23 @@ int launch_update_tc(Ctx* ctx, const Params& p, cudaStream_t stream);    // tcge
 // device helpers
 // ---------------------------------------------------------------------------------------------
 #ifdef __CUDACC__
+
+// Launch with (or without) the programmatic-stream-serialization attribute.
+template <typename Kern>
+inline cudaError_t launch_kernel(Kern kern, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, const Params& p,
+                                 bool pdl) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, p);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -146,6 +164,12 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
                  "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
+
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its
+// predecessor in the stream is still draining; everything it does before grid_dep_wait() must not touch memory the
+// predecessor may write.  Both instructions are no-ops for a normally launched kernel.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void record_fault(int* status, int code, int where) {
     if (status != nullptr) {

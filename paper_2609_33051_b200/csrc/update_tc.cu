@@ -162,6 +162,8 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    grid_dep_wait();                 // nothing above reads memory another kernel may write
+    grid_dep_launch_dependents();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_t = tmem_base;                          // T: 128 columns
     const uint32_t tmem_u = tmem_base + (NP <= 32 ? 0u : 128u); // UT: NP columns (re-uses consumed T columns if it fits)
@@ -442,8 +444,8 @@ int launch_update_tc(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)sm.total)) != cudaSuccess)
         return SKETCHSSM_CUDA_ERROR;
-    kern<<<dim3((unsigned)grid), kTcThreads, sm.total, stream>>>(p);
-    if ((ctx->last_cuda_error = cudaGetLastError()) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+    if ((ctx->last_cuda_error = launch_kernel(kern, dim3((unsigned)grid), dim3(kTcThreads), sm.total, stream, p, p.pdl != 0)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
     ctx->last_launches = 1;
     return SKETCHSSM_OK;
 }
