@@ -223,6 +223,24 @@ class Stack:
                     events.append(("decode" if t < L - 1 else "update", t, e0, e1))
         return launches
 
+    def run_decode_only(self):
+        """The L-1 decode steps of a window over every layer, back to back, no flush (the ring slots are simply
+        rewritten with the same tokens on the next pass)."""
+        L = self.w.buf_len
+        for t in range(L - 1):
+            for li, m in enumerate(self.layers):
+                tok = self.inputs[li][t]
+                m.decode_step(t, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], self.outs[li])
+        return (L - 1) * self.n_layers
+
+    def run_update_only(self):
+        """One flush per layer, back to back (full ring: n_before = L-1 plus the token)."""
+        L = self.w.buf_len
+        for li, m in enumerate(self.layers):
+            tok = self.inputs[li][L - 1]
+            m.state_update(L - 1, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], self.outs[li])
+        return self.n_layers
+
     # -- end-to-end: host buffers, copies inside the timed region ---------------------------------
     def setup_host(self):
         m = self.layers[0]
@@ -233,20 +251,30 @@ class Stack:
                 hb[k].copy_(tok[k])
             self.host_window.append(hb)
         self.staging = [m.new_token_buffers(pinned_host=False) for _ in range(2)]
+        self.host_out = [m.new_token_buffers(pinned_host=True)["out"] for _ in range(2)]
+        self.side_streams = [torch.cuda.Stream(device=self.device) for _ in range(2)]
 
     def run_window_host(self):
+        """One window with host token tensors.  Layer-steps alternate between two streams (each with its own device
+        staging and host output buffer) so that the upload of one layer-step overlaps the kernel and the download
+        of the previous one; a layer always uses the same stream, so its own steps stay ordered."""
         from paper_2609_33051_b200 import binding
         L = self.w.buf_len
         h2d = d2h = 0
-        i = 0
+        cur = torch.cuda.current_stream()
+        for s in self.side_streams:
+            s.wait_stream(cur)
         for t in range(L):
             hb = self.host_window[t]
-            for m in self.layers:
+            for li, m in enumerate(self.layers):
                 op = binding.OP_DECODE if t < L - 1 else binding.OP_UPDATE
-                m.step_host(op, t, hb, self.staging[i & 1])
-                i += 1
+                host = dict(hb)
+                host["out"] = self.host_out[li & 1]
+                m.step_host(op, t, host, self.staging[li & 1], stream=self.side_streams[li & 1])
                 h2d += sum(hb[k].numel() * hb[k].element_size() for k in ("q", "k", "v", "beta", "decay"))
-                d2h += hb["out"].numel() * hb["out"].element_size()
+                d2h += host["out"].numel() * host["out"].element_size()
+        for s in self.side_streams:
+            cur.wait_stream(s)
         return h2d, d2h
 
 
@@ -407,15 +435,38 @@ def main():
             if n:
                 kern[kind] = {"launches": n, "avg_us": 1e3 * ms / n, "share": ms / (agg["decode"][0] + agg["update"][0]),
                               "algorithmic_bytes_per_launch": by / n, "achieved_gbs": by / (ms * 1e-3) / 1e9}
+    # Back-to-back runs of one kernel between two events: the average launch duration as the stream sees it.
+    # An event between two launches removes the programmatic dependent launch overlap, so the bracketed figures
+    # above are the conservative ones; these are what a window actually pays per launch.
+    b2b = {}
+    if not args.no_launch_events:
+        reps = max(3, args.steps // 4)
+        ms_d, _, _ = timed_region(stack.run_decode_only, reps, 2)
+        n_d = (L - 1) * args.layers
+        by_d = sum(traffic.decode_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io) for t in range(L - 1)) / (L - 1)
+        b2b["decode"] = {"avg_us": 1e3 * ms_d / n_d, "achieved_gbs": by_d / (ms_d / n_d * 1e-3) / 1e9}
+        ms_u, _, _ = timed_region(stack.run_update_only, reps, 2)
+        by_u = traffic.update_bytes(w.kind, B, H, w.dk, w.dv, w.rank, L - 1, w.io)
+        b2b["update"] = {"avg_us": 1e3 * ms_u / args.layers, "achieved_gbs": by_u / (ms_u / args.layers * 1e-3) / 1e9}
+        stack.run_window("sketch", None)     # leave every layer at the start of a window again
+        for k in b2b:
+            if k in kern:
+                kern[k]["back_to_back_avg_us"] = b2b[k]["avg_us"]
+                kern[k]["back_to_back_achieved_gbs"] = b2b[k]["achieved_gbs"]
     dominant = max(kern, key=lambda k: kern[k]["share"]) if kern else None
     roofline = None
     if dominant:
         kname = "decode_kernel" if dominant == "decode" else "update_kernel"
-        roofline = {"bound": "hbm", "kernel": kname, "achieved": kern[dominant]["achieved_gbs"], "peak": peak,
-                    "unit": "GB/s", "frac": kern[dominant]["achieved_gbs"] / peak, "peak_source": peak_kind,
+        ach = b2b.get(dominant, {}).get("achieved_gbs", kern[dominant]["achieved_gbs"])
+        roofline = {"bound": "hbm", "kernel": kname, "achieved": ach, "peak": peak,
+                    "unit": "GB/s", "frac": ach / peak, "peak_source": peak_kind,
                     "traffic": ncu_traffic(kname, w.name, kern[dominant]["algorithmic_bytes_per_launch"]),
                     "algorithmic_bytes_per_launch": kern[dominant]["algorithmic_bytes_per_launch"],
-                    "frac_of_8TBs_nominal": kern[dominant]["achieved_gbs"] / 8000.0}
+                    "duration": "average over a run of back-to-back launches between two CUDA events "
+                                "(programmatic dependent launch overlaps heads and tails of consecutive launches)",
+                    "achieved_bracketed": kern[dominant]["achieved_gbs"],
+                    "frac_bracketed": kern[dominant]["achieved_gbs"] / peak,
+                    "frac_of_8TBs_nominal": ach / 8000.0}
 
     # ---- in-library full-read baseline (buffered replay that reads all of S every step) ----
     full = None
@@ -438,7 +489,8 @@ def main():
         ms_e2e, _, _ = timed_region(host_step, args.e2e_steps, 3)
         e2e = {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": bytes_io[0],
                "d2h_bytes_per_step": bytes_io[1], "ms_per_step": ms_e2e, "steps": args.e2e_steps,
-               "what": "sketchssm_step_host per layer-step: pinned host q,k,v,beta,decay -> device, kernel, o -> host"}
+               "what": "sketchssm_step_host per layer-step: pinned host q,k,v,beta,decay -> device, kernel, o -> host; "
+                       "layer-steps alternate between two streams so uploads overlap kernels and downloads"}
     for m in stack.layers:
         m.check_status()
 
