@@ -11,13 +11,13 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsketchssm.so")
 # (source, object suffix, extra defines); the lane-group decode kernel is compiled once per (recurrence kind, I/O type)
-UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []),
+UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []), ("update_tc_delta.cu", "", []),
          ("decode_static.cu", "", []), ("decode_mma.cu", "", []),
          *[("decode_fused.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
            for k in range(3) for io in range(2)],
          *[("decode_split.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
            for k in range(3) for io in range(2)]]
-HEADERS = [os.path.join(CSRC, "internal.cuh"), os.path.join(CSRC, "lanegroup.cuh"),
+HEADERS = [os.path.join(CSRC, "internal.cuh"), os.path.join(CSRC, "lanegroup.cuh"), os.path.join(CSRC, "tc_common.cuh"),
            os.path.join(ROOT, "include", "sketchssm.h")]
 
 

@@ -223,6 +223,11 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     if (p.update_impl == 0) {
         rc = launch_update_tc(ctx, p, static_cast<cudaStream_t>(stream));
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+
+    }
+    if (p.update_impl == 2) {       // opt-in: gated delta rule on tensor cores (measured slower than the CUDA-core kernel so far)
+        rc = launch_update_tc_delta(ctx, p, static_cast<cudaStream_t>(stream));
+        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
     }
     return launch_update(ctx, p, static_cast<cudaStream_t>(stream));
 }

@@ -151,6 +151,13 @@ def test_mamba2_tensor_core_variants(dv, rank, buf_len):
     check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"update_impl": 1}), "bf16")
 
 
+@pytest.mark.parametrize("rank,buf_len,steps", [(16, 16, 37), (8, 32, 70), (40, 12, 30)])
+def test_gdn_tensor_core_update(rank, buf_len, steps):
+    """The gated delta rule flush as tcgen05 contractions (WY form) against the oracle's token-by-token replay."""
+    w = synth.Workload("t", "gdn", 5, 3, 128, 128, rank, buf_len, 0, "bf16", 91, basis="qr")
+    check(run_schedule(w, steps, max_heads=10**9, tune={"update_impl": 2}), "bf16")
+
+
 def test_bf16_output_mode():
     w = synth.Workload("t", "gdn", 4, 2, 128, 128, 16, 8, 0, "bf16", 5, basis="qr")
     errs = run_schedule(w, 12, max_heads=10**9, out="bf16")
