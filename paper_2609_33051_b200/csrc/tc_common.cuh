@@ -31,6 +31,14 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar) {
                  : "memory");
 }
 
+// CTA-wide bounded wait: one warp polls the mbarrier, the others sleep in the block barrier instead of competing
+// for issue slots with the co-resident CTAs.  Returns false (to every thread) if the wait ran out.
+__device__ __forceinline__ bool cta_wait(uint64_t* bar, uint32_t phase) {
+    int bad = 0;
+    if (threadIdx.x < 32) bad = mbar_wait_bounded(bar, phase) ? 0 : 1;
+    return __syncthreads_or(bad) == 0;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -27,10 +27,10 @@ namespace {
 using namespace tc;
 
 struct TcSmem {
-    uint32_t a1_hi, a1_lo, b1, a2, b2_hi, b2_lo, w, bars, tmem_slot, total;
+    uint32_t a1_hi, a1_lo, b1, a2, b2_hi, b2_lo, w, stg, stg_head, bars, tmem_slot, total;
 };
 
-__host__ __device__ inline TcSmem make_tc_smem(int NH, int NP) {
+__host__ __device__ inline TcSmem make_tc_smem(int NH, int NP, int V = 64, int L = 16) {
     TcSmem s;
     const uint32_t kd1 = (uint32_t)(kTokBlock * NH);
     uint32_t off = 0;
@@ -40,11 +40,14 @@ __host__ __device__ inline TcSmem make_tc_smem(int NH, int NP) {
     s.a1_lo = off + 128u * kd1 * 2u;
     s.b1 = off + 2u * 128u * kd1 * 2u;
     s.a2 = off;
-    const uint32_t mma1_bytes = 3u * 128u * kd1 * 2u, mma2_bytes = 2u * 2u * 128u * kChunk * 2u;   // two chunk buffers, hi + lo
+    const uint32_t mma1_bytes = 3u * 128u * kd1 * 2u, mma2_bytes = 2u * 2u * 128u * 16u * 2u;   // two 16-row chunk buffers, hi + lo
     off += mma1_bytes > mma2_bytes ? mma1_bytes : mma2_bytes;
     s.b2_hi = off; off += (uint32_t)NP * kK * 2u;
     s.b2_lo = off; off += (uint32_t)NP * kK * 2u;
     s.w = off; off += 2u * 208u * 4u;                    // per head: w_s (64), total decay (16), beta_s (64), a_s (64)
+    // staging of the next tile's raw ring rows (first token block): per head keys [16][256 B], values [16][V*2 B], gates [2L] floats
+    s.stg_head = 16u * 256u + 16u * (uint32_t)V * 2u + (((uint32_t)(2 * L * 4) + 127u) & ~127u);
+    s.stg = off; off += (uint32_t)NH * s.stg_head;
     s.bars = off; off += 64u;
     s.tmem_slot = off; off += 64u;
     s.total = off;
@@ -65,7 +68,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
     const int R = p.R, H = p.H, B = p.B;
     const int NP = (R + NH + 15) & ~15;                   // sketch ranks + one query column per head, padded
     const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);
-    const TcSmem sm = make_tc_smem(NH, NP);
+    const TcSmem sm = make_tc_smem(NH, NP, V, p.L);
     __nv_bfloat16* sA1hi = reinterpret_cast<__nv_bfloat16*>(smem + sm.a1_hi);
     __nv_bfloat16* sA1lo = reinterpret_cast<__nv_bfloat16*>(smem + sm.a1_lo);
     __nv_bfloat16* sB1 = reinterpret_cast<__nv_bfloat16*>(smem + sm.b1);
@@ -73,7 +76,8 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
     __nv_bfloat16* sB2hi = reinterpret_cast<__nv_bfloat16*>(smem + sm.b2_hi);
     __nv_bfloat16* sB2lo = reinterpret_cast<__nv_bfloat16*>(smem + sm.b2_lo);
     float* sW = reinterpret_cast<float*>(smem + sm.w);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);     // [0] MMA 1, [1..2] MMA 2 chunk buffers, [3] MMA 2 all
+    unsigned char* sStg = smem + sm.stg;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);     // [0] MMA 1, [1..2] MMA 2 chunk buffers, [3] MMA 2 all, [4] staging
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.tmem_slot);
 
     const uint32_t tmem_cols = NP <= 32 ? 128u : 256u;
@@ -84,7 +88,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
-        for (int i = 0; i < 4; ++i) mbar_init(&bars[i], 1);
+        for (int i = 0; i < 5; ++i) mbar_init(&bars[i], 1);
         mbar_fence_init();
     }
     tc_fence_before();
@@ -116,8 +120,36 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
     const int my_head = tid / V;          // which head of the tile this thread's lane belongs to
     const int j = tid % V;
     int cur_h = -1;
-    uint32_t ph0 = 0, ph1[2] = {0, 0}, ph3 = 0;   // mbarrier phases
+    uint32_t ph0 = 0, ph1[2] = {0, 0}, ph3 = 0, ph4 = 0;   // mbarrier phases
     bool dead = false;
+
+    // Raw ring rows of a tile's first token block travel to shared memory by bulk copies issued one tile ahead, so that
+    // building the MMA-1 operands never waits on global memory.  Rows of later blocks (n > 16) are read directly.
+    const int rows0 = n_ring < kTokBlock ? n_ring : kTokBlock;
+    const bool tok0 = p.has_token && n_ring < kTokBlock;
+    const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
+    const uint32_t stg_bytes = (uint32_t)NH * ((uint32_t)rows0 * 256u + (uint32_t)rows0 * V * 2u + stg_gate_bytes +
+                                              (tok0 ? 256u + (uint32_t)V * 2u : 0u));
+    auto stage_tile = [&](int tile) {       // thread 0 only
+        const int h = tile / tiles_per_h;
+        const int b0 = (tile - h * tiles_per_h) * NH;
+        mbar_expect_tx(&bars[4], stg_bytes);
+        for (int hd = 0; hd < NH; ++hd) {
+            const size_t bw = (size_t)(b0 + hd) * H + h;
+            const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
+            unsigned char* dst = sStg + (size_t)hd * sm.stg_head;
+            if (rows0 > 0) {
+                bulk_g2s(dst, rh, (uint32_t)rows0 * 256u, &bars[4]);
+                bulk_g2s(dst + 4096, rh + p.rl.v_off, (uint32_t)rows0 * V * 2u, &bars[4]);
+            }
+            if (stg_gate_bytes) bulk_g2s(dst + 4096 + 16 * V * 2, rh + p.rl.beta_off, stg_gate_bytes, &bars[4]);
+            if (tok0) {
+                bulk_g2s(dst + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.k) + bw * K, 256u, &bars[4]);
+                bulk_g2s(dst + 4096 + (size_t)n_ring * V * 2, reinterpret_cast<const __nv_bfloat16*>(p.v) + bw * V, (uint32_t)V * 2u, &bars[4]);
+            }
+        }
+    };
+    if (tid == 0 && stg_bytes > 0 && tile0 < tile1) stage_tile(tile0);
 
     for (int tile = tile0; tile < tile1 && !dead; ++tile) {
         const int h = tile / tiles_per_h;
@@ -136,6 +168,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                 sB2lo[o2] = lo;
             }
             cur_h = h;
+            __syncthreads();     // the query columns written next overlap the zero padding written above
         }
         if (p.q != nullptr) {       // query columns R .. R+NH-1 (bf16-exact: lo = 0)
             for (int idx = tid; idx < K * NH; idx += kTcThreads) {
@@ -147,15 +180,18 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
         }
 
         // ---- token weights w_s = beta_s prod_{j>s} a_j and the total decay ----
-        // gates are fetched in parallel, then one thread per head runs the short serial scan from shared memory
+        // the staged rows and gates of this tile must have landed
+        if (stg_bytes > 0) {
+            if (!cta_wait(&bars[4], ph4)) { record_fault(p.status, kFaultUpdateWait, 6); dead = true; }
+            ph4 ^= 1;
+        }
         for (int idx = tid; idx < NH * 64; idx += kTcThreads) {
             const int hd = idx >> 6, s = idx & 63;
             if (s < n_tot) {
                 const size_t bw = (size_t)(b0 + hd) * H + h;
-                const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
-                sW[hd * 208 + 80 + s] = s < n_ring ? reinterpret_cast<const float*>(rh + p.rl.beta_off)[s] : p.beta[bw];
-                sW[hd * 208 + 144 + s] = s < n_ring ? reinterpret_cast<const float*>(rh + p.rl.decay_off)[s]
-                                                    : reinterpret_cast<const float*>(p.decay)[bw];
+                const float* sg = reinterpret_cast<const float*>(sStg + (size_t)hd * sm.stg_head + 4096 + 16 * V * 2);
+                sW[hd * 208 + 80 + s] = s < n_ring ? sg[s] : p.beta[bw];
+                sW[hd * 208 + 144 + s] = s < n_ring ? sg[p.L + s] : reinterpret_cast<const float*>(p.decay)[bw];
             }
         }
         __syncthreads();
@@ -167,18 +203,14 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             }
             sW[tid * 208 + 64] = suf;
         }
-        // prefetch the first chunk of S_0 while the operands are being prepared
         const float* Sg = p.state + bh * (size_t)K * V + j;
-        float s0[kChunk];
-#pragma unroll
-        for (int ii = 0; ii < kChunk; ++ii) s0[ii] = Sg[(size_t)ii * V];
         __syncthreads();
 
         // ---- MMA 1 over blocks of kTokBlock tokens per head ----
         const int n_blocks = (n_tot + kTokBlock - 1) / kTokBlock;
         for (int blk = 0; blk < n_blocks; ++blk) {
             if (blk > 0) {      // the previous block's MMAs must have read the operand buffers
-                if (!mbar_wait_bounded(&bars[0], ph0)) { record_fault(p.status, kFaultUpdateWait, 1); dead = true; }
+                if (!cta_wait(&bars[0], ph0)) { record_fault(p.status, kFaultUpdateWait, 1); dead = true; }
                 ph0 ^= 1;
                 tc_fence_after();
             }
@@ -190,7 +222,9 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                 const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
                 const size_t bk = (size_t)(b0 + hd) * H + h;
                 uint4 val = make_uint4(0, 0, 0, 0);
-                if (s < n_ring) {
+                if (blk == 0) {
+                    if (s < n_tot) val = *reinterpret_cast<const uint4*>(sStg + (size_t)hd * sm.stg_head + (size_t)s * 256 + a * 16);
+                } else if (s < n_ring) {
                     val = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + ((size_t)s * K + a * 8) * 2);
                 } else if (s < n_tot) {
                     val = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.k) + bk * K + a * 8);
@@ -207,7 +241,12 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                 uint4 vraw = make_uint4(0, 0, 0, 0);
                 float w = 0.f;
                 if (hd_lane == hd) {
-                    if (s < n_ring) {
+                    if (blk == 0) {
+                        if (s < n_tot) {
+                            vraw = *reinterpret_cast<const uint4*>(sStg + (size_t)hd * sm.stg_head + 4096 + (size_t)s * V * 2 + a * 16);
+                            w = sW[hd * 208 + s];
+                        }
+                    } else if (s < n_ring) {
                         vraw = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + p.rl.v_off + ((size_t)s * V + a * 8) * 2);
                         w = sW[hd * 208 + s];
                     } else if (s < n_tot) {
@@ -231,6 +270,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
+                if (blk == 0 && stg_bytes > 0 && tile + 1 < tile1) stage_tile(tile + 1);   // staging is free again
 #pragma unroll
                 for (int ks = 0; ks < KD1 / 16; ++ks) {
                     const uint64_t bd = make_desc(smem_u32(sB1) + ks * 2 * LBO1, LBO1, SBO);
@@ -241,45 +281,59 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             }
         }
         if (n_blocks > 0) {
-            if (!mbar_wait_bounded(&bars[0], ph0)) { record_fault(p.status, kFaultUpdateWait, 2); dead = true; }
+            if (!cta_wait(&bars[0], ph0)) { record_fault(p.status, kFaultUpdateWait, 2); dead = true; }
             ph0 ^= 1;
             tc_fence_after();
         }
-        dead = __syncthreads_or(dead ? 1 : 0) != 0;
         if (dead) break;
 
-        // ---- epilogue: S_new = d S_0 + T, written back; S_new hi/lo -> A operand of MMA 2, 32 rows at a time ----
+        // ---- epilogue: S_new = d S_0 + T, written back; S_new hi/lo -> A operand of MMA 2, 16 rows at a time ----
+        // The state rows of three chunks ahead are in flight in registers while a chunk is processed.
         const float dtot = n_tot > 0 ? sW[my_head * 208 + 64] : 1.f;
         float* So = p.state + bh * (size_t)K * V + j;
-        for (int c = 0; c < K / kChunk; ++c) {
-            float s0n[kChunk];
-            if (c + 1 < K / kChunk) {
+        constexpr int CH = 16, NCH = K / CH, PF = 3;
+        float sbuf[PF + 1][CH];
 #pragma unroll
-                for (int ii = 0; ii < kChunk; ++ii) s0n[ii] = Sg[(size_t)((c + 1) * kChunk + ii) * V];
+        for (int c = 0; c < PF; ++c) {
+#pragma unroll
+            for (int ii = 0; ii < CH; ++ii) sbuf[c][ii] = Sg[(size_t)(c * CH + ii) * V];
+        }
+        float t01[2 * CH];      // T columns of chunks 0 and 1: both are read before the first MMA 2 overwrites them with UT
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            if (c + PF < NCH) {
+#pragma unroll
+                for (int ii = 0; ii < CH; ++ii) sbuf[(c + PF) % (PF + 1)][ii] = Sg[(size_t)((c + PF) * CH + ii) * V];
             }
-            float t[kChunk];
+            float t[CH];
             if (n_blocks > 0) {
-                tmem_ld32(tmem_t + lane_sel + (uint32_t)(c * kChunk), t);
+                if (c == 0) tmem_ld32(tmem_t + lane_sel, t01);
+                if (c < 2) {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) t[ii] = t01[c * CH + ii];
+                } else {
+                    tmem_ld16(tmem_t + lane_sel + (uint32_t)(c * CH), t);
+                }
             } else {
 #pragma unroll
-                for (int ii = 0; ii < kChunk; ++ii) t[ii] = 0.f;
+                for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
             }
             if (c >= 2) {       // chunk buffer c&1 was read by the MMAs of chunk c-2
-                if (!mbar_wait_bounded(&bars[1 + (c & 1)], ph1[c & 1])) { record_fault(p.status, kFaultUpdateWait, 3); dead = true; }
+                if (!cta_wait(&bars[1 + (c & 1)], ph1[c & 1])) { record_fault(p.status, kFaultUpdateWait, 3); dead = true; }
                 ph1[c & 1] ^= 1;
             }
-            unsigned char* a2hi = sA2 + (size_t)(c & 1) * (2u * 128u * kChunk * 2u);
-            unsigned char* a2lo = a2hi + 128u * kChunk * 2u;
+            unsigned char* a2hi = sA2 + (size_t)(c & 1) * (2u * 128u * CH * 2u);
+            unsigned char* a2lo = a2hi + 128u * CH * 2u;
 #pragma unroll
-            for (int v8 = 0; v8 < kChunk / 8; ++v8) {
+            for (int v8 = 0; v8 < CH / 8; ++v8) {
                 uint32_t ohi[4], olo[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int i0 = v8 * 8 + 2 * e;
-                    const float x0 = fmaf(dtot, s0[i0], t[i0]), x1 = fmaf(dtot, s0[i0 + 1], t[i0 + 1]);
+                    const float x0 = fmaf(dtot, sbuf[c % (PF + 1)][i0], t[i0]), x1 = fmaf(dtot, sbuf[c % (PF + 1)][i0 + 1], t[i0 + 1]);
                     if (p.write_state) {
-                        So[(size_t)(c * kChunk + i0) * V] = x0;
-                        So[(size_t)(c * kChunk + i0 + 1) * V] = x1;
+                        So[(size_t)(c * CH + i0) * V] = x0;
+                        So[(size_t)(c * CH + i0 + 1) * V] = x1;
                     }
                     split_bf16x2(x0, x1, ohi[e], olo[e]);
                 }
@@ -292,29 +346,21 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < kChunk / 16; ++ks) {
-                    const uint32_t kb = (uint32_t)(c * (kChunk / 8) + ks * 2) * LBO2B;      // W rows of this K-step
-                    const uint64_t ahi = make_desc(smem_u32(a2hi) + ks * 2 * LBO2A, LBO2A, SBO);
-                    const uint64_t alo = make_desc(smem_u32(a2lo) + ks * 2 * LBO2A, LBO2A, SBO);
-                    const uint64_t bhi = make_desc(smem_u32(sB2hi) + kb, LBO2B, SBO);
-                    const uint64_t blo = make_desc(smem_u32(sB2lo) + kb, LBO2B, SBO);
-                    tc_mma_bf16(tmem_u, ahi, bhi, idesc2, (c | ks) ? 1u : 0u);
-                    tc_mma_bf16(tmem_u, alo, bhi, idesc2, 1u);
-                    tc_mma_bf16(tmem_u, ahi, blo, idesc2, 1u);
-                }
-                tc_commit(c + 1 < K / kChunk ? &bars[1 + (c & 1)] : &bars[3]);
-            }
-            if (c + 1 < K / kChunk) {
-#pragma unroll
-                for (int ii = 0; ii < kChunk; ++ii) s0[ii] = s0n[ii];
+                const uint32_t kb = (uint32_t)(c * (CH / 8)) * LBO2B;      // W rows of this K-step
+                const uint64_t ahi = make_desc(smem_u32(a2hi), LBO2A, SBO);
+                const uint64_t alo = make_desc(smem_u32(a2lo), LBO2A, SBO);
+                const uint64_t bhi = make_desc(smem_u32(sB2hi) + kb, LBO2B, SBO);
+                const uint64_t blo = make_desc(smem_u32(sB2lo) + kb, LBO2B, SBO);
+                tc_mma_bf16(tmem_u, ahi, bhi, idesc2, c ? 1u : 0u);
+                tc_mma_bf16(tmem_u, alo, bhi, idesc2, 1u);
+                tc_mma_bf16(tmem_u, ahi, blo, idesc2, 1u);
+                tc_commit(c + 1 < NCH ? &bars[1 + (c & 1)] : &bars[3]);
             }
         }
-        // drain: chunk 2's commit (buffer 0) is still pending on its barrier; the final commit covers everything
-        if (!mbar_wait_bounded(&bars[1], ph1[0])) { record_fault(p.status, kFaultUpdateWait, 4); dead = true; }
-        ph1[0] ^= 1;
-        if (!mbar_wait_bounded(&bars[3], ph3)) { record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
+        // drain: the final commit covers every MMA issued so far; chunk 6's commit on bars[1] completed with it
+        if (!cta_wait(&bars[3], ph3)) { record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
         ph3 ^= 1;
+        ph1[0] ^= 1;
         tc_fence_after();
 
         // ---- UT rows -> sketch and exact output ----
@@ -359,7 +405,7 @@ int launch_update_tc(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
             return SKETCHSSM_CUDA_ERROR;
         ctx->sm_count = sms;
     }
-    const TcSmem sm = make_tc_smem(NH, NP);
+    const TcSmem sm = make_tc_smem(NH, NP, c.dv, c.buf_len);
     const int tmem_cols = NP <= 32 ? 128 : 256;
     int ctas = (int)((228u * 1024u) / (sm.total + 1024u));
     if (ctas > 512 / tmem_cols) ctas = 512 / tmem_cols;     // tensor memory: 512 columns per SM

@@ -149,6 +149,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_gdn_kernel(const Params 
                 sB2lo[o2] = lo;
             }
             cur_h = h;
+            __syncthreads();     // the query columns written next overlap the zero padding written above
         }
         if (p.q != nullptr) {
             const int i = tid, g = R;
