@@ -288,10 +288,10 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
         if (dead) break;
 
         // ---- epilogue: S_new = d S_0 + T, written back; S_new hi/lo -> A operand of MMA 2, 16 rows at a time ----
-        // The state rows of three chunks ahead are in flight in registers while a chunk is processed.
+        // The state rows of the next two chunks are in flight in registers while a chunk is processed.
         const float dtot = n_tot > 0 ? sW[my_head * 208 + 64] : 1.f;
         float* So = p.state + bh * (size_t)K * V + j;
-        constexpr int CH = 16, NCH = K / CH, PF = 3;
+        constexpr int CH = 16, NCH = K / CH, PF = 2;
         float sbuf[PF + 1][CH];
 #pragma unroll
         for (int c = 0; c < PF; ++c) {
