@@ -220,10 +220,13 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     p.has_token = has_token ? 1 : 0;
     p.write_sketch = sketch ? 1 : 0;
     p.write_state = n_tot > 0 ? 1 : 0;
-    if (p.update_impl == 0) {
+    if (p.update_impl == 0 || p.update_impl == 3) {
+        if (p.update_impl == 0) {       // two warp groups per CTA; falls through outside its domain (rank + heads per tile > 32)
+            rc = launch_update_tc_ws(ctx, p, static_cast<cudaStream_t>(stream));
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        }
         rc = launch_update_tc(ctx, p, static_cast<cudaStream_t>(stream));
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-
     }
     if (p.update_impl == 2) {       // opt-in: gated delta rule on tensor cores (measured slower than the CUDA-core kernel so far)
         rc = launch_update_tc_delta(ctx, p, static_cast<cudaStream_t>(stream));

@@ -1,0 +1,733 @@
+// Warp-specialised state-update (flush) kernel for the Mamba-2 transition on tcgen05 + TMEM, sm_100a.
+//
+// Same arithmetic as the single-group tensor-core kernel (closed form of Eq. 3, sketch rows of Eq. 7):
+//     S_new = d S_0 + sum_s w_s k_s v_s^T,   U[g, :] = S_new^T omega_g,   o = S_new^T q,
+// with MMA 1 producing T = sum_s (w_s v_s) k_s^T in tensor memory and MMA 2 contracting the freshly formed
+// S_new rows with [Omega | q].  The difference is the schedule.  A CTA holds two warp groups of 128 threads and one
+// issue warp:
+//
+//   front group (warps 4-7), one tile AHEAD: turns the staged raw ring rows of tile i+1 into the MMA-1 operands
+//       (token weights, w_s v_s split into bf16 hi + lo, keys, query columns), issues MMA 1 into the other half of a
+//       double-buffered accumulator, and stores the sketch rows / exact output of tile i-1 from tensor memory;
+//   stream group (warps 0-3): streams the state of tile i in 16-row chunks (S_new = d S_0 + T, written back once),
+//       splits S_new into bf16 hi + lo in shared memory, warp by warp without a group barrier;
+//   issue warp (warp 8, one thread): issues MMA 2 for a chunk once its four warps have delivered it, and keeps a ring
+//       of shared-memory stages full of S_0 chunks by bulk copies (TMA) that run several chunks ahead and across tile
+//       boundaries, so the bytes in flight per SM do not depend on registers and the global loads never drain.
+//
+// Everything that used to sit serially between two tiles' state streams (operand building, MMA-1 latency, sketch
+// stores) now overlaps them.  The groups meet only through mbarriers; every wait is bounded.
+//
+// Domain: Mamba-2, bf16 I/O, K = 128, V in {64, 128}, rank <= 16 (the sketch accumulator [Omega | q | q'] then
+// re-uses the first 32 consumed columns of T, which keeps a CTA at 256 TMEM columns and two CTAs per SM).
+// W = [Omega | q-group A | q-group B]: consecutive tiles alternate between the two query groups, so the front group
+// can write the next tile's query columns while MMA 2 of the current tile still reads the buffer (it then also reads
+// half-written columns of the other group, whose outputs nobody uses).
+#include "internal.cuh"
+#include "tc_common.cuh"
+
+namespace sketchssm {
+
+namespace {
+
+using namespace tc;
+
+// Optional phase stamps of the first CTA into the work buffer (stream group: slots 0.., front group: slots 512..);
+// compiled out by default.
+#ifdef SKETCHSSM_PHASE_TIMING
+#define WS_STAMP(base, i)                                                                                      \
+    do {                                                                                                       \
+        if (gt == 0 && blockIdx.x == 0 && tile - tile0 >= 12 && tile - tile0 < 20)                             \
+            reinterpret_cast<long long*>(p.work)[(base) + (tile - tile0 - 12) * 32 + (i)] = clock64();         \
+    } while (0)
+#else
+#define WS_STAMP(base, i) do { } while (0)
+#endif
+
+constexpr int kWsThreads = 288;       // stream group (4 warps), front group (4 warps), issue warp
+constexpr int kGroup = 128;
+
+struct WsSmem {
+    uint32_t op, a2, b2, w, w_stride, stg, stg_head, stg_gate, stg_q, bars, misc, sst, sst_bytes, total;
+};
+
+constexpr int kMaxStages = 8;
+
+// operand set: a1_hi | a1_lo | b1, each 128 x KD1 bf16
+__host__ __device__ inline WsSmem make_ws_smem(int NH, int NP, int V, int L, int stages) {
+    WsSmem s;
+    const uint32_t kd1 = (uint32_t)(kTokBlock * NH);
+    uint32_t off = 0;
+    s.op = off; off += 3u * 128u * kd1 * 2u;
+    s.a2 = off; off += 2u * 2u * 128u * 16u * 2u;              // two 16-row chunk buffers, hi + lo
+    s.b2 = off; off += 2u * (uint32_t)NP * kK * 2u;             // hi | lo
+    s.w = off; s.w_stride = 2u * 208u * 4u; off += 2u * s.w_stride;     // per head: w_s (64), total decay; double-buffered
+    // staging of the next tile's raw rows: per head keys [16][256 B], values [16][V*2 B], gates [2L] floats, query row
+    s.stg_gate = 4096u + 16u * (uint32_t)V * 2u;
+    s.stg_q = s.stg_gate + (((uint32_t)(2 * L * 4) + 127u) & ~127u);
+    s.stg_head = s.stg_q + 256u;
+    s.stg = off; off += (uint32_t)NH * s.stg_head;
+    s.bars = off; off += 256u;
+    s.misc = off; off += 64u;
+    off = (off + 127u) & ~127u;
+    s.sst_bytes = 16u * 128u * 4u;                              // one stage: 16 state rows of every lane, fp32
+    s.sst = off; off += (uint32_t)stages * s.sst_bytes;
+    s.total = off;
+    return s;
+}
+
+// barrier slots
+enum { kBarT = 0, kBarPro = 2, kBarA2 = 4, kBarU = 6, kBarStg = 8, kBarBlk = 9, kBarA2Rdy = 10, kBarFull = 12,
+       kBarEmpty = 12 + kMaxStages, kNumBars = 12 + 2 * kMaxStages };
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// named barrier over one 128-thread group
+__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+
+// named barrier with an OR reduction of a per-thread flag
+__device__ __forceinline__ bool group_or(int id, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %2, 0;\n\t"
+        "bar.red.or.pred p, %1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(flag ? 1u : 0u)
+        : "memory");
+    return r != 0;
+}
+
+// group-wide bounded wait for a barrier that is usually NOT yet complete: one warp polls, the others sleep in the
+// named barrier.  Returns false to every thread of the group if the wait ran out.
+__device__ __forceinline__ bool group_wait(int id, int gt, uint64_t* bar, uint32_t phase) {
+    bool bad = false;
+    if (gt < 32) bad = !mbar_wait_bounded(bar, phase);
+    return !group_or(id, bad);
+}
+
+}  // namespace
+
+template <int V>
+__global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(const Params p) {
+    constexpr int K = kK;
+    constexpr int NH = 128 / V;
+    constexpr int KD1 = kTokBlock * NH;
+    constexpr uint32_t OPB = 128u * KD1 * 2u;              // bytes of one MMA-1 operand
+    extern __shared__ __align__(1024) unsigned char smem[];
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int wg = tid >> 7, gt = tid & 127;
+#ifdef SKETCHSSM_PHASE_TIMING
+    if (tid == 0) {
+        unsigned long long t_ns; unsigned smid;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
+        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        long long* rec = reinterpret_cast<long long*>(p.work) + 2048 + 4 * blockIdx.x;
+        rec[0] = (long long)t_ns; rec[2] = smid; rec[3] = clock64();
+    }
+#endif
+    const int R = p.R, H = p.H, B = p.B;
+    const int QA = (R + 7) & ~7;                          // first column of query group A; group B follows 8 columns later
+    const int NP = (QA + 16 + 15) & ~15;                  // <= 32 (checked by the launcher)
+    const int NS = p.stages;                              // state stages in shared memory (set by the launcher)
+    const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);
+    const WsSmem sm = make_ws_smem(NH, NP, V, p.L, NS);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.misc);
+    unsigned char* sStg = smem + sm.stg;
+
+    constexpr uint32_t tmem_cols = 256u;
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int i = 0; i < kNumBars; ++i) {
+            // chunk-ready and stage-empty barriers take one arrival per stream warp, the others a single arrival
+            const bool per_warp = (i >= kBarA2Rdy && i < kBarA2Rdy + 2) || i >= kBarEmpty;
+            mbar_init(&bars[i], per_warp ? 4 : 1);
+        }
+        mbar_fence_init();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    grid_dep_wait();                 // nothing above reads memory another kernel may write
+    grid_dep_launch_dependents();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+
+    // instruction descriptors: bf16 x bf16 -> fp32
+    const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+    const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)NP >> 3) << 17) | ((128u >> 4) << 24);
+    // canonical no-swizzle layouts (byte offsets)
+    //   MN-major (MMA 1): elem(mn, k) at (k%8)*16 + (mn%8)*2 + (mn/8)*128 + (k/8)*2048
+    //   K-major  (MMA 2): elem(mn, k) at (mn%8)*16 + (mn/8)*128 + (k/8)*LBO + (k%8)*2,  LBO = 16*MN
+    constexpr uint32_t LBO1 = 2048, SBO = 128, LBO2A = 2048;
+    const uint32_t LBO2B = (uint32_t)NP * 16u;
+
+    const int tiles_per_h = B / NH;
+    const long long n_tiles = (long long)H * tiles_per_h;
+    const int tile0 = (int)(n_tiles * blockIdx.x / gridDim.x);
+    const int tile1 = (int)(n_tiles * (blockIdx.x + 1) / gridDim.x);
+    const int n_blocks = (n_tot + kTokBlock - 1) / kTokBlock;
+
+    const int my_head = gt / V;           // which head of the tile this thread's TMEM lane belongs to
+    const int j = gt % V;
+
+    if (wg == 0) {
+        // =========================== stream group: S_0 -> S_new, MMA 2 ===========================
+        constexpr int CH = 16, NCH = K / CH;
+        const int lane = tid & 31;
+        uint32_t phT = 0, phP = 0, phA = 0;      // barrier phases, one bit per buffer
+        int gc = 0, stage = 0;                   // chunks consumed so far, their stage and its phase
+        uint32_t phF = 0;
+        bool bad = false;
+        for (int tile = tile0; tile < tile1 && !bad; ++tile) {
+            const int b = (tile - tile0) & 1;
+            const int h = tile / tiles_per_h;
+            const int b0 = (tile - h * tiles_per_h) * NH;
+            const size_t bh = (size_t)(b0 + my_head) * H + h;
+            float* So = p.state + bh * (size_t)K * V + j;
+            const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
+            WS_STAMP(0, 0);
+            // operands-ready (plain arrive: orders the front group's shared-memory writes) and MMA 1 complete
+            bad |= !mbar_wait_bounded(&bars[kBarPro + b], (phP >> b) & 1u);
+            bad |= !mbar_wait_bounded(&bars[kBarT + b], (phT >> b) & 1u);
+            phP ^= 1u << b;
+            phT ^= 1u << b;
+            tc_fence_after();
+            WS_STAMP(0, 1);
+            const float dtot = n_tot > 0 ? reinterpret_cast<const float*>(smem + sm.w + (uint32_t)b * sm.w_stride)[my_head * 208 + 64] : 1.f;
+            float t01[2 * CH];      // T columns of chunks 0 and 1: read before the first MMA 2 overwrites them with UT
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                if (c == 4) WS_STAMP(0, 12);
+                // this chunk's S_0 rows have landed in their stage; once in registers the stage is released
+                bad |= !mbar_wait_bounded(&bars[kBarFull + stage], phF);
+                if (c == 4) WS_STAMP(0, 13);
+                const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + my_head * CH * V + j;
+                float s0[CH];
+#pragma unroll
+                for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
+                float t[CH];
+                if (n_blocks > 0 && !bad) {
+                    if (c == 0) tmem_ld32(tmem_t + lane_sel, t01);
+                    if (c < 2) {
+#pragma unroll
+                        for (int ii = 0; ii < CH; ++ii) t[ii] = t01[c * CH + ii];
+                    } else {
+                        tmem_ld16(tmem_t + lane_sel + (uint32_t)(c * CH), t);
+                    }
+                } else {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
+                }
+                if (c == 4) WS_STAMP(0, 14);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[kBarEmpty + stage]);
+                if (gc >= 2) {       // chunk buffer c&1 was read by the MMAs issued two chunks ago
+                    bad |= !mbar_wait_bounded(&bars[kBarA2 + (c & 1)], (phA >> (c & 1)) & 1u);
+                    phA ^= 1u << (c & 1);
+                }
+                if (c == 4) WS_STAMP(0, 15);
+                unsigned char* a2hi = smem + sm.a2 + (size_t)(c & 1) * (2u * 128u * CH * 2u);
+                unsigned char* a2lo = a2hi + 128u * CH * 2u;
+#pragma unroll
+                for (int v8 = 0; v8 < CH / 8; ++v8) {
+                    uint32_t ohi[4], olo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i0 = v8 * 8 + 2 * e;
+                        const float x0 = fmaf(dtot, s0[i0], t[i0]), x1 = fmaf(dtot, s0[i0 + 1], t[i0 + 1]);
+                        if (p.write_state && !bad) {
+                            So[(size_t)(c * CH + i0) * V] = x0;
+                            So[(size_t)(c * CH + i0 + 1) * V] = x1;
+                        }
+                        split_bf16x2(x0, x1, ohi[e], olo[e]);
+                    }
+                    const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO2A;
+                    *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                    *reinterpret_cast<uint4*>(a2lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+                }
+                if (c == 4) WS_STAMP(0, 16);
+                // this warp's 32 rows of the chunk are written (and its T columns read): tell the issue warp
+                proxy_fence();
+                tc_fence_before();
+                bad = __any_sync(0xffffffffu, bad);
+                if (lane == 0 && !bad) mbar_arrive(&bars[kBarA2Rdy + (c & 1)]);
+                ++gc;
+                if (++stage == NS) { stage = 0; phF ^= 1u; }
+                WS_STAMP(0, 2 + c);
+            }
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 3);
+    } else if (wg == 2) {
+        // =========================== issue warp: S_0 stages (TMA) and MMA 2, one thread ===========================
+        if (gt == 0) {
+            constexpr int CH = 16, NCH = K / CH;
+            const int total_chunks = (tile1 - tile0) * NCH;
+            // producer cursor: the chunk to load next
+            int p_tile = tile0, p_c = 0, p_stage = 0;
+            const float* p_src[NH];
+            auto producer_tile = [&]() {
+                const int h = p_tile / tiles_per_h;
+                const int b0 = (p_tile - h * tiles_per_h) * NH;
+#pragma unroll
+                for (int hd = 0; hd < NH; ++hd) p_src[hd] = p.state + ((size_t)(b0 + hd) * H + h) * (size_t)K * V;
+            };
+            auto issue_chunk = [&]() {
+                uint64_t* bar = &bars[kBarFull + p_stage];
+                mbar_expect_tx(bar, sm.sst_bytes);
+#pragma unroll
+                for (int hd = 0; hd < NH; ++hd)
+                    bulk_g2s(smem + sm.sst + (size_t)p_stage * sm.sst_bytes + (size_t)hd * CH * V * 4,
+                             p_src[hd] + (size_t)p_c * CH * V, (uint32_t)(CH * V * 4), bar);
+                if (++p_stage == NS) p_stage = 0;
+                if (++p_c == NCH) {
+                    p_c = 0;
+                    ++p_tile;
+                    if (p_tile < tile1) producer_tile();
+                }
+            };
+            int issued = 0;
+            if (tile0 < tile1) producer_tile();
+            for (; issued < NS && issued < total_chunks; ++issued) issue_chunk();
+            uint32_t phR = 0, phE = 0;           // chunk-ready phases (bit per buffer), stage-empty phase
+            int stage = 0;
+            bool bad = false;
+            const uint32_t sB2 = smem_u32(smem + sm.b2);
+            for (int tile = tile0; tile < tile1 && !bad; ++tile) {
+                const int b = (tile - tile0) & 1;
+                const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    if (!mbar_wait_bounded(&bars[kBarA2Rdy + (c & 1)], (phR >> (c & 1)) & 1u)) { bad = true; break; }
+                    phR ^= 1u << (c & 1);
+                    tc_fence_after();
+                    const uint32_t a2 = smem_u32(smem + sm.a2) + (uint32_t)(c & 1) * (2u * 128u * CH * 2u);
+                    const uint32_t kb = (uint32_t)(c * (CH / 8)) * LBO2B;      // W rows of this K-step
+                    const uint64_t ahi = make_desc(a2, LBO2A, SBO);
+                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO2A, SBO);
+                    const uint64_t bhi = make_desc(sB2 + kb, LBO2B, SBO);
+                    const uint64_t blo = make_desc(sB2 + (uint32_t)NP * kK * 2u + kb, LBO2B, SBO);
+                    tc_mma_bf16(tmem_t, ahi, bhi, idesc2, c ? 1u : 0u);
+                    tc_mma_bf16(tmem_t, alo, bhi, idesc2, 1u);
+                    tc_mma_bf16(tmem_t, ahi, blo, idesc2, 1u);
+                    tc_commit(&bars[kBarA2 + (c & 1)]);
+                    if (c == NCH - 1) tc_commit(&bars[kBarU + b]);     // everything of this tile: UT is complete
+                    // the stage this chunk came from was released by all four stream warps before they wrote the chunk
+                    if (issued < total_chunks) {
+                        if (!mbar_wait_bounded(&bars[kBarEmpty + stage], phE)) { bad = true; break; }
+                        issue_chunk();
+                        ++issued;
+                    }
+                    if (++stage == NS) { stage = 0; phE ^= 1u; }
+                }
+            }
+            if (bad) record_fault(p.status, kFaultUpdateWait, 4);
+        }
+    } else {
+        // =========================== front group: operands, MMA 1, sketch stores ===========================
+        const int fwarp = gt >> 5;
+        int cur_h = -1;                       // head index whose Omega sits in W
+        int ops_built = 0;                    // MMA-1 operand sets written so far (single buffer)
+        int ut_stored = tile0;                // tiles below this one have their sketch rows stored
+        uint32_t phS = 0, phU = 0, phB = 0;
+        bool dead = false;
+
+        // Raw ring rows of a tile's first token block travel to shared memory by bulk copies issued one tile ahead.
+        // Rows of later blocks (n > 16) are read directly.
+        const int rows0 = n_ring < kTokBlock ? n_ring : kTokBlock;
+        const bool tok0 = p.has_token && n_ring < kTokBlock;
+        const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
+        const uint32_t stg_bytes = (uint32_t)NH * ((uint32_t)rows0 * 256u + (uint32_t)rows0 * V * 2u + stg_gate_bytes +
+                                                  (tok0 ? 256u + (uint32_t)V * 2u : 0u) + (p.q != nullptr ? 256u : 0u));
+        auto stage_tile = [&](int tile) {       // one thread
+            const int h = tile / tiles_per_h;
+            const int b0 = (tile - h * tiles_per_h) * NH;
+            mbar_expect_tx(&bars[kBarStg], stg_bytes);
+            for (int hd = 0; hd < NH; ++hd) {
+                const size_t bw = (size_t)(b0 + hd) * H + h;
+                const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
+                unsigned char* dst = sStg + (size_t)hd * sm.stg_head;
+                if (rows0 > 0) {
+                    bulk_g2s(dst, rh, (uint32_t)rows0 * 256u, &bars[kBarStg]);
+                    bulk_g2s(dst + 4096, rh + p.rl.v_off, (uint32_t)rows0 * V * 2u, &bars[kBarStg]);
+                }
+                if (stg_gate_bytes) bulk_g2s(dst + sm.stg_gate, rh + p.rl.beta_off, stg_gate_bytes, &bars[kBarStg]);
+                if (tok0) {
+                    bulk_g2s(dst + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.k) + bw * K, 256u, &bars[kBarStg]);
+                    bulk_g2s(dst + 4096 + (size_t)n_ring * V * 2, reinterpret_cast<const __nv_bfloat16*>(p.v) + bw * V, (uint32_t)V * 2u, &bars[kBarStg]);
+                }
+                if (p.q != nullptr) bulk_g2s(dst + sm.stg_q, reinterpret_cast<const __nv_bfloat16*>(p.q) + bw * K, 256u, &bars[kBarStg]);
+            }
+        };
+        // sketch rows and exact output of a finished tile: UT sits in the first NP columns of that tile's accumulator
+        auto store_ut = [&](int tile) -> bool {
+            const int b = (tile - tile0) & 1;
+            const int h = tile / tiles_per_h;
+            const int b0 = (tile - h * tiles_per_h) * NH;
+            const size_t bh = (size_t)(b0 + my_head) * H + h;
+            if (!group_wait(2, gt, &bars[kBarU + b], (phU >> b) & 1u)) return false;
+            phU ^= 1u << b;
+            tc_fence_after();
+            for (int g0 = 0; g0 < NP; g0 += 16) {
+                float u[16];
+                tmem_ld16(tmem_base + (uint32_t)b * 128u + lane_sel + (uint32_t)g0, u);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const int g = g0 + e;
+                    if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u[e];
+                    if (g == QA + 8 * b + my_head && p.out != nullptr) {
+                        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u[e]);
+                        else reinterpret_cast<float*>(p.out)[bh * V + j] = u[e];
+                    }
+                }
+            }
+            tc_fence_before();     // ordered before the next MMA 1 into this accumulator by the group barriers that follow
+            return true;
+        };
+
+        if (gt == 0 && stg_bytes > 0 && tile0 < tile1) stage_tile(tile0);
+        // W (padding columns, lo halves of the query columns) and the MMA-1 operands (off-diagonal head blocks) hold
+        // zeros that no tile ever overwrites: written once
+        for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGroup * 16u)
+            *reinterpret_cast<uint4*>(smem + sm.b2 + o) = make_uint4(0, 0, 0, 0);
+        for (uint32_t o = (uint32_t)gt * 16u; o < 3u * OPB; o += kGroup * 16u)
+            *reinterpret_cast<uint4*>(smem + sm.op + o) = make_uint4(0, 0, 0, 0);
+        group_sync(2);
+
+        for (int tile = tile0; tile < tile1 && !dead; ++tile) {
+            const int b = (tile - tile0) & 1;
+            const int h = tile / tiles_per_h;
+            const int b0 = (tile - h * tiles_per_h) * NH;
+            __nv_bfloat16* sB2hi = reinterpret_cast<__nv_bfloat16*>(smem + sm.b2);
+            __nv_bfloat16* sB2lo = sB2hi + (size_t)NP * kK;
+            float* sW = reinterpret_cast<float*>(smem + sm.w + (uint32_t)b * sm.w_stride);
+            unsigned char* sA1hi = smem + sm.op;
+            unsigned char* sA1lo = sA1hi + OPB;
+            unsigned char* sB1 = sA1lo + OPB;
+
+            WS_STAMP(512, 0);
+            // gates of the current token (one warp per head needs them for the weight scan): requested early
+            float tok_beta = 0.f, tok_a = 1.f;
+            if (fwarp < NH && p.has_token) {
+                const size_t bw = (size_t)(b0 + fwarp) * H + h;
+                tok_beta = p.beta[bw];
+                tok_a = reinterpret_cast<const float*>(p.decay)[bw];
+            }
+            // ---- W = [Omega | q | q'] hi/lo, K-major; the Omega part once per head index.  MMA 2 of the previous tile
+            // still reads W, so that tile is finished (and its sketch rows stored) first. ----
+            if (h != cur_h) {
+                if (tile > tile0) {
+                    if (!store_ut(tile - 1)) {
+                        if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+                        dead = true;
+                        break;
+                    }
+                    ut_stored = tile;
+                    group_sync(2);
+                }
+                const float* og = p.omega + (size_t)h * K * R;
+                if (!p.write_sketch) {
+                    // no sketch: the Omega columns stay zero (written once before the tile loop)
+                } else if ((R & 3) == 0) {
+                    // four ranks of one state row per step; all loads of a thread are in flight together
+                    const int per_row = R >> 2, items = K * per_row;
+                    for (int base = 0; base < items; base += 4 * kGroup) {
+                        float4 x[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int idx = base + u * kGroup + gt;
+                            x[u] = idx < items ? *reinterpret_cast<const float4*>(og + (size_t)idx * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int idx = base + u * kGroup + gt;
+                            if (idx < items) {
+                                const int i = idx / per_row, g4 = (idx - i * per_row) * 4;
+                                const float xv[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int g = g4 + e;
+                                    __nv_bfloat16 hi, lo;
+                                    split_bf16(xv[e], hi, lo);
+                                    const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO2B + (i & 7) * 2) >> 1;
+                                    sB2hi[o2] = hi;
+                                    sB2lo[o2] = lo;
+                                }
+                            }
+                        }
+                    }
+                } else {
+                    for (int idx = gt; idx < K * R; idx += kGroup) {
+                        const int i = idx / R, g = idx % R;
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(og[idx], hi, lo);
+                        const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO2B + (i & 7) * 2) >> 1;
+                        sB2hi[o2] = hi;
+                        sB2lo[o2] = lo;
+                    }
+                }
+                cur_h = h;
+            }
+            // the staged rows, gates and query rows of this tile must have landed
+            if (stg_bytes > 0) {
+                if (!group_wait(2, gt, &bars[kBarStg], phS)) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 6);
+                    dead = true;
+                    break;
+                }
+                phS ^= 1;
+            }
+            WS_STAMP(512, 1);
+            if (p.q != nullptr) {       // query columns of this tile's group (bf16-exact: lo = 0)
+                for (int idx = gt; idx < K * NH; idx += kGroup) {
+                    const int i = idx % K, hd = idx / K, g = QA + 8 * b + hd;
+                    const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO2B + (i & 7) * 2) >> 1;
+                    sB2hi[o2] = reinterpret_cast<const __nv_bfloat16*>(sStg + (size_t)hd * sm.stg_head + sm.stg_q)[i];
+                }
+            }
+            // ---- token weights w_s = beta_s prod_{j>s} a_j and the total decay: one warp per head, suffix scan ----
+            if (fwarp < NH) {
+                const int hd = fwarp, lane = gt & 31;
+                const float* sg = reinterpret_cast<const float*>(sStg + (size_t)hd * sm.stg_head + sm.stg_gate);
+                float suf = 1.f;          // product of the decays of all later tokens
+                for (int base = ((n_tot + 31) & ~31) - 32; base >= 0; base -= 32) {
+                    const int s = base + lane;
+                    float beta = 0.f, a = 1.f;
+                    if (s < n_ring) { beta = sg[s]; a = sg[p.L + s]; }
+                    else if (s < n_tot) { beta = tok_beta; a = tok_a; }
+                    // inclusive suffix product of a over lanes >= lane
+                    float incl = a;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const float other = __shfl_down_sync(0xffffffffu, incl, o);
+                        if (lane + o < 32) incl *= other;
+                    }
+                    float excl = __shfl_down_sync(0xffffffffu, incl, 1);
+                    if (lane == 31) excl = 1.f;
+                    if (s < n_tot) sW[hd * 208 + s] = beta * excl * suf;
+                    suf *= __shfl_sync(0xffffffffu, incl, 0);
+                }
+                if (lane == 0) sW[hd * 208 + 64] = suf;
+            }
+            proxy_fence();         // W is read by MMA 2 (async proxy)
+            group_sync(2);
+            WS_STAMP(512, 2);
+
+            // ---- MMA 1 over blocks of kTokBlock tokens per head ----
+            for (int blk = 0; blk < n_blocks; ++blk) {
+                if (ops_built > 0) {      // the previous MMA-1 block (of this or the previous tile) must have read the operand buffers
+                    if (!group_wait(2, gt, &bars[kBarBlk], phB)) {
+                        if (gt == 0) record_fault(p.status, kFaultUpdateWait, 1);
+                        dead = true;
+                        break;
+                    }
+                    phB ^= 1;
+                    tc_fence_after();
+                }
+                // Operand rows are written 16 bytes per thread; consecutive threads walk the 8 token rows of a core matrix
+                // first and then the next 8-element vector, so that a warp writes 512 contiguous bytes (no bank conflicts).
+                if (blk == 0) {
+                    // first block: rows come from the staging buffer; only the diagonal head blocks of A are written
+                    constexpr int NB = KD1 * (K / 8) / kGroup;          // B-operand vectors per thread
+                    uint4 kv[NB];
+#pragma unroll
+                    for (int r = 0; r < NB; ++r) {
+                        const int idx = gt + r * kGroup;
+                        const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
+                        const int hd = sp / kTokBlock, s = sp % kTokBlock;
+                        kv[r] = s < n_tot ? *reinterpret_cast<const uint4*>(sStg + (size_t)hd * sm.stg_head + (size_t)s * 256 + a * 16)
+                                          : make_uint4(0, 0, 0, 0);
+                    }
+                    constexpr int NA = NH * kTokBlock * (V / 8) / kGroup;      // diagonal A-operand vectors per thread
+                    uint4 vv[NA];
+                    float wv[NA];
+#pragma unroll
+                    for (int r = 0; r < NA; ++r) {
+                        const int it = gt + r * kGroup;
+                        const int t8 = it & 7, a = (it >> 3) % (V / 8), rest = it / V;
+                        const int hd = rest >> 1, s = (rest & 1) * 8 + t8;
+                        const bool live = s < n_tot;
+                        vv[r] = live ? *reinterpret_cast<const uint4*>(sStg + (size_t)hd * sm.stg_head + 4096 + (size_t)s * V * 2 + a * 16)
+                                     : make_uint4(0, 0, 0, 0);
+                        wv[r] = live ? sW[hd * 208 + s] : 0.f;
+                    }
+#pragma unroll
+                    for (int r = 0; r < NB; ++r) {
+                        const int idx = gt + r * kGroup;
+                        const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
+                        *reinterpret_cast<uint4*>(sB1 + (sp & 7) * 16 + a * SBO + (sp >> 3) * LBO1) = kv[r];
+                    }
+#pragma unroll
+                    for (int r = 0; r < NA; ++r) {
+                        const int it = gt + r * kGroup;
+                        const int t8 = it & 7, a = (it >> 3) % (V / 8), rest = it / V;
+                        const int hd = rest >> 1, sp = hd * kTokBlock + (rest & 1) * 8 + t8;
+                        const int a128 = hd * (V / 8) + a;
+                        const uint32_t vin[4] = {vv[r].x, vv[r].y, vv[r].z, vv[r].w};
+                        uint32_t ohi[4], olo[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float f0 = wv[r] * __uint_as_float(vin[e] << 16), f1 = wv[r] * __uint_as_float(vin[e] & 0xffff0000u);
+                            split_bf16x2(f0, f1, ohi[e], olo[e]);
+                        }
+                        const uint32_t off = (sp & 7) * 16 + a128 * SBO + (sp >> 3) * LBO1;
+                        *reinterpret_cast<uint4*>(sA1hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                        *reinterpret_cast<uint4*>(sA1lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+                    }
+                } else {
+                // later blocks (n > 16): rows are read from the ring in global memory
+                // B operand: keys, MN-major (mn = state row i, k = token slot)
+                for (int idx = gt; idx < KD1 * (K / 8); idx += kGroup) {
+                    const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
+                    const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
+                    const size_t bk = (size_t)(b0 + hd) * H + h;
+                    uint4 val = make_uint4(0, 0, 0, 0);
+                    if (s < n_ring) {
+                        val = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + ((size_t)s * K + a * 8) * 2);
+                    } else if (s < n_tot) {
+                        val = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.k) + bk * K + a * 8);
+                    }
+                    *reinterpret_cast<uint4*>(sB1 + (sp & 7) * 16 + a * SBO + (sp >> 3) * LBO1) = val;
+                }
+                // A operand: w_s v_s hi/lo, MN-major (mn = lane t = head*V + j, k = token slot), block diagonal over heads
+                for (int idx = gt; idx < KD1 * 16; idx += kGroup) {
+                    const int a128 = (idx >> 3) & 15, sp = (idx & 7) + 8 * (idx >> 7);
+                    const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
+                    const int hd_lane = a128 / (V / 8), a = a128 % (V / 8);
+                    if (hd_lane != hd) continue;          // off-diagonal blocks stay zero
+                    const size_t bk = (size_t)(b0 + hd) * H + h;
+                    uint4 vraw = make_uint4(0, 0, 0, 0);
+                    float w = 0.f;
+                    if (s < n_ring) {
+                        vraw = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + p.rl.v_off + ((size_t)s * V + a * 8) * 2);
+                        w = sW[hd * 208 + s];
+                    } else if (s < n_tot) {
+                        vraw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.v) + bk * V + a * 8);
+                        w = sW[hd * 208 + s];
+                    }
+                    const uint32_t vin[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
+                    uint32_t ohi[4], olo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float f0 = w * __uint_as_float(vin[e] << 16), f1 = w * __uint_as_float(vin[e] & 0xffff0000u);
+                        split_bf16x2(f0, f1, ohi[e], olo[e]);
+                    }
+                    const uint32_t off = (sp & 7) * 16 + a128 * SBO + (sp >> 3) * LBO1;
+                    *reinterpret_cast<uint4*>(sA1hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                    *reinterpret_cast<uint4*>(sA1lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+                }
+                }
+                proxy_fence();
+                tc_fence_before();
+                group_sync(2);
+                ++ops_built;
+                if (gt == 0) {
+                    tc_fence_after();
+                    if (blk == 0 && stg_bytes > 0 && tile + 1 < tile1) stage_tile(tile + 1);   // staging is free again
+                    const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
+#pragma unroll
+                    for (int ks = 0; ks < KD1 / 16; ++ks) {
+                        const uint64_t bd = make_desc(smem_u32(sB1) + ks * 2 * LBO1, LBO1, SBO);
+                        tc_mma_bf16(tmem_t, make_desc(smem_u32(sA1hi) + ks * 2 * LBO1, LBO1, SBO), bd, idesc1, (blk | ks) ? 1u : 0u);
+                        tc_mma_bf16(tmem_t, make_desc(smem_u32(sA1lo) + ks * 2 * LBO1, LBO1, SBO), bd, idesc1, 1u);
+                    }
+                    tc_commit(&bars[kBarBlk]);
+                    if (blk + 1 == n_blocks) tc_commit(&bars[kBarT + b]);
+                }
+            }
+            if (dead) break;
+            if (n_blocks == 0) {
+                // no token to replay: nothing reads the staging buffer after the query columns; T counts as zero
+                group_sync(2);
+                if (gt == 0) {
+                    if (stg_bytes > 0 && tile + 1 < tile1) stage_tile(tile + 1);
+                    mbar_arrive(&bars[kBarT + b]);
+                }
+            }
+            if (gt == 0) mbar_arrive(&bars[kBarPro + b]);      // after the group barrier: W, weights and decay are written
+            WS_STAMP(512, 3);
+
+            // ---- sketch rows and exact output of the previous tile, once the stream group has finished it ----
+            if (ut_stored < tile) {
+                if (!store_ut(tile - 1)) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+                    dead = true;
+                }
+                ut_stored = tile;
+            }
+            WS_STAMP(512, 4);
+        }
+        if (!dead && tile0 < tile1) {
+            if (!store_ut(tile1 - 1) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+#ifdef SKETCHSSM_PHASE_TIMING
+    if (tid == 0) {
+        unsigned long long t_ns;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
+        long long* rec = reinterpret_cast<long long*>(p.work) + 2048 + 4 * blockIdx.x;
+        rec[1] = (long long)t_ns; rec[3] = clock64() - rec[3];
+    }
+#endif
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// Returns SKETCHSSM_UNSUPPORTED_SHAPE when the configuration is outside this kernel's domain (the caller then
+// uses the single-group tensor-core kernel or the CUDA-core kernel).
+int launch_update_tc_ws(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+    const sketchssm_config& c = ctx->cfg;
+    if (c.kind != SKETCHSSM_MAMBA2 || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (c.dv != 64 && c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int NH = 128 / c.dv;
+    if (c.batch % NH != 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (c.rank > 16) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int NP = ((((c.rank + 7) & ~7) + 16) + 15) & ~15;      // [Omega | q | q'] <= 32 columns
+    Params p = p_in;
+    if (ctx->sm_count == 0) {
+        int dev = 0, sms = 0;
+        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return SKETCHSSM_CUDA_ERROR;
+        ctx->sm_count = sms;
+    }
+    // two CTAs per SM (tensor memory: 256 of the SM's 512 columns each) unless capped; the shared memory left after the
+    // operand buffers holds the ring of state stages
+    int ctas = 2;
+    if (p.max_warps_per_sm > 0 && p.max_warps_per_sm < 18) ctas = 1;
+    const uint32_t budget = (228u * 1024u) / (uint32_t)ctas - 1024u;
+    const WsSmem fixed = make_ws_smem(NH, NP, c.dv, c.buf_len, 0);
+    if (fixed.total + 2u * fixed.sst_bytes > budget) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    int stages = (int)((budget - fixed.total) / fixed.sst_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (p.stages >= 2 && p.stages < stages) stages = p.stages;
+    p.stages = stages;
+    const WsSmem sm = make_ws_smem(NH, NP, c.dv, c.buf_len, stages);
+    const long long n_tiles = (long long)c.batch * c.heads / NH;
+    long long grid = (long long)ctx->sm_count * ctas;
+    if (grid > n_tiles) grid = n_tiles;
+    auto kern = c.dv == 128 ? update_tc_ws_mamba2_kernel<128> : update_tc_ws_mamba2_kernel<64>;
+    if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)sm.total)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    if ((ctx->last_cuda_error = launch_kernel(kern, dim3((unsigned)grid), dim3(kWsThreads), sm.total, stream, p, p.pdl != 0)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    ctx->last_launches = 1;
+    return SKETCHSSM_OK;
+}
+
+}  // namespace sketchssm

@@ -149,6 +149,16 @@ def test_mamba2_tensor_core_variants(dv, rank, buf_len):
     w = synth.Workload("t", "mamba2", 6, 3, 128, dv, rank, buf_len, 0, "bf16", 77, basis="qr")
     check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"decode_mma": 1}), "bf16")
     check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"update_impl": 1}), "bf16")
+    check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"update_impl": 3}), "bf16")     # single-group tcgen05 kernel
+
+
+@pytest.mark.parametrize("tune", [{}, {"decode_max_warps_per_sm": 8}, {"pdl": 0}])
+@pytest.mark.parametrize("dv,batch,heads,buf_len", [(64, 64, 24, 16), (128, 40, 20, 8)])
+def test_mamba2_update_several_tiles_per_cta(tune, dv, batch, heads, buf_len):
+    """Warp-specialised tcgen05 update with every CTA walking several tiles (double-buffered accumulators, operand
+    sets and W buffers; head index changes inside a CTA's range), over two windows."""
+    w = synth.Workload("t", "mamba2", batch, heads, 128, dv, 16, buf_len, 0, "bf16", 79, basis="qr")
+    check(run_schedule(w, 2 * buf_len + 2, max_heads=96, tune=tune), "bf16")
 
 
 @pytest.mark.parametrize("rank,buf_len,steps", [(16, 16, 37), (8, 32, 70), (40, 12, 30)])
