@@ -88,7 +88,8 @@ typedef struct sketchssm_config {
 
 typedef struct sketchssm_sizes {
     size_t state_bytes, sketch_bytes, ring_bytes, omega_bytes, coef_bytes;
-    size_t status_bytes;     /* size of the status word block (16) */
+    size_t status_bytes;     /* size of the status block: 4 status ints, then the update kernel's tile-scheduler
+                                counters (4 + heads ints), rounded up to 16 bytes */
     size_t work_bytes;       /* per-head weight hand-off between the two decode kernels: B*H*(K+L) floats */
     size_t ring_head_bytes;  /* stride of one (b, h) ring block */
     size_t ring_v_offset, ring_beta_offset, ring_decay_offset; /* byte offsets inside a ring block (k is at 0) */
@@ -101,9 +102,11 @@ typedef struct sketchssm_buffers {
     void* ring;    /* ring   */
     void* omega;   /* Omega  */
     void* coef;    /* C      */
-    void* status;  /* int32[4], zero-initialised by the caller: [0] first device fault code
-                      (0 = none), [1] which wait, [2..3] reserved.  Kernels only ever write
-                      non-zero codes; sketchssm_read_status reads it back. */
+    void* status;  /* status_bytes, zero-initialised by the caller.  int32[0..3]: [0] first device fault code
+                      (0 = none), [1] which wait, [2..3] reserved; kernels only ever write non-zero codes
+                      there and sketchssm_read_status reads them back.  The ints after them are counters
+                      of the state-update kernel's tile scheduler: every launch leaves them zero again,
+                      and the caller never touches them after the initial zeroing. */
     void* work;    /* work_bytes of scratch for the decode calls (contents are transient: written and
                       consumed inside one call; calls that overlap on the GPU need separate contexts
                       with separate work buffers) */

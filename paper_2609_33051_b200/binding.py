@@ -129,7 +129,7 @@ class SketchSSM:
         self.ring = torch.zeros(self.sizes.ring_bytes, dtype=torch.uint8, device=d)
         self.omega = torch.zeros(self.H, self.K, self.R, dtype=torch.float32, device=d)
         self.coef = torch.zeros(self.H, self.R, self.K, dtype=torch.float32, device=d)
-        self.status = torch.zeros(4, dtype=torch.int32, device=d)
+        self.status = torch.zeros(self.sizes.status_bytes // 4, dtype=torch.int32, device=d)
         self.work = torch.zeros(self.sizes.work_bytes // 4, dtype=torch.float32, device=d)
         self.bind()
 

@@ -173,7 +173,7 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
     out->ring_bytes = bh * ctx->ring.head_bytes;
     out->omega_bytes = (size_t)c.heads * c.dk * c.rank * 4;
     out->coef_bytes = (size_t)c.heads * c.rank * c.dk * 4;
-    out->status_bytes = kStatusInts * sizeof(int32_t);
+    out->status_bytes = (((size_t)(kStatusInts + 4 + c.heads) * sizeof(int32_t)) + 15) & ~(size_t)15;   // status word + tile scheduler counters
     out->work_bytes = bh * (size_t)(c.dk + c.buf_len) * 4;
     out->ring_head_bytes = ctx->ring.head_bytes;
     out->ring_v_offset = ctx->ring.v_off;

@@ -37,14 +37,14 @@ using namespace tc;
 #ifdef SKETCHSSM_PHASE_TIMING
 #define WS_STAMP(base, i)                                                                                      \
     do {                                                                                                       \
-        if (gt == 0 && blockIdx.x == 0 && tile - tile0 >= 12 && tile - tile0 < 20)                             \
-            reinterpret_cast<long long*>(p.work)[(base) + (tile - tile0 - 12) * 32 + (i)] = clock64();         \
+        if (gt == 0 && blockIdx.x == 0 && k >= 0 && k < 8)                                                    \
+            reinterpret_cast<long long*>(p.work)[(base) + (k - 0) * 32  + (i)] = clock64();                    \
     } while (0)
 #else
 #define WS_STAMP(base, i) do { } while (0)
 #endif
 
-constexpr int kWsThreads = 288;       // stream group (4 warps), front group (4 warps), issue warp
+constexpr int kWsThreads = 320;       // stream group (4 warps), front group (4 warps), MMA-2 issue warp, state-load warp
 constexpr int kGroup = 128;
 
 struct WsSmem {
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
     extern __shared__ __align__(1024) unsigned char smem[];
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int wg = tid >> 7, gt = tid & 127;
+    const int gt = tid & 127;
 #ifdef SKETCHSSM_PHASE_TIMING
     if (tid == 0) {
         unsigned long long t_ns; unsigned smid;
@@ -148,6 +148,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
+        *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
         for (int i = 0; i < kNumBars; ++i) {
             // chunk-ready and stage-empty barriers take one arrival per stream warp, the others a single arrival
             const bool per_warp = (i >= kBarA2Rdy && i < kBarA2Rdy + 2) || i >= kBarEmpty;
@@ -174,14 +175,28 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 
     const int tiles_per_h = B / NH;
     const long long n_tiles = (long long)H * tiles_per_h;
-    const int tile0 = (int)(n_tiles * blockIdx.x / gridDim.x);
-    const int tile1 = (int)(n_tiles * (blockIdx.x + 1) / gridDim.x);
+    (void)n_tiles;
     const int n_blocks = (n_tot + kTokBlock - 1) / kTokBlock;
+
+    // Tiles are claimed at run time (see the front group); the CTA's sequence of tile numbers travels through a small
+    // ring in shared memory: entry k & 3 holds the k-th tile of this CTA (-1: no more), `seq_pub` counts entries.
+    volatile int* seq_ring = reinterpret_cast<volatile int*>(smem + sm.misc + 16);
+    volatile int* seq_pub = reinterpret_cast<volatile int*>(smem + sm.misc + 32);
+    auto seq_get = [&](int k) -> int {          // -2: the wait ran out
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+            if (*seq_pub > k) {
+                __threadfence_block();
+                return seq_ring[k & 3];
+            }
+            if (it > 32) __nanosleep(100);
+        }
+        return -2;
+    };
 
     const int my_head = gt / V;           // which head of the tile this thread's TMEM lane belongs to
     const int j = gt % V;
 
-    if (wg == 0) {
+    if (warp < 4) {
         // =========================== stream group: S_0 -> S_new, MMA 2 ===========================
         constexpr int CH = 16, NCH = K / CH;
         const int lane = tid & 31;
@@ -189,8 +204,13 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
         int gc = 0, stage = 0;                   // chunks consumed so far, their stage and its phase
         uint32_t phF = 0;
         bool bad = false;
-        for (int tile = tile0; tile < tile1 && !bad; ++tile) {
-            const int b = (tile - tile0) & 1;
+        for (int k = 0; !bad; ++k) {
+            const int tile = seq_get(k);
+            if (tile < 0) {
+                bad = tile < -1;
+                break;
+            }
+            const int b = k & 1;
             const int h = tile / tiles_per_h;
             const int b0 = (tile - h * tiles_per_h) * NH;
             const size_t bh = (size_t)(b0 + my_head) * H + h;
@@ -268,43 +288,20 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             }
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 3);
-    } else if (wg == 2) {
-        // =========================== issue warp: S_0 stages (TMA) and MMA 2, one thread ===========================
+    } else if (warp == 8) {
+        // =========================== MMA-2 issue warp (one thread) ===========================
         if (gt == 0) {
             constexpr int CH = 16, NCH = K / CH;
-            const int total_chunks = (tile1 - tile0) * NCH;
-            // producer cursor: the chunk to load next
-            int p_tile = tile0, p_c = 0, p_stage = 0;
-            const float* p_src[NH];
-            auto producer_tile = [&]() {
-                const int h = p_tile / tiles_per_h;
-                const int b0 = (p_tile - h * tiles_per_h) * NH;
-#pragma unroll
-                for (int hd = 0; hd < NH; ++hd) p_src[hd] = p.state + ((size_t)(b0 + hd) * H + h) * (size_t)K * V;
-            };
-            auto issue_chunk = [&]() {
-                uint64_t* bar = &bars[kBarFull + p_stage];
-                mbar_expect_tx(bar, sm.sst_bytes);
-#pragma unroll
-                for (int hd = 0; hd < NH; ++hd)
-                    bulk_g2s(smem + sm.sst + (size_t)p_stage * sm.sst_bytes + (size_t)hd * CH * V * 4,
-                             p_src[hd] + (size_t)p_c * CH * V, (uint32_t)(CH * V * 4), bar);
-                if (++p_stage == NS) p_stage = 0;
-                if (++p_c == NCH) {
-                    p_c = 0;
-                    ++p_tile;
-                    if (p_tile < tile1) producer_tile();
-                }
-            };
-            int issued = 0;
-            if (tile0 < tile1) producer_tile();
-            for (; issued < NS && issued < total_chunks; ++issued) issue_chunk();
-            uint32_t phR = 0, phE = 0;           // chunk-ready phases (bit per buffer), stage-empty phase
-            int stage = 0;
+            uint32_t phR = 0;                    // chunk-ready phases (bit per buffer)
             bool bad = false;
             const uint32_t sB2 = smem_u32(smem + sm.b2);
-            for (int tile = tile0; tile < tile1 && !bad; ++tile) {
-                const int b = (tile - tile0) & 1;
+            for (int k = 0; !bad; ++k) {
+                const int tile = seq_get(k);
+                if (tile < 0) {
+                    bad = tile < -1;
+                    break;
+                }
+                const int b = k & 1;
                 const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
@@ -322,25 +319,79 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                     tc_mma_bf16(tmem_t, ahi, blo, idesc2, 1u);
                     tc_commit(&bars[kBarA2 + (c & 1)]);
                     if (c == NCH - 1) tc_commit(&bars[kBarU + b]);     // everything of this tile: UT is complete
-                    // the stage this chunk came from was released by all four stream warps before they wrote the chunk
-                    if (issued < total_chunks) {
-                        if (!mbar_wait_bounded(&bars[kBarEmpty + stage], phE)) { bad = true; break; }
-                        issue_chunk();
-                        ++issued;
-                    }
-                    if (++stage == NS) { stage = 0; phE ^= 1u; }
                 }
             }
             if (bad) record_fault(p.status, kFaultUpdateWait, 4);
         }
+    } else if (warp == 9) {
+        // =========================== state-load warp: keeps the ring of S_0 stages full (one lane per head) ===========
+        constexpr int CH = 16, NCH = K / CH;
+        const int lane = gt & 31;
+        int stage = 0, round = 0;            // stage to fill next; how often the ring has wrapped
+        bool bad = false;
+        for (int k = 0; !bad; ++k) {
+            const int tile = seq_get(k);
+            if (tile < 0) {
+                bad = tile < -1;
+                break;
+            }
+            const int h = tile / tiles_per_h;
+            const int b0 = (tile - h * tiles_per_h) * NH;
+            const float* src = p.state + ((size_t)(b0 + (lane < NH ? lane : 0)) * H + h) * (size_t)K * V;
+            for (int c = 0; c < NCH; ++c) {
+                if (round > 0) {     // the stage was released by all four stream warps
+                    if (!mbar_wait_bounded(&bars[kBarEmpty + stage], (uint32_t)(round - 1) & 1u)) { bad = true; break; }
+                }
+                uint64_t* bar = &bars[kBarFull + stage];
+                if (lane == 0) mbar_expect_tx(bar, sm.sst_bytes);
+                __syncwarp();
+                if (lane < NH)
+                    bulk_g2s(smem + sm.sst + (size_t)stage * sm.sst_bytes + (size_t)lane * CH * V * 4,
+                             src + (size_t)c * CH * V, (uint32_t)(CH * V * 4), bar);
+                if (++stage == NS) { stage = 0; ++round; }
+            }
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 7);
     } else {
         // =========================== front group: operands, MMA 1, sketch stores ===========================
         const int fwarp = gt >> 5;
         int cur_h = -1;                       // head index whose Omega sits in W
         int ops_built = 0;                    // MMA-1 operand sets written so far (single buffer)
-        int ut_stored = tile0;                // tiles below this one have their sketch rows stored
+        int prev_tile = -1, last_b = 0;       // the tile whose sketch rows are still to be stored (-1: none) and its buffer
         uint32_t phS = 0, phU = 0, phB = 0;
         bool dead = false;
+
+        // ---- tile claiming (thread 0 of the group) ----
+        // Head index h owns a counter of tiles handed out.  A CTA keeps claiming tiles of the head index it works on
+        // (its Omega stays in shared memory); when that is exhausted it moves to the head index with the most tiles left.
+        // The claim for the tile after next is in flight while a tile's operands are built.  The last CTA to finish
+        // zeroes the counters again, so they are zero between launches.
+        int* sched = p.status + kStatusInts;  // [0] CTAs finished, [4 + h] tiles of head index h handed out
+        int* cnt = sched + 4;
+        int h_claim = (int)(((long long)blockIdx.x * H) / gridDim.x);
+        int t_raw = 0;
+        auto claim_issue = [&]() { t_raw = atomicAdd(&cnt[h_claim], 1); };
+        auto claim_resolve = [&]() -> int {   // tile number, or -1 when every tile has been handed out
+            for (int attempt = 0; attempt <= H; ++attempt) {
+                if (t_raw < tiles_per_h) return h_claim * tiles_per_h + t_raw;
+                int best = -1, best_c = tiles_per_h;
+                for (int i = 1; i <= H; ++i) {
+                    int hh = h_claim + i;
+                    if (hh >= H) hh -= H;
+                    const int c = *reinterpret_cast<volatile int*>(&cnt[hh]);
+                    if (c < best_c) { best_c = c; best = hh; }
+                }
+                if (best < 0) return -1;
+                h_claim = best;
+                t_raw = atomicAdd(&cnt[h_claim], 1);
+            }
+            return -1;
+        };
+        auto publish = [&](int k, int tile) {
+            seq_ring[k & 3] = tile;
+            __threadfence_block();
+            *seq_pub = k + 1;
+        };
 
         // Raw ring rows of a tile's first token block travel to shared memory by bulk copies issued one tile ahead.
         // Rows of later blocks (n > 16) are read directly.
@@ -370,8 +421,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             }
         };
         // sketch rows and exact output of a finished tile: UT sits in the first NP columns of that tile's accumulator
-        auto store_ut = [&](int tile) -> bool {
-            const int b = (tile - tile0) & 1;
+        auto store_ut = [&](int tile, int b) -> bool {
             const int h = tile / tiles_per_h;
             const int b0 = (tile - h * tiles_per_h) * NH;
             const size_t bh = (size_t)(b0 + my_head) * H + h;
@@ -395,7 +445,15 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             return true;
         };
 
-        if (gt == 0 && stg_bytes > 0 && tile0 < tile1) stage_tile(tile0);
+        if (gt == 0) {
+            claim_issue();
+            const int first = claim_resolve();
+            publish(0, first);
+            if (first >= 0) {
+                claim_issue();
+                if (stg_bytes > 0) stage_tile(first);
+            }
+        }
         // W (padding columns, lo halves of the query columns) and the MMA-1 operands (off-diagonal head blocks) hold
         // zeros that no tile ever overwrites: written once
         for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGroup * 16u)
@@ -404,8 +462,16 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             *reinterpret_cast<uint4*>(smem + sm.op + o) = make_uint4(0, 0, 0, 0);
         group_sync(2);
 
-        for (int tile = tile0; tile < tile1 && !dead; ++tile) {
-            const int b = (tile - tile0) & 1;
+        for (int k = 0; !dead; ++k) {
+            const int tile = seq_get(k);
+            if (tile < 0) {
+                if (tile < -1) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 8);
+                    dead = true;
+                }
+                break;
+            }
+            const int b = k & 1;
             const int h = tile / tiles_per_h;
             const int b0 = (tile - h * tiles_per_h) * NH;
             __nv_bfloat16* sB2hi = reinterpret_cast<__nv_bfloat16*>(smem + sm.b2);
@@ -426,13 +492,13 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             // ---- W = [Omega | q | q'] hi/lo, K-major; the Omega part once per head index.  MMA 2 of the previous tile
             // still reads W, so that tile is finished (and its sketch rows stored) first. ----
             if (h != cur_h) {
-                if (tile > tile0) {
-                    if (!store_ut(tile - 1)) {
+                if (prev_tile >= 0) {
+                    if (!store_ut(prev_tile, b ^ 1)) {
                         if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
                         dead = true;
                         break;
                     }
-                    ut_stored = tile;
+                    prev_tile = -1;
                     group_sync(2);
                 }
                 const float* og = p.omega + (size_t)h * K * R;
@@ -633,7 +699,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 ++ops_built;
                 if (gt == 0) {
                     tc_fence_after();
-                    if (blk == 0 && stg_bytes > 0 && tile + 1 < tile1) stage_tile(tile + 1);   // staging is free again
                     const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
 #pragma unroll
                     for (int ks = 0; ks < KD1 / 16; ++ks) {
@@ -643,6 +708,14 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                     }
                     tc_commit(&bars[kBarBlk]);
                     if (blk + 1 == n_blocks) tc_commit(&bars[kBarT + b]);
+                    if (blk == 0) {      // the staging buffer is free again: the next tile's rows may come in
+                        const int nxt = claim_resolve();
+                        publish(k + 1, nxt);
+                        if (nxt >= 0) {
+                            claim_issue();
+                            if (stg_bytes > 0) stage_tile(nxt);
+                        }
+                    }
                 }
             }
             if (dead) break;
@@ -650,25 +723,40 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 // no token to replay: nothing reads the staging buffer after the query columns; T counts as zero
                 group_sync(2);
                 if (gt == 0) {
-                    if (stg_bytes > 0 && tile + 1 < tile1) stage_tile(tile + 1);
                     mbar_arrive(&bars[kBarT + b]);
+                    const int nxt = claim_resolve();
+                    publish(k + 1, nxt);
+                    if (nxt >= 0) {
+                        claim_issue();
+                        if (stg_bytes > 0) stage_tile(nxt);
+                    }
                 }
             }
             if (gt == 0) mbar_arrive(&bars[kBarPro + b]);      // after the group barrier: W, weights and decay are written
             WS_STAMP(512, 3);
 
             // ---- sketch rows and exact output of the previous tile, once the stream group has finished it ----
-            if (ut_stored < tile) {
-                if (!store_ut(tile - 1)) {
+            if (prev_tile >= 0) {
+                if (!store_ut(prev_tile, b ^ 1)) {
                     if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
                     dead = true;
                 }
-                ut_stored = tile;
             }
+            prev_tile = tile;
+            last_b = b;
             WS_STAMP(512, 4);
         }
-        if (!dead && tile0 < tile1) {
-            if (!store_ut(tile1 - 1) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+        if (!dead && prev_tile >= 0) {
+            // the last tile used buffer (number of tiles - 1) & 1; phU tells which buffer has an odd number of stores
+            if (!store_ut(prev_tile, last_b) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+        }
+        if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
+            __threadfence();
+            if (atomicAdd(&sched[0], 1) == (int)gridDim.x - 1) {
+                for (int hh = 0; hh < H; ++hh) cnt[hh] = 0;
+                sched[0] = 0;
+                __threadfence();
+            }
         }
     }
 

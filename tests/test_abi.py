@@ -76,7 +76,7 @@ def test_sizes_and_ring_layout(lib, kind, io, K, V, L, expect_head):
     assert s.ring_v_offset == L * K * esz
     assert s.ring_beta_offset == s.ring_v_offset + L * V * esz
     assert s.ring_decay_offset == s.ring_beta_offset + L * 4
-    assert s.alignment == 16 and s.status_bytes == 16
+    assert s.alignment == 16 and s.status_bytes == ((4 + 4 + 5) * 4 + 15) // 16 * 16
     assert s.work_bytes == 15 * (K + L) * 4
     for off in (s.ring_head_bytes, s.ring_v_offset, s.ring_beta_offset, s.ring_decay_offset):
         assert off % 16 == 0
