@@ -5,9 +5,10 @@
 // and no per-CTA start-up cost is paid more than once per SM slot.  A warp owns one head at a time.  All of the
 // head's operands -- the sketch U, the buffered keys / values / gates of the ring and the current token's
 // q, k, v rows -- arrive in the warp's private shared-memory stage by 1-D bulk asynchronous copies (TMA, no
-// multicast) completing on the warp's mbarrier; the copies of the warp's next head are issued as soon as the
-// current one is done, and the token's scalar gates are fetched one head ahead, so no global-memory latency sits
-// on the per-head critical path except the stage itself.
+// multicast).  The stage is filled in two groups with an mbarrier each: what the ring sweep reads, and the sketch.
+// The next head's first group is issued right after the current head's sweep and its sketch right after the current
+// sketch has been used, each copy by its own lane, and the token's scalar gates are fetched one head ahead: the
+// loads of a head overlap the arithmetic of the one before it without a second stage.
 //
 // Arithmetic per head (Algorithm 1, non-flush step; Eq. 4):
 //   x <- q_t;  for s = t .. 1:  a_s = beta_s <k_s, x>;  x <- D_s (x - a_s k_s)   [Mamba-2: a_s = beta_s (prod_{j>s} a_j) <k_s, q_t>]
@@ -22,6 +23,17 @@
 namespace sketchssm {
 
 namespace {
+
+// Optional phase stamps (warp 0 of CTA 0 and of the middle CTA) into the work buffer; compiled out by default.
+#ifdef SKETCHSSM_PHASE_TIMING
+#define DEC_STAMP(i)                                                                                          \
+    do {                                                                                                      \
+        if (lane == 0 && warp == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2) && it < 8)             \
+            reinterpret_cast<long long*>(p.work)[(blockIdx.x == 0 ? 0 : 256) + it * 8 + (i)] = clock64();     \
+    } while (0)
+#else
+#define DEC_STAMP(i) do { } while (0)
+#endif
 
 struct StageLayout {
     uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
@@ -58,17 +70,16 @@ struct DecodeSmem {
     uint32_t coef_slot_bytes, bar_off, scratch_off, scratch_stride, stage_off, total;
 };
 
-__host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps, int stages, int full_read,
-                                                       uint32_t stage_bytes) {
+__host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps, int full_read, uint32_t stage_bytes) {
     DecodeSmem d;
     const int RP = (R + 7) & ~7;                       // coefficient rows padded to the reduction width
     d.coef_slot_bytes = full_read ? 0u : (uint32_t)(RP * K * 4);
     d.bar_off = 2u * d.coef_slot_bytes;
-    uint32_t off = d.bar_off + (((uint32_t)(nwarps * stages * 8) + 127u) & ~127u);
+    uint32_t off = d.bar_off + (((uint32_t)(nwarps * 2 * 8) + 127u) & ~127u);    // two mbarriers per warp
     d.scratch_stride = (uint32_t)((K + 80) * 4);       // per warp: q~ (full read) or c (K floats), then 64+ dot products
     d.scratch_off = off; off += (uint32_t)nwarps * d.scratch_stride;
     d.stage_off = off;
-    d.total = off + (uint32_t)(nwarps * stages) * stage_bytes;
+    d.total = off + (uint32_t)nwarps * stage_bytes;
     return d;
 }
 
@@ -86,14 +97,13 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
     const int nwarps = blockDim.x >> 5;
     const int R = p.R, L = p.L, H = p.H, B = p.B, n = p.n_before;
     const int RP = (R + 7) & ~7;
-    const int stages = p.stages;
 
     const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n, p.full_read);
-    const DecodeSmem ds = make_decode_smem(K, R, nwarps, stages, p.full_read, sl.total);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * stages;
+    const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, sl.total);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * 2;
     float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
     float* sP = sX + K;                                                                               // dot products
-    unsigned char* my_stage = smem + ds.stage_off + (size_t)warp * stages * sl.total;
+    unsigned char* my_stage = smem + ds.stage_off + (size_t)warp * sl.total;
 
     // contiguous range of items for this CTA; item = h * B + b
     const long long total = (long long)H * B;
@@ -103,7 +113,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
     const int h_last = item1 > item0 ? (item1 - 1) / B : h_first;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < nwarps * stages; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + ds.bar_off) + i, 1);
+        for (int i = 0; i < nwarps * 2; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + ds.bar_off) + i, 1);
         mbar_fence_init();
     }
     // coefficient maps of the (at most two) head indices of this range, rows padded with zeros.  C is a constant of
@@ -121,64 +131,88 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
     grid_dep_wait();                 // from here on the ring, the sketch and the token tensors are read
     grid_dep_launch_dependents();
 
-    const uint32_t tx_bytes = sl.u_bytes + sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes + 2u * sl.tqk_bytes +
-                              sl.tv_bytes + sl.tg_bytes;
-
-    auto issue = [&](int item, int st) {   // lane 0 only
-        uint64_t* bar = &bars[st];
-        unsigned char* sb = my_stage + (size_t)st * sl.total;
-        const int h = item / B, b = item - h * B;
-        const size_t bh = (size_t)b * H + h;
-        const unsigned char* rh = p.ring + bh * p.rl.head_bytes;
-        mbar_expect_tx(bar, tx_bytes);
-        bulk_g2s(sb + sl.tq_off, reinterpret_cast<const IO*>(p.q) + bh * K, sl.tqk_bytes, bar);
-        bulk_g2s(sb + sl.tk_off, reinterpret_cast<const IO*>(p.k) + bh * K, sl.tqk_bytes, bar);
-        bulk_g2s(sb + sl.tv_off, reinterpret_cast<const IO*>(p.v) + bh * V, sl.tv_bytes, bar);
-        if (sl.tg_bytes) bulk_g2s(sb + sl.tg_off, reinterpret_cast<const IO*>(p.decay) + bh * K, sl.tg_bytes, bar);
-        if (sl.k_bytes) {
-            bulk_g2s(sb + sl.k_off, rh, sl.k_bytes, bar);
-            bulk_g2s(sb + sl.gate_off, rh + p.rl.beta_off, sl.gate_bytes, bar);
-            if (sl.g_bytes) bulk_g2s(sb + sl.g_off, rh + p.rl.decay_off, sl.g_bytes, bar);
-            bulk_g2s(sb + sl.v_off, rh + p.rl.v_off, sl.v_bytes, bar);
+    // A warp's stage is filled by two groups of bulk copies, each completing on its own mbarrier: group A holds what
+    // the ring sweep reads (the token's rows and the buffered keys / values / gates), group B the sketch U.  Group A of
+    // the warp's next head is issued as soon as the sweep of the current head is over and group B as soon as U has been
+    // used, so the next head's loads overlap the rest of the current head's arithmetic without a second stage.
+    // Every copy is issued by its own lane from per-lane constants set up once (base pointer, bytes per head, target).
+    const uint32_t txA = sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes + 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
+    const uint32_t txB = sl.u_bytes;
+    const unsigned char* cp_base = nullptr;
+    size_t cp_stride = 0;
+    uint32_t cp_dst = 0, cp_bytes = 0;
+    switch (lane) {
+        case 0: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tq_off; cp_bytes = sl.tqk_bytes; break;
+        case 1: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tk_off; cp_bytes = sl.tqk_bytes; break;
+        case 2: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * sizeof(IO); cp_dst = sl.tv_off; cp_bytes = sl.tv_bytes; break;
+        case 3: cp_base = reinterpret_cast<const unsigned char*>(p.decay); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tg_off; cp_bytes = sl.tg_bytes; break;
+        case 4: cp_base = p.ring; cp_stride = p.rl.head_bytes; cp_dst = sl.k_off; cp_bytes = sl.k_bytes; break;
+        case 5: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sl.gate_off; cp_bytes = sl.gate_bytes; break;
+        case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_bytes = sl.v_bytes; break;
+        case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_bytes = sl.g_bytes; break;
+        case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * 4; cp_dst = sl.u_off; cp_bytes = sl.u_bytes; break;
+        default: break;
+    }
+    uint64_t* barA = &bars[0];
+    uint64_t* barB = &bars[1];
+    auto issue_a = [&](size_t bh) {      // whole warp
+        if (lane == 0) mbar_expect_tx(barA, txA);
+        __syncwarp();
+        if (lane < 8 && cp_bytes) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barA);
+    };
+    auto issue_b = [&](size_t bh) {      // whole warp
+        if (lane == 8 && cp_bytes) {
+            mbar_expect_tx(barB, txB);
+            bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barB);
         }
-        if (sl.u_bytes) bulk_g2s(sb + sl.u_off, p.sketch + bh * (size_t)R * V, sl.u_bytes, bar);
     };
 
+    // this warp's heads: items item0 + warp, item0 + warp + nwarps, ...; (head index, batch) advance without divisions
     const int n_items = item1 - item0;
     const int count = warp < n_items ? (n_items - warp + nwarps - 1) / nwarps : 0;
-    auto item_of = [&](int it) { return item0 + warp + it * nwarps; };
-
-    if (count > 0 && lane == 0) issue(item_of(0), 0);
+    int h = 0, b = 0;
+    if (count > 0) {
+        h = (item0 + warp) / B;
+        b = (item0 + warp) - h * B;
+    }
+    auto advance = [&](int& hh, int& bb) {
+        bb += nwarps;
+        while (bb >= B) { bb -= B; ++hh; }
+    };
+    int hn = h, bn = b;                 // the warp's next head
+    advance(hn, bn);
 
     // the token's scalar gates travel in registers, fetched one head ahead
-    auto scalar_gates = [&](int item, float& bt, float& dsc) {
-        const int h = item / B, b = item - h * B;
-        const size_t bh = (size_t)b * H + h;
+    auto scalar_gates = [&](size_t bh, float& bt, float& dsc) {
         bt = p.beta[bh];
         dsc = 1.f;
         if constexpr (KIND != SKETCHSSM_KDA) dsc = reinterpret_cast<const float*>(p.decay)[bh];
     };
     float bt_next = 0.f, dsc_next = 1.f;
-    if (count > 0) scalar_gates(item_of(0), bt_next, dsc_next);
+    if (count > 0) {
+        const size_t bh0 = (size_t)b * H + h;
+        issue_a(bh0);
+        issue_b(bh0);
+        scalar_gates(bh0, bt_next, dsc_next);
+    }
     bool dead = false;
 
     for (int it = 0; it < count; ++it) {
-        const int item = item_of(it);
-        const int st = stages == 2 ? (it & 1) : 0;
-        const uint32_t parity = stages == 2 ? ((it >> 1) & 1) : (it & 1);
-        if (stages == 2 && it + 1 < count && lane == 0) issue(item_of(it + 1), st ^ 1);
-
-        const int h = item / B, b = item - h * B;
+        const uint32_t parity = it & 1;
         const size_t bh = (size_t)b * H + h;
+        const size_t bh_next = (size_t)bn * H + hn;
+        const bool has_next = it + 1 < count;
         const float bt = bt_next, dsc = dsc_next;
-        if (it + 1 < count) scalar_gates(item_of(it + 1), bt_next, dsc_next);
+        if (has_next) scalar_gates(bh_next, bt_next, dsc_next);
 
-        if (!mbar_wait_bounded(&bars[st], parity)) {
+        DEC_STAMP(0);
+        if (!mbar_wait_bounded(barA, parity)) {
             record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
             dead = true;
             break;
         }
-        const unsigned char* sb = my_stage + (size_t)st * sl.total;
+        DEC_STAMP(1);
+        const unsigned char* sb = my_stage;
         const IO* sK = reinterpret_cast<const IO*>(sb + sl.k_off);
         const IO* sV = reinterpret_cast<const IO*>(sb + sl.v_off);
         const float* sBeta = reinterpret_cast<const float*>(sb + sl.gate_off);
@@ -278,6 +312,10 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
             }
         }
 
+        // the sweep is done with the ring part of the stage: the next head's group A may come in
+        __syncwarp();
+        if (has_next) issue_a(bh_next);
+        DEC_STAMP(2);
         if (!p.full_read) {
             // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
             const float* sC = reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
@@ -297,6 +335,11 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
             __syncwarp();
+            if (!mbar_wait_bounded(barB, parity)) {
+                record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
+                dead = true;
+                break;
+            }
             const float* sU = reinterpret_cast<const float*>(sb + sl.u_off);
 #pragma unroll 4
             for (int g = 0; g < R; ++g) {
@@ -306,6 +349,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
 #pragma unroll
                 for (int e = 0; e < EV; ++e) o[e] = fmaf(cg, uu[e], o[e]);
             }
+            __syncwarp();
+            if (has_next) issue_b(bh_next);
         } else {
             __syncwarp();
             store_io<EK>(sX, lane * EK, x);
@@ -325,20 +370,21 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
             }
         }
 
+        DEC_STAMP(3);
         if (p.out_bf16) {
             store_io<EV>(reinterpret_cast<__nv_bfloat16*>(p.out) + bh * V, lane * EV, o);
         } else {
             store_io<EV>(reinterpret_cast<float*>(p.out) + bh * V, lane * EV, o);
         }
 
-        __syncwarp();  // every lane is done with this stage and the scratch before either is reused
-        if (stages == 1 && it + 1 < count && lane == 0) issue(item_of(it + 1), 0);
+        __syncwarp();  // every lane is done with the scratch before it is reused
+        DEC_STAMP(4);
+        h = hn;
+        b = bn;
+        advance(hn, bn);
+        DEC_STAMP(5);
     }
-
-    if (dead && stages == 2) {   // bounded grace period for the other stage's copies before the CTA retires
-        mbar_wait_bounded(&bars[0], 0, 1u << 16);
-        mbar_wait_bounded(&bars[1], 0, 1u << 16);
-    }
+    (void)dead;
 }
 
 template <int KIND, typename IO, int K, int V>
@@ -353,14 +399,13 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
             return SKETCHSSM_CUDA_ERROR;
         ctx->sm_count = sms;
     }
-    // warps per CTA / stages / CTAs per SM: as many resident warps per SM as shared memory allows (capped),
-    // preferring a single stage (more heads in flight per byte of shared memory) and fewer, larger CTAs
+    // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
+    // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
-    const int want_st = (p.stages == 1 || p.stages == 2) ? p.stages : 1;
     int best_nw = 0, best_ctas = 1, best_warps = 0;
     for (int nw = 8; nw >= 1; --nw) {
         if (p.warps_per_cta && nw != p.warps_per_cta) continue;
-        const DecodeSmem d = make_decode_smem(K, p.R, nw, want_st, p.full_read, sl.total);
+        const DecodeSmem d = make_decode_smem(K, p.R, nw, p.full_read, sl.total);
         if (d.total > smem_budget) continue;
         int ctas = (int)((228u * 1024u) / (d.total + 1024u));
         if (ctas * nw > cap) ctas = cap / nw;
@@ -368,8 +413,7 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
         if (ctas * nw > best_warps) { best_warps = ctas * nw; best_nw = nw; best_ctas = ctas; }
     }
     if (best_nw == 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    p.stages = want_st;
-    const DecodeSmem d = make_decode_smem(K, p.R, best_nw, want_st, p.full_read, sl.total);
+    const DecodeSmem d = make_decode_smem(K, p.R, best_nw, p.full_read, sl.total);
     auto kern = decode_kernel<KIND, IO, K, V>;
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)d.total)) != cudaSuccess)
