@@ -35,6 +35,20 @@ namespace {
 #define DEC_STAMP(i) do { } while (0)
 #endif
 
+#ifdef SKETCHSSM_PHASE_TIMING
+// bounded wait that also counts its polls
+__device__ __forceinline__ bool mbar_wait_counted(uint64_t* bar, uint32_t parity, unsigned long long& polls) {
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        ++polls;
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    return false;
+}
+#define DEC_WAIT(bar, parity) mbar_wait_counted(bar, parity, poll_count)
+#else
+#define DEC_WAIT(bar, parity) mbar_wait_bounded(bar, parity)
+#endif
+
 struct StageLayout {
     uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
     uint32_t k_off, k_bytes;        // n buffered keys
@@ -85,8 +99,9 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
 
 }  // namespace
 
-template <int KIND, typename IO, int K, int V>
-__global__ void __launch_bounds__(256) decode_kernel(const Params p) {
+// RT: the sketch rank as a compile-time constant (loops over ranks unroll fully), or 0 for any rank.
+template <int KIND, typename IO, int K, int V, int RT>
+__global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
     constexpr int EV = V / 32;
     constexpr int NB = 8;                               // dot products per transposing reduction
@@ -95,7 +110,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
-    const int R = p.R, L = p.L, H = p.H, B = p.B, n = p.n_before;
+    const int R = RT ? RT : p.R;
+    const int L = p.L, H = p.H, B = p.B, n = p.n_before;
     const int RP = (R + 7) & ~7;
 
     const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n, p.full_read);
@@ -196,6 +212,9 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
         scalar_gates(bh0, bt_next, dsc_next);
     }
     bool dead = false;
+#ifdef SKETCHSSM_PHASE_TIMING
+    unsigned long long poll_count = 0;
+#endif
 
     for (int it = 0; it < count; ++it) {
         const uint32_t parity = it & 1;
@@ -206,7 +225,7 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
         if (has_next) scalar_gates(bh_next, bt_next, dsc_next);
 
         DEC_STAMP(0);
-        if (!mbar_wait_bounded(barA, parity)) {
+        if (!DEC_WAIT(barA, parity)) {
             record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
             dead = true;
             break;
@@ -261,7 +280,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
         // ---- buffered tokens ----
         if constexpr (KIND == SKETCHSSM_MAMBA2) {
             // independent dot products <k_s, q_t>, eight per transposing reduction; lane l ends up with slot s0 + l/4
-            for (int s0 = 0; s0 < n; s0 += NB) {
+            int s0 = 0;
+            for (; s0 + 4 < n; s0 += NB) {      // blocks of eight while more than four slots remain
                 float part[NB];
 #pragma unroll
                 for (int i = 0; i < NB; ++i) {
@@ -274,6 +294,20 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
                 }
                 group_reduce_transpose<32, NB>(part, lane);
                 if ((lane & 3) == 0) sP[s0 + (lane >> 2)] = part[0];
+            }
+            if (s0 < n) {                       // one to four slots left: lane l ends up with slot s0 + l/8
+                float part[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float kr[EK];
+                    load_io<EK>(sK, min(s0 + i, n - 1) * K + lane * EK, kr);
+                    float acc = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EK; ++e) acc = fmaf(kr[e], q0[e], acc);
+                    part[i] = acc;
+                }
+                group_reduce_transpose<32, 4>(part, lane);
+                if ((lane & 7) == 0) sP[s0 + (lane >> 3)] = part[0];
             }
             __syncwarp();
 #pragma unroll 4
@@ -320,7 +354,8 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
             // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
             const float* sC = reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
             __syncwarp();
-            for (int g0 = 0; g0 < RP; g0 += NB) {
+#pragma unroll
+            for (int g0 = 0; g0 < (RT ? ((RT + 7) & ~7) : RP); g0 += NB) {
                 float part[NB];
 #pragma unroll
                 for (int i = 0; i < NB; ++i) {
@@ -335,13 +370,13 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
             __syncwarp();
-            if (!mbar_wait_bounded(barB, parity)) {
+            if (!DEC_WAIT(barB, parity)) {
                 record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
                 dead = true;
                 break;
             }
             const float* sU = reinterpret_cast<const float*>(sb + sl.u_off);
-#pragma unroll 4
+#pragma unroll (RT ? RT : 4)
             for (int g = 0; g < R; ++g) {
                 const float cg = sX[g];
                 float uu[EV];
@@ -385,6 +420,9 @@ __global__ void __launch_bounds__(256) decode_kernel(const Params p) {
         DEC_STAMP(5);
     }
     (void)dead;
+#ifdef SKETCHSSM_PHASE_TIMING
+    if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(p.work) + 1000, poll_count);
+#endif
 }
 
 template <int KIND, typename IO, int K, int V>
@@ -402,6 +440,16 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
     // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
+    auto kern = p.R == 16 ? decode_kernel<KIND, IO, K, V, 16> : decode_kernel<KIND, IO, K, V, 0>;
+    // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does
+    static int regs_per_thread[2] = {0, 0};
+    int& regs = regs_per_thread[p.R == 16 ? 1 : 0];
+    if (regs == 0) {
+        cudaFuncAttributes fa;
+        if ((ctx->last_cuda_error = cudaFuncGetAttributes(&fa, kern)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        regs = fa.numRegs > 0 ? fa.numRegs : 64;
+    }
+    const int reg_warps = 65536 / (regs * 32);          // warps the register file holds
     int best_nw = 0, best_ctas = 1, best_warps = 0;
     for (int nw = 8; nw >= 1; --nw) {
         if (p.warps_per_cta && nw != p.warps_per_cta) continue;
@@ -409,12 +457,12 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
         if (d.total > smem_budget) continue;
         int ctas = (int)((228u * 1024u) / (d.total + 1024u));
         if (ctas * nw > cap) ctas = cap / nw;
+        if (ctas * nw > reg_warps) ctas = reg_warps / nw;
         if (ctas < 1) continue;
         if (ctas * nw > best_warps) { best_warps = ctas * nw; best_nw = nw; best_ctas = ctas; }
     }
     if (best_nw == 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
     const DecodeSmem d = make_decode_smem(K, p.R, best_nw, p.full_read, sl.total);
-    auto kern = decode_kernel<KIND, IO, K, V>;
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)d.total)) != cudaSuccess)
         return SKETCHSSM_CUDA_ERROR;
