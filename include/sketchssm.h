@@ -214,9 +214,9 @@ int sketchssm_last_launch_count(const sketchssm_ctx* ctx);
  * the decode kernels serves for its head; 0 = library default), "decode_stages" (1 or 2 shared-memory
  * stages per lane group; 0 = library default), "decode_warps_per_cta", "decode_max_warps_per_sm",
  * "decode_lanes_per_head", "decode_l2_prefetch", "decode_mma" (1 = tensor-core dot products in the
- * warp-per-head decode where supported; 0 = off, the default), "update_impl" (0 = tensor cores for Mamba-2 and CUDA
- * cores otherwise, the default; 1 = CUDA cores only; 2 = as 0 plus the tensor-core kernel for GDN; 3 = as 0 but with the
- * single-warp-group tensor-core kernel for Mamba-2 instead of the warp-specialised one), "decode_impl" (0 = two kernels; 1 = one fused
+ * warp-per-head decode where supported; 0 = off, the default), "update_impl" (0 = warp-specialised tensor-core kernels for Mamba-2 and
+ * GDN where their shape limits allow and CUDA cores otherwise, the default; 1 = CUDA cores only; 2 = as 0 but the
+ * single-group tensor-core kernel for GDN; 3 = single-group tensor-core kernel for Mamba-2, CUDA cores for GDN), "decode_impl" (0 = two kernels; 1 = one fused
  * kernel with a warp per head, the default; 2 = one fused kernel with 8 or 16 lanes per head).  Results depend on these
  * only through floating-point summation order. */
 int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value);

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsketchssm.so")
 # (source, object suffix, extra defines); the lane-group decode kernel is compiled once per (recurrence kind, I/O type)
-UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []), ("update_tc_ws.cu", "", []), ("update_tc_delta.cu", "", []),
+UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []), ("update_tc_ws.cu", "", []), ("update_tc_ws_gdn.cu", "", []), ("update_tc_delta.cu", "", []),
          ("decode_static.cu", "", []), ("decode_mma.cu", "", []),
          *[("decode_fused.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
            for k in range(3) for io in range(2)],

@@ -228,7 +228,11 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
         rc = launch_update_tc(ctx, p, static_cast<cudaStream_t>(stream));
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
     }
-    if (p.update_impl == 2) {       // opt-in: gated delta rule on tensor cores (measured slower than the CUDA-core kernel so far)
+    if (p.update_impl == 0 || p.update_impl == 4) {       // gated delta rule: warp-specialised tensor-core kernel (1..16 tokens, rank <= 16)
+        rc = launch_update_tc_ws_gdn(ctx, p, static_cast<cudaStream_t>(stream));
+        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+    }
+    if (p.update_impl == 2) {       // gated delta rule, single-group tensor-core kernel (slower than the CUDA-core kernel)
         rc = launch_update_tc_delta(ctx, p, static_cast<cudaStream_t>(stream));
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
     }

@@ -68,7 +68,7 @@ struct Params {
     int l2_prefetch;     // decode (group kernel): request the following item's operands into L2
     int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
     int update_impl;      // 0: tensor cores for Mamba-2, CUDA cores otherwise; 1: CUDA cores only; 2: also the GDN tensor-core kernel;
-                          // 3: as 0 but without the warp-specialised Mamba-2 kernel
+                          // 3: as 0 but without the warp-specialised kernels (single-group Mamba-2 kernel, CUDA cores for GDN)
     int decode_mma;       // warp-per-head decode: 1 = tensor-core dot products where supported
     int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
 };
@@ -94,6 +94,7 @@ int launch_decode_group_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream)
 int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);       // CUDA cores, every configuration
 int launch_update_tc(Ctx* ctx, const Params& p, cudaStream_t stream);    // tcgen05 tensor cores, Mamba-2; UNSUPPORTED_SHAPE outside its domain
 int launch_update_tc_ws(Ctx* ctx, const Params& p, cudaStream_t stream); // same, two warp groups per CTA (operand building overlaps the state stream)
+int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p, cudaStream_t stream); // gated delta rule, warp-specialised, two passes over the state
 int launch_update_tc_delta(Ctx* ctx, const Params& p, cudaStream_t stream);  // tcgen05 tensor cores, gated delta rule; same convention
 
 // ---------------------------------------------------------------------------------------------

@@ -1,0 +1,845 @@
+// Warp-specialised state-update (flush) kernel for the gated delta rule (GDN) on tcgen05 + TMEM, sm_100a.
+//
+// Replaying n tokens of S_s = a_s S_{s-1} + k_s e_s^T,  e_s = beta_s (v_s - (a_s S_{s-1})^T k_s)  (Eq. 1, 3), unrolled
+// over the window (the WY form of Appendix C, Eq. 41-42, applied to the state), is
+//     P     = K S_0                                  n x V     raw keys against the old state
+//     E'    = T1 (V - C P)                           n x V     T1 = Dn (I + Bd A)^{-1} Bd,  C = diag(prod_{i<=s} a_i),
+//                                                              A_sj = (prod_{j<i<=s} a_i) <k_j, k_s> (j < s),  Dn = diag(prod_{i>s} a_i)
+//     S_new = (prod_i a_i) S_0 + K^T E'              K x V
+//     [U | o] = S_new^T [Omega | q]                            (Eq. 7 and the exact output of the flush step)
+// Every product of decays is built by multiplication (no quotients), and all tensor-core operands that come from the
+// ring are the raw bf16 keys, so those products are exact; fp32 operands (S_0, S_new, E') are split into bf16 hi + lo.
+//
+// Tile = one head (K = V = 128); TMEM lane = value column j.  The state is streamed twice through a ring of
+// shared-memory stages filled by bulk copies (TMA): pass A contracts S_0 with the keys (P), pass B forms S_new from
+// S_0 (read again, from L2) and K^T E' and contracts it with [Omega | q].  The CTA is specialised like the Mamba-2
+// kernel: a front group builds the ring-only operands (Gram matrix, T1, key layouts) one tile ahead and stores the
+// sketch rows of the tile before; a stream group does the per-element work of both passes and the small E' step;
+// one thread issues every MMA; one warp keeps the stages full.  Passes of consecutive tiles are interleaved
+// (A(i+1) runs between E'(i) and B(i)), so no MMA round trip is waited for.
+//
+// Domain: GDN, bf16 I/O, K = V = 128, 1..16 tokens per flush, rank <= 16.
+#include "internal.cuh"
+#include "tc_common.cuh"
+
+namespace sketchssm {
+
+namespace {
+
+using namespace tc;
+
+// Optional phase stamps of the first CTA into the work buffer; compiled out by default.
+#ifdef SKETCHSSM_PHASE_TIMING
+#define G_STAMP(base, k, i)                                                                              \
+    do {                                                                                                 \
+        if ((tid & 127) == 0 && blockIdx.x == 0 && (k) >= 8 && (k) < 16)                                   \
+            reinterpret_cast<long long*>(p.work)[(base) + ((k) - 8) * 16 + (i)] = clock64();             \
+    } while (0)
+#else
+#define G_STAMP(base, k, i) do { } while (0)
+#endif
+
+constexpr int kGThreads = 320;       // stream group (4 warps), front group (4 warps), MMA issue warp, state-load warp
+constexpr int kGrp = 128;
+constexpr int kNTok = 16;            // tokens per flush
+constexpr int kGStages = 8;
+constexpr int kGS = 20;              // row stride (floats) of the small n x n work matrices
+constexpr int kA2 = 2;               // chunk buffers between the stream group and the MMA issue warp
+
+struct GSmem {
+    uint32_t a2, e, w, set, set_stride, set_bt, set_vv, set_t1, set_gates, stg, stg_v, stg_gate, stg_q, mats, bars, misc, sst,
+        sst_bytes, total;
+};
+
+__host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
+    GSmem s;
+    uint32_t off = 0;
+    s.a2 = off; off += (uint32_t)kA2 * 2u * 128u * 16u * 2u;      // 16-row chunk buffers, hi + lo
+    s.e = off; off += 2u * 128u * 16u * 2u;                       // E' hi + lo (same layout as a chunk buffer)
+    s.w = off; off += 2u * (uint32_t)NP * kK * 2u;                // [Omega | q | q'] hi | lo
+    // per-tile operand set, double-buffered: keys as B operand of pass A (K-major) and of K^T E' (MN-major),
+    // raw value rows, T1, gates (C diagonal, total decay)
+    s.set = off;
+    s.set_bt = 4096u; s.set_vv = 8192u; s.set_t1 = 12288u; s.set_gates = 13312u; s.set_stride = 13440u;
+    off += 2u * s.set_stride;
+    // staging of the next tile's raw rows: keys [16][256 B], values [16][256 B], gates [2L] floats, query row
+    s.stg_v = 4096u;
+    s.stg_gate = 8192u;
+    s.stg_q = s.stg_gate + (((uint32_t)(2 * L * 4) + 127u) & ~127u);
+    s.stg = off; off += s.stg_q + 256u;
+    s.mats = off; off += 4u * (uint32_t)kNTok * kGS * 4u + 256u;  // Gram / A, decay products, T, beta / alpha / dn
+    s.bars = off; off += 384u;
+    s.misc = off; off += 64u;
+    off = (off + 127u) & ~127u;
+    s.sst_bytes = 16u * 128u * 4u;
+    s.sst = off; off += (uint32_t)stages * s.sst_bytes;
+    s.total = off;
+    return s;
+}
+
+enum { gPro = 0, gPfull = 2, gTfull = 4, gUfull = 6, gBufFree = 8, gA2free = 10, gA2rdy = 10 + kA2, gErdy = 10 + 2 * kA2,
+       gStg = 11 + 2 * kA2, gProW = 12 + 2 * kA2, gFull = 14 + 2 * kA2, gEmpty = 14 + 2 * kA2 + kGStages,
+       gNumBars = 14 + 2 * kA2 + 2 * kGStages };
+
+__device__ __forceinline__ void g_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void g_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ bool g_or(int id, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %2, 0;\n\t"
+        "bar.red.or.pred p, %1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(flag ? 1u : 0u)
+        : "memory");
+    return r != 0;
+}
+// group-wide bounded wait: one warp polls, the others sleep in the named barrier
+__device__ __forceinline__ bool g_wait(int id, int gt, uint64_t* bar, uint32_t phase) {
+    bool bad = false;
+    if (gt < 32) bad = !mbar_wait_bounded(bar, phase);
+    return !g_or(id, bad);
+}
+
+__device__ __forceinline__ void g_ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void g_ldmatrix_x2(uint32_t addr, uint32_t (&r)[2]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void g_mma_16816(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Params p) {
+    constexpr int K = kK, V = 128, CH = 16, NCH = K / CH;
+    extern __shared__ __align__(1024) unsigned char smem[];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gt = tid & 127;
+    const int R = p.R, H = p.H, B = p.B;
+    const int QA = (R + 7) & ~7;                          // first column of query group A; group B follows 8 columns later
+    const int NP = (QA + 16 + 15) & ~15;                  // <= 32 (checked by the launcher)
+    const int NS = p.stages;
+    const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);     // 1..16 (checked by the launcher)
+    const GSmem sm = make_gsmem(NP, p.L, NS);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.misc);
+    unsigned char* sStg = smem + sm.stg;
+
+    constexpr uint32_t tmem_cols = 256u;
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
+        for (int i = 0; i < gNumBars; ++i) {
+            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty;     // one arrival per stream warp
+            mbar_init(&bars[i], per_warp ? 4 : 1);
+        }
+        mbar_fence_init();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    grid_dep_wait();                 // nothing above reads memory another kernel may write
+    grid_dep_launch_dependents();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+
+    // instruction descriptors: bf16 x bf16 -> fp32, M = 128
+    const uint32_t idescP = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);                 // K-major x K-major, N = 16
+    const uint32_t idescT = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);    // K-major x MN-major, N = 128
+    const uint32_t idescU = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)NP >> 3) << 17) | ((128u >> 4) << 24);        // K-major x K-major, N = NP
+    // canonical no-swizzle layouts (byte offsets)
+    //   K-major : elem(mn, k) at (mn%8)*16 + (mn/8)*128 + (k/8)*LBO + (k%8)*2,  LBO = 16*MN
+    //   MN-major: elem(mn, k) at (k%8)*16 + (mn%8)*2 + (mn/8)*128 + (k/8)*2048
+    constexpr uint32_t SBO = 128, LBO_M = 2048, LBO_BP = 256;
+    const uint32_t LBO_W = (uint32_t)NP * 16u;
+
+    const int tiles_per_h = B;
+
+    // the CTA's sequence of tile numbers (claimed at run time by the front group) travels through a small ring
+    volatile int* seq_ring = reinterpret_cast<volatile int*>(smem + sm.misc + 16);
+    volatile int* seq_pub = reinterpret_cast<volatile int*>(smem + sm.misc + 32);
+    auto seq_get = [&](int k) -> int {          // -2: the wait ran out
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+            if (*seq_pub > k) {
+                __threadfence_block();
+                return seq_ring[k & 3];
+            }
+            if (it > 32) __nanosleep(100);
+        }
+        return -2;
+    };
+    // A published tile number carries a flag when its head index differs from the tile before it: W is then rewritten
+    // between the two tiles, so their passes are not interleaved (pass B of the earlier tile runs first).
+    constexpr int kSepFlag = 1 << 30;
+    auto set_ptr = [&](int b) { return smem + sm.set + (uint32_t)b * sm.set_stride; };
+
+    const int j = gt;                 // value column of this thread's TMEM lane (stream and front groups)
+
+    if (warp < 4) {
+        // =========================== stream group ===========================
+        uint32_t phPro = 0, phProW = 0, phP = 0, phT = 0, phA = 0, phF = 0;
+        float dt0 = 1.f, dt1 = 1.f;          // total decay of the tile in each operand set, read when E' is formed
+        int gc = 0, stage = 0;
+        bool bad = false;
+
+        // one pass over the 8 chunks of a tile: pass A delivers S_0 chunks (hi + lo) for P = K S_0; pass B forms
+        // S_new = d S_0 + T, writes it back and delivers it for [U | o]
+        auto do_pass = [&](bool is_b, int tile, int b) {
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            float* So = p.state + bh * (size_t)K * V + j;
+            const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
+            const float dtot = is_b ? (b ? dt1 : dt0) : 1.f;
+            float t01[2 * CH];
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
+                const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
+                float s0[CH];
+#pragma unroll
+                for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
+                float t[CH];
+                if (is_b && !bad) {
+                    if (c == 0) tmem_ld32(tmem_t + lane_sel, t01);
+                    if (c < 2) {
+#pragma unroll
+                        for (int ii = 0; ii < CH; ++ii) t[ii] = t01[c * CH + ii];
+                    } else {
+                        tmem_ld16(tmem_t + lane_sel + (uint32_t)(c * CH), t);
+                    }
+                } else {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) g_arrive(&bars[gEmpty + stage]);
+                const int ab = c & (kA2 - 1);
+                if (gc >= kA2) {     // the chunk buffer was read by the MMAs issued kA2 chunks ago
+                    bad |= !mbar_wait_bounded(&bars[gA2free + ab], (phA >> ab) & 1u);
+                    phA ^= 1u << ab;
+                }
+                unsigned char* a2hi = smem + sm.a2 + (size_t)ab * (2u * 128u * CH * 2u);
+                unsigned char* a2lo = a2hi + 128u * CH * 2u;
+#pragma unroll
+                for (int v8 = 0; v8 < CH / 8; ++v8) {
+                    uint32_t ohi[4], olo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i0 = v8 * 8 + 2 * e;
+                        const float x0 = fmaf(dtot, s0[i0], t[i0]), x1 = fmaf(dtot, s0[i0 + 1], t[i0 + 1]);
+                        if (is_b && !bad) {
+                            So[(size_t)(c * CH + i0) * V] = x0;
+                            So[(size_t)(c * CH + i0 + 1) * V] = x1;
+                        }
+                        split_bf16x2(x0, x1, ohi[e], olo[e]);
+                    }
+                    const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO_M;
+                    *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                    *reinterpret_cast<uint4*>(a2lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+                }
+                proxy_fence();
+                tc_fence_before();
+                bad = __any_sync(0xffffffffu, bad);
+                if (lane == 0 && !bad) g_arrive(&bars[gA2rdy + ab]);
+                ++gc;
+                if (++stage == NS) { stage = 0; phF ^= 1u; }
+            }
+        };
+        // E'[s, j] = sum_t T1[s, t] (v_t[j] - C_t P[t, j]) -> hi + lo A operand of K^T E' (chunk-buffer layout)
+        auto do_e = [&](int b) {
+            bad |= !mbar_wait_bounded(&bars[gPfull + b], (phP >> b) & 1u);
+            phP ^= 1u << b;
+            tc_fence_after();
+            const unsigned char* set = set_ptr(b);
+            const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(set + sm.set_vv);
+            const float* sT1 = reinterpret_cast<const float*>(set + sm.set_t1);
+            const float* sC = reinterpret_cast<const float*>(set + sm.set_gates);
+            if (b) dt1 = sC[kNTok]; else dt0 = sC[kNTok];
+            float x[kNTok];
+            if (!bad) tmem_ld16(tmem_base + (uint32_t)b * 128u + lane_sel, x);
+#pragma unroll
+            for (int t = 0; t < kNTok; ++t) x[t] = fmaf(-sC[t], x[t], __bfloat162float(sV[t * V + j]));
+            float e[kNTok];
+#pragma unroll
+            for (int s = 0; s < kNTok; ++s) {
+                float acc = 0.f;
+#pragma unroll
+                for (int t4 = 0; t4 < kNTok / 4; ++t4) {
+                    const float4 tt = *reinterpret_cast<const float4*>(sT1 + s * kNTok + t4 * 4);
+                    acc = fmaf(tt.x, x[t4 * 4], acc);
+                    acc = fmaf(tt.y, x[t4 * 4 + 1], acc);
+                    acc = fmaf(tt.z, x[t4 * 4 + 2], acc);
+                    acc = fmaf(tt.w, x[t4 * 4 + 3], acc);
+                }
+                e[s] = acc;
+            }
+            unsigned char* ehi = smem + sm.e;
+            unsigned char* elo = ehi + 128u * CH * 2u;
+#pragma unroll
+            for (int v8 = 0; v8 < 2; ++v8) {
+                uint32_t ohi[4], olo[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) split_bf16x2(e[v8 * 8 + 2 * q], e[v8 * 8 + 2 * q + 1], ohi[q], olo[q]);
+                const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO_M;
+                *reinterpret_cast<uint4*>(ehi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                *reinterpret_cast<uint4*>(elo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+            }
+            proxy_fence();
+            tc_fence_before();
+            bad = __any_sync(0xffffffffu, bad);
+            if (lane == 0 && !bad) g_arrive(&bars[gErdy]);
+        };
+        auto wait_pro = [&](int b) {
+            bad |= !mbar_wait_bounded(&bars[gPro + b], (phPro >> b) & 1u);
+            phPro ^= 1u << b;
+        };
+
+        int cur = seq_get(0);
+        if (cur >= 0) {
+            cur &= kSepFlag - 1;
+            wait_pro(0);
+            do_pass(false, cur, 0);
+            do_e(0);
+            for (int k = 0; !bad; ++k) {
+                const int b = k & 1;
+                const int raw = seq_get(k + 1);
+                if (raw < -1) { bad = true; break; }
+                const int nxt = raw < 0 ? -1 : (raw & (kSepFlag - 1));
+                const bool sep = raw >= 0 && (raw & kSepFlag) != 0;
+                G_STAMP(0, k, 0);
+                if (nxt >= 0 && !sep) {
+                    wait_pro(b ^ 1);
+                    G_STAMP(0, k, 1);
+                    do_pass(false, nxt, b ^ 1);
+                }
+                G_STAMP(0, k, 2);
+                bad |= !mbar_wait_bounded(&bars[gProW + b], (phProW >> b) & 1u);     // this tile's query column (and Omega) are in W
+                phProW ^= 1u << b;
+                bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);
+                phT ^= 1u << b;
+                tc_fence_after();
+                G_STAMP(0, k, 3);
+                do_pass(true, cur, b);
+                G_STAMP(0, k, 4);
+                if (nxt < 0) break;
+                if (sep) {
+                    wait_pro(b ^ 1);
+                    do_pass(false, nxt, b ^ 1);
+                }
+                do_e(b ^ 1);
+                G_STAMP(0, k, 5);
+                cur = nxt;
+            }
+        } else if (cur < -1) {
+            bad = true;
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 3);
+    } else if (warp == 8) {
+        // =========================== MMA issue warp (one thread) ===========================
+        if (lane == 0) {
+            uint32_t phR = 0, phE = 0, phBuf = 0;
+            bool bad = false;
+            const uint32_t sW = smem_u32(smem + sm.w);
+            const uint32_t a2base = smem_u32(smem + sm.a2);
+            auto pass_a = [&](int k) {          // P(b) = K S_0, chunk by chunk
+                const int b = k & 1;
+                if (k >= 2) {                   // the accumulator half still holds the sketch rows of tile k - 2 until they are stored
+                    if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; return; }
+                    phBuf ^= 1u << b;
+                    tc_fence_after();
+                }
+                const uint32_t tmem_p = tmem_base + (uint32_t)b * 128u;
+                const uint32_t bp = smem_u32(set_ptr(b));
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const int ab = c & (kA2 - 1);
+                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; return; }
+                    phR ^= 1u << ab;
+                    tc_fence_after();
+                    const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
+                    const uint64_t ahi = make_desc(a2, LBO_M, SBO);
+                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
+                    const uint64_t bk = make_desc(bp + (uint32_t)(c * 2) * LBO_BP, LBO_BP, SBO);
+                    tc_mma_bf16(tmem_p, ahi, bk, idescP, c ? 1u : 0u);
+                    tc_mma_bf16(tmem_p, alo, bk, idescP, 1u);
+                    tc_commit(&bars[gA2free + ab]);
+                    if (c == NCH - 1) tc_commit(&bars[gPfull + b]);
+                }
+            };
+            auto step_e = [&](int k) {          // T(b) = E'^T-contraction with the keys: T[j, i] = sum_s E'[s, j] k_s[i]
+                const int b = k & 1;
+                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; return; }
+                phE ^= 1u;
+                tc_fence_after();
+                const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
+                const uint32_t e = smem_u32(smem + sm.e);
+                const uint64_t bt = make_desc(smem_u32(set_ptr(b) + sm.set_bt), LBO_M, SBO);
+                tc_mma_bf16(tmem_t, make_desc(e, LBO_M, SBO), bt, idescT, 0u);
+                tc_mma_bf16(tmem_t, make_desc(e + 128u * CH * 2u, LBO_M, SBO), bt, idescT, 1u);
+                tc_commit(&bars[gTfull + b]);
+            };
+            auto pass_b = [&](int k) {          // [U | o](b) = S_new^T [Omega | q]
+                const int b = k & 1;
+                const uint32_t tmem_u = tmem_base + (uint32_t)b * 128u;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const int ab = c & (kA2 - 1);
+                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; return; }
+                    phR ^= 1u << ab;
+                    tc_fence_after();
+                    const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
+                    const uint32_t kb = (uint32_t)(c * (CH / 8)) * LBO_W;
+                    const uint64_t ahi = make_desc(a2, LBO_M, SBO);
+                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
+                    const uint64_t bhi = make_desc(sW + kb, LBO_W, SBO);
+                    const uint64_t blo = make_desc(sW + (uint32_t)NP * kK * 2u + kb, LBO_W, SBO);
+                    tc_mma_bf16(tmem_u, ahi, bhi, idescU, c ? 1u : 0u);
+                    tc_mma_bf16(tmem_u, alo, bhi, idescU, 1u);
+                    tc_mma_bf16(tmem_u, ahi, blo, idescU, 1u);
+                    tc_commit(&bars[gA2free + ab]);
+                    if (c == NCH - 1) tc_commit(&bars[gUfull + b]);
+                }
+            };
+            int cur = seq_get(0);
+            if (cur >= 0) {
+                pass_a(0);
+                if (!bad) step_e(0);
+                for (int k = 0; !bad; ++k) {
+                    const int raw = seq_get(k + 1);
+                    if (raw < -1) { bad = true; break; }
+                    const bool sep = raw >= 0 && (raw & kSepFlag) != 0;
+                    if (raw >= 0 && !sep) pass_a(k + 1);
+                    if (bad) break;
+                    pass_b(k);
+                    if (raw < 0 || bad) break;
+                    if (sep) pass_a(k + 1);
+                    if (bad) break;
+                    step_e(k + 1);
+                }
+            } else if (cur < -1) {
+                bad = true;
+            }
+            if (bad) record_fault(p.status, kFaultUpdateWait, 4);
+        }
+    } else if (warp == 9) {
+        // =========================== state-load warp: keeps the ring of S_0 stages full ===========================
+        int stage = 0, round = 0;
+        bool bad = false;
+        auto load_tile = [&](int tile) {
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const float* src = p.state + ((size_t)bb * H + h) * (size_t)K * V;
+            for (int c = 0; c < NCH; ++c) {
+                if (round > 0) {     // the stage was released by all four stream warps
+                    if (!mbar_wait_bounded(&bars[gEmpty + stage], (uint32_t)(round - 1) & 1u)) { bad = true; return; }
+                }
+                uint64_t* bar = &bars[gFull + stage];
+                if (lane == 0) {
+                    mbar_expect_tx(bar, sm.sst_bytes);
+                    bulk_g2s(smem + sm.sst + (size_t)stage * sm.sst_bytes, src + (size_t)c * CH * V, (uint32_t)(CH * V * 4), bar);
+                }
+                if (++stage == NS) { stage = 0; ++round; }
+            }
+        };
+        int cur = seq_get(0);
+        if (cur >= 0) {
+            cur &= kSepFlag - 1;
+            load_tile(cur);                       // pass A of the first tile
+            for (int k = 0; !bad; ++k) {
+                const int raw = seq_get(k + 1);
+                if (raw < -1) { bad = true; break; }
+                const int nxt = raw < 0 ? -1 : (raw & (kSepFlag - 1));
+                const bool sep = raw >= 0 && (raw & kSepFlag) != 0;
+                if (nxt >= 0 && !sep) load_tile(nxt);     // pass A of the next tile
+                if (bad) break;
+                load_tile(cur);                   // pass B of this tile (its state is read again, from L2)
+                if (nxt < 0) break;
+                if (sep) load_tile(nxt);
+                cur = nxt;
+            }
+        } else if (cur < -1) {
+            bad = true;
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 7);
+    } else {
+        // =========================== front group: ring-only operands, sketch stores ===========================
+        const int fwarp = gt >> 5;
+        int cur_h = -1;
+        int pend0 = -1, pend1 = -1;           // tiles whose sketch rows are still to be stored: older, newer
+        uint32_t phS = 0, phU = 0, phTf = 0;
+        bool dead = false;
+        float* sGm = reinterpret_cast<float*>(smem + sm.mats);
+        float* sPm = sGm + kNTok * kGS;
+        float* sTm = sPm + kNTok * kGS;
+        float* sBeta = sTm + kNTok * kGS;
+        float* sAlpha = sBeta + kNTok;
+        float* sDn = sAlpha + kNTok;
+        float* sCum = sDn + kNTok;
+        __nv_bfloat16* sWhi = reinterpret_cast<__nv_bfloat16*>(smem + sm.w);
+        __nv_bfloat16* sWlo = sWhi + (size_t)NP * kK;
+
+        // ---- tile claiming (thread 0 of the group): per-head-index counters behind the status words ----
+        int* sched = p.status + kStatusInts;
+        int* cnt = sched + 4;
+        int h_claim = (int)(((long long)blockIdx.x * H) / gridDim.x);
+        int t_raw = 0;
+        auto claim_issue = [&]() { t_raw = atomicAdd(&cnt[h_claim], 1); };
+        auto claim_resolve = [&]() -> int {
+            for (int attempt = 0; attempt <= H; ++attempt) {
+                if (t_raw < tiles_per_h) return h_claim * tiles_per_h + t_raw;
+                int best = -1, best_c = tiles_per_h;
+                for (int i = 1; i <= H; ++i) {
+                    int hh = h_claim + i;
+                    if (hh >= H) hh -= H;
+                    const int c = *reinterpret_cast<volatile int*>(&cnt[hh]);
+                    if (c < best_c) { best_c = c; best = hh; }
+                }
+                if (best < 0) return -1;
+                h_claim = best;
+                t_raw = atomicAdd(&cnt[h_claim], 1);
+            }
+            return -1;
+        };
+        auto publish = [&](int k, int tile) {
+            seq_ring[k & 3] = tile;
+            __threadfence_block();
+            *seq_pub = k + 1;
+        };
+
+        const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
+        const uint32_t stg_bytes = (uint32_t)n_ring * 512u + stg_gate_bytes + (p.has_token ? 512u : 0u) + (p.q != nullptr ? 256u : 0u);
+        auto stage_tile = [&](int tile) {       // one thread
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bw = (size_t)bb * H + h;
+            const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
+            mbar_expect_tx(&bars[gStg], stg_bytes);
+            if (n_ring > 0) {
+                bulk_g2s(sStg, rh, (uint32_t)n_ring * 256u, &bars[gStg]);
+                bulk_g2s(sStg + sm.stg_v, rh + p.rl.v_off, (uint32_t)n_ring * 256u, &bars[gStg]);
+                bulk_g2s(sStg + sm.stg_gate, rh + p.rl.beta_off, stg_gate_bytes, &bars[gStg]);
+            }
+            if (p.has_token) {
+                bulk_g2s(sStg + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.k) + bw * K, 256u, &bars[gStg]);
+                bulk_g2s(sStg + sm.stg_v + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.v) + bw * V, 256u, &bars[gStg]);
+            }
+            if (p.q != nullptr) bulk_g2s(sStg + sm.stg_q, reinterpret_cast<const __nv_bfloat16*>(p.q) + bw * K, 256u, &bars[gStg]);
+        };
+        // sketch rows and exact output of a finished tile; afterwards its accumulator half is free for the issue warp
+        auto store_ut = [&](int tile, int b) -> bool {
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            if (!g_wait(2, gt, &bars[gUfull + b], (phU >> b) & 1u)) return false;
+            phU ^= 1u << b;
+            tc_fence_after();
+            for (int g0 = 0; g0 < NP; g0 += 16) {
+                float u[16];
+                tmem_ld16(tmem_base + (uint32_t)b * 128u + lane_sel + (uint32_t)g0, u);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const int g = g0 + e;
+                    if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u[e];
+                    if (g == QA + 8 * b && p.out != nullptr) {
+                        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u[e]);
+                        else reinterpret_cast<float*>(p.out)[bh * V + j] = u[e];
+                    }
+                }
+            }
+            tc_fence_before();
+            g_sync(2);
+            if (gt == 0) g_arrive(&bars[gBufFree + b]);
+            return true;
+        };
+
+        if (gt == 0) {
+            claim_issue();
+            const int first = claim_resolve();
+            publish(0, first);
+            if (first >= 0) {
+                claim_issue();
+                stage_tile(first);
+            }
+        }
+        // W padding columns and lo halves of the query columns hold zeros that no tile overwrites: written once
+        for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGrp * 16u)
+            *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
+        g_sync(2);
+
+        for (int k = 0; !dead; ++k) {
+            const int raw_tile = seq_get(k);
+            if (raw_tile < 0) {
+                if (raw_tile < -1) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 8);
+                    dead = true;
+                }
+                break;
+            }
+            const int tile = raw_tile & (kSepFlag - 1);
+            const int b = k & 1;
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            unsigned char* set = set_ptr(b);
+
+            G_STAMP(256, k, 0);
+            // gates of the current token: requested early
+            float tok_beta = 0.f, tok_a = 1.f;
+            if (gt < kNTok && p.has_token) {
+                tok_beta = p.beta[bh];
+                tok_a = reinterpret_cast<const float*>(p.decay)[bh];
+            }
+            // the operand set of tile k - 2 is free once its K^T E' has completed (E' was formed before it was issued)
+            if (k >= 2) {
+                if (!g_wait(2, gt, &bars[gTfull + b], (phTf >> b) & 1u)) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 9);
+                    dead = true;
+                    break;
+                }
+                phTf ^= 1u << b;
+            }
+            // the staged rows, gates and query row of this tile must have landed
+            if (!g_wait(2, gt, &bars[gStg], phS)) {
+                if (gt == 0) record_fault(p.status, kFaultUpdateWait, 6);
+                dead = true;
+                break;
+            }
+            phS ^= 1;
+            G_STAMP(256, k, 1);
+
+            // ---- key layouts, value rows, query column, gates ----
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int idx = gt + r * kGrp;
+                const int t8 = idx & 7, a = (idx >> 3) & 15, s = (idx >> 7) * 8 + t8;
+                uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+                if (s < n_tot) {
+                    kv = *reinterpret_cast<const uint4*>(sStg + (size_t)s * 256 + a * 16);
+                    vv = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)s * 256 + a * 16);
+                }
+                *reinterpret_cast<uint4*>(set + (s & 7) * 16 + (s >> 3) * SBO + a * LBO_BP) = kv;                 // K-major: (n = s, k = i)
+                *reinterpret_cast<uint4*>(set + sm.set_bt + (s & 7) * 16 + a * SBO + (s >> 3) * LBO_M) = kv;      // MN-major: (mn = i, k = s)
+                *reinterpret_cast<uint4*>(set + sm.set_vv + (size_t)s * 256 + a * 16) = vv;
+            }
+            __nv_bfloat16 q_elem = __float2bfloat16_rn(0.f);         // written into W after the tile two before is done with it
+            if (p.q != nullptr) q_elem = reinterpret_cast<const __nv_bfloat16*>(sStg + sm.stg_q)[gt];
+            if (gt < kNTok) {
+                const int s = gt;
+                const float* sg = reinterpret_cast<const float*>(sStg + sm.stg_gate);
+                float bt = 0.f, al = 1.f;
+                if (s < n_ring) { bt = sg[s]; al = sg[p.L + s]; }
+                else if (s < n_tot) { bt = tok_beta; al = tok_a; }
+                sBeta[s] = bt;
+                sAlpha[s] = al;
+            }
+            for (int idx = gt; idx < kNTok * kGS; idx += kGrp) sTm[idx] = 0.f;
+            g_sync(2);
+
+            // ---- products of decays (no quotients) and the Gram matrix <k_s, k_j> ----
+            if (gt < kNTok) {
+                const int s = gt;
+                float pr = 1.f;                                   // Pm(j, s) = prod_{j < i <= s} alpha_i, for j = s-1 .. 0
+                for (int jj = s - 1; jj >= 0; --jj) {
+                    pr *= sAlpha[jj + 1];
+                    sPm[s * kGS + jj] = pr;
+                }
+                sCum[s] = s < n_tot ? pr * sAlpha[0] : 0.f;       // prod_{i <= s} alpha_i
+                float dn = 1.f;
+                for (int i = s + 1; i < n_tot; ++i) dn *= sAlpha[i];
+                sDn[s] = s < n_tot ? dn : 0.f;
+            }
+            if (fwarp >= 2) {     // 16 x 16 Gram matrix from the staged keys, one 16 x 8 block per warp
+                const int nt = fwarp - 2;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * 256u + (uint32_t)(lane >> 4) * 16u;
+                const uint32_t bbase = smem_u32(sStg) + (uint32_t)(nt * 8 + (lane & 7)) * 256u + (uint32_t)((lane >> 3) & 1) * 16u;
+#pragma unroll
+                for (int ks = 0; ks < K / 16; ++ks) {
+                    uint32_t a[4], bbv[2];
+                    g_ldmatrix_x4(abase + ks * 32, a);
+                    g_ldmatrix_x2(bbase + ks * 32, bbv);
+                    g_mma_16816(acc, a, bbv);
+                }
+                const int r0 = lane >> 2, c0 = nt * 8 + (lane & 3) * 2;
+                sGm[r0 * kGS + c0] = acc[0];
+                sGm[r0 * kGS + c0 + 1] = acc[1];
+                sGm[(r0 + 8) * kGS + c0] = acc[2];
+                sGm[(r0 + 8) * kGS + c0 + 1] = acc[3];
+            }
+            g_sync(2);
+            G_STAMP(256, k, 2);
+            // beta_s A_sj in place of the Gram entries (strictly lower triangle)
+            if (gt < n_tot) {
+                const int s = gt;
+                const float bs = sBeta[s];
+                for (int jj = 0; jj < s; ++jj) sGm[s * kGS + jj] *= bs * sPm[s * kGS + jj];
+            }
+            g_sync(2);
+            G_STAMP(256, k, 3);
+            // ---- T = (I + Bd A)^{-1} Bd by forward substitution: one column per thread, held in registers ----
+            if (gt < kNTok) {
+                const int c = gt;
+                float tcol[kNTok];
+#pragma unroll
+                for (int s = 0; s < kNTok; ++s) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int j4 = 0; j4 < (s + 3) / 4; ++j4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(sGm + s * kGS + j4 * 4);
+                        if (j4 * 4 + 0 < s) acc = fmaf(l4.x, tcol[j4 * 4 + 0], acc);
+                        if (j4 * 4 + 1 < s) acc = fmaf(l4.y, tcol[j4 * 4 + 1], acc);
+                        if (j4 * 4 + 2 < s) acc = fmaf(l4.z, tcol[j4 * 4 + 2], acc);
+                        if (j4 * 4 + 3 < s) acc = fmaf(l4.w, tcol[j4 * 4 + 3], acc);
+                    }
+                    tcol[s] = (s >= n_tot || s < c || c >= n_tot) ? 0.f : (s == c ? 1.f : -acc);
+                }
+                const float bc = sBeta[c];
+#pragma unroll
+                for (int s = 0; s < kNTok; ++s) sTm[s * kGS + c] = tcol[s] * bc;
+            }
+            g_sync(2);
+            G_STAMP(256, k, 4);
+            // ---- T1 = Dn T (rows and columns beyond the tokens are zero), C diagonal, total decay ----
+            {
+                float* sT1 = reinterpret_cast<float*>(set + sm.set_t1);
+                float* sC = reinterpret_cast<float*>(set + sm.set_gates);
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int idx = gt + r * kGrp;
+                    const int s = idx >> 4, t = idx & 15;
+                    sT1[idx] = sDn[s] * sTm[s * kGS + t];
+                }
+                if (gt < kNTok) sC[gt] = sCum[gt];
+                if (gt == 0) sC[kNTok] = sCum[n_tot - 1];
+            }
+            proxy_fence();         // key layouts and W are read by MMAs (async proxy)
+            g_sync(2);
+            if (gt == 0) {
+                g_arrive(&bars[gPro + b]);
+                // the staging buffer has been read: claim / publish the next tile and let its rows come in
+                const int nxt = claim_resolve();
+                publish(k + 1, nxt);
+                if (nxt >= 0) {
+                    claim_issue();
+                    stage_tile(nxt);
+                }
+            }
+            G_STAMP(256, k, 5);
+
+            // ---- sketch rows and exact output of earlier tiles.  Tile k - 2 used the same query group and accumulator
+            // half as this tile; on a change of head index W is rewritten, so tile k - 1 is finished as well. ----
+            if (pend0 >= 0) {
+                if (!store_ut(pend0, b)) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+                    dead = true;
+                    break;
+                }
+                pend0 = -1;
+            }
+            if (h != cur_h) {
+                if (pend1 >= 0) {
+                    if (!store_ut(pend1, b ^ 1)) {
+                        if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+                        dead = true;
+                        break;
+                    }
+                    pend1 = -1;
+                }
+                if (p.write_sketch) {
+                    const float* og = p.omega + (size_t)h * K * R;
+                    for (int idx = gt; idx < K * R; idx += kGrp) {
+                        const int i = idx / R, g = idx - i * R;
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(og[idx], hi, lo);
+                        const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
+                        sWhi[o2] = hi;
+                        sWlo[o2] = lo;
+                    }
+                }
+                cur_h = h;
+            }
+            if (p.q != nullptr) {
+                const int i = gt, g = QA + 8 * b;
+                const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
+                sWhi[o2] = q_elem;
+            }
+            proxy_fence();
+            g_sync(2);
+            if (gt == 0) g_arrive(&bars[gProW + b]);
+            pend0 = pend1;
+            pend1 = tile;
+            G_STAMP(256, k, 6);
+        }
+        if (!dead) {      // the last one or two tiles; the newer one used buffer (tiles - 1) & 1
+            const int done = *seq_pub - 1;                    // number of tiles this CTA processed
+            if (pend0 >= 0 && !store_ut(pend0, done & 1)) { if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
+            if (!dead && pend1 >= 0 && !store_ut(pend1, (done - 1) & 1) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+        }
+        if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
+            __threadfence();
+            if (atomicAdd(&sched[0], 1) == (int)gridDim.x - 1) {
+                for (int hh = 0; hh < H; ++hh) cnt[hh] = 0;
+                sched[0] = 0;
+                __threadfence();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// Returns SKETCHSSM_UNSUPPORTED_SHAPE outside this kernel's domain (the caller then uses another kernel).
+int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+    const sketchssm_config& c = ctx->cfg;
+    if (c.kind != SKETCHSSM_GDN || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK || c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (c.rank > 16) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    Params p = p_in;
+    const int n_tot = p.n_before + (p.has_token ? 1 : 0);
+    if (n_tot < 1 || n_tot > kNTok) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int NP = ((((c.rank + 7) & ~7) + 16) + 15) & ~15;
+    if (ctx->sm_count == 0) {
+        int dev = 0, sms = 0;
+        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return SKETCHSSM_CUDA_ERROR;
+        ctx->sm_count = sms;
+    }
+    int ctas = 2;                                             // tensor memory: 256 of the SM's 512 columns per CTA
+    if (p.max_warps_per_sm > 0 && p.max_warps_per_sm < 20) ctas = 1;
+    const uint32_t budget = (228u * 1024u) / (uint32_t)ctas - 1024u;
+    const GSmem fixed = make_gsmem(NP, c.buf_len, 0);
+    if (fixed.total + 2u * fixed.sst_bytes > budget) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    int stages = (int)((budget - fixed.total) / fixed.sst_bytes);
+    if (stages > kGStages) stages = kGStages;
+    if (p.stages >= 2 && p.stages < stages) stages = p.stages;
+    p.stages = stages;
+    const GSmem sm = make_gsmem(NP, c.buf_len, stages);
+    const long long n_tiles = (long long)c.batch * c.heads;
+    long long grid = (long long)ctx->sm_count * ctas;
+    if (grid > n_tiles) grid = n_tiles;
+    auto kern = update_tc_ws_gdn_kernel;
+    if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)sm.total)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    if ((ctx->last_cuda_error = launch_kernel(kern, dim3((unsigned)grid), dim3(kGThreads), sm.total, stream, p, p.pdl != 0)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    ctx->last_launches = 1;
+    return SKETCHSSM_OK;
+}
+
+}  // namespace sketchssm

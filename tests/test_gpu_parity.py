@@ -168,6 +168,15 @@ def test_gdn_tensor_core_update(rank, buf_len, steps):
     check(run_schedule(w, steps, max_heads=10**9, tune={"update_impl": 2}), "bf16")
 
 
+@pytest.mark.parametrize("tune", [{}, {"decode_max_warps_per_sm": 10}, {"pdl": 0}])
+@pytest.mark.parametrize("batch,heads,rank,buf_len", [(5, 3, 16, 16), (40, 20, 16, 16), (33, 7, 8, 12), (6, 2, 5, 4)])
+def test_gdn_warp_specialised_update(tune, batch, heads, rank, buf_len):
+    """Warp-specialised tcgen05 flush of the gated delta rule (two passes over the state, interleaved across tiles,
+    tiles claimed at run time) against the oracle's token-by-token replay, over two windows."""
+    w = synth.Workload("t", "gdn", batch, heads, 128, 128, rank, buf_len, 0, "bf16", 93, basis="qr")
+    check(run_schedule(w, 2 * buf_len + 3, max_heads=96, tune=tune), "bf16")
+
+
 def test_bf16_output_mode():
     w = synth.Workload("t", "gdn", 4, 2, 128, 128, 16, 8, 0, "bf16", 5, basis="qr")
     errs = run_schedule(w, 12, max_heads=10**9, out="bf16")
