@@ -18,8 +18,9 @@
 // Everything that used to sit serially between two tiles' state streams (operand building, MMA-1 latency, sketch
 // stores) now overlaps them.  The groups meet only through mbarriers; every wait is bounded.
 //
-// Domain: Mamba-2, bf16 I/O, K = 128, V in {64, 128}, rank <= 16 (the sketch accumulator [Omega | q | q'] then
-// re-uses the first 32 consumed columns of T, which keeps a CTA at 256 TMEM columns and two CTAs per SM).
+// Domain: Mamba-2, bf16 I/O, K = 128, V in {64, 128}, rank <= 32 (the sketch accumulator [Omega | q | q'] re-uses
+// the first 32 or 48 columns of T, read ahead by the stream group, which keeps a CTA at 256 TMEM columns and two
+// CTAs per SM).
 // W = [Omega | q-group A | q-group B]: consecutive tiles alternate between the two query groups, so the front group
 // can write the next tile's query columns while MMA 2 of the current tile still reads the buffer (it then also reads
 // half-written columns of the other group, whose outputs nobody uses).
@@ -37,8 +38,8 @@ using namespace tc;
 #ifdef SKETCHSSM_PHASE_TIMING
 #define WS_STAMP(base, i)                                                                                      \
     do {                                                                                                       \
-        if (gt == 0 && blockIdx.x == 0 && k >= 0 && k < 8)                                                    \
-            reinterpret_cast<long long*>(p.work)[(base) + (k - 0) * 32  + (i)] = clock64();                    \
+        if (gt == 0 && blockIdx.x == 0 && k >= 8 && k < 16)                                                   \
+            reinterpret_cast<long long*>(p.work)[(base) + (k - 8) * 32  + (i)] = clock64();                    \
     } while (0)
 #else
 #define WS_STAMP(base, i) do { } while (0)
@@ -48,13 +49,13 @@ constexpr int kWsThreads = 320;       // stream group (4 warps), front group (4 
 constexpr int kGroup = 128;
 
 struct WsSmem {
-    uint32_t op, a2, b2, w, w_stride, stg, stg_head, stg_gate, stg_q, bars, misc, sst, sst_bytes, total;
+    uint32_t op, a2, b2, w, w_stride, stg, stg_tile_head, stg_q, stg_blk, stg_blk_head, stg_blk_stride, bars, misc, sst, sst_bytes, total;
 };
 
 constexpr int kMaxStages = 8;
 
 // operand set: a1_hi | a1_lo | b1, each 128 x KD1 bf16
-__host__ __device__ inline WsSmem make_ws_smem(int NH, int NP, int V, int L, int stages) {
+__host__ __device__ inline WsSmem make_ws_smem(int NH, int NP, int V, int L, int stages, int stg_bufs) {
     WsSmem s;
     const uint32_t kd1 = (uint32_t)(kTokBlock * NH);
     uint32_t off = 0;
@@ -62,11 +63,14 @@ __host__ __device__ inline WsSmem make_ws_smem(int NH, int NP, int V, int L, int
     s.a2 = off; off += 2u * 2u * 128u * 16u * 2u;              // two 16-row chunk buffers, hi + lo
     s.b2 = off; off += 2u * (uint32_t)NP * kK * 2u;             // hi | lo
     s.w = off; s.w_stride = 2u * 208u * 4u; off += 2u * s.w_stride;     // per head: w_s (64), total decay; double-buffered
-    // staging of the next tile's raw rows: per head keys [16][256 B], values [16][V*2 B], gates [2L] floats, query row
-    s.stg_gate = 4096u + 16u * (uint32_t)V * 2u;
-    s.stg_q = s.stg_gate + (((uint32_t)(2 * L * 4) + 127u) & ~127u);
-    s.stg_head = s.stg_q + 256u;
-    s.stg = off; off += (uint32_t)NH * s.stg_head;
+    // staging of raw ring rows, filled by bulk copies ahead of use: per head and tile the gates [2L] floats and the query
+    // row; per head and block of 16 tokens the keys [16][256 B] and values [16][V*2 B], in one or two block buffers
+    s.stg_q = ((uint32_t)(2 * L * 4) + 127u) & ~127u;
+    s.stg_tile_head = s.stg_q + 256u;
+    s.stg = off; off += (uint32_t)NH * s.stg_tile_head;
+    s.stg_blk_head = 4096u + 16u * (uint32_t)V * 2u;
+    s.stg_blk_stride = (uint32_t)NH * s.stg_blk_head;
+    s.stg_blk = off; off += (uint32_t)stg_bufs * s.stg_blk_stride;
     s.bars = off; off += 256u;
     s.misc = off; off += 64u;
     off = (off + 127u) & ~127u;
@@ -77,8 +81,8 @@ __host__ __device__ inline WsSmem make_ws_smem(int NH, int NP, int V, int L, int
 }
 
 // barrier slots
-enum { kBarT = 0, kBarPro = 2, kBarA2 = 4, kBarU = 6, kBarStg = 8, kBarBlk = 9, kBarA2Rdy = 10, kBarFull = 12,
-       kBarEmpty = 12 + kMaxStages, kNumBars = 12 + 2 * kMaxStages };
+enum { kBarT = 0, kBarPro = 2, kBarA2 = 4, kBarU = 6, kBarStg = 8, kBarBlk = 10, kBarA2Rdy = 11, kBarFull = 13,
+       kBarEmpty = 13 + kMaxStages, kNumBars = 13 + 2 * kMaxStages };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -111,7 +115,8 @@ __device__ __forceinline__ bool group_wait(int id, int gt, uint64_t* bar, uint32
 
 }  // namespace
 
-template <int V>
+// WIDE: the sketch accumulator [Omega | q | q'] takes 48 columns (rank 17..32) instead of 32.
+template <int V, bool WIDE>
 __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(const Params p) {
     constexpr int K = kK;
     constexpr int NH = 128 / V;
@@ -132,10 +137,11 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 #endif
     const int R = p.R, H = p.H, B = p.B;
     const int QA = (R + 7) & ~7;                          // first column of query group A; group B follows 8 columns later
-    const int NP = (QA + 16 + 15) & ~15;                  // <= 32 (checked by the launcher)
+    const int NP = (QA + 16 + 15) & ~15;                  // 32, or 48 in the WIDE instantiation (chosen by the launcher)
     const int NS = p.stages;                              // state stages in shared memory (set by the launcher)
     const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);
-    const WsSmem sm = make_ws_smem(NH, NP, V, p.L, NS);
+    const int stg_bufs = n_tot > kTokBlock ? 2 : 1;      // staging block buffers (the launcher sizes shared memory the same way)
+    const WsSmem sm = make_ws_smem(NH, NP, V, p.L, NS, stg_bufs);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.misc);
     unsigned char* sStg = smem + sm.stg;
@@ -225,7 +231,10 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             tc_fence_after();
             WS_STAMP(0, 1);
             const float dtot = n_tot > 0 ? reinterpret_cast<const float*>(smem + sm.w + (uint32_t)b * sm.w_stride)[my_head * 208 + 64] : 1.f;
-            float t01[2 * CH];      // T columns of chunks 0 and 1: read before the first MMA 2 overwrites them with UT
+            // T columns that UT will occupy (chunks 0 and 1, and chunk 2 when UT is 48 wide) are read before the first
+            // MMA 2 overwrites them
+            float t01[2 * CH];
+            float t2[WIDE ? CH : 1];
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 if (c == 4) WS_STAMP(0, 12);
@@ -238,10 +247,16 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
                 float t[CH];
                 if (n_blocks > 0 && !bad) {
-                    if (c == 0) tmem_ld32(tmem_t + lane_sel, t01);
+                    if (c == 0) {
+                        tmem_ld32(tmem_t + lane_sel, t01);
+                        if constexpr (WIDE) tmem_ld16(tmem_t + lane_sel + 32u, t2);
+                    }
                     if (c < 2) {
 #pragma unroll
                         for (int ii = 0; ii < CH; ++ii) t[ii] = t01[c * CH + ii];
+                    } else if (WIDE && c == 2) {
+#pragma unroll
+                        for (int ii = 0; ii < CH; ++ii) t[ii] = t2[WIDE ? ii : 0];
                     } else {
                         tmem_ld16(tmem_t + lane_sel + (uint32_t)(c * CH), t);
                     }
@@ -358,7 +373,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
         int cur_h = -1;                       // head index whose Omega sits in W
         int ops_built = 0;                    // MMA-1 operand sets written so far (single buffer)
         int prev_tile = -1, last_b = 0;       // the tile whose sketch rows are still to be stored (-1: none) and its buffer
-        uint32_t phS = 0, phU = 0, phB = 0;
+        uint32_t phU = 0, phB = 0;
         bool dead = false;
 
         // ---- tile claiming (thread 0 of the group) ----
@@ -393,33 +408,80 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             *seq_pub = k + 1;
         };
 
-        // Raw ring rows of a tile's first token block travel to shared memory by bulk copies issued one tile ahead.
-        // Rows of later blocks (n > 16) are read directly.
-        const int rows0 = n_ring < kTokBlock ? n_ring : kTokBlock;
-        const bool tok0 = p.has_token && n_ring < kTokBlock;
+        // Raw ring rows travel to shared memory block by block (16 tokens per head) by bulk copies that run ahead of
+        // their use: with one block per tile the next tile's block is requested while this tile's operands are built,
+        // with several blocks per tile two block buffers alternate.  A tile's gates and query rows come with its first block.
+        const int n_stage_blocks = n_blocks > 0 ? n_blocks : 1;       // a tile without tokens still stages its query rows
         const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
-        const uint32_t stg_bytes = (uint32_t)NH * ((uint32_t)rows0 * 256u + (uint32_t)rows0 * V * 2u + stg_gate_bytes +
-                                                  (tok0 ? 256u + (uint32_t)V * 2u : 0u) + (p.q != nullptr ? 256u : 0u));
-        auto stage_tile = [&](int tile) {       // one thread
+        auto block_bytes = [&](int blk) -> uint32_t {
+            int rows = n_ring - blk * kTokBlock;
+            rows = rows < 0 ? 0 : (rows > kTokBlock ? kTokBlock : rows);
+            const bool tok = p.has_token && n_ring / kTokBlock == blk;
+            uint32_t by = (uint32_t)rows * 256u + (uint32_t)rows * V * 2u + (tok ? 256u + (uint32_t)V * 2u : 0u);
+            if (blk == 0) by += stg_gate_bytes + (p.q != nullptr ? 256u : 0u);
+            return (uint32_t)NH * by;
+        };
+        const bool staging = block_bytes(0) > 0;
+        // One bulk copy per lane of the group's first warp: lane = head * 6 + kind, kind = block keys, block values,
+        // token key, token value, gates, query row.  Base pointer and bytes per (batch, head) are per-lane constants.
+        const int cp_hd = gt / 6, cp_kind = gt - cp_hd * 6;
+        const unsigned char* cp_base = nullptr;
+        size_t cp_stride = 0;
+        if (gt < 6 * NH) {
+            switch (cp_kind) {
+                case 0: cp_base = p.ring; cp_stride = p.rl.head_bytes; break;
+                case 1: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; break;
+                case 2: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; break;
+                case 3: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; break;
+                case 4: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; break;
+                default: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; break;
+            }
+        }
+        auto stage_block = [&](int tile, int blk, int buf) {       // first warp of the group
             const int h = tile / tiles_per_h;
             const int b0 = (tile - h * tiles_per_h) * NH;
-            mbar_expect_tx(&bars[kBarStg], stg_bytes);
-            for (int hd = 0; hd < NH; ++hd) {
-                const size_t bw = (size_t)(b0 + hd) * H + h;
-                const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
-                unsigned char* dst = sStg + (size_t)hd * sm.stg_head;
-                if (rows0 > 0) {
-                    bulk_g2s(dst, rh, (uint32_t)rows0 * 256u, &bars[kBarStg]);
-                    bulk_g2s(dst + 4096, rh + p.rl.v_off, (uint32_t)rows0 * V * 2u, &bars[kBarStg]);
-                }
-                if (stg_gate_bytes) bulk_g2s(dst + sm.stg_gate, rh + p.rl.beta_off, stg_gate_bytes, &bars[kBarStg]);
-                if (tok0) {
-                    bulk_g2s(dst + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.k) + bw * K, 256u, &bars[kBarStg]);
-                    bulk_g2s(dst + 4096 + (size_t)n_ring * V * 2, reinterpret_cast<const __nv_bfloat16*>(p.v) + bw * V, (uint32_t)V * 2u, &bars[kBarStg]);
-                }
-                if (p.q != nullptr) bulk_g2s(dst + sm.stg_q, reinterpret_cast<const __nv_bfloat16*>(p.q) + bw * K, 256u, &bars[kBarStg]);
+            int rows = n_ring - blk * kTokBlock;
+            rows = rows < 0 ? 0 : (rows > kTokBlock ? kTokBlock : rows);
+            const bool tok = p.has_token && n_ring / kTokBlock == blk;
+            const int tok_row = n_ring - blk * kTokBlock;
+            uint64_t* bar = &bars[kBarStg + buf];
+            if (gt == 0) mbar_expect_tx(bar, block_bytes(blk));
+            __syncwarp();
+            if (gt < 6 * NH) {
+                const size_t bw = (size_t)(b0 + cp_hd) * H + h;
+                const uint32_t blk_dst = sm.stg_blk + (uint32_t)buf * sm.stg_blk_stride + (uint32_t)cp_hd * sm.stg_blk_head;
+                const uint32_t tile_dst = sm.stg + (uint32_t)cp_hd * sm.stg_tile_head;
+                uint32_t bytes = 0, dst = 0, src_off = 0;
+                if (cp_kind == 0) { bytes = (uint32_t)rows * 256u; dst = blk_dst; src_off = (uint32_t)blk * kTokBlock * 256u; }
+                else if (cp_kind == 1) { bytes = (uint32_t)rows * V * 2u; dst = blk_dst + 4096u; src_off = (uint32_t)blk * kTokBlock * V * 2u; }
+                else if (cp_kind == 2) { bytes = tok ? 256u : 0u; dst = blk_dst + (uint32_t)tok_row * 256u; }
+                else if (cp_kind == 3) { bytes = tok ? (uint32_t)V * 2u : 0u; dst = blk_dst + 4096u + (uint32_t)tok_row * V * 2u; }
+                else if (cp_kind == 4) { bytes = blk == 0 ? stg_gate_bytes : 0u; dst = tile_dst; }
+                else { bytes = (blk == 0 && p.q != nullptr) ? 256u : 0u; dst = tile_dst + sm.stg_q; }
+                if (bytes) bulk_g2s(smem + dst, cp_base + bw * cp_stride + src_off, bytes, bar);
             }
         };
+        // producer cursor of the staging ring (kept by every lane of the first warp): the next block to request, and how
+        // many tiles have been published
+        int sq_tile = 0, sq_blk = 0, sq_idx = 0, pub_k = 0;
+        auto stage_next = [&]() {           // first warp: request the next block in sequence; entering a new tile claims it
+            if (sq_tile < 0) return;
+            if (sq_blk == 0) {              // the claim issued a tile ago is resolved only now, the one after it goes out
+                int nxt = 0;
+                if (gt == 0) {
+                    nxt = claim_resolve();
+                    publish(pub_k, nxt);
+                    if (nxt >= 0) claim_issue();
+                }
+                ++pub_k;
+                sq_tile = __shfl_sync(0xffffffffu, nxt, 0);
+                if (sq_tile < 0) return;
+            }
+            if (staging) stage_block(sq_tile, sq_blk, sq_idx % stg_bufs);
+            ++sq_idx;
+            if (++sq_blk == n_stage_blocks) sq_blk = 0;
+        };
+        int cq_idx = 0;                     // blocks consumed by the group so far
         // sketch rows and exact output of a finished tile: UT sits in the first NP columns of that tile's accumulator
         auto store_ut = [&](int tile, int b) -> bool {
             const int h = tile / tiles_per_h;
@@ -445,14 +507,10 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             return true;
         };
 
-        if (gt == 0) {
-            claim_issue();
-            const int first = claim_resolve();
-            publish(0, first);
-            if (first >= 0) {
-                claim_issue();
-                if (stg_bytes > 0) stage_tile(first);
-            }
+        if (gt < 32) {
+            if (gt == 0) claim_issue();
+            stage_next();
+            if (stg_bufs > 1 && n_stage_blocks > 1) stage_next();
         }
         // W (padding columns, lo halves of the query columns) and the MMA-1 operands (off-diagonal head blocks) hold
         // zeros that no tile ever overwrites: written once
@@ -544,27 +602,26 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 }
                 cur_h = h;
             }
-            // the staged rows, gates and query rows of this tile must have landed
-            if (stg_bytes > 0) {
-                if (!group_wait(2, gt, &bars[kBarStg], phS)) {
+            // the first block of this tile (with its gates and query rows) must have landed
+            if (staging) {
+                if (!group_wait(2, gt, &bars[kBarStg + cq_idx % stg_bufs], (uint32_t)(cq_idx / stg_bufs) & 1u)) {
                     if (gt == 0) record_fault(p.status, kFaultUpdateWait, 6);
                     dead = true;
                     break;
                 }
-                phS ^= 1;
             }
             WS_STAMP(512, 1);
             if (p.q != nullptr) {       // query columns of this tile's group (bf16-exact: lo = 0)
                 for (int idx = gt; idx < K * NH; idx += kGroup) {
                     const int i = idx % K, hd = idx / K, g = QA + 8 * b + hd;
                     const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO2B + (i & 7) * 2) >> 1;
-                    sB2hi[o2] = reinterpret_cast<const __nv_bfloat16*>(sStg + (size_t)hd * sm.stg_head + sm.stg_q)[i];
+                    sB2hi[o2] = reinterpret_cast<const __nv_bfloat16*>(sStg + (size_t)hd * sm.stg_tile_head + sm.stg_q)[i];
                 }
             }
             // ---- token weights w_s = beta_s prod_{j>s} a_j and the total decay: one warp per head, suffix scan ----
             if (fwarp < NH) {
                 const int hd = fwarp, lane = gt & 31;
-                const float* sg = reinterpret_cast<const float*>(sStg + (size_t)hd * sm.stg_head + sm.stg_gate);
+                const float* sg = reinterpret_cast<const float*>(sStg + (size_t)hd * sm.stg_tile_head);
                 float suf = 1.f;          // product of the decays of all later tokens
                 for (int base = ((n_tot + 31) & ~31) - 32; base >= 0; base -= 32) {
                     const int s = base + lane;
@@ -602,8 +659,17 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 }
                 // Operand rows are written 16 bytes per thread; consecutive threads walk the 8 token rows of a core matrix
                 // first and then the next 8-element vector, so that a warp writes 512 contiguous bytes (no bank conflicts).
-                if (blk == 0) {
-                    // first block: rows come from the staging buffer; only the diagonal head blocks of A are written
+                {
+                    // rows come from the block's staging buffer; only the diagonal head blocks of A are written
+                    if (blk > 0 && staging) {      // (the first block was waited for above)
+                        if (!group_wait(2, gt, &bars[kBarStg + cq_idx % stg_bufs], (uint32_t)(cq_idx / stg_bufs) & 1u)) {
+                            if (gt == 0) record_fault(p.status, kFaultUpdateWait, 6);
+                            dead = true;
+                            break;
+                        }
+                    }
+                    const unsigned char* sBlk = smem + sm.stg_blk + (size_t)(cq_idx % stg_bufs) * sm.stg_blk_stride;
+                    const int s_base = blk * kTokBlock;
                     constexpr int NB = KD1 * (K / 8) / kGroup;          // B-operand vectors per thread
                     uint4 kv[NB];
 #pragma unroll
@@ -611,8 +677,8 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                         const int idx = gt + r * kGroup;
                         const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
                         const int hd = sp / kTokBlock, s = sp % kTokBlock;
-                        kv[r] = s < n_tot ? *reinterpret_cast<const uint4*>(sStg + (size_t)hd * sm.stg_head + (size_t)s * 256 + a * 16)
-                                          : make_uint4(0, 0, 0, 0);
+                        kv[r] = s_base + s < n_tot ? *reinterpret_cast<const uint4*>(sBlk + (size_t)hd * sm.stg_blk_head + (size_t)s * 256 + a * 16)
+                                                   : make_uint4(0, 0, 0, 0);
                     }
                     constexpr int NA = NH * kTokBlock * (V / 8) / kGroup;      // diagonal A-operand vectors per thread
                     uint4 vv[NA];
@@ -622,10 +688,10 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                         const int it = gt + r * kGroup;
                         const int t8 = it & 7, a = (it >> 3) % (V / 8), rest = it / V;
                         const int hd = rest >> 1, s = (rest & 1) * 8 + t8;
-                        const bool live = s < n_tot;
-                        vv[r] = live ? *reinterpret_cast<const uint4*>(sStg + (size_t)hd * sm.stg_head + 4096 + (size_t)s * V * 2 + a * 16)
+                        const bool live = s_base + s < n_tot;
+                        vv[r] = live ? *reinterpret_cast<const uint4*>(sBlk + (size_t)hd * sm.stg_blk_head + 4096 + (size_t)s * V * 2 + a * 16)
                                      : make_uint4(0, 0, 0, 0);
-                        wv[r] = live ? sW[hd * 208 + s] : 0.f;
+                        wv[r] = live ? sW[hd * 208 + s_base + s] : 0.f;
                     }
 #pragma unroll
                     for (int r = 0; r < NB; ++r) {
@@ -650,48 +716,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                         *reinterpret_cast<uint4*>(sA1hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
                         *reinterpret_cast<uint4*>(sA1lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
                     }
-                } else {
-                // later blocks (n > 16): rows are read from the ring in global memory
-                // B operand: keys, MN-major (mn = state row i, k = token slot)
-                for (int idx = gt; idx < KD1 * (K / 8); idx += kGroup) {
-                    const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
-                    const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
-                    const size_t bk = (size_t)(b0 + hd) * H + h;
-                    uint4 val = make_uint4(0, 0, 0, 0);
-                    if (s < n_ring) {
-                        val = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + ((size_t)s * K + a * 8) * 2);
-                    } else if (s < n_tot) {
-                        val = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.k) + bk * K + a * 8);
-                    }
-                    *reinterpret_cast<uint4*>(sB1 + (sp & 7) * 16 + a * SBO + (sp >> 3) * LBO1) = val;
-                }
-                // A operand: w_s v_s hi/lo, MN-major (mn = lane t = head*V + j, k = token slot), block diagonal over heads
-                for (int idx = gt; idx < KD1 * 16; idx += kGroup) {
-                    const int a128 = (idx >> 3) & 15, sp = (idx & 7) + 8 * (idx >> 7);
-                    const int hd = sp / kTokBlock, s = blk * kTokBlock + sp % kTokBlock;
-                    const int hd_lane = a128 / (V / 8), a = a128 % (V / 8);
-                    if (hd_lane != hd) continue;          // off-diagonal blocks stay zero
-                    const size_t bk = (size_t)(b0 + hd) * H + h;
-                    uint4 vraw = make_uint4(0, 0, 0, 0);
-                    float w = 0.f;
-                    if (s < n_ring) {
-                        vraw = *reinterpret_cast<const uint4*>(p.ring + bk * p.rl.head_bytes + p.rl.v_off + ((size_t)s * V + a * 8) * 2);
-                        w = sW[hd * 208 + s];
-                    } else if (s < n_tot) {
-                        vraw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.v) + bk * V + a * 8);
-                        w = sW[hd * 208 + s];
-                    }
-                    const uint32_t vin[4] = {vraw.x, vraw.y, vraw.z, vraw.w};
-                    uint32_t ohi[4], olo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float f0 = w * __uint_as_float(vin[e] << 16), f1 = w * __uint_as_float(vin[e] & 0xffff0000u);
-                        split_bf16x2(f0, f1, ohi[e], olo[e]);
-                    }
-                    const uint32_t off = (sp & 7) * 16 + a128 * SBO + (sp >> 3) * LBO1;
-                    *reinterpret_cast<uint4*>(sA1hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
-                    *reinterpret_cast<uint4*>(sA1lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
-                }
+                    ++cq_idx;
                 }
                 proxy_fence();
                 tc_fence_before();
@@ -707,32 +732,24 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                         tc_mma_bf16(tmem_t, make_desc(smem_u32(sA1lo) + ks * 2 * LBO1, LBO1, SBO), bd, idesc1, 1u);
                     }
                     tc_commit(&bars[kBarBlk]);
-                    if (blk + 1 == n_blocks) tc_commit(&bars[kBarT + b]);
-                    if (blk == 0) {      // the staging buffer is free again: the next tile's rows may come in
-                        const int nxt = claim_resolve();
-                        publish(k + 1, nxt);
-                        if (nxt >= 0) {
-                            claim_issue();
-                            if (stg_bytes > 0) stage_tile(nxt);
-                        }
+                    if (blk + 1 == n_blocks) {
+                        tc_commit(&bars[kBarT + b]);
+                        mbar_arrive(&bars[kBarPro + b]);      // after the group barrier: W, weights and decay are written
                     }
                 }
+                if (gt < 32) stage_next();        // the block buffer just read is free again
             }
             if (dead) break;
             if (n_blocks == 0) {
                 // no token to replay: nothing reads the staging buffer after the query columns; T counts as zero
+                ++cq_idx;
                 group_sync(2);
                 if (gt == 0) {
                     mbar_arrive(&bars[kBarT + b]);
-                    const int nxt = claim_resolve();
-                    publish(k + 1, nxt);
-                    if (nxt >= 0) {
-                        claim_issue();
-                        if (stg_bytes > 0) stage_tile(nxt);
-                    }
+                    mbar_arrive(&bars[kBarPro + b]);
                 }
+                if (gt < 32) stage_next();
             }
-            if (gt == 0) mbar_arrive(&bars[kBarPro + b]);      // after the group barrier: W, weights and decay are written
             WS_STAMP(512, 3);
 
             // ---- sketch rows and exact output of the previous tile, once the stream group has finished it ----
@@ -783,8 +800,8 @@ int launch_update_tc_ws(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
     if (c.dv != 64 && c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
     const int NH = 128 / c.dv;
     if (c.batch % NH != 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    if (c.rank > 16) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    const int NP = ((((c.rank + 7) & ~7) + 16) + 15) & ~15;      // [Omega | q | q'] <= 32 columns
+    if (c.rank > 32) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int NP = ((((c.rank + 7) & ~7) + 16) + 15) & ~15;      // [Omega | q | q']: 32 or 48 columns
     Params p = p_in;
     if (ctx->sm_count == 0) {
         int dev = 0, sms = 0;
@@ -798,17 +815,20 @@ int launch_update_tc_ws(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
     int ctas = 2;
     if (p.max_warps_per_sm > 0 && p.max_warps_per_sm < 18) ctas = 1;
     const uint32_t budget = (228u * 1024u) / (uint32_t)ctas - 1024u;
-    const WsSmem fixed = make_ws_smem(NH, NP, c.dv, c.buf_len, 0);
+    const int n_tot = p.n_before + (p.has_token ? 1 : 0);
+    const int stg_bufs = n_tot > kTokBlock ? 2 : 1;
+    const WsSmem fixed = make_ws_smem(NH, NP, c.dv, c.buf_len, 0, stg_bufs);
     if (fixed.total + 2u * fixed.sst_bytes > budget) return SKETCHSSM_UNSUPPORTED_SHAPE;
     int stages = (int)((budget - fixed.total) / fixed.sst_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (p.stages >= 2 && p.stages < stages) stages = p.stages;
     p.stages = stages;
-    const WsSmem sm = make_ws_smem(NH, NP, c.dv, c.buf_len, stages);
+    const WsSmem sm = make_ws_smem(NH, NP, c.dv, c.buf_len, stages, stg_bufs);
     const long long n_tiles = (long long)c.batch * c.heads / NH;
     long long grid = (long long)ctx->sm_count * ctas;
     if (grid > n_tiles) grid = n_tiles;
-    auto kern = c.dv == 128 ? update_tc_ws_mamba2_kernel<128> : update_tc_ws_mamba2_kernel<64>;
+    auto kern = NP > 32 ? (c.dv == 128 ? update_tc_ws_mamba2_kernel<128, true> : update_tc_ws_mamba2_kernel<64, true>)
+                        : (c.dv == 128 ? update_tc_ws_mamba2_kernel<128, false> : update_tc_ws_mamba2_kernel<64, false>);
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)sm.total)) != cudaSuccess)
         return SKETCHSSM_CUDA_ERROR;

@@ -153,11 +153,12 @@ def test_mamba2_tensor_core_variants(dv, rank, buf_len):
 
 
 @pytest.mark.parametrize("tune", [{}, {"decode_max_warps_per_sm": 8}, {"pdl": 0}])
-@pytest.mark.parametrize("dv,batch,heads,buf_len", [(64, 64, 24, 16), (128, 40, 20, 8)])
-def test_mamba2_update_several_tiles_per_cta(tune, dv, batch, heads, buf_len):
+@pytest.mark.parametrize("dv,batch,heads,buf_len,rank", [(64, 64, 24, 16, 16), (128, 40, 20, 8, 16), (64, 64, 24, 16, 32),
+                                                         (128, 24, 10, 12, 24), (64, 48, 12, 40, 8)])
+def test_mamba2_update_several_tiles_per_cta(tune, dv, batch, heads, buf_len, rank):
     """Warp-specialised tcgen05 update with every CTA walking several tiles (double-buffered accumulators, operand
     sets and W buffers; head index changes inside a CTA's range), over two windows."""
-    w = synth.Workload("t", "mamba2", batch, heads, 128, dv, 16, buf_len, 0, "bf16", 79, basis="qr")
+    w = synth.Workload("t", "mamba2", batch, heads, 128, dv, rank, buf_len, 0, "bf16", 79, basis="qr")
     check(run_schedule(w, 2 * buf_len + 2, max_heads=96, tune=tune), "bf16")
 
 
