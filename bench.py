@@ -196,9 +196,10 @@ class Stack:
         return per * self.n_layers
 
     def run_window(self, mode: str = "sketch", events=None):
-        """One step: L tokens through every layer.  mode: "sketch" (decode_step + state_update) or
-        "full_read" (full_read_decode + state_update without the sketch write).  `events`, if given, receives
-        (kind, n_before, start_event, end_event) per launch."""
+        """One step: L tokens through every layer.  mode: "sketch" (decode_step + state_update),
+        "full_read" (full_read_decode + state_update without the sketch write) or "standard" (no buffering: the
+        state is read, updated with the one token and written back at every step; the flush kernel with an empty
+        ring and no sketch).  `events`, if given, receives (kind, n_before, start_event, end_event) per launch."""
         from paper_2609_33051_b200.binding import NO_SKETCH
         L = self.w.buf_len
         launches = 0
@@ -209,7 +210,9 @@ class Stack:
                     e0 = torch.cuda.Event(enable_timing=True)
                     e1 = torch.cuda.Event(enable_timing=True)
                     e0.record()
-                if t < L - 1:
+                if mode == "standard":
+                    m.state_update(0, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], o, flags=NO_SKETCH)
+                elif t < L - 1:
                     if mode == "sketch":
                         m.decode_step(t, tok["q"], tok["k"], tok["v"], tok["beta"], tok["decay"], o)
                     else:
@@ -475,6 +478,11 @@ def main():
         full = {"value": world * tokens_per_step / (ms_full * 1e-3), "unit": UNIT, "ms_per_step": ms_full,
                 "what": "sketchssm_full_read_decode x (L-1) + sketchssm_state_update(NO_SKETCH) per layer and window",
                 "sketch_speedup": ms_full / ms_step}
+        # the execution without a buffer: full state read + write per token (what the paper calls the standard decode)
+        ms_std, _, _ = timed_region(lambda: stack.run_window("standard", None), max(3, args.steps // 4), 3)
+        full["standard"] = {"value": world * tokens_per_step / (ms_std * 1e-3), "unit": UNIT, "ms_per_step": ms_std,
+                            "what": "sketchssm_state_update(n_before = 0, token, NO_SKETCH) at every step",
+                            "sketch_speedup": ms_std / ms_step}
         stack.run_window("sketch", None)     # leave a fresh sketch behind
 
     # ---- end to end through the C ABI with host buffers ----

@@ -89,7 +89,7 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
     const int RP = (R + 7) & ~7;                       // coefficient rows padded to the reduction width
     d.coef_slot_bytes = full_read ? 0u : (uint32_t)(RP * K * 4);
     d.bar_off = 2u * d.coef_slot_bytes;
-    uint32_t off = d.bar_off + (((uint32_t)(nwarps * 2 * 8) + 127u) & ~127u);    // two mbarriers per warp
+    uint32_t off = d.bar_off + (((uint32_t)(nwarps * 2 * 8 + 16) + 127u) & ~127u);    // two mbarriers per warp, the head counter
     d.scratch_stride = (uint32_t)((K + 80) * 4);       // per warp: q~ (full read) or c (K floats), then 64+ dot products
     d.scratch_off = off; off += (uint32_t)nwarps * d.scratch_stride;
     d.stage_off = off;
@@ -130,6 +130,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < nwarps * 2; ++i) mbar_init(reinterpret_cast<uint64_t*>(smem + ds.bar_off) + i, 1);
+        *reinterpret_cast<int*>(smem + ds.bar_off + (size_t)nwarps * 16) = nwarps;
         mbar_fence_init();
     }
     // coefficient maps of the (at most two) head indices of this range, rows padded with zeros.  C is a constant of
@@ -183,20 +184,25 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         }
     };
 
-    // this warp's heads: items item0 + warp, item0 + warp + nwarps, ...; (head index, batch) advance without divisions
+    // The CTA's heads are handed to its warps at run time (a counter in shared memory): a warp claims its next head
+    // when it starts the current one, so the warps of a CTA finish within one head of each other whatever the count.
+    // The range spans at most two head indices, so (head index, batch) follow from the item number without divisions.
     const int n_items = item1 - item0;
-    const int count = warp < n_items ? (n_items - warp + nwarps - 1) / nwarps : 0;
-    int h = 0, b = 0;
-    if (count > 0) {
-        h = (item0 + warp) / B;
-        b = (item0 + warp) - h * B;
-    }
-    auto advance = [&](int& hh, int& bb) {
-        bb += nwarps;
-        while (bb >= B) { bb -= B; ++hh; }
+    int* item_ctr = reinterpret_cast<int*>(smem + ds.bar_off + (size_t)nwarps * 16);
+    const int second_h_start = (h_first + 1) * B;      // first item of the range's second head index
+    auto claim = [&]() -> int {            // whole warp; returns an item number, or item1 when none is left
+        int v = 0;
+        if (lane == 0) v = atomicAdd(item_ctr, 1);
+        v = __shfl_sync(0xffffffffu, v, 0);
+        return v < n_items ? item0 + v : item1;
     };
-    int hn = h, bn = b;                 // the warp's next head
-    advance(hn, bn);
+    auto head_of = [&](int item, int& hh, int& bb) {
+        hh = item >= second_h_start ? h_first + 1 : h_first;
+        bb = item - hh * B;
+    };
+    int item = warp < n_items ? item0 + warp : item1;      // the first head of every warp is fixed (the counter starts at nwarps)
+    int h = 0, b = 0, hn = 0, bn = 0;
+    if (item < item1) head_of(item, h, b);
 
     // the token's scalar gates travel in registers, fetched one head ahead
     auto scalar_gates = [&](size_t bh, float& bt, float& dsc) {
@@ -205,7 +211,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         if constexpr (KIND != SKETCHSSM_KDA) dsc = reinterpret_cast<const float*>(p.decay)[bh];
     };
     float bt_next = 0.f, dsc_next = 1.f;
-    if (count > 0) {
+    if (item < item1) {
         const size_t bh0 = (size_t)b * H + h;
         issue_a(bh0);
         issue_b(bh0);
@@ -216,11 +222,13 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     unsigned long long poll_count = 0;
 #endif
 
-    for (int it = 0; it < count; ++it) {
+    for (int it = 0; item < item1; ++it) {
         const uint32_t parity = it & 1;
         const size_t bh = (size_t)b * H + h;
+        const int item_next = claim();
+        const bool has_next = item_next < item1;
+        if (has_next) head_of(item_next, hn, bn);
         const size_t bh_next = (size_t)bn * H + hn;
-        const bool has_next = it + 1 < count;
         const float bt = bt_next, dsc = dsc_next;
         if (has_next) scalar_gates(bh_next, bt_next, dsc_next);
 
@@ -414,9 +422,9 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 
         __syncwarp();  // every lane is done with the scratch before it is reused
         DEC_STAMP(4);
+        item = item_next;
         h = hn;
         b = bn;
-        advance(hn, bn);
         DEC_STAMP(5);
     }
     (void)dead;
