@@ -18,6 +18,13 @@
 // one thread issues every MMA; one warp keeps the stages full.  Passes of consecutive tiles are interleaved
 // (A(i+1) runs between E'(i) and B(i)), so no MMA round trip is waited for.
 //
+// The sketch rows never need S_new as a tensor-core operand: [U | o] = d S_0^T W + E'^T (K W) with W = [Omega | q], so
+// pass A contracts the S_0 chunks with W as well (same hi + lo operand as for P), the small product K W is formed by
+// the front group, and the correction E'^T (K W) rides along with K^T E'.  Pass B is then only
+// S_new = d S_0 + K^T E' written back: no split, no operand hand-off, no MMA.
+// Tensor memory per CTA (256 columns): two 64-column slots [U0 (32) | P (16), later the correction (32)] for
+// alternating tiles, and one 128-column accumulator for K^T E'.
+//
 // Domain: GDN, bf16 I/O, K = V = 128, 1..16 tokens per flush, rank <= 16.
 #include "internal.cuh"
 #include "tc_common.cuh"
@@ -47,8 +54,8 @@ constexpr int kGS = 20;              // row stride (floats) of the small n x n w
 constexpr int kA2 = 2;               // chunk buffers between the stream group and the MMA issue warp
 
 struct GSmem {
-    uint32_t a2, e, w, set, set_stride, set_bt, set_vv, set_t1, set_gates, stg, stg_v, stg_gate, stg_q, mats, bars, misc, sst,
-        sst_bytes, total;
+    uint32_t a2, e, w, set, set_stride, set_bt, set_vv, set_t1, set_bc, set_gates, stg, stg_v, stg_gate, stg_q, mats, bars,
+        misc, sst, sst_bytes, total;
 };
 
 __host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
@@ -58,9 +65,9 @@ __host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
     s.e = off; off += 2u * 128u * 16u * 2u;                       // E' hi + lo (same layout as a chunk buffer)
     s.w = off; off += 2u * (uint32_t)NP * kK * 2u;                // [Omega | q | q'] hi | lo
     // per-tile operand set, double-buffered: keys as B operand of pass A (K-major) and of K^T E' (MN-major),
-    // raw value rows, T1, gates (C diagonal, total decay)
+    // raw value rows, T1, K [Omega | q] hi | lo (B operand of the sketch correction), gates (C diagonal, total decay)
     s.set = off;
-    s.set_bt = 4096u; s.set_vv = 8192u; s.set_t1 = 12288u; s.set_gates = 13312u; s.set_stride = 13440u;
+    s.set_bt = 4096u; s.set_vv = 8192u; s.set_t1 = 12288u; s.set_bc = 13312u; s.set_gates = 15360u; s.set_stride = 15488u;
     off += 2u * s.set_stride;
     // staging of the next tile's raw rows: keys [16][256 B], values [16][256 B], gates [2L] floats, query row
     s.stg_v = 4096u;
@@ -77,7 +84,7 @@ __host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
     return s;
 }
 
-enum { gPro = 0, gPfull = 2, gTfull = 4, gUfull = 6, gBufFree = 8, gA2free = 10, gA2rdy = 10 + kA2, gErdy = 10 + 2 * kA2,
+enum { gPro = 0, gPfull = 2, gTfull = 4, gBdone = 6, gBufFree = 8, gA2free = 10, gA2rdy = 10 + kA2, gErdy = 10 + 2 * kA2,
        gStg = 11 + 2 * kA2, gProW = 12 + 2 * kA2, gFull = 14 + 2 * kA2, gEmpty = 14 + 2 * kA2 + kGStages,
        gNumBars = 14 + 2 * kA2 + 2 * kGStages };
 
@@ -145,7 +152,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     if (tid == 0) {
         *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
         for (int i = 0; i < gNumBars; ++i) {
-            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty;     // one arrival per stream warp
+            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty || i == gBdone || i == gBdone + 1;     // one arrival per stream warp
             mbar_init(&bars[i], per_warp ? 4 : 1);
         }
         mbar_fence_init();
@@ -192,20 +199,14 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 
     if (warp < 4) {
         // =========================== stream group ===========================
-        uint32_t phPro = 0, phProW = 0, phP = 0, phT = 0, phA = 0, phF = 0;
+        uint32_t phPro = 0, phP = 0, phT = 0, phA = 0, phF = 0;
         float dt0 = 1.f, dt1 = 1.f;          // total decay of the tile in each operand set, read when E' is formed
         int gc = 0, stage = 0;
         bool bad = false;
 
-        // one pass over the 8 chunks of a tile: pass A delivers S_0 chunks (hi + lo) for P = K S_0; pass B forms
-        // S_new = d S_0 + T, writes it back and delivers it for [U | o]
-        auto do_pass = [&](bool is_b, int tile, int b) {
-            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
-            const size_t bh = (size_t)bb * H + h;
-            float* So = p.state + bh * (size_t)K * V + j;
-            const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
-            const float dtot = is_b ? (b ? dt1 : dt0) : 1.f;
-            float t01[2 * CH];
+        // pass A over the 8 chunks of a tile: the S_0 chunks are split into bf16 hi + lo and handed to the issue warp,
+        // which contracts them with [Omega | q] (U0) and with the keys (P)
+        auto pass_a = [&]() {
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
@@ -213,19 +214,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 float s0[CH];
 #pragma unroll
                 for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
-                float t[CH];
-                if (is_b && !bad) {
-                    if (c == 0) tmem_ld32(tmem_t + lane_sel, t01);
-                    if (c < 2) {
-#pragma unroll
-                        for (int ii = 0; ii < CH; ++ii) t[ii] = t01[c * CH + ii];
-                    } else {
-                        tmem_ld16(tmem_t + lane_sel + (uint32_t)(c * CH), t);
-                    }
-                } else {
-#pragma unroll
-                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
-                }
                 __syncwarp();
                 if (lane == 0) g_arrive(&bars[gEmpty + stage]);
                 const int ab = c & (kA2 - 1);
@@ -239,26 +227,50 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 for (int v8 = 0; v8 < CH / 8; ++v8) {
                     uint32_t ohi[4], olo[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int i0 = v8 * 8 + 2 * e;
-                        const float x0 = fmaf(dtot, s0[i0], t[i0]), x1 = fmaf(dtot, s0[i0 + 1], t[i0 + 1]);
-                        if (is_b && !bad) {
-                            So[(size_t)(c * CH + i0) * V] = x0;
-                            So[(size_t)(c * CH + i0 + 1) * V] = x1;
-                        }
-                        split_bf16x2(x0, x1, ohi[e], olo[e]);
-                    }
+                    for (int e = 0; e < 4; ++e) split_bf16x2(s0[v8 * 8 + 2 * e], s0[v8 * 8 + 2 * e + 1], ohi[e], olo[e]);
                     const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO_M;
                     *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
                     *reinterpret_cast<uint4*>(a2lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
                 }
                 proxy_fence();
-                tc_fence_before();
                 bad = __any_sync(0xffffffffu, bad);
                 if (lane == 0 && !bad) g_arrive(&bars[gA2rdy + ab]);
                 ++gc;
                 if (++stage == NS) { stage = 0; phF ^= 1u; }
             }
+        };
+        // pass B: S_new = d S_0 + K^T E', written back; nothing is handed on
+        auto pass_b = [&](int tile, int b) {
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            float* So = p.state + bh * (size_t)K * V + j;
+            const float dtot = b ? dt1 : dt0;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
+                const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
+                float s0[CH];
+#pragma unroll
+                for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
+                float t[CH];
+                if (!bad) {
+                    tmem_ld16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), t);
+                } else {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) g_arrive(&bars[gEmpty + stage]);
+                if (!bad) {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = fmaf(dtot, s0[ii], t[ii]);
+                }
+                if (++stage == NS) { stage = 0; phF ^= 1u; }
+            }
+            // this warp has read its lanes of K^T E': the accumulator may be overwritten, the tile's sketch rows stored
+            tc_fence_before();
+            bad = __any_sync(0xffffffffu, bad);
+            if (lane == 0 && !bad) g_arrive(&bars[gBdone + b]);
         };
         // E'[s, j] = sum_t T1[s, t] (v_t[j] - C_t P[t, j]) -> hi + lo A operand of K^T E' (chunk-buffer layout)
         auto do_e = [&](int b) {
@@ -271,7 +283,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const float* sC = reinterpret_cast<const float*>(set + sm.set_gates);
             if (b) dt1 = sC[kNTok]; else dt0 = sC[kNTok];
             float x[kNTok];
-            if (!bad) tmem_ld16(tmem_base + (uint32_t)b * 128u + lane_sel, x);
+            if (!bad) tmem_ld16(tmem_base + (uint32_t)b * 64u + 32u + lane_sel, x);
 #pragma unroll
             for (int t = 0; t < kNTok; ++t) x[t] = fmaf(-sC[t], x[t], __bfloat162float(sV[t * V + j]));
             float e[kNTok];
@@ -313,34 +325,27 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         if (cur >= 0) {
             cur &= kSepFlag - 1;
             wait_pro(0);
-            do_pass(false, cur, 0);
+            pass_a();
             do_e(0);
             for (int k = 0; !bad; ++k) {
                 const int b = k & 1;
                 const int raw = seq_get(k + 1);
                 if (raw < -1) { bad = true; break; }
                 const int nxt = raw < 0 ? -1 : (raw & (kSepFlag - 1));
-                const bool sep = raw >= 0 && (raw & kSepFlag) != 0;
                 G_STAMP(0, k, 0);
-                if (nxt >= 0 && !sep) {
+                if (nxt >= 0) {
                     wait_pro(b ^ 1);
                     G_STAMP(0, k, 1);
-                    do_pass(false, nxt, b ^ 1);
+                    pass_a();
                 }
                 G_STAMP(0, k, 2);
-                bad |= !mbar_wait_bounded(&bars[gProW + b], (phProW >> b) & 1u);     // this tile's query column (and Omega) are in W
-                phProW ^= 1u << b;
                 bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);
                 phT ^= 1u << b;
                 tc_fence_after();
                 G_STAMP(0, k, 3);
-                do_pass(true, cur, b);
+                pass_b(cur, b);
                 G_STAMP(0, k, 4);
                 if (nxt < 0) break;
-                if (sep) {
-                    wait_pro(b ^ 1);
-                    do_pass(false, nxt, b ^ 1);
-                }
                 do_e(b ^ 1);
                 G_STAMP(0, k, 5);
                 cur = nxt;
@@ -356,46 +361,16 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             bool bad = false;
             const uint32_t sW = smem_u32(smem + sm.w);
             const uint32_t a2base = smem_u32(smem + sm.a2);
-            auto pass_a = [&](int k) {          // P(b) = K S_0, chunk by chunk
+            auto pass_a = [&](int k) {          // U0(b) = S_0^T [Omega | q] and P(b) = (K S_0)^T, chunk by chunk
                 const int b = k & 1;
-                if (k >= 2) {                   // the accumulator half still holds the sketch rows of tile k - 2 until they are stored
+                if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
                     if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; return; }
                     phBuf ^= 1u << b;
                     tc_fence_after();
                 }
-                const uint32_t tmem_p = tmem_base + (uint32_t)b * 128u;
+                const uint32_t tmem_u0 = tmem_base + (uint32_t)b * 64u;
+                const uint32_t tmem_p = tmem_u0 + 32u;
                 const uint32_t bp = smem_u32(set_ptr(b));
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int ab = c & (kA2 - 1);
-                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; return; }
-                    phR ^= 1u << ab;
-                    tc_fence_after();
-                    const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
-                    const uint64_t ahi = make_desc(a2, LBO_M, SBO);
-                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
-                    const uint64_t bk = make_desc(bp + (uint32_t)(c * 2) * LBO_BP, LBO_BP, SBO);
-                    tc_mma_bf16(tmem_p, ahi, bk, idescP, c ? 1u : 0u);
-                    tc_mma_bf16(tmem_p, alo, bk, idescP, 1u);
-                    tc_commit(&bars[gA2free + ab]);
-                    if (c == NCH - 1) tc_commit(&bars[gPfull + b]);
-                }
-            };
-            auto step_e = [&](int k) {          // T(b) = E'^T-contraction with the keys: T[j, i] = sum_s E'[s, j] k_s[i]
-                const int b = k & 1;
-                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; return; }
-                phE ^= 1u;
-                tc_fence_after();
-                const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
-                const uint32_t e = smem_u32(smem + sm.e);
-                const uint64_t bt = make_desc(smem_u32(set_ptr(b) + sm.set_bt), LBO_M, SBO);
-                tc_mma_bf16(tmem_t, make_desc(e, LBO_M, SBO), bt, idescT, 0u);
-                tc_mma_bf16(tmem_t, make_desc(e + 128u * CH * 2u, LBO_M, SBO), bt, idescT, 1u);
-                tc_commit(&bars[gTfull + b]);
-            };
-            auto pass_b = [&](int k) {          // [U | o](b) = S_new^T [Omega | q]
-                const int b = k & 1;
-                const uint32_t tmem_u = tmem_base + (uint32_t)b * 128u;
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     const int ab = c & (kA2 - 1);
@@ -406,14 +381,38 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     const uint32_t kb = (uint32_t)(c * (CH / 8)) * LBO_W;
                     const uint64_t ahi = make_desc(a2, LBO_M, SBO);
                     const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
-                    const uint64_t bhi = make_desc(sW + kb, LBO_W, SBO);
-                    const uint64_t blo = make_desc(sW + (uint32_t)NP * kK * 2u + kb, LBO_W, SBO);
-                    tc_mma_bf16(tmem_u, ahi, bhi, idescU, c ? 1u : 0u);
-                    tc_mma_bf16(tmem_u, alo, bhi, idescU, 1u);
-                    tc_mma_bf16(tmem_u, ahi, blo, idescU, 1u);
+                    const uint64_t whi = make_desc(sW + kb, LBO_W, SBO);
+                    const uint64_t wlo = make_desc(sW + (uint32_t)NP * kK * 2u + kb, LBO_W, SBO);
+                    const uint64_t bk = make_desc(bp + (uint32_t)(c * 2) * LBO_BP, LBO_BP, SBO);
+                    tc_mma_bf16(tmem_u0, ahi, whi, idescU, c ? 1u : 0u);
+                    tc_mma_bf16(tmem_u0, alo, whi, idescU, 1u);
+                    tc_mma_bf16(tmem_u0, ahi, wlo, idescU, 1u);
+                    tc_mma_bf16(tmem_p, ahi, bk, idescP, c ? 1u : 0u);
+                    tc_mma_bf16(tmem_p, alo, bk, idescP, 1u);
                     tc_commit(&bars[gA2free + ab]);
-                    if (c == NCH - 1) tc_commit(&bars[gUfull + b]);
+                    if (c == NCH - 1) tc_commit(&bars[gPfull + b]);
                 }
+            };
+            auto step_e = [&](int k) {          // T = K^T E' (128 columns) and the sketch correction E'^T (K W) over the spent P
+                const int b = k & 1;
+                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; return; }
+                phE ^= 1u;
+                tc_fence_after();
+                const uint32_t tmem_t = tmem_base + 128u;
+                const uint32_t tmem_c = tmem_base + (uint32_t)b * 64u + 32u;
+                const uint32_t e = smem_u32(smem + sm.e);
+                const uint64_t ehi = make_desc(e, LBO_M, SBO);
+                const uint64_t elo = make_desc(e + 128u * CH * 2u, LBO_M, SBO);
+                const uint64_t bt = make_desc(smem_u32(set_ptr(b) + sm.set_bt), LBO_M, SBO);
+                const uint32_t bc = smem_u32(set_ptr(b) + sm.set_bc);
+                const uint64_t bchi = make_desc(bc, 512u, SBO);
+                const uint64_t bclo = make_desc(bc + 1024u, 512u, SBO);
+                tc_mma_bf16(tmem_t, ehi, bt, idescT, 0u);
+                tc_mma_bf16(tmem_t, elo, bt, idescT, 1u);
+                tc_mma_bf16(tmem_c, ehi, bchi, idescU, 0u);
+                tc_mma_bf16(tmem_c, elo, bchi, idescU, 1u);
+                tc_mma_bf16(tmem_c, ehi, bclo, idescU, 1u);
+                tc_commit(&bars[gTfull + b]);
             };
             int cur = seq_get(0);
             if (cur >= 0) {
@@ -422,14 +421,9 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 for (int k = 0; !bad; ++k) {
                     const int raw = seq_get(k + 1);
                     if (raw < -1) { bad = true; break; }
-                    const bool sep = raw >= 0 && (raw & kSepFlag) != 0;
-                    if (raw >= 0 && !sep) pass_a(k + 1);
-                    if (bad) break;
-                    pass_b(k);
+                    if (raw >= 0) pass_a(k + 1);
                     if (raw < 0 || bad) break;
-                    if (sep) pass_a(k + 1);
-                    if (bad) break;
-                    step_e(k + 1);
+                    step_e(k + 1);       // the stream group forms E'(k + 1) after its pass B of tile k
                 }
             } else if (cur < -1) {
                 bad = true;
@@ -480,7 +474,9 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         const int fwarp = gt >> 5;
         int cur_h = -1;
         int pend0 = -1, pend1 = -1;           // tiles whose sketch rows are still to be stored: older, newer
-        uint32_t phS = 0, phU = 0, phTf = 0;
+        int pk0 = 0, pk1 = 0;                 // their positions in this CTA's tile sequence
+        float pd0 = 1.f, pd1 = 1.f;           // and their total decays
+        uint32_t phS = 0;
         bool dead = false;
         float* sGm = reinterpret_cast<float*>(smem + sm.mats);
         float* sPm = sGm + kNTok * kGS;
@@ -539,22 +535,26 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             if (p.q != nullptr) bulk_g2s(sStg + sm.stg_q, reinterpret_cast<const __nv_bfloat16*>(p.q) + bw * K, 256u, &bars[gStg]);
         };
         // sketch rows and exact output of a finished tile; afterwards its accumulator half is free for the issue warp
-        auto store_ut = [&](int tile, int b) -> bool {
+        auto store_ut = [&](int tile, int kk, float dtile) -> bool {
+            const int b = kk & 1;
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bh = (size_t)bb * H + h;
-            if (!g_wait(2, gt, &bars[gUfull + b], (phU >> b) & 1u)) return false;
-            phU ^= 1u << b;
+            // pass B of that tile is over (so K^T E' and the correction are complete and read)
+            if (!g_wait(2, gt, &bars[gBdone + b], (uint32_t)(kk >> 1) & 1u)) return false;
             tc_fence_after();
+            const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
             for (int g0 = 0; g0 < NP; g0 += 16) {
-                float u[16];
-                tmem_ld16(tmem_base + (uint32_t)b * 128u + lane_sel + (uint32_t)g0, u);
+                float u0[16], cr[16];
+                tmem_ld16(slot + (uint32_t)g0, u0);
+                tmem_ld16(slot + 32u + (uint32_t)g0, cr);
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
                     const int g = g0 + e;
-                    if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u[e];
+                    const float u = fmaf(dtile, u0[e], cr[e]);      // [U | o] = d S_0^T W + E'^T (K W)
+                    if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u;
                     if (g == QA + 8 * b && p.out != nullptr) {
-                        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u[e]);
-                        else reinterpret_cast<float*>(p.out)[bh * V + j] = u[e];
+                        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
+                        else reinterpret_cast<float*>(p.out)[bh * V + j] = u;
                     }
                 }
             }
@@ -576,6 +576,15 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         // W padding columns and lo halves of the query columns hold zeros that no tile overwrites: written once
         for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGrp * 16u)
             *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
+        // staged key rows beyond the tokens of a flush are never written by the copies: zero them once, so that the
+        // products formed from all 16 rows stay finite
+        for (uint32_t o = (uint32_t)gt * 16u; o < 4096u; o += kGrp * 16u)
+            if ((int)(o >> 8) >= n_tot) *reinterpret_cast<uint4*>(sStg + o) = make_uint4(0, 0, 0, 0);
+        if (gt < 2 * 128) {
+            const int sb = gt >> 6;           // 64 threads per set: 2 KB of K W operand each
+            if (sb < 2) *reinterpret_cast<uint4*>(set_ptr(sb) + sm.set_bc + (uint32_t)(gt & 63) * 32u) = make_uint4(0, 0, 0, 0),
+                        *reinterpret_cast<uint4*>(set_ptr(sb) + sm.set_bc + (uint32_t)(gt & 63) * 32u + 16u) = make_uint4(0, 0, 0, 0);
+        }
         g_sync(2);
 
         for (int k = 0; !dead; ++k) {
@@ -602,12 +611,11 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             }
             // the operand set of tile k - 2 is free once its K^T E' has completed (E' was formed before it was issued)
             if (k >= 2) {
-                if (!g_wait(2, gt, &bars[gTfull + b], (phTf >> b) & 1u)) {
+                if (!g_wait(2, gt, &bars[gTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
                     if (gt == 0) record_fault(p.status, kFaultUpdateWait, 9);
                     dead = true;
                     break;
                 }
-                phTf ^= 1u << b;
             }
             // the staged rows, gates and query row of this tile must have landed
             if (!g_wait(2, gt, &bars[gStg], phS)) {
@@ -649,14 +657,22 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             // ---- products of decays (no quotients) and the Gram matrix <k_s, k_j> ----
             if (gt < kNTok) {
                 const int s = gt;
+                float al[kNTok];
+#pragma unroll
+                for (int i = 0; i < kNTok; ++i) al[i] = sAlpha[i];
                 float pr = 1.f;                                   // Pm(j, s) = prod_{j < i <= s} alpha_i, for j = s-1 .. 0
-                for (int jj = s - 1; jj >= 0; --jj) {
-                    pr *= sAlpha[jj + 1];
-                    sPm[s * kGS + jj] = pr;
+#pragma unroll
+                for (int jj = kNTok - 2; jj >= 0; --jj) {
+                    if (jj < s) {
+                        pr *= al[jj + 1];
+                        sPm[s * kGS + jj] = pr;
+                    }
                 }
-                sCum[s] = s < n_tot ? pr * sAlpha[0] : 0.f;       // prod_{i <= s} alpha_i
+                sCum[s] = s < n_tot ? pr * al[0] : 0.f;           // prod_{i <= s} alpha_i
                 float dn = 1.f;
-                for (int i = s + 1; i < n_tot; ++i) dn *= sAlpha[i];
+#pragma unroll
+                for (int i = 1; i < kNTok; ++i)
+                    if (i > s && i < n_tot) dn *= al[i];
                 sDn[s] = s < n_tot ? dn : 0.f;
             }
             if (fwarp >= 2) {     // 16 x 16 Gram matrix from the staged keys, one 16 x 8 block per warp
@@ -723,7 +739,72 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 if (gt < kNTok) sC[gt] = sCum[gt];
                 if (gt == 0) sC[kNTok] = sCum[n_tot - 1];
             }
-            proxy_fence();         // key layouts and W are read by MMAs (async proxy)
+            // ---- W = [Omega | q | q'] (and Omega in fp32 for the product below): the Omega part once per head index.
+            // Pass A of the previous tile still reads W, so it is waited for first. ----
+            if (h != cur_h) {
+                if (k >= 1) {
+                    if (!g_wait(2, gt, &bars[gPfull + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) {
+                        if (gt == 0) record_fault(p.status, kFaultUpdateWait, 10);
+                        dead = true;
+                        break;
+                    }
+                }
+                if (p.write_sketch) {
+                    const float* og = p.omega + (size_t)h * K * R;
+                    for (int idx = gt; idx < K * R; idx += kGrp) {
+                        const int i = idx / R, g = idx - i * R;
+                        const float x = og[idx];
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(x, hi, lo);
+                        const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
+                        sWhi[o2] = hi;
+                        sWlo[o2] = lo;
+                    }
+                }
+                cur_h = h;
+                g_sync(2);
+            }
+            if (p.q != nullptr) {
+                const int i = gt, g = QA + 8 * b;
+                const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
+                sWhi[o2] = q_elem;
+            }
+            // ---- K W: 16 tokens x [Omega | q | q'] as mma.sync products of the staged keys with the hi and lo halves of W
+            // (whose K-major core matrices are exactly the 8 x 8 B fragments), hi + lo, the B operand of the sketch
+            // correction; one block of 8 columns per warp ----
+            proxy_fence();
+            g_sync(2);             // the query column and (after a change of head index) Omega are in W
+            {
+                const int nt = fwarp;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * 256u + (uint32_t)(lane >> 4) * 16u;
+                const uint32_t wbase = smem_u32(smem + sm.w) + (uint32_t)nt * SBO + (uint32_t)(lane & 7) * 16u + (uint32_t)((lane >> 3) & 1) * LBO_W;
+#pragma unroll
+                for (int ks = 0; ks < K / 16; ++ks) {
+                    uint32_t a[4], bh2[2], bl2[2];
+                    g_ldmatrix_x4(abase + ks * 32, a);
+                    g_ldmatrix_x2(wbase + (uint32_t)(ks * 2) * LBO_W, bh2);
+                    g_ldmatrix_x2(wbase + (uint32_t)NP * kK * 2u + (uint32_t)(ks * 2) * LBO_W, bl2);
+                    g_mma_16816(acc, a, bh2);
+                    g_mma_16816(acc, a, bl2);
+                }
+                __nv_bfloat16* bchi = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bc);
+                __nv_bfloat16* bclo = bchi + 512;
+                auto put = [&](int s, int g, float x) {
+                    __nv_bfloat16 hi, lo;
+                    split_bf16(x, hi, lo);
+                    const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (s >> 3) * 512 + (s & 7) * 2) >> 1;
+                    bchi[o2] = hi;
+                    bclo[o2] = lo;
+                };
+                const int r0 = lane >> 2, c0 = nt * 8 + (lane & 3) * 2;
+                put(r0, c0, acc[0]);
+                put(r0, c0 + 1, acc[1]);
+                put(r0 + 8, c0, acc[2]);
+                put(r0 + 8, c0 + 1, acc[3]);
+            }
+            const float d_cur = sCum[n_tot - 1];
+            proxy_fence();         // operand sets and W are read by MMAs (async proxy)
             g_sync(2);
             if (gt == 0) {
                 g_arrive(&bars[gPro + b]);
@@ -737,54 +818,21 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             }
             G_STAMP(256, k, 5);
 
-            // ---- sketch rows and exact output of earlier tiles.  Tile k - 2 used the same query group and accumulator
-            // half as this tile; on a change of head index W is rewritten, so tile k - 1 is finished as well. ----
+            // ---- sketch rows and exact output of tile k - 2 (it used the same slot of tensor memory as this tile) ----
             if (pend0 >= 0) {
-                if (!store_ut(pend0, b)) {
+                if (!store_ut(pend0, pk0, pd0)) {
                     if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
                     dead = true;
                     break;
                 }
-                pend0 = -1;
             }
-            if (h != cur_h) {
-                if (pend1 >= 0) {
-                    if (!store_ut(pend1, b ^ 1)) {
-                        if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
-                        dead = true;
-                        break;
-                    }
-                    pend1 = -1;
-                }
-                if (p.write_sketch) {
-                    const float* og = p.omega + (size_t)h * K * R;
-                    for (int idx = gt; idx < K * R; idx += kGrp) {
-                        const int i = idx / R, g = idx - i * R;
-                        __nv_bfloat16 hi, lo;
-                        split_bf16(og[idx], hi, lo);
-                        const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
-                        sWhi[o2] = hi;
-                        sWlo[o2] = lo;
-                    }
-                }
-                cur_h = h;
-            }
-            if (p.q != nullptr) {
-                const int i = gt, g = QA + 8 * b;
-                const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
-                sWhi[o2] = q_elem;
-            }
-            proxy_fence();
-            g_sync(2);
-            if (gt == 0) g_arrive(&bars[gProW + b]);
-            pend0 = pend1;
-            pend1 = tile;
+            pend0 = pend1; pk0 = pk1; pd0 = pd1;
+            pend1 = tile; pk1 = k; pd1 = d_cur;
             G_STAMP(256, k, 6);
         }
-        if (!dead) {      // the last one or two tiles; the newer one used buffer (tiles - 1) & 1
-            const int done = *seq_pub - 1;                    // number of tiles this CTA processed
-            if (pend0 >= 0 && !store_ut(pend0, done & 1)) { if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
-            if (!dead && pend1 >= 0 && !store_ut(pend1, (done - 1) & 1) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
+        if (!dead) {      // the last one or two tiles
+            if (pend0 >= 0 && !store_ut(pend0, pk0, pd0)) { if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
+            if (!dead && pend1 >= 0 && !store_ut(pend1, pk1, pd1) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
         }
         if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
             __threadfence();
