@@ -518,21 +518,38 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 
         const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
         const uint32_t stg_bytes = (uint32_t)n_ring * 512u + stg_gate_bytes + (p.has_token ? 512u : 0u) + (p.q != nullptr ? 256u : 0u);
-        auto stage_tile = [&](int tile) {       // one thread
+        // one bulk copy per lane of the group's first warp, from per-lane constants: ring keys, ring values, ring gates,
+        // token key, token value, query row
+        const unsigned char* cp_base = nullptr;
+        size_t cp_stride = 0;
+        uint32_t cp_dst = 0, cp_bytes = 0;
+        switch (gt) {
+            case 0: cp_base = p.ring; cp_stride = p.rl.head_bytes; cp_dst = 0; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 1: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 2: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_gate; cp_bytes = stg_gate_bytes; break;
+            case 3: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
+            case 4: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; cp_dst = sm.stg_v + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
+            case 5: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; cp_dst = sm.stg_q; cp_bytes = p.q != nullptr ? 256u : 0u; break;
+            default: break;
+        }
+        auto stage_tile = [&](int tile) {       // first warp of the group
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bw = (size_t)bb * H + h;
-            const unsigned char* rh = p.ring + bw * p.rl.head_bytes;
-            mbar_expect_tx(&bars[gStg], stg_bytes);
-            if (n_ring > 0) {
-                bulk_g2s(sStg, rh, (uint32_t)n_ring * 256u, &bars[gStg]);
-                bulk_g2s(sStg + sm.stg_v, rh + p.rl.v_off, (uint32_t)n_ring * 256u, &bars[gStg]);
-                bulk_g2s(sStg + sm.stg_gate, rh + p.rl.beta_off, stg_gate_bytes, &bars[gStg]);
+            if (gt == 0) mbar_expect_tx(&bars[gStg], stg_bytes);
+            __syncwarp();
+            if (cp_bytes) bulk_g2s(sStg + cp_dst, cp_base + bw * cp_stride, cp_bytes, &bars[gStg]);
+        };
+        // thread 0 resolves the claim, publishes it as entry k of the sequence and issues the next claim; the warp then
+        // requests the tile's rows
+        auto next_tile = [&](int k) {          // first warp of the group
+            int nxt = 0;
+            if (gt == 0) {
+                nxt = claim_resolve();
+                publish(k, nxt);
+                if (nxt >= 0) claim_issue();
             }
-            if (p.has_token) {
-                bulk_g2s(sStg + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.k) + bw * K, 256u, &bars[gStg]);
-                bulk_g2s(sStg + sm.stg_v + (size_t)n_ring * 256, reinterpret_cast<const __nv_bfloat16*>(p.v) + bw * V, 256u, &bars[gStg]);
-            }
-            if (p.q != nullptr) bulk_g2s(sStg + sm.stg_q, reinterpret_cast<const __nv_bfloat16*>(p.q) + bw * K, 256u, &bars[gStg]);
+            nxt = __shfl_sync(0xffffffffu, nxt, 0);
+            if (nxt >= 0) stage_tile(nxt);
         };
         // sketch rows and exact output of a finished tile; afterwards its accumulator half is free for the issue warp
         auto store_ut = [&](int tile, int kk, float dtile) -> bool {
@@ -564,14 +581,9 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             return true;
         };
 
-        if (gt == 0) {
-            claim_issue();
-            const int first = claim_resolve();
-            publish(0, first);
-            if (first >= 0) {
-                claim_issue();
-                stage_tile(first);
-            }
+        if (gt < 32) {
+            if (gt == 0) claim_issue();
+            next_tile(0);
         }
         // W padding columns and lo halves of the query columns hold zeros that no tile overwrites: written once
         for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGrp * 16u)
@@ -806,16 +818,8 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const float d_cur = sCum[n_tot - 1];
             proxy_fence();         // operand sets and W are read by MMAs (async proxy)
             g_sync(2);
-            if (gt == 0) {
-                g_arrive(&bars[gPro + b]);
-                // the staging buffer has been read: claim / publish the next tile and let its rows come in
-                const int nxt = claim_resolve();
-                publish(k + 1, nxt);
-                if (nxt >= 0) {
-                    claim_issue();
-                    stage_tile(nxt);
-                }
-            }
+            if (gt == 0) g_arrive(&bars[gPro + b]);
+            if (gt < 32) next_tile(k + 1);      // the staging buffer has been read: the next tile's rows may come in
             G_STAMP(256, k, 5);
 
             // ---- sketch rows and exact output of tile k - 2 (it used the same slot of tensor memory as this tile) ----
