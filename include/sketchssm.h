@@ -106,7 +106,9 @@ typedef struct sketchssm_buffers {
                       (0 = none), [1] which wait, [2..3] reserved; kernels only ever write non-zero codes
                       there and sketchssm_read_status reads them back.  The ints after them are counters
                       of the state-update kernel's tile scheduler: every launch leaves them zero again,
-                      and the caller never touches them after the initial zeroing. */
+                      and the caller never touches them after the initial zeroing.  Two state updates that
+                      overlap on the GPU therefore need separate contexts with separate status blocks
+                      (as they do anyway: they would update the same state). */
     void* work;    /* work_bytes of scratch for the decode calls (contents are transient: written and
                       consumed inside one call; calls that overlap on the GPU need separate contexts
                       with separate work buffers) */
@@ -212,13 +214,16 @@ int sketchssm_last_launch_count(const sketchssm_ctx* ctx);
 
 /* Optional launch tuning, host-only.  Keys: "decode_batches_per_cta" (batch entries one CTA of
  * the decode kernels serves for its head; 0 = library default), "decode_stages" (1 or 2 shared-memory
- * stages per lane group; 0 = library default), "decode_warps_per_cta", "decode_max_warps_per_sm",
- * "decode_lanes_per_head", "decode_l2_prefetch", "decode_mma" (1 = tensor-core dot products in the
- * warp-per-head decode where supported; 0 = off, the default), "update_impl" (0 = warp-specialised tensor-core kernels for Mamba-2 and
- * GDN where their shape limits allow and CUDA cores otherwise, the default; 1 = CUDA cores only; 2 = as 0 but the
- * single-group tensor-core kernel for GDN; 3 = single-group tensor-core kernel for Mamba-2, CUDA cores for GDN), "decode_impl" (0 = two kernels; 1 = one fused
- * kernel with a warp per head, the default; 2 = one fused kernel with 8 or 16 lanes per head).  Results depend on these
- * only through floating-point summation order. */
+ * stages per lane group of the lane-group decode kernels; for the warp-specialised update kernels an upper
+ * bound >= 2 on their shared-memory stages of state rows; 0 = library default), "decode_warps_per_cta",
+ * "decode_max_warps_per_sm" (also caps the update kernels' CTAs per SM), "decode_lanes_per_head",
+ * "decode_l2_prefetch", "decode_mma" (1 = tensor-core dot products in the warp-per-head decode where
+ * supported; 0 = off, the default), "update_impl" (0 = warp-specialised tensor-core kernels for Mamba-2 and GDN
+ * where their shape limits allow and CUDA cores otherwise, the default; 1 = CUDA cores only; 2 = as 0 but the
+ * single-group tensor-core kernel for GDN; 3 = as 0 but the single-group tensor-core kernel for Mamba-2 and CUDA
+ * cores for GDN), "decode_impl" (0 = two kernels; 1 = one fused kernel with a warp per head, the default;
+ * 2 = one fused kernel with 8 or 16 lanes per head), "pdl" (1 = programmatic dependent launch, the default).
+ * Results depend on these only through floating-point summation order. */
 int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value);
 
 const char* sketchssm_status_string(int status);

@@ -220,23 +220,25 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     p.has_token = has_token ? 1 : 0;
     p.write_sketch = sketch ? 1 : 0;
     p.write_state = n_tot > 0 ? 1 : 0;
-    if (p.update_impl == 0 || p.update_impl == 3) {
-        if (p.update_impl == 0) {       // two warp groups per CTA; falls through outside its domain (rank + heads per tile > 32)
-            rc = launch_update_tc_ws(ctx, p, static_cast<cudaStream_t>(stream));
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (p.update_impl != 1) {
+        // Mamba-2: warp-specialised tensor-core kernel, then the single-group one (ranks above 32); 3 skips the former
+        if (p.update_impl != 3) {
+            rc = launch_update_tc_ws(ctx, p, cs);
             if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
         }
-        rc = launch_update_tc(ctx, p, static_cast<cudaStream_t>(stream));
+        rc = launch_update_tc(ctx, p, cs);
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        // gated delta rule: warp-specialised tensor-core kernel (1..16 tokens, rank <= 16); 2 selects the single-group one
+        if (p.update_impl == 0) {
+            rc = launch_update_tc_ws_gdn(ctx, p, cs);
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        } else if (p.update_impl == 2) {
+            rc = launch_update_tc_delta(ctx, p, cs);
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        }
     }
-    if (p.update_impl == 0 || p.update_impl == 4) {       // gated delta rule: warp-specialised tensor-core kernel (1..16 tokens, rank <= 16)
-        rc = launch_update_tc_ws_gdn(ctx, p, static_cast<cudaStream_t>(stream));
-        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-    }
-    if (p.update_impl == 2) {       // gated delta rule, single-group tensor-core kernel (slower than the CUDA-core kernel)
-        rc = launch_update_tc_delta(ctx, p, static_cast<cudaStream_t>(stream));
-        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-    }
-    return launch_update(ctx, p, static_cast<cudaStream_t>(stream));
+    return launch_update(ctx, p, cs);
 }
 
 int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
