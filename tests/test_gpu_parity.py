@@ -178,6 +178,44 @@ def test_gdn_warp_specialised_update(tune, batch, heads, rank, buf_len):
     check(run_schedule(w, 2 * buf_len + 3, max_heads=96, tune=tune), "bf16")
 
 
+@pytest.mark.parametrize("kind,dv,buf_len,fills", [("mamba2", 64, 32, (0, 1, 15, 16, 17, 31)), ("mamba2", 128, 64, (16, 32, 47, 48, 63)),
+                                                    ("gdn", 128, 16, (0, 1, 7, 15)), ("gdn", 128, 32, (3, 15, 16, 31))])
+def test_flush_at_any_ring_fill(kind, dv, buf_len, fills):
+    """state_update with n_before tokens in the ring plus the current token, for fills around the tensor-core kernels'
+    block boundaries (16 tokens per block) and beyond their domains, and a replay without a current token."""
+    dev = _device()
+    w = synth.Workload("t", kind, 6, 3, 128, dv, 16, buf_len, 0, "bf16", 23, basis="qr")
+    bs, hs = harness.select_heads(w, 10**9)
+    toks = [synth.step_inputs(w, 0, t) for t in range(buf_len)]
+    for n_before in fills:
+        for with_token in ((True, False) if n_before > 0 else (True,)):
+            m, S0, Om, C, _ = make_layer(w)
+            m.state_update(0)
+            o = m.new_output()
+            S = S0[bs, hs].astype(np.float64)
+            Om_s = Om[hs].astype(np.float64)
+            ring = []
+            for t in range(n_before):
+                tt = harness.token_tensors(w, toks[t], dev)
+                m.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+                ring.append(harness.oracle_token(toks[t], bs, hs))
+            x = toks[n_before if with_token else n_before - 1]
+            tt = harness.token_tensors(w, x, dev)
+            q = x["q"][bs, hs].astype(np.float64)
+            if with_token:
+                ring.append(harness.oracle_token(x, bs, hs))
+                m.state_update(n_before, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+                S_ref, U_ref, o_ref = orc.state_update(w.kind, S, ring, Om_s, q)
+                got_o = o.float().cpu().numpy()[bs, hs]
+                assert harness.rel_err(got_o, o_ref) <= TOL["bf16"], (n_before, with_token)
+            else:
+                m.state_update(n_before)
+                S_ref, U_ref, _ = orc.state_update(w.kind, S, ring, Om_s, q)
+            m.check_status()
+            assert harness.rel_err(m.state.cpu().numpy()[bs, hs], S_ref) <= FP32_GUARD, (n_before, with_token)
+            assert harness.rel_err(m.sketch.cpu().numpy()[bs, hs].transpose(0, 2, 1), U_ref) <= FP32_GUARD, (n_before, with_token)
+
+
 def test_bf16_output_mode():
     w = synth.Workload("t", "gdn", 4, 2, 128, 128, 16, 8, 0, "bf16", 5, basis="qr")
     errs = run_schedule(w, 12, max_heads=10**9, out="bf16")
