@@ -326,6 +326,7 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-full-read", action="store_true")
+    ap.add_argument("--skip-graph", action="store_true")
     ap.add_argument("--tune", default="", help="comma list key=value passed to sketchssm_tune")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -416,6 +417,25 @@ def main():
     for m in stack.layers:
         m.check_status()
     value = job_value(tokens_per_step, world, ms_step)
+
+    # ---- the same step captured once in a CUDA graph and replayed (no host work between launches) ----
+    graph = None
+    if not args.skip_graph:
+        try:
+            g = torch.cuda.CUDAGraph()
+            cap_stream = torch.cuda.Stream()
+            cap_stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.graph(g, stream=cap_stream):
+                stack.run_window("sketch", None)
+            torch.cuda.current_stream().wait_stream(cap_stream)
+            ms_graph, _, _ = timed_region(g.replay, args.steps, args.warmup)
+            for m in stack.layers:
+                m.check_status()
+            graph = {"value": job_value(tokens_per_step, world, ms_graph), "unit": UNIT, "ms_per_step": ms_graph,
+                     "what": "one window over all layers captured in a CUDA graph (programmatic dependent launch edges "
+                             "included) and replayed"}
+        except Exception as exc:      # capture is a convenience measurement: report why it is missing
+            graph = {"unavailable": f"{type(exc).__name__}: {exc}"[:200]}
 
     # ---- the same region again with every launch bracketed by events: per-kernel durations ----
     events = None if args.no_launch_events else []
@@ -518,7 +538,7 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks,
                 "e2e": e2e, "gpu_launches": launches_per_step[0] * args.steps, "roofline": roofline,
-                "kernels": kern, "ms_per_step_with_launch_events": ms_step_instrumented, "full_read_baseline": full, "cpu_baseline": cpu,
+                "kernels": kern, "ms_per_step_with_launch_events": ms_step_instrumented, "full_read_baseline": full, "graph_replay": graph, "cpu_baseline": cpu,
                 "per_gpu_heads": B * H}
         print(json.dumps(line))
     if dist is not None:

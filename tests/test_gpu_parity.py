@@ -358,3 +358,41 @@ def test_repeat_runs_are_bitwise_identical():
         outs.append((o.clone(), m.state.clone(), m.sketch.clone()))
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+
+
+def test_window_replays_from_a_cuda_graph():
+    """Every call only enqueues work on the given stream, so a window can be captured in a CUDA graph; replaying it
+    reproduces the eager results bit for bit (the update kernels' run-time tile scheduler leaves its counters zero)."""
+    dev = _device()
+    w = synth.Workload("t", "mamba2", 8, 4, 128, 64, 16, 8, 0, "bf16", 31, basis="qr")
+    toks = [harness.token_tensors(w, synth.step_inputs(w, 0, t), dev) for t in range(w.buf_len)]
+
+    def window(m, outs):
+        for t, tt in enumerate(toks):
+            if t < w.buf_len - 1:
+                m.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], outs[t])
+            else:
+                m.state_update(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], outs[t])
+
+    me, *_ = make_layer(w)
+    mg, *_ = make_layer(w)
+    me.state_update(0); mg.state_update(0)
+    oe = [me.new_output() for _ in toks]
+    og = [mg.new_output() for _ in toks]
+    window(mg, og)                                  # warm-up outside capture (first-call set-up), then restore
+    torch.cuda.synchronize()
+    mg.state.copy_(me.state); mg.sketch.copy_(me.sketch)
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=s):
+        window(mg, og)
+    torch.cuda.current_stream().wait_stream(s)
+    for rep in range(2):                            # two windows eagerly and from the graph
+        window(me, oe)
+        g.replay()
+        torch.cuda.synchronize()
+        for a, b in zip(oe, og):
+            assert torch.equal(a, b)
+        assert torch.equal(me.state, mg.state) and torch.equal(me.sketch, mg.sketch)
+    me.check_status(); mg.check_status()
