@@ -46,11 +46,12 @@ using namespace tc;
 #define G_STAMP(base, k, i) do { } while (0)
 #endif
 
-constexpr int kGThreads = 320;       // stream group (4 warps), front group (4 warps), MMA issue warp, state-load warp
+constexpr int kGThreads = 448;       // pass-A group (4 warps), front group (4 warps), MMA issue warp, state-load warp, pass-B group (4 warps)
 constexpr int kGrp = 128;
 constexpr int kNTok = 16;            // tokens per flush
 constexpr int kGStages = 8;
 constexpr int kGS = 20;              // row stride (floats) of the small n x n work matrices
+constexpr uint32_t kKeyRow = 272u;   // bytes between staged key rows: 256 + 16, so that the 8 rows of an ldmatrix fall in different banks
 constexpr int kA2 = 2;               // chunk buffers between the stream group and the MMA issue warp
 
 struct GSmem {
@@ -69,9 +70,9 @@ __host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
     s.set = off;
     s.set_bt = 4096u; s.set_vv = 8192u; s.set_t1 = 12288u; s.set_bc = 13312u; s.set_gates = 15360u; s.set_stride = 15488u;
     off += 2u * s.set_stride;
-    // staging of the next tile's raw rows: keys [16][256 B], values [16][256 B], gates [2L] floats, query row
-    s.stg_v = 4096u;
-    s.stg_gate = 8192u;
+    // staging of the next tile's raw rows: keys [16][kKeyRow], values [16][256 B], gates [2L] floats, query row
+    s.stg_v = (uint32_t)kNTok * kKeyRow;
+    s.stg_gate = s.stg_v + 4096u;
     s.stg_q = s.stg_gate + (((uint32_t)(2 * L * 4) + 127u) & ~127u);
     s.stg = off; off += s.stg_q + 256u;
     s.mats = off; off += 4u * (uint32_t)kNTok * kGS * 4u + 256u;  // Gram / A, decay products, T, beta / alpha / dn
@@ -152,7 +153,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     if (tid == 0) {
         *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
         for (int i = 0; i < gNumBars; ++i) {
-            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty || i == gBdone || i == gBdone + 1;     // one arrival per stream warp
+            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty || (i >= gBdone && i < gBdone + 4);     // one arrival per warp of a stream group (gBdone, gBufFree too)
             mbar_init(&bars[i], per_warp ? 4 : 1);
         }
         mbar_fence_init();
@@ -195,21 +196,22 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     constexpr int kSepFlag = 1 << 30;
     auto set_ptr = [&](int b) { return smem + sm.set + (uint32_t)b * sm.set_stride; };
 
-    const int j = gt;                 // value column of this thread's TMEM lane (stream and front groups)
+    const int j = (warp & 3) * 32 + lane;      // value column = TMEM lane of this thread (both stream groups and the front group)
+    volatile float* sDt = reinterpret_cast<volatile float*>(smem + sm.misc + 40);      // total decay of the tile in each operand set
 
     if (warp < 4) {
-        // =========================== stream group ===========================
+        // =========================== pass-A group: S_0 chunks -> operands, and the E' step ===========================
         uint32_t phPro = 0, phP = 0, phT = 0, phA = 0, phF = 0;
-        float dt0 = 1.f, dt1 = 1.f;          // total decay of the tile in each operand set, read when E' is formed
         int gc = 0, stage = 0;
         bool bad = false;
 
-        // pass A over the 8 chunks of a tile: the S_0 chunks are split into bf16 hi + lo and handed to the issue warp,
-        // which contracts them with [Omega | q] (U0) and with the keys (P)
+        int kst = 0;
         auto pass_a = [&]() {
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
+                if (c == 3 || c == 4) G_STAMP(0, kst, 6 + (c - 3) * 4);
                 bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
+                if (c == 3 || c == 4) G_STAMP(0, kst, 7 + (c - 3) * 4);
                 const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
                 float s0[CH];
 #pragma unroll
@@ -221,6 +223,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     bad |= !mbar_wait_bounded(&bars[gA2free + ab], (phA >> ab) & 1u);
                     phA ^= 1u << ab;
                 }
+                if (c == 3 || c == 4) G_STAMP(0, kst, 8 + (c - 3) * 4);
                 unsigned char* a2hi = smem + sm.a2 + (size_t)ab * (2u * 128u * CH * 2u);
                 unsigned char* a2lo = a2hi + 128u * CH * 2u;
 #pragma unroll
@@ -235,42 +238,10 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 proxy_fence();
                 bad = __any_sync(0xffffffffu, bad);
                 if (lane == 0 && !bad) g_arrive(&bars[gA2rdy + ab]);
+                if (c == 3 || c == 4) G_STAMP(0, kst, 9 + (c - 3) * 4);
                 ++gc;
                 if (++stage == NS) { stage = 0; phF ^= 1u; }
             }
-        };
-        // pass B: S_new = d S_0 + K^T E', written back; nothing is handed on
-        auto pass_b = [&](int tile, int b) {
-            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
-            const size_t bh = (size_t)bb * H + h;
-            float* So = p.state + bh * (size_t)K * V + j;
-            const float dtot = b ? dt1 : dt0;
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
-                const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
-                float s0[CH];
-#pragma unroll
-                for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
-                float t[CH];
-                if (!bad) {
-                    tmem_ld16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), t);
-                } else {
-#pragma unroll
-                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
-                }
-                __syncwarp();
-                if (lane == 0) g_arrive(&bars[gEmpty + stage]);
-                if (!bad) {
-#pragma unroll
-                    for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = fmaf(dtot, s0[ii], t[ii]);
-                }
-                if (++stage == NS) { stage = 0; phF ^= 1u; }
-            }
-            // this warp has read its lanes of K^T E': the accumulator may be overwritten, the tile's sketch rows stored
-            tc_fence_before();
-            bad = __any_sync(0xffffffffu, bad);
-            if (lane == 0 && !bad) g_arrive(&bars[gBdone + b]);
         };
         // E'[s, j] = sum_t T1[s, t] (v_t[j] - C_t P[t, j]) -> hi + lo A operand of K^T E' (chunk-buffer layout)
         auto do_e = [&](int b) {
@@ -281,7 +252,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(set + sm.set_vv);
             const float* sT1 = reinterpret_cast<const float*>(set + sm.set_t1);
             const float* sC = reinterpret_cast<const float*>(set + sm.set_gates);
-            if (b) dt1 = sC[kNTok]; else dt0 = sC[kNTok];
+            if (lane == 0) sDt[b] = sC[kNTok];
             float x[kNTok];
             if (!bad) tmem_ld16(tmem_base + (uint32_t)b * 64u + 32u + lane_sel, x);
 #pragma unroll
@@ -323,7 +294,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 
         int cur = seq_get(0);
         if (cur >= 0) {
-            cur &= kSepFlag - 1;
             wait_pro(0);
             pass_a();
             do_e(0);
@@ -331,50 +301,121 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const int b = k & 1;
                 const int raw = seq_get(k + 1);
                 if (raw < -1) { bad = true; break; }
-                const int nxt = raw < 0 ? -1 : (raw & (kSepFlag - 1));
+                if (raw < 0) break;
                 G_STAMP(0, k, 0);
-                if (nxt >= 0) {
-                    wait_pro(b ^ 1);
-                    G_STAMP(0, k, 1);
-                    pass_a();
-                }
+                wait_pro(b ^ 1);
+                G_STAMP(0, k, 1);
+                kst = k;
+                pass_a();
                 G_STAMP(0, k, 2);
+                // the E' operand buffer is read by K^T E' of tile k: that must be complete before it is rewritten
                 bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);
                 phT ^= 1u << b;
-                tc_fence_after();
                 G_STAMP(0, k, 3);
-                pass_b(cur, b);
-                G_STAMP(0, k, 4);
-                if (nxt < 0) break;
                 do_e(b ^ 1);
                 G_STAMP(0, k, 5);
-                cur = nxt;
             }
         } else if (cur < -1) {
             bad = true;
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 3);
+    } else if (warp >= 10) {
+        // =========================== pass-B group: S_new = d S_0 + K^T E' written back, then the sketch rows ===========================
+        // S_0 is read a second time here, with plain loads one chunk ahead (the lines are in L2 since pass A), so the
+        // stage ring serves pass A alone.
+        uint32_t phT = 0;
+        bool bad = false;
+        for (int k = 0; !bad; ++k) {
+            const int raw = seq_get(k);
+            if (raw < 0) { bad = raw < -1; break; }
+            const int tile = raw & (kSepFlag - 1);
+            const int b = k & 1;
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            float* So = p.state + bh * (size_t)K * V + j;
+            float sn[CH];
+#pragma unroll
+            for (int ii = 0; ii < CH; ++ii) sn[ii] = __ldcg(So + (size_t)ii * V);
+            G_STAMP(128, k, 0);
+            bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);      // K^T E' and the sketch correction are complete
+            phT ^= 1u << b;
+            G_STAMP(128, k, 1);
+            tc_fence_after();
+            const float dtot = sDt[b];
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                float s0[CH];
+#pragma unroll
+                for (int ii = 0; ii < CH; ++ii) s0[ii] = sn[ii];
+                if (c + 1 < NCH) {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) sn[ii] = __ldcg(So + (size_t)((c + 1) * CH + ii) * V);
+                }
+                float t[CH];
+                if (!bad) {
+                    tmem_ld16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), t);
+                } else {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
+                }
+                if (!bad) {
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = fmaf(dtot, s0[ii], t[ii]);
+                }
+            }
+            G_STAMP(128, k, 2);
+            // this warp has read its lanes of K^T E': the accumulator may be overwritten
+            tc_fence_before();
+            bad = __any_sync(0xffffffffu, bad);
+            if (lane == 0 && !bad) g_arrive(&bars[gBdone + b]);
+            // [U | o] = d S_0^T W + E'^T (K W) from the tile's slot of tensor memory
+            if (!bad) {
+                const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
+                for (int g0 = 0; g0 < NP; g0 += 16) {
+                    float u0[16], cr[16];
+                    tmem_ld16(slot + (uint32_t)g0, u0);
+                    tmem_ld16(slot + 32u + (uint32_t)g0, cr);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int g = g0 + e;
+                        const float u = fmaf(dtot, u0[e], cr[e]);
+                        if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u;
+                        if (g == QA + 8 * b && p.out != nullptr) {
+                            if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
+                            else reinterpret_cast<float*>(p.out)[bh * V + j] = u;
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) g_arrive(&bars[gBufFree + b]);       // the slot is free for pass A of tile k + 2
+            }
+            G_STAMP(128, k, 3);
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 11);
     } else if (warp == 8) {
         // =========================== MMA issue warp (one thread) ===========================
         if (lane == 0) {
             uint32_t phR = 0, phE = 0, phBuf = 0;
             bool bad = false;
+            int where = 4;                  // which wait gave up (reported through the status words)
             const uint32_t sW = smem_u32(smem + sm.w);
             const uint32_t a2base = smem_u32(smem + sm.a2);
             auto pass_a = [&](int k) {          // U0(b) = S_0^T [Omega | q] and P(b) = (K S_0)^T, chunk by chunk
                 const int b = k & 1;
                 if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
-                    if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; return; }
+                    if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 4100 + k; return; }
                     phBuf ^= 1u << b;
                     tc_fence_after();
                 }
                 const uint32_t tmem_u0 = tmem_base + (uint32_t)b * 64u;
                 const uint32_t tmem_p = tmem_u0 + 32u;
                 const uint32_t bp = smem_u32(set_ptr(b));
+                G_STAMP(384, k, 0);
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     const int ab = c & (kA2 - 1);
-                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; return; }
+                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 4000 + 10 * k + c; return; }
                     phR ^= 1u << ab;
                     tc_fence_after();
                     const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
@@ -392,11 +433,17 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     tc_commit(&bars[gA2free + ab]);
                     if (c == NCH - 1) tc_commit(&bars[gPfull + b]);
                 }
+                G_STAMP(384, k, 1);
             };
             auto step_e = [&](int k) {          // T = K^T E' (128 columns) and the sketch correction E'^T (K W) over the spent P
                 const int b = k & 1;
-                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; return; }
+                G_STAMP(384, k, 2);
+                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; where = 4200 + k; return; }
                 phE ^= 1u;
+                G_STAMP(384, k, 3);
+                if (k >= 1) {                   // the pass-B group must have read K^T E' of the tile before
+                    if (!mbar_wait_bounded(&bars[gBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 4300 + k; return; }
+                }
                 tc_fence_after();
                 const uint32_t tmem_t = tmem_base + 128u;
                 const uint32_t tmem_c = tmem_base + (uint32_t)b * 64u + 32u;
@@ -413,6 +460,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 tc_mma_bf16(tmem_c, elo, bchi, idescU, 1u);
                 tc_mma_bf16(tmem_c, ehi, bclo, idescU, 1u);
                 tc_commit(&bars[gTfull + b]);
+                G_STAMP(384, k, 4);
             };
             int cur = seq_get(0);
             if (cur >= 0) {
@@ -428,7 +476,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             } else if (cur < -1) {
                 bad = true;
             }
-            if (bad) record_fault(p.status, kFaultUpdateWait, 4);
+            if (bad) record_fault(p.status, kFaultUpdateWait, where);
         }
     } else if (warp == 9) {
         // =========================== state-load warp: keeps the ring of S_0 stages full ===========================
@@ -452,18 +500,12 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         int cur = seq_get(0);
         if (cur >= 0) {
             cur &= kSepFlag - 1;
-            load_tile(cur);                       // pass A of the first tile
+            load_tile(cur);
             for (int k = 0; !bad; ++k) {
                 const int raw = seq_get(k + 1);
                 if (raw < -1) { bad = true; break; }
-                const int nxt = raw < 0 ? -1 : (raw & (kSepFlag - 1));
-                const bool sep = raw >= 0 && (raw & kSepFlag) != 0;
-                if (nxt >= 0 && !sep) load_tile(nxt);     // pass A of the next tile
-                if (bad) break;
-                load_tile(cur);                   // pass B of this tile (its state is read again, from L2)
-                if (nxt < 0) break;
-                if (sep) load_tile(nxt);
-                cur = nxt;
+                if (raw < 0) break;
+                load_tile(raw & (kSepFlag - 1));
             }
         } else if (cur < -1) {
             bad = true;
@@ -473,9 +515,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         // =========================== front group: ring-only operands, sketch stores ===========================
         const int fwarp = gt >> 5;
         int cur_h = -1;
-        int pend0 = -1, pend1 = -1;           // tiles whose sketch rows are still to be stored: older, newer
-        int pk0 = 0, pk1 = 0;                 // their positions in this CTA's tile sequence
-        float pd0 = 1.f, pd1 = 1.f;           // and their total decays
         uint32_t phS = 0;
         bool dead = false;
         float* sGm = reinterpret_cast<float*>(smem + sm.mats);
@@ -518,18 +557,21 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 
         const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
         const uint32_t stg_bytes = (uint32_t)n_ring * 512u + stg_gate_bytes + (p.has_token ? 512u : 0u) + (p.q != nullptr ? 256u : 0u);
-        // one bulk copy per lane of the group's first warp, from per-lane constants: ring keys, ring values, ring gates,
-        // token key, token value, query row
+        // one bulk copy per lane of the group's first warp, from per-lane constants: lanes 0..15 one key row each (ring
+        // rows, then the token's), lanes 16..19 ring values, ring gates, token value, query row
         const unsigned char* cp_base = nullptr;
         size_t cp_stride = 0;
         uint32_t cp_dst = 0, cp_bytes = 0;
+        if (gt < n_ring) {
+            cp_base = p.ring + (size_t)gt * 256u; cp_stride = p.rl.head_bytes; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
+        } else if (gt == n_ring && p.has_token) {
+            cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
+        }
         switch (gt) {
-            case 0: cp_base = p.ring; cp_stride = p.rl.head_bytes; cp_dst = 0; cp_bytes = (uint32_t)n_ring * 256u; break;
-            case 1: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
-            case 2: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_gate; cp_bytes = stg_gate_bytes; break;
-            case 3: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
-            case 4: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; cp_dst = sm.stg_v + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
-            case 5: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; cp_dst = sm.stg_q; cp_bytes = p.q != nullptr ? 256u : 0u; break;
+            case 16: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 17: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_gate; cp_bytes = stg_gate_bytes; break;
+            case 18: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; cp_dst = sm.stg_v + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
+            case 19: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; cp_dst = sm.stg_q; cp_bytes = p.q != nullptr ? 256u : 0u; break;
             default: break;
         }
         auto stage_tile = [&](int tile) {       // first warp of the group
@@ -552,35 +594,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             if (nxt >= 0) stage_tile(nxt);
         };
         // sketch rows and exact output of a finished tile; afterwards its accumulator half is free for the issue warp
-        auto store_ut = [&](int tile, int kk, float dtile) -> bool {
-            const int b = kk & 1;
-            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
-            const size_t bh = (size_t)bb * H + h;
-            // pass B of that tile is over (so K^T E' and the correction are complete and read)
-            if (!g_wait(2, gt, &bars[gBdone + b], (uint32_t)(kk >> 1) & 1u)) return false;
-            tc_fence_after();
-            const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
-            for (int g0 = 0; g0 < NP; g0 += 16) {
-                float u0[16], cr[16];
-                tmem_ld16(slot + (uint32_t)g0, u0);
-                tmem_ld16(slot + 32u + (uint32_t)g0, cr);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int g = g0 + e;
-                    const float u = fmaf(dtile, u0[e], cr[e]);      // [U | o] = d S_0^T W + E'^T (K W)
-                    if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u;
-                    if (g == QA + 8 * b && p.out != nullptr) {
-                        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
-                        else reinterpret_cast<float*>(p.out)[bh * V + j] = u;
-                    }
-                }
-            }
-            tc_fence_before();
-            g_sync(2);
-            if (gt == 0) g_arrive(&bars[gBufFree + b]);
-            return true;
-        };
-
         if (gt < 32) {
             if (gt == 0) claim_issue();
             next_tile(0);
@@ -590,8 +603,8 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
         // staged key rows beyond the tokens of a flush are never written by the copies: zero them once, so that the
         // products formed from all 16 rows stay finite
-        for (uint32_t o = (uint32_t)gt * 16u; o < 4096u; o += kGrp * 16u)
-            if ((int)(o >> 8) >= n_tot) *reinterpret_cast<uint4*>(sStg + o) = make_uint4(0, 0, 0, 0);
+        for (uint32_t o = (uint32_t)gt * 16u; o < (uint32_t)kNTok * kKeyRow; o += kGrp * 16u)
+            if ((int)(o / kKeyRow) >= n_tot) *reinterpret_cast<uint4*>(sStg + o) = make_uint4(0, 0, 0, 0);
         if (gt < 2 * 128) {
             const int sb = gt >> 6;           // 64 threads per set: 2 KB of K W operand each
             if (sb < 2) *reinterpret_cast<uint4*>(set_ptr(sb) + sm.set_bc + (uint32_t)(gt & 63) * 32u) = make_uint4(0, 0, 0, 0),
@@ -645,7 +658,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const int t8 = idx & 7, a = (idx >> 3) & 15, s = (idx >> 7) * 8 + t8;
                 uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
                 if (s < n_tot) {
-                    kv = *reinterpret_cast<const uint4*>(sStg + (size_t)s * 256 + a * 16);
+                    kv = *reinterpret_cast<const uint4*>(sStg + (size_t)s * kKeyRow + a * 16);
                     vv = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)s * 256 + a * 16);
                 }
                 *reinterpret_cast<uint4*>(set + (s & 7) * 16 + (s >> 3) * SBO + a * LBO_BP) = kv;                 // K-major: (n = s, k = i)
@@ -690,8 +703,8 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             if (fwarp >= 2) {     // 16 x 16 Gram matrix from the staged keys, one 16 x 8 block per warp
                 const int nt = fwarp - 2;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * 256u + (uint32_t)(lane >> 4) * 16u;
-                const uint32_t bbase = smem_u32(sStg) + (uint32_t)(nt * 8 + (lane & 7)) * 256u + (uint32_t)((lane >> 3) & 1) * 16u;
+                const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * kKeyRow + (uint32_t)(lane >> 4) * 16u;
+                const uint32_t bbase = smem_u32(sStg) + (uint32_t)(nt * 8 + (lane & 7)) * kKeyRow + (uint32_t)((lane >> 3) & 1) * 16u;
 #pragma unroll
                 for (int ks = 0; ks < K / 16; ++ks) {
                     uint32_t a[4], bbv[2];
@@ -789,7 +802,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             {
                 const int nt = fwarp;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * 256u + (uint32_t)(lane >> 4) * 16u;
+                const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * kKeyRow + (uint32_t)(lane >> 4) * 16u;
                 const uint32_t wbase = smem_u32(smem + sm.w) + (uint32_t)nt * SBO + (uint32_t)(lane & 7) * 16u + (uint32_t)((lane >> 3) & 1) * LBO_W;
 #pragma unroll
                 for (int ks = 0; ks < K / 16; ++ks) {
@@ -815,28 +828,13 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 put(r0 + 8, c0, acc[2]);
                 put(r0 + 8, c0 + 1, acc[3]);
             }
-            const float d_cur = sCum[n_tot - 1];
             proxy_fence();         // operand sets and W are read by MMAs (async proxy)
             g_sync(2);
             if (gt == 0) g_arrive(&bars[gPro + b]);
             if (gt < 32) next_tile(k + 1);      // the staging buffer has been read: the next tile's rows may come in
             G_STAMP(256, k, 5);
 
-            // ---- sketch rows and exact output of tile k - 2 (it used the same slot of tensor memory as this tile) ----
-            if (pend0 >= 0) {
-                if (!store_ut(pend0, pk0, pd0)) {
-                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
-                    dead = true;
-                    break;
-                }
-            }
-            pend0 = pend1; pk0 = pk1; pd0 = pd1;
-            pend1 = tile; pk1 = k; pd1 = d_cur;
             G_STAMP(256, k, 6);
-        }
-        if (!dead) {      // the last one or two tiles
-            if (pend0 >= 0 && !store_ut(pend0, pk0, pd0)) { if (gt == 0) record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
-            if (!dead && pend1 >= 0 && !store_ut(pend1, pk1, pd1) && gt == 0) record_fault(p.status, kFaultUpdateWait, 5);
         }
         if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
             __threadfence();
@@ -872,7 +870,7 @@ int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
         ctx->sm_count = sms;
     }
     int ctas = 2;                                             // tensor memory: 256 of the SM's 512 columns per CTA
-    if (p.max_warps_per_sm > 0 && p.max_warps_per_sm < 20) ctas = 1;
+    if (p.max_warps_per_sm > 0 && p.max_warps_per_sm < 28) ctas = 1;
     const uint32_t budget = (228u * 1024u) / (uint32_t)ctas - 1024u;
     const GSmem fixed = make_gsmem(NP, c.buf_len, 0);
     if (fixed.total + 2u * fixed.sst_bytes > budget) return SKETCHSSM_UNSUPPORTED_SHAPE;
