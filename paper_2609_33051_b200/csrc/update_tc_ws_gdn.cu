@@ -64,11 +64,13 @@ __host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
     uint32_t off = 0;
     s.a2 = off; off += (uint32_t)kA2 * 2u * 128u * 16u * 2u;      // 16-row chunk buffers, hi + lo
     s.e = off; off += 2u * 128u * 16u * 2u;                       // E' hi + lo (same layout as a chunk buffer)
-    s.w = off; off += 2u * (uint32_t)NP * kK * 2u;                // [Omega | q | q'] hi | lo
-    // per-tile operand set, double-buffered: keys as B operand of pass A (K-major) and of K^T E' (MN-major),
-    // raw value rows, T1, K [Omega | q] hi | lo (B operand of the sketch correction), gates (C diagonal, total decay)
+    // B operand of pass A, hi halves: 64 rows [keys of even tiles (16) | Omega | q | q' (NP = 32) | keys of odd tiles (16)],
+    // so that a tile's 48-row window [keys | W] or [W | keys] is one operand; then the lo halves of [Omega | q | q']
+    s.w = off; off += (64u + (uint32_t)NP) * kK * 2u;
+    // per-tile operand set, double-buffered: keys as B operand of K^T E' (MN-major), raw value rows, T1,
+    // K [Omega | q] hi | lo (B operand of the sketch correction), gates (C diagonal, total decay)
     s.set = off;
-    s.set_bt = 4096u; s.set_vv = 8192u; s.set_t1 = 12288u; s.set_bc = 13312u; s.set_gates = 15360u; s.set_stride = 15488u;
+    s.set_bt = 0u; s.set_vv = 4096u; s.set_t1 = 8192u; s.set_bc = 9216u; s.set_gates = 11264u; s.set_stride = 11392u;
     off += 2u * s.set_stride;
     // staging of the next tile's raw rows: keys [16][kKeyRow], values [16][256 B], gates [2L] floats, query row
     s.stg_v = (uint32_t)kNTok * kKeyRow;
@@ -167,14 +169,16 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
 
     // instruction descriptors: bf16 x bf16 -> fp32, M = 128
-    const uint32_t idescP = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);                 // K-major x K-major, N = 16
     const uint32_t idescT = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);    // K-major x MN-major, N = 128
     const uint32_t idescU = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)NP >> 3) << 17) | ((128u >> 4) << 24);        // K-major x K-major, N = NP
+    const uint32_t idescA = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)(NP + 16) >> 3) << 17) | ((128u >> 4) << 24);   // K-major x K-major, N = NP + 16
     // canonical no-swizzle layouts (byte offsets)
     //   K-major : elem(mn, k) at (mn%8)*16 + (mn/8)*128 + (k/8)*LBO + (k%8)*2,  LBO = 16*MN
     //   MN-major: elem(mn, k) at (k%8)*16 + (mn%8)*2 + (mn/8)*128 + (k/8)*2048
-    constexpr uint32_t SBO = 128, LBO_M = 2048, LBO_BP = 256;
-    const uint32_t LBO_W = (uint32_t)NP * 16u;
+    constexpr uint32_t SBO = 128, LBO_M = 2048;
+    constexpr uint32_t LBO_WH = 64u * 16u;                // hi halves: 64 rows
+    const uint32_t LBO_WL = (uint32_t)NP * 16u;           // lo halves: NP rows
+    const uint32_t w_lo_off = 64u * kK * 2u;              // byte offset of the lo halves in the W region
 
     const int tiles_per_h = B;
 
@@ -205,13 +209,10 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         int gc = 0, stage = 0;
         bool bad = false;
 
-        int kst = 0;
         auto pass_a = [&]() {
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-                if (c == 3 || c == 4) G_STAMP(0, kst, 6 + (c - 3) * 4);
                 bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
-                if (c == 3 || c == 4) G_STAMP(0, kst, 7 + (c - 3) * 4);
                 const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
                 float s0[CH];
 #pragma unroll
@@ -223,7 +224,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     bad |= !mbar_wait_bounded(&bars[gA2free + ab], (phA >> ab) & 1u);
                     phA ^= 1u << ab;
                 }
-                if (c == 3 || c == 4) G_STAMP(0, kst, 8 + (c - 3) * 4);
                 unsigned char* a2hi = smem + sm.a2 + (size_t)ab * (2u * 128u * CH * 2u);
                 unsigned char* a2lo = a2hi + 128u * CH * 2u;
 #pragma unroll
@@ -238,7 +238,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 proxy_fence();
                 bad = __any_sync(0xffffffffu, bad);
                 if (lane == 0 && !bad) g_arrive(&bars[gA2rdy + ab]);
-                if (c == 3 || c == 4) G_STAMP(0, kst, 9 + (c - 3) * 4);
                 ++gc;
                 if (++stage == NS) { stage = 0; phF ^= 1u; }
             }
@@ -254,7 +253,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const float* sC = reinterpret_cast<const float*>(set + sm.set_gates);
             if (lane == 0) sDt[b] = sC[kNTok];
             float x[kNTok];
-            if (!bad) tmem_ld16(tmem_base + (uint32_t)b * 64u + 32u + lane_sel, x);
+            if (!bad) tmem_ld16(tmem_base + (uint32_t)b * 64u + (b ? 32u : 16u) + lane_sel, x);
 #pragma unroll
             for (int t = 0; t < kNTok; ++t) x[t] = fmaf(-sC[t], x[t], __bfloat162float(sV[t * V + j]));
             float e[kNTok];
@@ -305,7 +304,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 G_STAMP(0, k, 0);
                 wait_pro(b ^ 1);
                 G_STAMP(0, k, 1);
-                kst = k;
                 pass_a();
                 G_STAMP(0, k, 2);
                 // the E' operand buffer is read by K^T E' of tile k: that must be complete before it is rewritten
@@ -373,8 +371,8 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
                 for (int g0 = 0; g0 < NP; g0 += 16) {
                     float u0[16], cr[16];
-                    tmem_ld16(slot + (uint32_t)g0, u0);
-                    tmem_ld16(slot + 32u + (uint32_t)g0, cr);
+                    tmem_ld16(slot + (b ? 0u : 32u) + (uint32_t)g0, u0);
+                    tmem_ld16(slot + (b ? 32u : 0u) + (uint32_t)g0, cr);
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                         const int g = g0 + e;
@@ -401,16 +399,20 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             int where = 4;                  // which wait gave up (reported through the status words)
             const uint32_t sW = smem_u32(smem + sm.w);
             const uint32_t a2base = smem_u32(smem + sm.a2);
-            auto pass_a = [&](int k) {          // U0(b) = S_0^T [Omega | q] and P(b) = (K S_0)^T, chunk by chunk
+            // [P | U0](b) = S_0^T [K^T | Omega | q] chunk by chunk.  The keys of even tiles sit before [Omega | q] in the
+            // operand and those of odd tiles after it, so each tile multiplies one 48-row window; the accumulator columns
+            // follow the window: even tiles [free 16 | P 16 | U0 32], odd tiles [U0 32 | P 16 | free 16].
+            auto pass_a = [&](int k) {
                 const int b = k & 1;
                 if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
                     if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 4100 + k; return; }
                     phBuf ^= 1u << b;
                     tc_fence_after();
                 }
-                const uint32_t tmem_u0 = tmem_base + (uint32_t)b * 64u;
-                const uint32_t tmem_p = tmem_u0 + 32u;
-                const uint32_t bp = smem_u32(set_ptr(b));
+                const uint32_t slot = tmem_base + (uint32_t)b * 64u;
+                const uint32_t tmem_win = slot + (b ? 0u : 16u);
+                const uint32_t tmem_u0 = slot + (b ? 0u : 32u);
+                const uint32_t win = sW + (b ? 2u : 0u) * SBO;
                 G_STAMP(384, k, 0);
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
@@ -419,17 +421,13 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     phR ^= 1u << ab;
                     tc_fence_after();
                     const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
-                    const uint32_t kb = (uint32_t)(c * (CH / 8)) * LBO_W;
                     const uint64_t ahi = make_desc(a2, LBO_M, SBO);
                     const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
-                    const uint64_t whi = make_desc(sW + kb, LBO_W, SBO);
-                    const uint64_t wlo = make_desc(sW + (uint32_t)NP * kK * 2u + kb, LBO_W, SBO);
-                    const uint64_t bk = make_desc(bp + (uint32_t)(c * 2) * LBO_BP, LBO_BP, SBO);
-                    tc_mma_bf16(tmem_u0, ahi, whi, idescU, c ? 1u : 0u);
-                    tc_mma_bf16(tmem_u0, alo, whi, idescU, 1u);
+                    const uint64_t whi = make_desc(win + (uint32_t)(c * (CH / 8)) * LBO_WH, LBO_WH, SBO);
+                    const uint64_t wlo = make_desc(sW + w_lo_off + (uint32_t)(c * (CH / 8)) * LBO_WL, LBO_WL, SBO);
+                    tc_mma_bf16(tmem_win, ahi, whi, idescA, c ? 1u : 0u);
+                    tc_mma_bf16(tmem_win, alo, whi, idescA, 1u);
                     tc_mma_bf16(tmem_u0, ahi, wlo, idescU, 1u);
-                    tc_mma_bf16(tmem_p, ahi, bk, idescP, c ? 1u : 0u);
-                    tc_mma_bf16(tmem_p, alo, bk, idescP, 1u);
                     tc_commit(&bars[gA2free + ab]);
                     if (c == NCH - 1) tc_commit(&bars[gPfull + b]);
                 }
@@ -446,7 +444,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 }
                 tc_fence_after();
                 const uint32_t tmem_t = tmem_base + 128u;
-                const uint32_t tmem_c = tmem_base + (uint32_t)b * 64u + 32u;
+                const uint32_t tmem_c = tmem_base + (uint32_t)b * 64u + (b ? 32u : 0u);      // over the spent P and the free columns
                 const uint32_t e = smem_u32(smem + sm.e);
                 const uint64_t ehi = make_desc(e, LBO_M, SBO);
                 const uint64_t elo = make_desc(e + 128u * CH * 2u, LBO_M, SBO);
@@ -525,7 +523,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         float* sDn = sAlpha + kNTok;
         float* sCum = sDn + kNTok;
         __nv_bfloat16* sWhi = reinterpret_cast<__nv_bfloat16*>(smem + sm.w);
-        __nv_bfloat16* sWlo = sWhi + (size_t)NP * kK;
+        __nv_bfloat16* sWlo = sWhi + (size_t)64 * kK;
 
         // ---- tile claiming (thread 0 of the group): per-head-index counters behind the status words ----
         int* sched = p.status + kStatusInts;
@@ -599,7 +597,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             next_tile(0);
         }
         // W padding columns and lo halves of the query columns hold zeros that no tile overwrites: written once
-        for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGrp * 16u)
+        for (uint32_t o = (uint32_t)gt * 16u; o < (64u + (uint32_t)NP) * kK * 2u; o += kGrp * 16u)
             *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
         // staged key rows beyond the tokens of a flush are never written by the copies: zero them once, so that the
         // products formed from all 16 rows stay finite
@@ -661,7 +659,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     kv = *reinterpret_cast<const uint4*>(sStg + (size_t)s * kKeyRow + a * 16);
                     vv = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)s * 256 + a * 16);
                 }
-                *reinterpret_cast<uint4*>(set + (s & 7) * 16 + (s >> 3) * SBO + a * LBO_BP) = kv;                 // K-major: (n = s, k = i)
+                *reinterpret_cast<uint4*>(smem + sm.w + (s & 7) * 16 + ((s >> 3) + (b ? 6 : 0)) * SBO + a * LBO_WH) = kv;   // K-major, rows (b ? 48 : 0) + s of W
                 *reinterpret_cast<uint4*>(set + sm.set_bt + (s & 7) * 16 + a * SBO + (s >> 3) * LBO_M) = kv;      // MN-major: (mn = i, k = s)
                 *reinterpret_cast<uint4*>(set + sm.set_vv + (size_t)s * 256 + a * 16) = vv;
             }
@@ -781,9 +779,9 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                         const float x = og[idx];
                         __nv_bfloat16 hi, lo;
                         split_bf16(x, hi, lo);
-                        const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
-                        sWhi[o2] = hi;
-                        sWlo[o2] = lo;
+                        const uint32_t oc = (g & 7) * 16 + (g >> 3) * SBO + (i & 7) * 2;
+                        sWhi[(oc + 2u * SBO + (i >> 3) * LBO_WH) >> 1] = hi;
+                        sWlo[(oc + (i >> 3) * LBO_WL) >> 1] = lo;
                     }
                 }
                 cur_h = h;
@@ -791,7 +789,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             }
             if (p.q != nullptr) {
                 const int i = gt, g = QA + 8 * b;
-                const uint32_t o2 = ((g & 7) * 16 + (g >> 3) * SBO + (i >> 3) * LBO_W + (i & 7) * 2) >> 1;
+                const uint32_t o2 = ((g & 7) * 16 + ((g >> 3) + 2) * SBO + (i >> 3) * LBO_WH + (i & 7) * 2) >> 1;
                 sWhi[o2] = q_elem;
             }
             // ---- K W: 16 tokens x [Omega | q | q'] as mma.sync products of the staged keys with the hi and lo halves of W
@@ -803,13 +801,15 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const int nt = fwarp;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t abase = smem_u32(sStg) + (uint32_t)(lane & 15) * kKeyRow + (uint32_t)(lane >> 4) * 16u;
-                const uint32_t wbase = smem_u32(smem + sm.w) + (uint32_t)nt * SBO + (uint32_t)(lane & 7) * 16u + (uint32_t)((lane >> 3) & 1) * LBO_W;
+                const uint32_t wrow = smem_u32(smem + sm.w) + (uint32_t)nt * SBO + (uint32_t)(lane & 7) * 16u;
+                const uint32_t whbase = wrow + 2u * SBO + (uint32_t)((lane >> 3) & 1) * LBO_WH;
+                const uint32_t wlbase = wrow + w_lo_off + (uint32_t)((lane >> 3) & 1) * LBO_WL;
 #pragma unroll
                 for (int ks = 0; ks < K / 16; ++ks) {
                     uint32_t a[4], bh2[2], bl2[2];
                     g_ldmatrix_x4(abase + ks * 32, a);
-                    g_ldmatrix_x2(wbase + (uint32_t)(ks * 2) * LBO_W, bh2);
-                    g_ldmatrix_x2(wbase + (uint32_t)NP * kK * 2u + (uint32_t)(ks * 2) * LBO_W, bl2);
+                    g_ldmatrix_x2(whbase + (uint32_t)(ks * 2) * LBO_WH, bh2);
+                    g_ldmatrix_x2(wlbase + (uint32_t)(ks * 2) * LBO_WL, bl2);
                     g_mma_16816(acc, a, bh2);
                     g_mma_16816(acc, a, bl2);
                 }
