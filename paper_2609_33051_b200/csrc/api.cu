@@ -229,7 +229,7 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
         }
         rc = launch_update_tc(ctx, p, cs);
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        // gated delta rule: warp-specialised tensor-core kernel (1..16 tokens, rank <= 16); 2 selects the single-group one
+        // gated delta rule: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 16, rank <= 16); 2 selects the single-group one
         if (p.update_impl == 0) {
             rc = launch_update_tc_ws_gdn(ctx, p, cs);
             if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;

@@ -71,6 +71,7 @@ struct Params {
                           // 3: as 0 but without the warp-specialised kernels (single-group Mamba-2 kernel, CUDA cores for GDN)
     int decode_mma;       // warp-per-head decode: 1 = tensor-core dot products where supported
     int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
+    int tok_base;         // update (GDN tensor-core kernel): first ring row of this pass when a flush is replayed in blocks of 16 tokens
 };
 
 int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head

@@ -10,22 +10,28 @@
 // Every product of decays is built by multiplication (no quotients), and all tensor-core operands that come from the
 // ring are the raw bf16 keys, so those products are exact; fp32 operands (S_0, S_new, E') are split into bf16 hi + lo.
 //
-// Tile = one head (K = V = 128); TMEM lane = value column j.  The state is streamed twice through a ring of
-// shared-memory stages filled by bulk copies (TMA): pass A contracts S_0 with the keys (P), pass B forms S_new from
-// S_0 (read again, from L2) and K^T E' and contracts it with [Omega | q].  The CTA is specialised like the Mamba-2
-// kernel: a front group builds the ring-only operands (Gram matrix, T1, key layouts) one tile ahead and stores the
-// sketch rows of the tile before; a stream group does the per-element work of both passes and the small E' step;
-// one thread issues every MMA; one warp keeps the stages full.  Passes of consecutive tiles are interleaved
-// (A(i+1) runs between E'(i) and B(i)), so no MMA round trip is waited for.
+// Tile = one head (K = V = 128); TMEM lane = value column j.  The state is read twice: pass A contracts S_0 (from a ring
+// of shared-memory stages filled by bulk copies) with the keys (P) and with W = [Omega | q]; pass B forms
+// S_new = d S_0 + K^T E' from S_0 read again (plain loads, from L2) and writes it back.  The CTA is specialised:
+//   front group (4 warps)   ring-only operands two tiles ahead: key layouts, Gram matrix, T1, K W, tile claiming
+//   pass-A group (4 warps)  S_0 chunks -> bf16 hi + lo operands, then the small E' step
+//   pass-B group (4 warps)  S_new written back, then the sketch rows and the exact output from tensor memory
+//   one thread issues every MMA; one warp keeps the stages full.
+// Pass A of tile i + 1 runs while pass B of tile i does, so no MMA round trip is waited for.
 //
-// The sketch rows never need S_new as a tensor-core operand: [U | o] = d S_0^T W + E'^T (K W) with W = [Omega | q], so
-// pass A contracts the S_0 chunks with W as well (same hi + lo operand as for P), the small product K W is formed by
-// the front group, and the correction E'^T (K W) rides along with K^T E'.  Pass B is then only
-// S_new = d S_0 + K^T E' written back: no split, no operand hand-off, no MMA.
-// Tensor memory per CTA (256 columns): two 64-column slots [U0 (32) | P (16), later the correction (32)] for
-// alternating tiles, and one 128-column accumulator for K^T E'.
+// The sketch rows never need S_new as a tensor-core operand: [U | o] = d S_0^T W + E'^T (K W), so pass A contracts the
+// S_0 chunks with the keys and W in one product (the keys sit next to W in shared memory: a 48-row operand window per
+// tile), the small product K W is formed by the front group, and the correction E'^T (K W) rides along with K^T E'.
+// Pass B is then only S_new = d S_0 + K^T E': no split, no operand hand-off, no MMA.
+// Tensor memory per CTA (256 columns): two 64-column slots for alternating tiles ([U0 32 | P 16 | free 16] or
+// [free 16 | P 16 | U0 32]; the correction later goes over P and the free columns), and one 128-column accumulator
+// for K^T E'.
 //
-// Domain: GDN, bf16 I/O, K = V = 128, 1..16 tokens per flush, rank <= 16.
+// Shared memory is the busiest unit of this kernel (load/store data pipe ~70 % busy): the staged key rows are padded so
+// that ldmatrix reads them without bank conflicts.
+//
+// Domain: GDN, bf16 I/O, K = V = 128, rank <= 16; 1..16 tokens per pass, up to 64 tokens per flush in blocks of 16
+// (one pass over the state per block).
 #include "internal.cuh"
 #include "tc_common.cuh"
 
@@ -139,7 +145,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     const int QA = (R + 7) & ~7;                          // first column of query group A; group B follows 8 columns later
     const int NP = (QA + 16 + 15) & ~15;                  // <= 32 (checked by the launcher)
     const int NS = p.stages;
-    const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);     // 1..16 (checked by the launcher)
+    const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);     // 1..16 per pass (the launcher sees to it)
     const GSmem sm = make_gsmem(NP, p.L, NS);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.misc);
@@ -396,7 +402,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         if (lane == 0) {
             uint32_t phR = 0, phE = 0, phBuf = 0;
             bool bad = false;
-            int where = 4;                  // which wait gave up (reported through the status words)
+            int where = 4;                  // which wait gave up (status detail): 41 slot free, 42 chunk ready, 43 E' ready, 44 K^T E' read
             const uint32_t sW = smem_u32(smem + sm.w);
             const uint32_t a2base = smem_u32(smem + sm.a2);
             // [P | U0](b) = S_0^T [K^T | Omega | q] chunk by chunk.  The keys of even tiles sit before [Omega | q] in the
@@ -405,7 +411,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             auto pass_a = [&](int k) {
                 const int b = k & 1;
                 if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
-                    if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 4100 + k; return; }
+                    if (!mbar_wait_bounded(&bars[gBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 41; return; }
                     phBuf ^= 1u << b;
                     tc_fence_after();
                 }
@@ -417,7 +423,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     const int ab = c & (kA2 - 1);
-                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 4000 + 10 * k + c; return; }
+                    if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 42; return; }
                     phR ^= 1u << ab;
                     tc_fence_after();
                     const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
@@ -436,11 +442,11 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             auto step_e = [&](int k) {          // T = K^T E' (128 columns) and the sketch correction E'^T (K W) over the spent P
                 const int b = k & 1;
                 G_STAMP(384, k, 2);
-                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; where = 4200 + k; return; }
+                if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; where = 43; return; }
                 phE ^= 1u;
                 G_STAMP(384, k, 3);
                 if (k >= 1) {                   // the pass-B group must have read K^T E' of the tile before
-                    if (!mbar_wait_bounded(&bars[gBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 4300 + k; return; }
+                    if (!mbar_wait_bounded(&bars[gBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 44; return; }
                 }
                 tc_fence_after();
                 const uint32_t tmem_t = tmem_base + 128u;
@@ -561,12 +567,12 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         size_t cp_stride = 0;
         uint32_t cp_dst = 0, cp_bytes = 0;
         if (gt < n_ring) {
-            cp_base = p.ring + (size_t)gt * 256u; cp_stride = p.rl.head_bytes; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
+            cp_base = p.ring + (size_t)(p.tok_base + gt) * 256u; cp_stride = p.rl.head_bytes; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
         } else if (gt == n_ring && p.has_token) {
             cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
         }
         switch (gt) {
-            case 16: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 16: cp_base = p.ring + p.rl.v_off + (size_t)p.tok_base * 256u; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
             case 17: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_gate; cp_bytes = stg_gate_bytes; break;
             case 18: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; cp_dst = sm.stg_v + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
             case 19: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; cp_dst = sm.stg_q; cp_bytes = p.q != nullptr ? 256u : 0u; break;
@@ -669,7 +675,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const int s = gt;
                 const float* sg = reinterpret_cast<const float*>(sStg + sm.stg_gate);
                 float bt = 0.f, al = 1.f;
-                if (s < n_ring) { bt = sg[s]; al = sg[p.L + s]; }
+                if (s < n_ring) { bt = sg[p.tok_base + s]; al = sg[p.L + p.tok_base + s]; }
                 else if (s < n_tot) { bt = tok_beta; al = tok_a; }
                 sBeta[s] = bt;
                 sAlpha[s] = al;
@@ -853,22 +859,11 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     }
 }
 
-// Returns SKETCHSSM_UNSUPPORTED_SHAPE outside this kernel's domain (the caller then uses another kernel).
-int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+// One pass of the kernel over all tiles: ring rows tok_base .. tok_base + n_before - 1 (and the current token).
+static int launch_gdn_pass(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
     const sketchssm_config& c = ctx->cfg;
-    if (c.kind != SKETCHSSM_GDN || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK || c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    if (c.rank > 16) return SKETCHSSM_UNSUPPORTED_SHAPE;
     Params p = p_in;
-    const int n_tot = p.n_before + (p.has_token ? 1 : 0);
-    if (n_tot < 1 || n_tot > kNTok) return SKETCHSSM_UNSUPPORTED_SHAPE;
     const int NP = ((((c.rank + 7) & ~7) + 16) + 15) & ~15;
-    if (ctx->sm_count == 0) {
-        int dev = 0, sms = 0;
-        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
-        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
-            return SKETCHSSM_CUDA_ERROR;
-        ctx->sm_count = sms;
-    }
     int ctas = 2;                                             // tensor memory: 256 of the SM's 512 columns per CTA
     if (p.max_warps_per_sm > 0 && p.max_warps_per_sm < 28) ctas = 1;
     const uint32_t budget = (228u * 1024u) / (uint32_t)ctas - 1024u;
@@ -888,7 +883,42 @@ int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
         return SKETCHSSM_CUDA_ERROR;
     if ((ctx->last_cuda_error = launch_kernel(kern, dim3((unsigned)grid), dim3(kGThreads), sm.total, stream, p, p.pdl != 0)) != cudaSuccess)
         return SKETCHSSM_CUDA_ERROR;
-    ctx->last_launches = 1;
+    return SKETCHSSM_OK;
+}
+
+// Returns SKETCHSSM_UNSUPPORTED_SHAPE outside this kernel's domain (the caller then uses another kernel).  A flush of more
+// than 16 tokens is replayed in blocks of 16: every block is one pass over the state, and only the last one (which holds
+// the current token) writes the sketch and the exact output.
+int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+    const sketchssm_config& c = ctx->cfg;
+    if (c.kind != SKETCHSSM_GDN || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK || c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (c.rank > 16) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int n_tot = p_in.n_before + (p_in.has_token ? 1 : 0);
+    if (n_tot < 1 || n_tot > 4 * kNTok) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (ctx->sm_count == 0) {
+        int dev = 0, sms = 0;
+        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return SKETCHSSM_CUDA_ERROR;
+        ctx->sm_count = sms;
+    }
+    const int passes = (n_tot + kNTok - 1) / kNTok;
+    for (int ps = 0; ps < passes; ++ps) {
+        Params p = p_in;
+        p.tok_base = ps * kNTok;
+        if (ps + 1 < passes) {          // 16 ring rows, state only
+            p.n_before = kNTok;
+            p.has_token = 0;
+            p.q = nullptr;
+            p.out = nullptr;
+            p.write_sketch = 0;
+        } else {
+            p.n_before = p_in.n_before - ps * kNTok;
+        }
+        const int rc = launch_gdn_pass(ctx, p, stream);
+        if (rc != SKETCHSSM_OK) return rc;
+    }
+    ctx->last_launches = passes;
     return SKETCHSSM_OK;
 }
 

@@ -69,7 +69,8 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32"):
             m.state_update(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
             S, U, ref = orc.state_update(w.kind, S, ring, Om_s, q)
             ring = []
-        assert m.last_launch_count() in (1, 2)   # the two-kernel decode launches twice
+        # the two-kernel decode launches twice; a GDN flush of more than 16 tokens is one launch per block of 16
+        assert 1 <= m.last_launch_count() <= max(2, (w.buf_len + 15) // 16)
         got = o_dev.float().cpu().numpy()[bs, hs]
         assert np.all(np.isfinite(got))
         worst = max(worst, harness.rel_err(got, ref))
@@ -170,10 +171,12 @@ def test_gdn_tensor_core_update(rank, buf_len, steps):
 
 
 @pytest.mark.parametrize("tune", [{}, {"decode_max_warps_per_sm": 10}, {"pdl": 0}])
-@pytest.mark.parametrize("batch,heads,rank,buf_len", [(5, 3, 16, 16), (40, 20, 16, 16), (33, 7, 8, 12), (6, 2, 5, 4)])
+@pytest.mark.parametrize("batch,heads,rank,buf_len", [(5, 3, 16, 16), (40, 20, 16, 16), (33, 7, 8, 12), (6, 2, 5, 4),
+                                                      (12, 4, 16, 32), (7, 3, 12, 40), (5, 2, 16, 64)])
 def test_gdn_warp_specialised_update(tune, batch, heads, rank, buf_len):
     """Warp-specialised tcgen05 flush of the gated delta rule (two passes over the state, interleaved across tiles,
-    tiles claimed at run time) against the oracle's token-by-token replay, over two windows."""
+    tiles claimed at run time; windows of more than 16 tokens replayed in blocks of 16) against the oracle's
+    token-by-token replay, over two windows."""
     w = synth.Workload("t", "gdn", batch, heads, 128, 128, rank, buf_len, 0, "bf16", 93, basis="qr")
     check(run_schedule(w, 2 * buf_len + 3, max_heads=96, tune=tune), "bf16")
 
