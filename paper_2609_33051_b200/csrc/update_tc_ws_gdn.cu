@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         bool bad = false;
 
         auto pass_a = [&]() {
-#pragma unroll
+#pragma unroll 2
             for (int c = 0; c < NCH; ++c) {
                 bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
                 const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             G_STAMP(128, k, 1);
             tc_fence_after();
             const float dtot = sDt[b];
-#pragma unroll
+#pragma unroll 2
             for (int c = 0; c < NCH; ++c) {
                 float s0[CH];
 #pragma unroll
@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const uint32_t tmem_u0 = slot + (b ? 0u : 32u);
                 const uint32_t win = sW + (b ? 2u : 0u) * SBO;
                 G_STAMP(384, k, 0);
-#pragma unroll
+#pragma unroll 2
                 for (int c = 0; c < NCH; ++c) {
                     const int ab = c & (kA2 - 1);
                     if (!mbar_wait_bounded(&bars[gA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 42; return; }
