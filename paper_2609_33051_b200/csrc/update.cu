@@ -25,6 +25,26 @@ struct PaddedRow {
     __host__ __device__ static constexpr int at(int i) { return i + 4 * (i / RP); }
 };
 
+// Packed pairs of fp32 (sm_100: one instruction for two independent IEEE operations): the replay loops are bound by
+// instruction issue, and a column's rows are independent.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 struct UpdateSmem {
     uint32_t k_off, g_off, v_off, beta_off, dec_off, q_off, om_off, total;
 };
@@ -143,62 +163,71 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const Params p) {
         __syncthreads();
         if (n_tot > 0) {
             const float d = s_total;
+            f32x2 c2[RP / 2];
 #pragma unroll
-            for (int ii = 0; ii < RP; ++ii) col[ii] *= d;
+            for (int i2 = 0; i2 < RP / 2; ++i2) c2[i2] = pack2(col[2 * i2] * d, col[2 * i2 + 1] * d);
             for (int s = 0; s < n_tot; ++s) {
                 const float w = sBeta[s] * sV[s * kVT + jl];
+                const f32x2 w2 = pack2(w, w);
                 const float4* kp = reinterpret_cast<const float4*>(sK + s * PR::stride + part * (RP + 4));
 #pragma unroll
                 for (int i4 = 0; i4 < RP / 4; ++i4) {
                     const float4 kq = kp[i4];
-                    col[4 * i4 + 0] = fmaf(kq.x, w, col[4 * i4 + 0]);
-                    col[4 * i4 + 1] = fmaf(kq.y, w, col[4 * i4 + 1]);
-                    col[4 * i4 + 2] = fmaf(kq.z, w, col[4 * i4 + 2]);
-                    col[4 * i4 + 3] = fmaf(kq.w, w, col[4 * i4 + 3]);
+                    c2[2 * i4] = fma2(pack2(kq.x, kq.y), w2, c2[2 * i4]);
+                    c2[2 * i4 + 1] = fma2(pack2(kq.z, kq.w), w2, c2[2 * i4 + 1]);
                 }
             }
+#pragma unroll
+            for (int i2 = 0; i2 < RP / 2; ++i2) unpack2(c2[i2], col[2 * i2], col[2 * i2 + 1]);
         }
     } else {
+        f32x2 c2[RP / 2];
+#pragma unroll
+        for (int i2 = 0; i2 < RP / 2; ++i2) c2[i2] = pack2(col[2 * i2], col[2 * i2 + 1]);
         for (int s = 0; s < n_tot; ++s) {
             const float4* kp = reinterpret_cast<const float4*>(sK + s * PR::stride + part * (RP + 4));
-            float dot0 = 0.f, dot1 = 0.f;
+            f32x2 k2[RP / 2];
+#pragma unroll
+            for (int i4 = 0; i4 < RP / 4; ++i4) {
+                const float4 kq = kp[i4];
+                k2[2 * i4] = pack2(kq.x, kq.y);
+                k2[2 * i4 + 1] = pack2(kq.z, kq.w);
+            }
+            f32x2 dot01 = pack2(0.f, 0.f), dot23 = dot01;
             if constexpr (KIND == SKETCHSSM_GDN) {
                 const float a = sDec[s];
+                const f32x2 a2 = pack2(a, a);
 #pragma unroll
                 for (int i4 = 0; i4 < RP / 4; ++i4) {
-                    const float4 kq = kp[i4];
-                    col[4 * i4 + 0] *= a; col[4 * i4 + 1] *= a; col[4 * i4 + 2] *= a; col[4 * i4 + 3] *= a;
-                    dot0 = fmaf(kq.x, col[4 * i4 + 0], dot0);
-                    dot1 = fmaf(kq.y, col[4 * i4 + 1], dot1);
-                    dot0 = fmaf(kq.z, col[4 * i4 + 2], dot0);
-                    dot1 = fmaf(kq.w, col[4 * i4 + 3], dot1);
+                    c2[2 * i4] = mul2(c2[2 * i4], a2);
+                    c2[2 * i4 + 1] = mul2(c2[2 * i4 + 1], a2);
+                    dot01 = fma2(k2[2 * i4], c2[2 * i4], dot01);
+                    dot23 = fma2(k2[2 * i4 + 1], c2[2 * i4 + 1], dot23);
                 }
             } else {
                 const float4* gp = reinterpret_cast<const float4*>(sG + s * PR::stride + part * (RP + 4));
 #pragma unroll
                 for (int i4 = 0; i4 < RP / 4; ++i4) {
-                    const float4 kq = kp[i4];
                     const float4 gq = gp[i4];
-                    col[4 * i4 + 0] *= gq.x; col[4 * i4 + 1] *= gq.y; col[4 * i4 + 2] *= gq.z; col[4 * i4 + 3] *= gq.w;
-                    dot0 = fmaf(kq.x, col[4 * i4 + 0], dot0);
-                    dot1 = fmaf(kq.y, col[4 * i4 + 1], dot1);
-                    dot0 = fmaf(kq.z, col[4 * i4 + 2], dot0);
-                    dot1 = fmaf(kq.w, col[4 * i4 + 3], dot1);
+                    c2[2 * i4] = mul2(c2[2 * i4], pack2(gq.x, gq.y));
+                    c2[2 * i4 + 1] = mul2(c2[2 * i4 + 1], pack2(gq.z, gq.w));
+                    dot01 = fma2(k2[2 * i4], c2[2 * i4], dot01);
+                    dot23 = fma2(k2[2 * i4 + 1], c2[2 * i4 + 1], dot23);
                 }
             }
-            float dot = dot0 + dot1;
+            float d0, d1, d2, d3;
+            unpack2(dot01, d0, d1);
+            unpack2(dot23, d2, d3);
+            float dot = (d0 + d2) + (d1 + d3);
             dot += __shfl_xor_sync(0xffffffffu, dot, 8);
             dot += __shfl_xor_sync(0xffffffffu, dot, 16);
             const float e = sBeta[s] * (sV[s * kVT + jl] - dot);
+            const f32x2 e2 = pack2(e, e);
 #pragma unroll
-            for (int i4 = 0; i4 < RP / 4; ++i4) {
-                const float4 kq = kp[i4];
-                col[4 * i4 + 0] = fmaf(kq.x, e, col[4 * i4 + 0]);
-                col[4 * i4 + 1] = fmaf(kq.y, e, col[4 * i4 + 1]);
-                col[4 * i4 + 2] = fmaf(kq.z, e, col[4 * i4 + 2]);
-                col[4 * i4 + 3] = fmaf(kq.w, e, col[4 * i4 + 3]);
-            }
+            for (int i2 = 0; i2 < RP / 2; ++i2) c2[i2] = fma2(k2[i2], e2, c2[i2]);
         }
+#pragma unroll
+        for (int i2 = 0; i2 < RP / 2; ++i2) unpack2(c2[i2], col[2 * i2], col[2 * i2 + 1]);
     }
 
     // ---- write the updated tile back ----
