@@ -58,7 +58,7 @@ constexpr int kNTok = 16;            // tokens per flush
 constexpr int kGStages = 8;
 constexpr int kGS = 20;              // row stride (floats) of the small n x n work matrices
 constexpr uint32_t kKeyRow = 272u;   // bytes between staged key rows: 256 + 16, so that the 8 rows of an ldmatrix fall in different banks
-constexpr int kA2 = 2;               // chunk buffers between the stream group and the MMA issue warp
+constexpr int kA2 = 2;               // chunk buffers between the pass-A group and the MMA issue warp
 
 struct GSmem {
     uint32_t a2, e, w, set, set_stride, set_bt, set_vv, set_t1, set_bc, set_gates, stg, stg_v, stg_gate, stg_q, mats, bars,
@@ -475,7 +475,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     if (raw < -1) { bad = true; break; }
                     if (raw >= 0) pass_a(k + 1);
                     if (raw < 0 || bad) break;
-                    step_e(k + 1);       // the stream group forms E'(k + 1) after its pass B of tile k
+                    step_e(k + 1);       // the pass-A group forms E'(k + 1) right after pass A of tile k + 1
                 }
             } else if (cur < -1) {
                 bad = true;
@@ -516,7 +516,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 7);
     } else {
-        // =========================== front group: ring-only operands, sketch stores ===========================
+        // =========================== front group: ring-only operands, tile claiming ===========================
         const int fwarp = gt >> 5;
         int cur_h = -1;
         uint32_t phS = 0;
@@ -597,7 +597,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             nxt = __shfl_sync(0xffffffffu, nxt, 0);
             if (nxt >= 0) stage_tile(nxt);
         };
-        // sketch rows and exact output of a finished tile; afterwards its accumulator half is free for the issue warp
+        // the first tile: claimed, published and its rows requested before anything else
         if (gt < 32) {
             if (gt == 0) claim_issue();
             next_tile(0);
