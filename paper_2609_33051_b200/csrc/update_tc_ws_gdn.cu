@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             for (int s = 0; s < kNTok; ++s) {
                 float acc = 0.f;
 #pragma unroll
-                for (int t4 = 0; t4 < kNTok / 4; ++t4) {
+                for (int t4 = 0; t4 <= s / 4; ++t4) {      // T1 is lower triangular
                     const float4 tt = *reinterpret_cast<const float4*>(sT1 + s * kNTok + t4 * 4);
                     acc = fmaf(tt.x, x[t4 * 4], acc);
                     acc = fmaf(tt.y, x[t4 * 4 + 1], acc);
