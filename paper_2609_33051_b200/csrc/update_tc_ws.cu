@@ -657,8 +657,9 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                     phB ^= 1;
                     tc_fence_after();
                 }
-                // Operand rows are written 16 bytes per thread; consecutive threads walk the 8 token rows of a core matrix
-                // first and then the next 8-element vector, so that a warp writes 512 contiguous bytes (no bank conflicts).
+                // Operand rows are moved 16 bytes per thread.  The 8 lanes of a quarter warp take the 8 token rows of a core
+                // matrix, each at a different 8-element vector (a diagonal), so that neither the reads of the staged rows
+                // (row pitch 256 or 128 bytes) nor the writes of the core matrices meet in a bank.
                 {
                     // rows come from the block's staging buffer; only the diagonal head blocks of A are written
                     if (blk > 0 && staging) {      // (the first block was waited for above)
@@ -675,7 +676,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 #pragma unroll
                     for (int r = 0; r < NB; ++r) {
                         const int idx = gt + r * kGroup;
-                        const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
+                        const int a = ((idx >> 3) + (idx & 7)) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
                         const int hd = sp / kTokBlock, s = sp % kTokBlock;
                         kv[r] = s_base + s < n_tot ? *reinterpret_cast<const uint4*>(sBlk + (size_t)hd * sm.stg_blk_head + (size_t)s * 256 + a * 16)
                                                    : make_uint4(0, 0, 0, 0);
@@ -686,7 +687,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 #pragma unroll
                     for (int r = 0; r < NA; ++r) {
                         const int it = gt + r * kGroup;
-                        const int t8 = it & 7, a = (it >> 3) % (V / 8), rest = it / V;
+                        const int t8 = it & 7, a = ((it >> 3) + t8) % (V / 8), rest = it / V;
                         const int hd = rest >> 1, s = (rest & 1) * 8 + t8;
                         const bool live = s_base + s < n_tot;
                         vv[r] = live ? *reinterpret_cast<const uint4*>(sBlk + (size_t)hd * sm.stg_blk_head + 4096 + (size_t)s * V * 2 + a * 16)
@@ -696,13 +697,13 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 #pragma unroll
                     for (int r = 0; r < NB; ++r) {
                         const int idx = gt + r * kGroup;
-                        const int a = (idx >> 3) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
+                        const int a = ((idx >> 3) + (idx & 7)) % (K / 8), sp = (idx & 7) + 8 * (idx / (8 * (K / 8)));
                         *reinterpret_cast<uint4*>(sB1 + (sp & 7) * 16 + a * SBO + (sp >> 3) * LBO1) = kv[r];
                     }
 #pragma unroll
                     for (int r = 0; r < NA; ++r) {
                         const int it = gt + r * kGroup;
-                        const int t8 = it & 7, a = (it >> 3) % (V / 8), rest = it / V;
+                        const int t8 = it & 7, a = ((it >> 3) + t8) % (V / 8), rest = it / V;
                         const int hd = rest >> 1, sp = hd * kTokBlock + (rest & 1) * 8 + t8;
                         const int a128 = hd * (V / 8) + a;
                         const uint32_t vin[4] = {vv[r].x, vv[r].y, vv[r].z, vv[r].w};

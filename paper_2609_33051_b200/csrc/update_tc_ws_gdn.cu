@@ -659,7 +659,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 const int idx = gt + r * kGrp;
-                const int t8 = idx & 7, a = (idx >> 3) & 15, s = (idx >> 7) * 8 + t8;
+                const int t8 = idx & 7, a = ((idx >> 3) + t8) & 15, s = (idx >> 7) * 8 + t8;      // a diagonal: the 8 rows of a quarter warp at 8 different vectors (no bank conflicts at a 256-byte pitch)
                 uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
                 if (s < n_tot) {
                     kv = *reinterpret_cast<const uint4*>(sStg + (size_t)s * kKeyRow + a * 16);
