@@ -422,12 +422,15 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             return (uint32_t)NH * by;
         };
         const bool staging = block_bytes(0) > 0;
-        // One bulk copy per lane of the group's first warp: lane = head * 6 + kind, kind = block keys, block values,
-        // token key, token value, gates, query row.  Base pointer and bytes per (batch, head) are per-lane constants.
-        const int cp_hd = gt / 6, cp_kind = gt - cp_hd * 6;
+        // One bulk copy per thread, spread over the four warps of the group (a warp's copies are issued one after the
+        // other, ~400 cycles each, so four warps issue a block's copies four times as fast): copy number
+        // c = head * 6 + kind, kind = block keys, block values, token key, token value, gates, query row, belongs to lane
+        // c / 4 of warp c % 4.  Base pointer and bytes per (batch, head) are per-thread constants.
+        const int cp_c = (gt & 31) < 3 * NH ? (gt & 31) * 4 + (gt >> 5) : 6 * NH;
+        const int cp_hd = cp_c / 6, cp_kind = cp_c - cp_hd * 6;
         const unsigned char* cp_base = nullptr;
         size_t cp_stride = 0;
-        if (gt < 6 * NH) {
+        if (cp_c < 6 * NH) {
             switch (cp_kind) {
                 case 0: cp_base = p.ring; cp_stride = p.rl.head_bytes; break;
                 case 1: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; break;
@@ -437,7 +440,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 default: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; break;
             }
         }
-        auto stage_block = [&](int tile, int blk, int buf) {       // first warp of the group
+        auto stage_block = [&](int tile, int blk, int buf) {       // whole group
             const int h = tile / tiles_per_h;
             const int b0 = (tile - h * tiles_per_h) * NH;
             int rows = n_ring - blk * kTokBlock;
@@ -445,9 +448,9 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             const bool tok = p.has_token && n_ring / kTokBlock == blk;
             const int tok_row = n_ring - blk * kTokBlock;
             uint64_t* bar = &bars[kBarStg + buf];
-            if (gt == 0) mbar_expect_tx(bar, block_bytes(blk));
+            if (gt == 0) mbar_expect_tx(bar, block_bytes(blk));      // (the phase cannot complete before this arrival, whatever the order of the copies)
             __syncwarp();
-            if (gt < 6 * NH) {
+            if (cp_c < 6 * NH) {
                 const size_t bw = (size_t)(b0 + cp_hd) * H + h;
                 const uint32_t blk_dst = sm.stg_blk + (uint32_t)buf * sm.stg_blk_stride + (uint32_t)cp_hd * sm.stg_blk_head;
                 const uint32_t tile_dst = sm.stg + (uint32_t)cp_hd * sm.stg_tile_head;
@@ -461,20 +464,20 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 if (bytes) bulk_g2s(smem + dst, cp_base + bw * cp_stride + src_off, bytes, bar);
             }
         };
-        // producer cursor of the staging ring (kept by every lane of the first warp): the next block to request, and how
+        // producer cursor of the staging ring (kept by every thread of the group): the next block to request, and how
         // many tiles have been published
         int sq_tile = 0, sq_blk = 0, sq_idx = 0, pub_k = 0;
-        auto stage_next = [&]() {           // first warp: request the next block in sequence; entering a new tile claims it
+        auto stage_next = [&]() {           // whole group: request the next block in sequence; entering a new tile claims it
             if (sq_tile < 0) return;
             if (sq_blk == 0) {              // the claim issued a tile ago is resolved only now, the one after it goes out
-                int nxt = 0;
                 if (gt == 0) {
-                    nxt = claim_resolve();
+                    const int nxt = claim_resolve();
                     publish(pub_k, nxt);
                     if (nxt >= 0) claim_issue();
                 }
+                group_sync(2);              // the published entry is the hand-off to the other threads
+                sq_tile = seq_ring[pub_k & 3];
                 ++pub_k;
-                sq_tile = __shfl_sync(0xffffffffu, nxt, 0);
                 if (sq_tile < 0) return;
             }
             if (staging) stage_block(sq_tile, sq_blk, sq_idx % stg_bufs);
@@ -507,11 +510,9 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             return true;
         };
 
-        if (gt < 32) {
-            if (gt == 0) claim_issue();
-            stage_next();
-            if (stg_bufs > 1 && n_stage_blocks > 1) stage_next();
-        }
+        if (gt == 0) claim_issue();
+        stage_next();
+        if (stg_bufs > 1 && n_stage_blocks > 1) stage_next();
         // W (padding columns, lo halves of the query columns) and the MMA-1 operands (off-diagonal head blocks) hold
         // zeros that no tile ever overwrites: written once
         for (uint32_t o = (uint32_t)gt * 16u; o < 2u * (uint32_t)NP * kK * 2u; o += kGroup * 16u)
@@ -738,7 +739,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                         mbar_arrive(&bars[kBarPro + b]);      // after the group barrier: W, weights and decay are written
                     }
                 }
-                if (gt < 32) stage_next();        // the block buffer just read is free again
+                stage_next();        // the block buffer just read is free again
             }
             if (dead) break;
             if (n_blocks == 0) {
@@ -749,7 +750,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                     mbar_arrive(&bars[kBarT + b]);
                     mbar_arrive(&bars[kBarPro + b]);
                 }
-                if (gt < 32) stage_next();
+                stage_next();
             }
             WS_STAMP(512, 3);
 
