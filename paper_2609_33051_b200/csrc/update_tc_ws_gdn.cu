@@ -561,47 +561,47 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
 
         const uint32_t stg_gate_bytes = n_ring > 0 ? (uint32_t)(2 * p.L * 4) : 0u;
         const uint32_t stg_bytes = (uint32_t)n_ring * 512u + stg_gate_bytes + (p.has_token ? 512u : 0u) + (p.q != nullptr ? 256u : 0u);
-        // one bulk copy per lane of the group's first warp, from per-lane constants: lanes 0..15 one key row each (ring
-        // rows, then the token's), lanes 16..19 ring values, ring gates, token value, query row
+        // One bulk copy per thread from per-thread constants, spread over the four warps of the group (a warp's copies are
+        // issued one after the other, ~400 cycles each): copy number c belongs to lane c / 4 of warp c % 4; copies 0..15
+        // one key row each (ring rows, then the token's), 16..19 ring values, ring gates, token value, query row.
+        const int cp_c = (gt & 31) < 5 ? (gt & 31) * 4 + (gt >> 5) : 32;
         const unsigned char* cp_base = nullptr;
         size_t cp_stride = 0;
         uint32_t cp_dst = 0, cp_bytes = 0;
-        if (gt < n_ring) {
-            cp_base = p.ring + (size_t)(p.tok_base + gt) * 256u; cp_stride = p.rl.head_bytes; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
-        } else if (gt == n_ring && p.has_token) {
-            cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)gt * kKeyRow; cp_bytes = 256u;
+        if (cp_c < n_ring) {
+            cp_base = p.ring + (size_t)(p.tok_base + cp_c) * 256u; cp_stride = p.rl.head_bytes; cp_dst = (uint32_t)cp_c * kKeyRow; cp_bytes = 256u;
+        } else if (cp_c == n_ring && p.has_token) {
+            cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)cp_c * kKeyRow; cp_bytes = 256u;
         }
-        switch (gt) {
+        switch (cp_c) {
             case 16: cp_base = p.ring + p.rl.v_off + (size_t)p.tok_base * 256u; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
             case 17: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_gate; cp_bytes = stg_gate_bytes; break;
             case 18: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; cp_dst = sm.stg_v + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
             case 19: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; cp_dst = sm.stg_q; cp_bytes = p.q != nullptr ? 256u : 0u; break;
             default: break;
         }
-        auto stage_tile = [&](int tile) {       // first warp of the group
+        auto stage_tile = [&](int tile) {       // whole group
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bw = (size_t)bb * H + h;
-            if (gt == 0) mbar_expect_tx(&bars[gStg], stg_bytes);
+            if (gt == 0) mbar_expect_tx(&bars[gStg], stg_bytes);      // (the phase cannot complete before this arrival, whatever the order of the copies)
             __syncwarp();
             if (cp_bytes) bulk_g2s(sStg + cp_dst, cp_base + bw * cp_stride, cp_bytes, &bars[gStg]);
         };
-        // thread 0 resolves the claim, publishes it as entry k of the sequence and issues the next claim; the warp then
+        // thread 0 resolves the claim, publishes it as entry k of the sequence and issues the next claim; the group then
         // requests the tile's rows
-        auto next_tile = [&](int k) {          // first warp of the group
-            int nxt = 0;
+        auto next_tile = [&](int k) {          // whole group
             if (gt == 0) {
-                nxt = claim_resolve();
+                const int nxt = claim_resolve();
                 publish(k, nxt);
                 if (nxt >= 0) claim_issue();
             }
-            nxt = __shfl_sync(0xffffffffu, nxt, 0);
-            if (nxt >= 0) stage_tile(nxt);
+            g_sync(2);                         // the published entry is the hand-off to the other threads
+            const int nxt = seq_ring[k & 3];
+            if (nxt >= 0) stage_tile(nxt & (kSepFlag - 1));
         };
         // the first tile: claimed, published and its rows requested before anything else
-        if (gt < 32) {
-            if (gt == 0) claim_issue();
-            next_tile(0);
-        }
+        if (gt == 0) claim_issue();
+        next_tile(0);
         // W padding columns and lo halves of the query columns hold zeros that no tile overwrites: written once
         for (uint32_t o = (uint32_t)gt * 16u; o < (64u + (uint32_t)NP) * kK * 2u; o += kGrp * 16u)
             *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
@@ -837,7 +837,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             proxy_fence();         // operand sets and W are read by MMAs (async proxy)
             g_sync(2);
             if (gt == 0) g_arrive(&bars[gPro + b]);
-            if (gt < 32) next_tile(k + 1);      // the staging buffer has been read: the next tile's rows may come in
+            next_tile(k + 1);      // the staging buffer has been read: the next tile's rows may come in
             G_STAMP(256, k, 5);
 
             G_STAMP(256, k, 6);
