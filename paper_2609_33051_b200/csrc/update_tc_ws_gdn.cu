@@ -201,9 +201,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         }
         return -2;
     };
-    // A published tile number carries a flag when its head index differs from the tile before it: W is then rewritten
-    // between the two tiles, so their passes are not interleaved (pass B of the earlier tile runs first).
-    constexpr int kSepFlag = 1 << 30;
     auto set_ptr = [&](int b) { return smem + sm.set + (uint32_t)b * sm.set_stride; };
 
     const int j = (warp & 3) * 32 + lane;      // value column = TMEM lane of this thread (both stream groups and the front group)
@@ -332,7 +329,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         for (int k = 0; !bad; ++k) {
             const int raw = seq_get(k);
             if (raw < 0) { bad = raw < -1; break; }
-            const int tile = raw & (kSepFlag - 1);
+            const int tile = raw;
             const int b = k & 1;
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bh = (size_t)bb * H + h;
@@ -503,13 +500,12 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         };
         int cur = seq_get(0);
         if (cur >= 0) {
-            cur &= kSepFlag - 1;
             load_tile(cur);
             for (int k = 0; !bad; ++k) {
                 const int raw = seq_get(k + 1);
                 if (raw < -1) { bad = true; break; }
                 if (raw < 0) break;
-                load_tile(raw & (kSepFlag - 1));
+                load_tile(raw);
             }
         } else if (cur < -1) {
             bad = true;
@@ -597,7 +593,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             }
             g_sync(2);                         // the published entry is the hand-off to the other threads
             const int nxt = seq_ring[k & 3];
-            if (nxt >= 0) stage_tile(nxt & (kSepFlag - 1));
+            if (nxt >= 0) stage_tile(nxt);
         };
         // the first tile: claimed, published and its rows requested before anything else
         if (gt == 0) claim_issue();
@@ -625,7 +621,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 }
                 break;
             }
-            const int tile = raw_tile & (kSepFlag - 1);
+            const int tile = raw_tile;
             const int b = k & 1;
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bh = (size_t)bb * H + h;
