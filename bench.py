@@ -38,7 +38,7 @@ UNIT = "tokens/s/layer"
 NCU_TRAFFIC_CAPTURES = {
     ("decode_kernel", "c2_mamba2"): (118.04e6, 0.5 * (traffic.decode_bytes("mamba2", 256, 64, 128, 64, 16, 4, "bf16")
                                                       + traffic.decode_bytes("mamba2", 256, 64, 128, 64, 16, 5, "bf16"))),
-    ("update_kernel", "c2_mamba2"): (1194.11e6, float(traffic.update_bytes("mamba2", 256, 64, 128, 64, 16, 15, "bf16"))),
+    ("update_kernel", "c2_mamba2"): (1194.56e6, float(traffic.update_bytes("mamba2", 256, 64, 128, 64, 16, 15, "bf16"))),
 }
 
 
