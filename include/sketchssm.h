@@ -126,7 +126,14 @@ int sketchssm_destroy(sketchssm_ctx* ctx);
 int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out);
 
 /* Record the caller's device buffers (all seven required, 16-byte aligned).  The context
- * stores the pointers only; the caller keeps ownership and must keep them alive. */
+ * stores the pointers only; the caller keeps ownership and must keep them alive.
+ * Between calls on a context its sketch is written by sketchssm_state_update only.  The library's kernels
+ * are launched with programmatic dependent launch, and a decode step that does not directly follow a state
+ * update (or a bind) of its own context requests sketch rows before it waits for its predecessor in the
+ * stream.  So a sketch buffer must not be shared between contexts, and work of the caller that writes the
+ * sketch (a kernel, a copy that restores a checkpoint) must be followed by sketchssm_bind, which makes
+ * the next decode step wait first, or by a stream synchronisation.  With the tune key "pdl" = 0 every
+ * kernel waits for its predecessor as usual. */
 int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* bufs);
 
 /* Flush step of Algorithm 1: (optionally) append the current token, replay every buffered

@@ -90,6 +90,10 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     p.has_token = 1;
     p.append = (flags & SKETCHSSM_NO_APPEND) ? 0 : 1;
     p.full_read = full_read;
+    // Only a state update writes the sketch.  Unless that was the previous call on this context (it may still be running:
+    // programmatic dependent launch), a decode step may read U before it waits for its predecessor in the stream.
+    p.early_sketch = (!full_read && !ctx->sketch_fresh) ? 1 : 0;
+    ctx->sketch_fresh = false;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
     if (ctx->tune_decode_impl == 1) {
@@ -143,6 +147,7 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     c->bound = false;
     c->bufs = sketchssm_buffers{};
     c->last_launches = 0;
+    c->sketch_fresh = true;
     c->last_cuda_error = cudaSuccess;
     c->tune_batches_per_cta = 0;
     c->tune_stages = 0;
@@ -191,6 +196,7 @@ int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* b) {
     }
     ctx->bufs = *b;
     ctx->bound = true;
+    ctx->sketch_fresh = true;       // whatever filled the buffers may still be running
     return SKETCHSSM_OK;
 }
 
@@ -220,6 +226,7 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     p.has_token = has_token ? 1 : 0;
     p.write_sketch = sketch ? 1 : 0;
     p.write_state = n_tot > 0 ? 1 : 0;
+    ctx->sketch_fresh = true;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (p.update_impl != 1) {
         // Mamba-2: warp-specialised tensor-core kernel, then the single-group one (ranks above 32); 3 skips the former

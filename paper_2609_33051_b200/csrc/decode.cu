@@ -145,8 +145,6 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         }
     }
     __syncthreads();
-    grid_dep_wait();                 // from here on the ring, the sketch and the token tensors are read
-    grid_dep_launch_dependents();
 
     // A warp's stage is filled by two groups of bulk copies, each completing on its own mbarrier: group A holds what
     // the ring sweep reads (the token's rows and the buffered keys / values / gates), group B the sketch U.  Group A of
@@ -211,10 +209,18 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         if constexpr (KIND != SKETCHSSM_KDA) dsc = reinterpret_cast<const float*>(p.decay)[bh];
     };
     float bt_next = 0.f, dsc_next = 1.f;
+    // Only a state update writes the sketch; unless one may still be running (the caller of the launcher knows), the first
+    // head's sketch rows are requested before the predecessor in the stream is waited for, so they travel during its tail.
+    const bool early_u = p.early_sketch != 0;
+    if (item < item1 && early_u) issue_b((size_t)b * H + h);
+    grid_dep_wait();                 // from here on the ring and the token tensors (and otherwise the sketch) are read
+    // Dependents are released only now: a successor that reads its sketch early must not start before this kernel has
+    // seen its own predecessor (possibly a state update) complete.
+    grid_dep_launch_dependents();
     if (item < item1) {
         const size_t bh0 = (size_t)b * H + h;
         issue_a(bh0);
-        issue_b(bh0);
+        if (!early_u) issue_b(bh0);
         scalar_gates(bh0, bt_next, dsc_next);
     }
     bool dead = false;

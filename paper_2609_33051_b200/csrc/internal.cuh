@@ -30,6 +30,7 @@ struct Ctx {
     int sm_count;       // filled lazily on first launch
     int max_smem_optin; // ditto
     int last_launches;
+    bool sketch_fresh;  // the last hot-path call on this context was a state update that wrote the sketch (or none was made yet)
     cudaError_t last_cuda_error;  // of the most recent failing runtime call
 };
 
@@ -71,6 +72,8 @@ struct Params {
                           // 3: as 0 but without the warp-specialised kernels (single-group Mamba-2 kernel, CUDA cores for GDN)
     int decode_mma;       // warp-per-head decode: 1 = tensor-core dot products where supported
     int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
+    int early_sketch;     // decode: the first head's sketch rows may be requested before the predecessor in the stream is
+                          // waited for (no kernel that may still be running writes the sketch)
     int tok_base;         // update (GDN tensor-core kernel): first ring row of this pass when a flush is replayed in blocks of 16 tokens
 };
 

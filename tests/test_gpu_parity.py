@@ -399,3 +399,38 @@ def test_window_replays_from_a_cuda_graph():
             assert torch.equal(a, b)
         assert torch.equal(me.state, mg.state) and torch.equal(me.sketch, mg.sketch)
     me.check_status(); mg.check_status()
+
+
+@pytest.mark.parametrize("kind,dv", [("mamba2", 64), ("gdn", 128)])
+def test_decode_after_update_sees_the_new_sketch_with_dependent_launch(kind, dv):
+    """With programmatic dependent launch a decode step requests sketch rows before it waits for its predecessor in
+    the stream, unless that predecessor is a state update of its own context (the only writer of the sketch).  Windows
+    run back to back without synchronisation, and a decode step issued directly after a flush, give bit-identical
+    results with dependent launch on and off."""
+    dev = _device()
+    w = synth.Workload("t", kind, 64, 8, 128, dv, 16, 8, 0, "bf16", 37, basis="qr")
+    toks = [harness.token_tensors(w, synth.step_inputs(w, 0, t), dev) for t in range(w.buf_len)]
+    results = []
+    for pdl in (1, 0):
+        m, *_ = make_layer(w)
+        m.tune("pdl", pdl)
+        m.state_update(0)
+        outs = [m.new_output() for _ in range(3 * w.buf_len + 1)]
+        i = 0
+        for rep in range(3):
+            for t, tt in enumerate(toks):
+                if t < w.buf_len - 1:
+                    m.decode_step(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], outs[i])
+                else:
+                    m.state_update(t, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], outs[i])
+                i += 1
+        # directly after the flush: a decode step over the first three (still stored) ring slots, nothing appended
+        tt = toks[3]
+        m.decode_step(3, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], outs[i], flags=1)
+        torch.cuda.synchronize()
+        m.check_status()
+        results.append(([o.clone() for o in outs], m.state.clone(), m.sketch.clone()))
+    (oa, sa, ua), (ob, sb, ub) = results
+    for a, b in zip(oa, ob):
+        assert torch.equal(a, b)
+    assert torch.equal(sa, sb) and torch.equal(ua, ub)
