@@ -486,7 +486,9 @@ def main():
                     "traffic": ncu_traffic(kname, w.name, kern[dominant]["algorithmic_bytes_per_launch"]),
                     "algorithmic_bytes_per_launch": kern[dominant]["algorithmic_bytes_per_launch"],
                     "duration": "average over a run of back-to-back launches between two CUDA events "
-                                "(programmatic dependent launch overlaps heads and tails of consecutive launches)",
+                                "(programmatic dependent launch overlaps heads and tails of consecutive launches; in "
+                                "this run the n = 0 launches, 1 of L-1, also request their sketch rows before the "
+                                "dependency wait, which after a flush in a window they do not)",
                     "achieved_bracketed": kern[dominant]["achieved_gbs"],
                     "frac_bracketed": kern[dominant]["achieved_gbs"] / peak,
                     "frac_of_8TBs_nominal": ach / 8000.0}
