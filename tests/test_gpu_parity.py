@@ -182,7 +182,8 @@ def test_gdn_warp_specialised_update(tune, batch, heads, rank, buf_len):
 
 
 @pytest.mark.parametrize("kind,dv,buf_len,fills", [("mamba2", 64, 32, (0, 1, 15, 16, 17, 31)), ("mamba2", 128, 64, (16, 32, 47, 48, 63)),
-                                                    ("gdn", 128, 16, (0, 1, 7, 15)), ("gdn", 128, 32, (3, 15, 16, 31))])
+                                                    ("gdn", 128, 16, (0, 1, 7, 15)), ("gdn", 128, 32, (3, 15, 16, 31)),
+                                                    ("gdn", 128, 64, (17, 32, 33, 48, 63))])
 def test_flush_at_any_ring_fill(kind, dv, buf_len, fills):
     """state_update with n_before tokens in the ring plus the current token, for fills around the tensor-core kernels'
     block boundaries (16 tokens per block) and beyond their domains, and a replay without a current token."""
