@@ -422,11 +422,16 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             return (uint32_t)NH * by;
         };
         const bool staging = block_bytes(0) > 0;
-        // One bulk copy per thread, spread over the four warps of the group (a warp's copies are issued one after the
-        // other, ~400 cycles each, so four warps issue a block's copies four times as fast): copy number
-        // c = head * 6 + kind, kind = block keys, block values, token key, token value, gates, query row, belongs to lane
-        // c / 4 of warp c % 4.  Base pointer and bytes per (batch, head) are per-thread constants.
-        const int cp_c = (gt & 31) < 3 * NH ? (gt & 31) * 4 + (gt >> 5) : 6 * NH;
+        // One bulk copy per thread, spread over the warps of the group (a warp's copies are issued one after the other,
+        // ~400 cycles each): copy number c = head * 6 + kind, kind = block keys, block values, token key, token value,
+        // gates, query row.  With one token block per tile all four warps share the copies (lane c / 4 of warp c % 4) and
+        // thread 0 issues MMA 1; with several blocks per tile, where the front group is the limit, the first three warps
+        // share them (lane c / 3 of warp c % 3) and the fourth warp issues MMA 1 meanwhile.  Base pointer and bytes per
+        // (batch, head) are per-thread constants.
+        const bool split_issue = n_blocks > 1;
+        const int mma_thread = split_issue ? 3 * 32 : 0;
+        const int cp_c = split_issue ? (((gt >> 5) < 3 && (gt & 31) < 2 * NH) ? (gt & 31) * 3 + (gt >> 5) : 6 * NH)
+                                     : ((gt & 31) < 3 * NH ? (gt & 31) * 4 + (gt >> 5) : 6 * NH);
         const int cp_hd = cp_c / 6, cp_kind = cp_c - cp_hd * 6;
         const unsigned char* cp_base = nullptr;
         size_t cp_stride = 0;
@@ -724,7 +729,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 tc_fence_before();
                 group_sync(2);
                 ++ops_built;
-                if (gt == 0) {
+                if (gt == mma_thread) {
                     tc_fence_after();
                     const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
 #pragma unroll
