@@ -10,22 +10,23 @@
 // Every product of decays is built by multiplication (no quotients), and all tensor-core operands that come from the
 // ring are the raw bf16 keys, so those products are exact; fp32 operands (S_0, S_new, E') are split into bf16 hi + lo.
 //
-// Tile = one head (K = V = 128); TMEM lane = value column j.  The state is read twice: pass A contracts S_0 (from a ring
-// of shared-memory stages filled by bulk copies) with the keys (P) and with W = [Omega | q]; pass B forms
-// S_new = d S_0 + K^T E' from S_0 read again (plain loads, from L2) and writes it back.  The CTA is specialised:
+// Tile = one head (K = V = 128); TMEM lane = value column j.  The state is read once: pass A takes the S_0 chunks from a
+// ring of shared-memory stages filled by bulk copies, contracts them with the keys (P) and with W = [Omega | q], and
+// leaves d S_0 in the accumulator of K^T E' (tcgen05.st), so that the MMAs of the E' step turn it into S_new; pass B
+// only writes that accumulator back.  The CTA is specialised:
 //   front group (4 warps)   ring-only operands two tiles ahead: key layouts, Gram matrix, T1, K W, tile claiming
-//   pass-A group (4 warps)  S_0 chunks -> bf16 hi + lo operands, then the small E' step
+//   pass-A group (4 warps)  S_0 chunks -> bf16 hi + lo operands and d S_0 into tensor memory, then the small E' step
 //   pass-B group (4 warps)  S_new written back, then the sketch rows and the exact output from tensor memory
 //   one thread issues every MMA; one warp keeps the stages full.
-// Pass A of tile i + 1 runs while pass B of tile i does, so no MMA round trip is waited for.
+// Pass A of tile i + 1 runs while pass B of tile i does (it follows pass B through the accumulator half by half), so no
+// MMA round trip is waited for.
 //
 // The sketch rows never need S_new as a tensor-core operand: [U | o] = d S_0^T W + E'^T (K W), so pass A contracts the
 // S_0 chunks with the keys and W in one product (the keys sit next to W in shared memory: a 48-row operand window per
 // tile), the small product K W is formed by the front group, and the correction E'^T (K W) rides along with K^T E'.
-// Pass B is then only S_new = d S_0 + K^T E': no split, no operand hand-off, no MMA.
 // Tensor memory per CTA (256 columns): two 64-column slots for alternating tiles ([U0 32 | P 16 | free 16] or
 // [free 16 | P 16 | U0 32]; the correction later goes over P and the free columns), and one 128-column accumulator
-// for K^T E'.
+// for d S_0 + K^T E'.
 //
 // Shared memory is the busiest unit of this kernel (load/store data pipe ~70 % busy): the staged key rows are padded so
 // that ldmatrix reads them without bank conflicts.
@@ -95,7 +96,7 @@ __host__ __device__ inline GSmem make_gsmem(int NP, int L, int stages) {
 
 enum { gPro = 0, gPfull = 2, gTfull = 4, gBdone = 6, gBufFree = 8, gA2free = 10, gA2rdy = 10 + kA2, gErdy = 10 + 2 * kA2,
        gStg = 11 + 2 * kA2, gProW = 12 + 2 * kA2, gFull = 14 + 2 * kA2, gEmpty = 14 + 2 * kA2 + kGStages,
-       gNumBars = 14 + 2 * kA2 + 2 * kGStages };
+       gTfree = 14 + 2 * kA2 + 2 * kGStages, gNumBars = 16 + 2 * kA2 + 2 * kGStages };
 
 __device__ __forceinline__ void g_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
     if (tid == 0) {
         *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
         for (int i = 0; i < gNumBars; ++i) {
-            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty || (i >= gBdone && i < gBdone + 4);     // one arrival per warp of a stream group (gBdone, gBufFree too)
+            const bool per_warp = (i >= gA2rdy && i <= gErdy) || i >= gEmpty /* gTfree too */ || (i >= gBdone && i < gBdone + 4);     // one arrival per warp of a stream group (gBdone, gBufFree too)
             mbar_init(&bars[i], per_warp ? 4 : 1);
         }
         mbar_fence_init();
@@ -212,9 +213,19 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         int gc = 0, stage = 0;
         bool bad = false;
 
-        auto pass_a = [&]() {
+        uint32_t phTf = 0;
+        // pass A of a tile with operand set b; `later`: not the CTA's first tile, so the K^T E' accumulator still holds
+        // the tile before until the pass-B group has read it (half by half)
+        auto pass_a = [&](int b, bool later) {
+            const float dtile = reinterpret_cast<const float*>(set_ptr(b) + sm.set_gates)[kNTok];
 #pragma unroll 2
             for (int c = 0; c < NCH; ++c) {
+                if (later && (c == 0 || c == NCH / 2)) {
+                    const int hf = c ? 1 : 0;
+                    bad |= !mbar_wait_bounded(&bars[gTfree + hf], (phTf >> hf) & 1u);
+                    phTf ^= 1u << hf;
+                    tc_fence_after();
+                }
                 bad |= !mbar_wait_bounded(&bars[gFull + stage], phF);
                 const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
                 float s0[CH];
@@ -222,6 +233,12 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
                 __syncwarp();
                 if (lane == 0) g_arrive(&bars[gEmpty + stage]);
+                {   // d S_0 goes into the K^T E' accumulator, so that the MMAs leave S_new there: pass B reads S_0 no more
+                    float ds[CH];
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) ds[ii] = dtile * s0[ii];
+                    if (!bad) tmem_st16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), ds);
+                }
                 const int ab = c & (kA2 - 1);
                 if (gc >= kA2) {     // the chunk buffer was read by the MMAs issued kA2 chunks ago
                     bad |= !mbar_wait_bounded(&bars[gA2free + ab], (phA >> ab) & 1u);
@@ -285,6 +302,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 *reinterpret_cast<uint4*>(elo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
             }
             proxy_fence();
+            tmem_st_wait();            // the d S_0 columns of pass A are in tensor memory
             tc_fence_before();
             bad = __any_sync(0xffffffffu, bad);
             if (lane == 0 && !bad) g_arrive(&bars[gErdy]);
@@ -297,7 +315,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         int cur = seq_get(0);
         if (cur >= 0) {
             wait_pro(0);
-            pass_a();
+            pass_a(0, false);
             do_e(0);
             for (int k = 0; !bad; ++k) {
                 const int b = k & 1;
@@ -307,7 +325,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 G_STAMP(0, k, 0);
                 wait_pro(b ^ 1);
                 G_STAMP(0, k, 1);
-                pass_a();
+                pass_a(b ^ 1, true);
                 G_STAMP(0, k, 2);
                 // the E' operand buffer is read by K^T E' of tile k: that must be complete before it is rewritten
                 bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);
@@ -321,9 +339,8 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 3);
     } else if (warp >= 10) {
-        // =========================== pass-B group: S_new = d S_0 + K^T E' written back, then the sketch rows ===========================
-        // S_0 is read a second time here, with plain loads one chunk ahead (the lines are in L2 since pass A), so the
-        // stage ring serves pass A alone.
+        // =========================== pass-B group: S_new written back, then the sketch rows ===========================
+        // Pass A left d S_0 in the K^T E' accumulator, so the accumulator holds S_new: nothing is read from memory here.
         uint32_t phT = 0;
         bool bad = false;
         for (int k = 0; !bad; ++k) {
@@ -334,9 +351,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bh = (size_t)bb * H + h;
             float* So = p.state + bh * (size_t)K * V + j;
-            float sn[CH];
-#pragma unroll
-            for (int ii = 0; ii < CH; ++ii) sn[ii] = __ldcg(So + (size_t)ii * V);
             G_STAMP(128, k, 0);
             bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);      // K^T E' and the sketch correction are complete
             phT ^= 1u << b;
@@ -345,23 +359,16 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const float dtot = sDt[b];
 #pragma unroll 2
             for (int c = 0; c < NCH; ++c) {
-                float s0[CH];
-#pragma unroll
-                for (int ii = 0; ii < CH; ++ii) s0[ii] = sn[ii];
-                if (c + 1 < NCH) {
-#pragma unroll
-                    for (int ii = 0; ii < CH; ++ii) sn[ii] = __ldcg(So + (size_t)((c + 1) * CH + ii) * V);
-                }
-                float t[CH];
                 if (!bad) {
+                    float t[CH];
                     tmem_ld16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), t);
-                } else {
+                    if (c == NCH / 2 - 1 || c == NCH - 1) {      // this warp is done with a half of the accumulator
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) g_arrive(&bars[gTfree + (c == NCH - 1 ? 1 : 0)]);
+                    }
 #pragma unroll
-                    for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
-                }
-                if (!bad) {
-#pragma unroll
-                    for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = fmaf(dtot, s0[ii], t[ii]);
+                    for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = t[ii];
                 }
             }
             G_STAMP(128, k, 2);
@@ -455,7 +462,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const uint32_t bc = smem_u32(set_ptr(b) + sm.set_bc);
                 const uint64_t bchi = make_desc(bc, 512u, SBO);
                 const uint64_t bclo = make_desc(bc + 1024u, 512u, SBO);
-                tc_mma_bf16(tmem_t, ehi, bt, idescT, 0u);
+                tc_mma_bf16(tmem_t, ehi, bt, idescT, 1u);      // onto d S_0, which pass A left there
                 tc_mma_bf16(tmem_t, elo, bt, idescT, 1u);
                 tc_mma_bf16(tmem_c, ehi, bchi, idescU, 0u);
                 tc_mma_bf16(tmem_c, elo, bchi, idescU, 1u);
