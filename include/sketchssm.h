@@ -30,6 +30,9 @@
  *     records a code in the caller's status word (see sketchssm_buffers.status).
  *   - The window phase is the caller's: `n_before` (tokens already buffered) is
  *     the same for the whole batch.
+ *   - Every call that touches the GPU makes config.device the calling thread's current CUDA device
+ *     and leaves it current on return; a caller that drives several GPUs from one thread must not
+ *     assume that its previous device is still selected.
  *
  * Layouts (B = batch, H = heads, K = dk, V = dv, r = rank, L = buf_len; "io" is
  * float or bfloat16 as configured):
@@ -132,8 +135,9 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out);
  * update (or a bind) of its own context requests sketch rows before it waits for its predecessor in the
  * stream.  So a sketch buffer must not be shared between contexts, and work of the caller that writes the
  * sketch (a kernel, a copy that restores a checkpoint) must be followed by sketchssm_bind, which makes
- * the next decode step wait first, or by a stream synchronisation.  With the tune key "pdl" = 0 every
- * kernel waits for its predecessor as usual. */
+ * the next decode step wait first, or by a stream synchronisation.  A decode step recorded into a stream
+ * capture always waits first (a replayed graph may follow a state update that is still running).  With the
+ * tune key "pdl" = 0 every kernel waits for its predecessor as usual. */
 int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* bufs);
 
 /* Flush step of Algorithm 1: (optionally) append the current token, replay every buffered
@@ -161,8 +165,9 @@ int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const
 
 /* Exact decode step that reads the whole state: o = S_0^T q~_t + sum_s a_s v_s (Eq. 4).
  * Same arguments and ring behaviour as sketchssm_decode_step; U and C are not read.
- * Both decode calls run as two kernels: the first forms the buffer weights a_s and the coefficients
- * (c_t, or q~_t for the full read) into `work`, the second forms the weighted sum of rows. */
+ * By default both decode calls run as one kernel with a warp per (batch, head) and leave `work` alone; with the
+ * tune key "decode_impl" = 0 they run as two kernels, the first of which forms the buffer weights a_s and the
+ * coefficients (c_t, or q~_t for the full read) into `work` and the second the weighted sum of rows. */
 int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
                                const void* v, const void* beta, const void* decay, void* out,
                                uint32_t flags, void* stream);
@@ -213,6 +218,15 @@ int sketchssm_step_host(sketchssm_ctx* ctx, int op, int n_before, const void* ho
  * four status ints. */
 int sketchssm_read_status(sketchssm_ctx* ctx, int32_t detail[4], void* stream);
 
+/* Self-test of the failure-reporting path (no counterpart in the paper).  Every device wait of the hot-path kernels
+ * is bounded and reports through the status block when its limit is reached; in normal operation none ever does.
+ * This call launches one warp that waits, for at most `poll_limit` polls (1..65536), on a barrier phase that nothing
+ * completes -- no copy is issued, so nothing is in flight when it gives up -- and then records the fault code 4 with
+ * `where` as the place.  Afterwards sketchssm_read_status returns SKETCHSSM_DEVICE_TIMEOUT with detail = {4, where, ..}.
+ * The status block keeps its first fault: zero its first four ints before going on with normal calls.  The GPU
+ * context stays usable; nothing traps or hangs. */
+int sketchssm_selftest_wait_timeout(sketchssm_ctx* ctx, int poll_limit, int where, void* stream);
+
 /* Text of the CUDA runtime error behind the most recent SKETCHSSM_CUDA_ERROR of this context. */
 const char* sketchssm_last_cuda_error(const sketchssm_ctx* ctx);
 
@@ -220,16 +234,14 @@ const char* sketchssm_last_cuda_error(const sketchssm_ctx* ctx);
 int sketchssm_last_launch_count(const sketchssm_ctx* ctx);
 
 /* Optional launch tuning, host-only.  Keys: "decode_batches_per_cta" (batch entries one CTA of
- * the decode kernels serves for its head; 0 = library default), "decode_stages" (1 or 2 shared-memory
- * stages per lane group of the lane-group decode kernels; for the warp-specialised update kernels an upper
+ * the two-kernel decode serves for its head; 0 = library default), "decode_stages" (1 or 2 shared-memory
+ * stages per lane group of the two-kernel decode; for the warp-specialised update kernels an upper
  * bound >= 2 on their shared-memory stages of state rows; 0 = library default), "decode_warps_per_cta",
- * "decode_max_warps_per_sm" (also caps the update kernels' CTAs per SM), "decode_lanes_per_head",
- * "decode_l2_prefetch", "decode_mma" (1 = tensor-core dot products in the warp-per-head decode where
- * supported; 0 = off, the default), "update_impl" (0 = warp-specialised tensor-core kernels for Mamba-2 and GDN
- * where their shape limits allow and CUDA cores otherwise, the default; 1 = CUDA cores only; 2 = as 0 but the
- * single-group tensor-core kernel for GDN; 3 = as 0 but the single-group tensor-core kernel for Mamba-2 and CUDA
- * cores for GDN), "decode_impl" (0 = two kernels; 1 = one fused kernel with a warp per head, the default;
- * 2 = one fused kernel with 8 or 16 lanes per head), "pdl" (1 = programmatic dependent launch, the default).
+ * "decode_max_warps_per_sm" (also caps the update kernels' CTAs per SM), "update_impl" (0 = warp-specialised
+ * tensor-core kernels where their shape limits allow and CUDA cores otherwise, the default; 1 = CUDA cores
+ * only; 3 = as 0 but the single-group tensor-core kernel for Mamba-2 and CUDA cores for the delta-rule kinds),
+ * "decode_impl" (0 = two kernels; 1 = one fused kernel with a warp per head, the default), "pdl"
+ * (1 = programmatic dependent launch, the default).
  * Results depend on these only through floating-point summation order. */
 int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value);
 

@@ -26,7 +26,7 @@ EXPORTED = (
     "sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode",
     "sketchssm_read_status", "sketchssm_last_launch_count", "sketchssm_tune",
     "sketchssm_status_string", "sketchssm_version", "sketchssm_last_cuda_error", "sketchssm_step_host",
-    "sketchssm_decode_step_static",
+    "sketchssm_decode_step_static", "sketchssm_selftest_wait_timeout",
 )
 OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 
@@ -78,6 +78,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
                  "sketchssm_decode_step_static"):
         getattr(lib, name).argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u32, vp]
     lib.sketchssm_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.POINTER(Staging), u32, vp]
+    lib.sketchssm_selftest_wait_timeout.argtypes = [vp, i32, i32, vp]
     lib.sketchssm_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32 * 4), vp]
     lib.sketchssm_last_launch_count.argtypes = [vp]
     lib.sketchssm_tune.argtypes = [vp, ctypes.c_char_p, i32]
@@ -228,6 +229,11 @@ class SketchSSM:
                                           ctypes.byref(st), flags, self._stream(stream))
         self._check("sketchssm_step_host", rc)
         return host["out"]
+
+    def selftest_wait_timeout(self, poll_limit: int = 2048, where: int = 99, stream=None):
+        """sketchssm_selftest_wait_timeout: one warp whose bounded wait runs out and reports through the status block."""
+        self._check("sketchssm_selftest_wait_timeout",
+                    self.lib.sketchssm_selftest_wait_timeout(self._ctx, poll_limit, where, self._stream(stream)))
 
     def read_status(self, stream=None):
         detail = (ctypes.c_int32 * 4)()

@@ -10,11 +10,9 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsketchssm.so")
-# (source, object suffix, extra defines); the lane-group decode kernel is compiled once per (recurrence kind, I/O type)
-UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []), ("update_tc_ws.cu", "", []), ("update_tc_ws_gdn.cu", "", []), ("update_tc_delta.cu", "", []),
-         ("decode_static.cu", "", []), ("decode_mma.cu", "", []),
-         *[("decode_fused.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
-           for k in range(3) for io in range(2)],
+# (source, object suffix, extra defines); the two-kernel decode is compiled once per (recurrence kind, I/O type)
+UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []),
+         ("update_tc_ws.cu", "", []), ("update_tc_ws_gdn.cu", "", []), ("decode_static.cu", "", []), ("selftest.cu", "", []),
          *[("decode_split.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
            for k in range(3) for io in range(2)]]
 HEADERS = [os.path.join(CSRC, "internal.cuh"), os.path.join(CSRC, "lanegroup.cuh"), os.path.join(CSRC, "tc_common.cuh"),
@@ -42,7 +40,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(objdir, exist_ok=True)
     flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
              "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-    flags += os.environ.get("SKETCHSSM_NVCC_FLAGS", "").split()     # e.g. -DSKETCHSSM_PHASE_TIMING for kernel phase stamps
     if verbose:
         flags += ["-Xptxas", "-v"]
     procs, objs = [], []

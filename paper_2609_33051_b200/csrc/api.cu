@@ -9,13 +9,10 @@ struct sketchssm_ctx : public Ctx {
     int tune_batches_per_cta;
     int tune_stages;
     int tune_warps_per_cta;
-    int tune_lanes_per_head;
-    int tune_decode_impl;   // 0: two kernels (weights + output rows), 1: warp-per-head kernel, 2: fused lane-group kernel
+    int tune_decode_impl;   // 0: two kernels (weights + output rows), 1: warp-per-head kernel
     int tune_max_warps;
     int tune_update_impl;
-    int tune_decode_mma;
     int tune_pdl;
-    int tune_l2_prefetch;   // lane-group kernel: 1 (default) / 0
 };
 
 namespace {
@@ -57,11 +54,8 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.batches_per_cta = ctx->tune_batches_per_cta;
     p.stages = ctx->tune_stages;
     p.warps_per_cta = ctx->tune_warps_per_cta;
-    p.lanes_per_head = ctx->tune_lanes_per_head;
-    p.l2_prefetch = ctx->tune_l2_prefetch;
     p.max_warps_per_sm = ctx->tune_max_warps;
     p.update_impl = ctx->tune_update_impl;
-    p.decode_mma = ctx->tune_decode_mma;
     p.pdl = ctx->tune_pdl;
     return p;
 }
@@ -73,16 +67,15 @@ int set_device(const sketchssm_ctx* ctx) {
     return SKETCHSSM_OK;
 }
 
-int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q, const void* k, const void* v,
-                  const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+// Argument checks shared by every decode entry point, then the parameter block of a decode launch.
+int decode_params(sketchssm_ctx* ctx, int full_read, int n_before, const void* q, const void* k, const void* v,
+                  const void* beta, const void* decay, void* out, uint32_t flags, Params* out_p) {
     if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
     ctx->last_launches = 0;
     if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
     if (n_before < 0 || n_before > ctx->cfg.buf_len - 1) return SKETCHSSM_INVALID_ARG;
     if (flags & ~SKETCHSSM_NO_APPEND) return SKETCHSSM_INVALID_ARG;
-    int rc = check_token_ptrs(q, k, v, beta, decay, out);
-    if (rc != SKETCHSSM_OK) return rc;
-    rc = set_device(ctx);
+    const int rc = check_token_ptrs(q, k, v, beta, decay, out);
     if (rc != SKETCHSSM_OK) return rc;
     Params p = base_params(ctx);
     p.q = q; p.k = k; p.v = v; p.beta = static_cast<const float*>(beta); p.decay = decay; p.out = out;
@@ -90,29 +83,30 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     p.has_token = 1;
     p.append = (flags & SKETCHSSM_NO_APPEND) ? 0 : 1;
     p.full_read = full_read;
+    *out_p = p;
+    return SKETCHSSM_OK;
+}
+
+int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q, const void* k, const void* v,
+                  const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    Params p;
+    int rc = decode_params(ctx, full_read, n_before, q, k, v, beta, decay, out, flags, &p);
+    if (rc != SKETCHSSM_OK) return rc;
+    rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
     // Only a state update writes the sketch.  Unless that was the previous call on this context (it may still be running:
     // programmatic dependent launch), a decode step may read U before it waits for its predecessor in the stream.
     p.early_sketch = (!full_read && !ctx->sketch_fresh) ? 1 : 0;
     ctx->sketch_fresh = false;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (p.early_sketch) {
+        // A step recorded into a stream capture is replayed after whatever the graph's previous launch left running,
+        // which may be a state update of this context: the recorded node always waits first.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(cs, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) p.early_sketch = 0;
+    }
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
-    if (ctx->tune_decode_impl == 1) {
-        if (p.decode_mma) {
-            const int rc = launch_decode_mma(ctx, p, cs);
-            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        }
-        return launch_decode(ctx, p, cs);
-    }
-    if (ctx->tune_decode_impl == 2) {
-        switch (ctx->cfg.kind) {
-            case SKETCHSSM_MAMBA2:
-                return bf ? launch_decode_group_mamba2_bf16(ctx, p, cs) : launch_decode_group_mamba2_f32(ctx, p, cs);
-            case SKETCHSSM_GDN:
-                return bf ? launch_decode_group_gdn_bf16(ctx, p, cs) : launch_decode_group_gdn_f32(ctx, p, cs);
-            default:
-                return bf ? launch_decode_group_kda_bf16(ctx, p, cs) : launch_decode_group_kda_f32(ctx, p, cs);
-        }
-    }
+    if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
     switch (ctx->cfg.kind) {
         case SKETCHSSM_MAMBA2:
             return bf ? launch_decode_split_mamba2_bf16(ctx, p, cs) : launch_decode_split_mamba2_f32(ctx, p, cs);
@@ -152,12 +146,9 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     c->tune_batches_per_cta = 0;
     c->tune_stages = 0;
     c->tune_warps_per_cta = 0;
-    c->tune_lanes_per_head = 0;
     c->tune_decode_impl = 1;
-    c->tune_l2_prefetch = 1;
     c->tune_max_warps = 0;
     c->tune_update_impl = 0;
-    c->tune_decode_mma = 0;
     c->tune_pdl = 1;
     *out = c;
     return SKETCHSSM_OK;
@@ -236,12 +227,9 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
         }
         rc = launch_update_tc(ctx, p, cs);
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        // gated delta rule: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 16, rank <= 16); 2 selects the single-group one
+        // gated delta rule: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 16, rank <= 16)
         if (p.update_impl == 0) {
             rc = launch_update_tc_ws_gdn(ctx, p, cs);
-            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        } else if (p.update_impl == 2) {
-            rc = launch_update_tc_delta(ctx, p, cs);
             if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
         }
     }
@@ -260,24 +248,15 @@ int sketchssm_full_read_decode(sketchssm_ctx* ctx, int n_before, const void* q, 
 
 int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
                                  const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
-    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
-    ctx->last_launches = 0;
-    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
-    if (n_before < 0 || n_before > ctx->cfg.buf_len - 1) return SKETCHSSM_INVALID_ARG;
-    if (flags & ~SKETCHSSM_NO_APPEND) return SKETCHSSM_INVALID_ARG;
-    int rc = check_token_ptrs(q, k, v, beta, decay, out);
+    Params p;
+    int rc = decode_params(ctx, 0, n_before, q, k, v, beta, decay, out, flags, &p);
     if (rc != SKETCHSSM_OK) return rc;
-    if ((size_t)ctx->cfg.batch * ctx->cfg.heads * (size_t)(ctx->cfg.dk + ctx->cfg.buf_len) * sizeof(float) >
-        (size_t)SKETCHSSM_STATIC_WORK_BYTES)
-        return SKETCHSSM_UNSUPPORTED_SHAPE;     // would not fit the library's static array
+    // the size limit of the library's static array is checked (on the host, before any CUDA call) by the launcher
+    const sketchssm_config& c = ctx->cfg;
+    if ((size_t)c.batch * c.heads * (size_t)(c.dk + c.buf_len) * sizeof(float) > (size_t)SKETCHSSM_STATIC_WORK_BYTES)
+        return SKETCHSSM_UNSUPPORTED_SHAPE;
     rc = set_device(ctx);
     if (rc != SKETCHSSM_OK) return rc;
-    Params p = base_params(ctx);
-    p.q = q; p.k = k; p.v = v; p.beta = static_cast<const float*>(beta); p.decay = decay; p.out = out;
-    p.n_before = n_before;
-    p.has_token = 1;
-    p.append = (flags & SKETCHSSM_NO_APPEND) ? 0 : 1;
-    p.full_read = 0;
     return launch_decode_static(ctx, p, static_cast<cudaStream_t>(stream));
 }
 
@@ -332,6 +311,16 @@ int sketchssm_read_status(sketchssm_ctx* ctx, int32_t detail[4], void* stream) {
     return host[0] == 0 ? SKETCHSSM_OK : SKETCHSSM_DEVICE_TIMEOUT;
 }
 
+int sketchssm_selftest_wait_timeout(sketchssm_ctx* ctx, int poll_limit, int where, void* stream) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    ctx->last_launches = 0;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    if (poll_limit < 1 || poll_limit > (1 << 16)) return SKETCHSSM_INVALID_ARG;
+    const int rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    return launch_wait_probe(ctx, poll_limit, where, static_cast<cudaStream_t>(stream));
+}
+
 const char* sketchssm_last_cuda_error(const sketchssm_ctx* ctx) {
     return ctx == nullptr ? "no context" : cudaGetErrorString(ctx->last_cuda_error);
 }
@@ -347,11 +336,8 @@ int sketchssm_tune(sketchssm_ctx* ctx, const char* key, int value) {
     if (eq(key, "decode_batches_per_cta")) { ctx->tune_batches_per_cta = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_stages")) { ctx->tune_stages = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_warps_per_cta")) { ctx->tune_warps_per_cta = value; return SKETCHSSM_OK; }
-    if (eq(key, "decode_lanes_per_head")) { ctx->tune_lanes_per_head = value; return SKETCHSSM_OK; }
-    if (eq(key, "decode_l2_prefetch")) { ctx->tune_l2_prefetch = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_max_warps_per_sm")) { ctx->tune_max_warps = value; return SKETCHSSM_OK; }
     if (eq(key, "pdl")) { ctx->tune_pdl = value; return SKETCHSSM_OK; }
-    if (eq(key, "decode_mma")) { ctx->tune_decode_mma = value; return SKETCHSSM_OK; }
     if (eq(key, "update_impl")) { ctx->tune_update_impl = value; return SKETCHSSM_OK; }
     if (eq(key, "decode_impl")) { ctx->tune_decode_impl = value; return SKETCHSSM_OK; }
     return SKETCHSSM_INVALID_ARG;

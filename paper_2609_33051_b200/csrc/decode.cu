@@ -24,30 +24,8 @@ namespace sketchssm {
 
 namespace {
 
-// Optional phase stamps (warp 0 of CTA 0 and of the middle CTA) into the work buffer; compiled out by default.
-#ifdef SKETCHSSM_PHASE_TIMING
-#define DEC_STAMP(i)                                                                                          \
-    do {                                                                                                      \
-        if (lane == 0 && warp == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2) && it < 8)             \
-            reinterpret_cast<long long*>(p.work)[(blockIdx.x == 0 ? 0 : 256) + it * 8 + (i)] = clock64();     \
-    } while (0)
-#else
-#define DEC_STAMP(i) do { } while (0)
-#endif
 
-#ifdef SKETCHSSM_PHASE_TIMING
-// bounded wait that also counts its polls
-__device__ __forceinline__ bool mbar_wait_counted(uint64_t* bar, uint32_t parity, unsigned long long& polls) {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        ++polls;
-        if (mbar_try_wait(bar, parity)) return true;
-    }
-    return false;
-}
-#define DEC_WAIT(bar, parity) mbar_wait_counted(bar, parity, poll_count)
-#else
 #define DEC_WAIT(bar, parity) mbar_wait_bounded(bar, parity)
-#endif
 
 struct StageLayout {
     uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
@@ -223,10 +201,9 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         if (!early_u) issue_b(bh0);
         scalar_gates(bh0, bt_next, dsc_next);
     }
-    bool dead = false;
-#ifdef SKETCHSSM_PHASE_TIMING
-    unsigned long long poll_count = 0;
-#endif
+    // A wait that runs out ends the warp's loop; the decision is taken by vote so that all lanes leave together.
+    // pendA / pendB: parity of a phase whose copies may still be in flight when the loop is left that way (-1: none).
+    int pendA = -1, pendB = -1;
 
     for (int it = 0; item < item1; ++it) {
         const uint32_t parity = it & 1;
@@ -238,13 +215,12 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         const float bt = bt_next, dsc = dsc_next;
         if (has_next) scalar_gates(bh_next, bt_next, dsc_next);
 
-        DEC_STAMP(0);
-        if (!DEC_WAIT(barA, parity)) {
-            record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
-            dead = true;
+        if (__any_sync(0xffffffffu, !DEC_WAIT(barA, parity))) {
+            if (lane == 0) record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
+            pendA = (int)parity;
+            pendB = p.full_read ? -1 : (int)parity;
             break;
         }
-        DEC_STAMP(1);
         const unsigned char* sb = my_stage;
         const IO* sK = reinterpret_cast<const IO*>(sb + sl.k_off);
         const IO* sV = reinterpret_cast<const IO*>(sb + sl.v_off);
@@ -363,7 +339,6 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         // the sweep is done with the ring part of the stage: the next head's group A may come in
         __syncwarp();
         if (has_next) issue_a(bh_next);
-        DEC_STAMP(2);
         if (!p.full_read) {
             // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
             const float* sC = reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
@@ -384,9 +359,10 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
             __syncwarp();
-            if (!DEC_WAIT(barB, parity)) {
-                record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
-                dead = true;
+            if (__any_sync(0xffffffffu, !DEC_WAIT(barB, parity))) {
+                if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
+                pendB = (int)parity;
+                pendA = has_next ? (int)(parity ^ 1u) : -1;
                 break;
             }
             const float* sU = reinterpret_cast<const float*>(sb + sl.u_off);
@@ -419,7 +395,6 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
             }
         }
 
-        DEC_STAMP(3);
         if (p.out_bf16) {
             store_io<EV>(reinterpret_cast<__nv_bfloat16*>(p.out) + bh * V, lane * EV, o);
         } else {
@@ -427,16 +402,14 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         }
 
         __syncwarp();  // every lane is done with the scratch before it is reused
-        DEC_STAMP(4);
         item = item_next;
         h = hn;
         b = bn;
-        DEC_STAMP(5);
     }
-    (void)dead;
-#ifdef SKETCHSSM_PHASE_TIMING
-    if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long*>(p.work) + 1000, poll_count);
-#endif
+    // Left on a timeout: bulk copies already issued into this warp's stage get a short, bounded grace period, so that
+    // they do not land in shared memory that has meanwhile been handed to another CTA.
+    if (pendA >= 0) mbar_wait_bounded(barA, (uint32_t)pendA, 1u << 14);
+    if (pendB >= 0) mbar_wait_bounded(barB, (uint32_t)pendB, 1u << 14);
 }
 
 template <int KIND, typename IO, int K, int V>

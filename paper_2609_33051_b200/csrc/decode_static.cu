@@ -4,6 +4,8 @@
 // has been sized and frozen up front, a plug-in that is handed its tensors and has no allocator of its own, a
 // stream-ordered region where cudaMalloc would synchronise the device -- and for them a fixed array that every
 // GPU loading the library carries until exit is the only place such scratch can come from.
+#include <atomic>
+
 #include "internal.cuh"
 
 namespace sketchssm {
@@ -18,7 +20,8 @@ constexpr int kMaxDevices = 64;
 static __device__ __align__(256) float g_static_work[kStaticWorkFloats];
 
 // Device address of g_static_work per device ordinal, resolved on the first call made with that device current.
-float* g_static_work_ptr[kMaxDevices] = {nullptr};
+// Atomic because any calling thread may be the first on a device; two threads that race both store the same address.
+std::atomic<float*> g_static_work_ptr[kMaxDevices];
 
 }  // namespace
 
@@ -29,7 +32,8 @@ int launch_decode_static(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
     int dev = -1;
     if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
     if (dev < 0 || dev >= kMaxDevices) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    if (g_static_work_ptr[dev] == nullptr) {
+    float* work = g_static_work_ptr[dev].load(std::memory_order_acquire);
+    if (work == nullptr) {
         // one-time set-up for this device (it is the current one): ask the runtime where the array lives here
         float* ptr = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_work);
@@ -37,10 +41,11 @@ int launch_decode_static(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
             ctx->last_cuda_error = e;
             return SKETCHSSM_CUDA_ERROR;
         }
-        g_static_work_ptr[dev] = ptr;
+        g_static_work_ptr[dev].store(ptr, std::memory_order_release);
+        work = ptr;
     }
     Params p = p_in;
-    p.work = g_static_work_ptr[dev];
+    p.work = work;
     p.wstride = c.dk + c.buf_len;
     const bool bf = c.io_dtype == SKETCHSSM_BF16;
     switch (c.kind) {

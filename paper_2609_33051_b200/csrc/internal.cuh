@@ -16,6 +16,7 @@ constexpr int kStatusInts = 4;
 constexpr int kFaultDecodeWait = 1;
 constexpr int kFaultFullReadWait = 2;
 constexpr int kFaultUpdateWait = 3;
+constexpr int kFaultProbeWait = 4;     // the self-test kernel's wait (sketchssm_selftest_wait_timeout)
 
 struct RingLayout {
     size_t head_bytes, v_off, beta_off, decay_off;
@@ -65,12 +66,9 @@ struct Params {
     int batches_per_cta;
     int stages;
     int warps_per_cta;   // decode: 0 = library default
-    int lanes_per_head;  // decode (group kernel): 8 or 16; 0 = library default
-    int l2_prefetch;     // decode (group kernel): request the following item's operands into L2
     int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
-    int update_impl;      // 0: tensor cores for Mamba-2, CUDA cores otherwise; 1: CUDA cores only; 2: also the GDN tensor-core kernel;
-                          // 3: as 0 but without the warp-specialised kernels (single-group Mamba-2 kernel, CUDA cores for GDN)
-    int decode_mma;       // warp-per-head decode: 1 = tensor-core dot products where supported
+    int update_impl;      // 0: warp-specialised tensor-core kernels where their shape limits allow, CUDA cores otherwise;
+                          // 1: CUDA cores only; 3: single-group tensor-core kernel for Mamba-2, CUDA cores otherwise
     int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
     int early_sketch;     // decode: the first head's sketch rows may be requested before the predecessor in the stream is
                           // waited for (no kernel that may still be running writes the sketch)
@@ -78,8 +76,6 @@ struct Params {
 };
 
 int launch_decode(Ctx* ctx, const Params& p, cudaStream_t stream);        // one warp per head
-int launch_decode_mma(Ctx* ctx, const Params& p, cudaStream_t stream);    // Mamba-2 with tensor-core dot products; UNSUPPORTED_SHAPE outside its domain
-// 8 or 16 lanes per head, one entry per recurrence kind
 // two-kernel decode with the weight hand-off in the library's static device array
 int launch_decode_static(Ctx* ctx, const Params& p, cudaStream_t stream);
 // decode as two kernels (weights, then output rows), one entry per (kind, I/O type)
@@ -89,17 +85,11 @@ int launch_decode_split_gdn_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_split_gdn_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_split_kda_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_split_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_decode_group_mamba2_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_decode_group_mamba2_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_decode_group_gdn_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_decode_group_gdn_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_decode_group_kda_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
-int launch_decode_group_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);       // CUDA cores, every configuration
+int launch_wait_probe(Ctx* ctx, int poll_limit, int where, cudaStream_t stream);   // self-test: a bounded wait that runs out
 int launch_update_tc(Ctx* ctx, const Params& p, cudaStream_t stream);    // tcgen05 tensor cores, Mamba-2; UNSUPPORTED_SHAPE outside its domain
 int launch_update_tc_ws(Ctx* ctx, const Params& p, cudaStream_t stream); // same, two warp groups per CTA (operand building overlaps the state stream)
 int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p, cudaStream_t stream); // gated delta rule, warp-specialised, two passes over the state
-int launch_update_tc_delta(Ctx* ctx, const Params& p, cudaStream_t stream);  // tcgen05 tensor cores, gated delta rule; same convention
 
 // ---------------------------------------------------------------------------------------------
 // device helpers

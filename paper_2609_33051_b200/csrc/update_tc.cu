@@ -26,15 +26,6 @@ namespace {
 
 using namespace tc;
 
-// Optional phase stamps of two CTAs (first and middle of the grid) into the work buffer; compiled out by default.
-#ifdef SKETCHSSM_PHASE_TIMING
-#define PHASE_STAMP(i)                                                                                       \
-    do {                                                                                                     \
-        if (tid == 0 && stamp_base != nullptr && tile - tile0 < 8) stamp_base[(tile - tile0) * 32 + (i)] = clock64(); \
-    } while (0)
-#else
-#define PHASE_STAMP(i) do { } while (0)
-#endif
 
 struct TcSmem {
     uint32_t a1_hi, a1_lo, b1, a2, b2_hi, b2_lo, w, stg, stg_head, bars, tmem_slot, total;
@@ -161,13 +152,7 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
     };
     if (tid == 0 && stg_bytes > 0 && tile0 < tile1) stage_tile(tile0);
 
-#ifdef SKETCHSSM_PHASE_TIMING
-    long long* stamp_base = nullptr;
-    if (blockIdx.x == 0) stamp_base = reinterpret_cast<long long*>(p.work);
-    else if (blockIdx.x == gridDim.x / 2) stamp_base = reinterpret_cast<long long*>(p.work) + 256;
-#endif
     for (int tile = tile0; tile < tile1 && !dead; ++tile) {
-        PHASE_STAMP(0);
         const int h = tile / tiles_per_h;
         const int b0 = (tile - h * tiles_per_h) * NH;
         const size_t bh = (size_t)(b0 + my_head) * H + h;
@@ -195,14 +180,12 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             }
         }
 
-        PHASE_STAMP(1);
         // ---- token weights w_s = beta_s prod_{j>s} a_j and the total decay ----
         // the staged rows and gates of this tile must have landed
         if (stg_bytes > 0) {
             if (!cta_wait(&bars[4], ph4)) { record_fault(p.status, kFaultUpdateWait, 6); dead = true; }
             ph4 ^= 1;
         }
-        PHASE_STAMP(2);
         for (int idx = tid; idx < NH * 64; idx += kTcThreads) {
             const int hd = idx >> 6, s = idx & 63;
             if (s < n_tot) {
@@ -223,7 +206,6 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
         }
         const float* Sg = p.state + bh * (size_t)K * V + j;
         __syncthreads();
-        PHASE_STAMP(3);
 
         // ---- MMA 1 over blocks of kTokBlock tokens per head ----
         const int n_blocks = (n_tot + kTokBlock - 1) / kTokBlock;
@@ -287,7 +269,6 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             proxy_fence();
             tc_fence_before();
             __syncthreads();
-            PHASE_STAMP(4);
             if (tid == 0) {
                 tc_fence_after();
                 if (blk == 0 && stg_bytes > 0 && tile + 1 < tile1) stage_tile(tile + 1);   // staging is free again
@@ -306,7 +287,6 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
             tc_fence_after();
         }
         if (dead) break;
-        PHASE_STAMP(5);
 
         // ---- epilogue: S_new = d S_0 + T, written back; S_new hi/lo -> A operand of MMA 2, 16 rows at a time ----
         // The state rows of the next two chunks are in flight in registers while a chunk is processed.
@@ -377,14 +357,12 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
                 tc_mma_bf16(tmem_u, ahi, blo, idesc2, 1u);
                 tc_commit(c + 1 < NCH ? &bars[1 + (c & 1)] : &bars[3]);
             }
-            PHASE_STAMP(6 + c);
         }
         // drain: the final commit covers every MMA issued so far; chunk 6's commit on bars[1] completed with it
         if (!cta_wait(&bars[3], ph3)) { record_fault(p.status, kFaultUpdateWait, 5); dead = true; }
         ph3 ^= 1;
         ph1[0] ^= 1;
         tc_fence_after();
-        PHASE_STAMP(14);
 
         // ---- UT rows -> sketch and exact output ----
         for (int g0 = 0; g0 < NP; g0 += 16) {
@@ -403,7 +381,6 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
         tc_fence_before();
         dead = __syncthreads_or(dead ? 1 : 0) != 0;   // T / UT are free again; also publishes any fault
         tc_fence_after();
-        PHASE_STAMP(15);
     }
 
     __syncthreads();

@@ -33,18 +33,6 @@ namespace {
 
 using namespace tc;
 
-// Optional phase stamps of the first CTA into the work buffer (stream group: slots 0.., front group: slots 512..);
-// compiled out by default.
-#ifdef SKETCHSSM_PHASE_TIMING
-#define WS_STAMP(base, i)                                                                                      \
-    do {                                                                                                       \
-        if (gt == 0 && blockIdx.x == 0 && k >= 8 && k < 16)                                                   \
-            reinterpret_cast<long long*>(p.work)[(base) + (k - 8) * 32  + (i)] = clock64();                    \
-    } while (0)
-#else
-#define WS_STAMP(base, i) do { } while (0)
-#endif
-
 constexpr int kWsThreads = 320;       // stream group (4 warps), front group (4 warps), MMA-2 issue warp, state-load warp
 constexpr int kGroup = 128;
 
@@ -126,15 +114,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int gt = tid & 127;
-#ifdef SKETCHSSM_PHASE_TIMING
-    if (tid == 0) {
-        unsigned long long t_ns; unsigned smid;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
-        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        long long* rec = reinterpret_cast<long long*>(p.work) + 2048 + 4 * blockIdx.x;
-        rec[0] = (long long)t_ns; rec[2] = smid; rec[3] = clock64();
-    }
-#endif
     const int R = p.R, H = p.H, B = p.B;
     const int QA = (R + 7) & ~7;                          // first column of query group A; group B follows 8 columns later
     const int NP = (QA + 16 + 15) & ~15;                  // 32, or 48 in the WIDE instantiation (chosen by the launcher)
@@ -222,14 +201,12 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             const size_t bh = (size_t)(b0 + my_head) * H + h;
             float* So = p.state + bh * (size_t)K * V + j;
             const uint32_t tmem_t = tmem_base + (uint32_t)b * 128u;
-            WS_STAMP(0, 0);
             // operands-ready (plain arrive: orders the front group's shared-memory writes) and MMA 1 complete
             bad |= !mbar_wait_bounded(&bars[kBarPro + b], (phP >> b) & 1u);
             bad |= !mbar_wait_bounded(&bars[kBarT + b], (phT >> b) & 1u);
             phP ^= 1u << b;
             phT ^= 1u << b;
             tc_fence_after();
-            WS_STAMP(0, 1);
             const float dtot = n_tot > 0 ? reinterpret_cast<const float*>(smem + sm.w + (uint32_t)b * sm.w_stride)[my_head * 208 + 64] : 1.f;
             // T columns that UT will occupy (chunks 0 and 1, and chunk 2 when UT is 48 wide) are read before the first
             // MMA 2 overwrites them
@@ -237,10 +214,8 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             float t2[WIDE ? CH : 1];
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-                if (c == 4) WS_STAMP(0, 12);
                 // this chunk's S_0 rows have landed in their stage; once in registers the stage is released
                 bad |= !mbar_wait_bounded(&bars[kBarFull + stage], phF);
-                if (c == 4) WS_STAMP(0, 13);
                 const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + my_head * CH * V + j;
                 float s0[CH];
 #pragma unroll
@@ -264,14 +239,12 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 #pragma unroll
                     for (int ii = 0; ii < CH; ++ii) t[ii] = 0.f;
                 }
-                if (c == 4) WS_STAMP(0, 14);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[kBarEmpty + stage]);
                 if (gc >= 2) {       // chunk buffer c&1 was read by the MMAs issued two chunks ago
                     bad |= !mbar_wait_bounded(&bars[kBarA2 + (c & 1)], (phA >> (c & 1)) & 1u);
                     phA ^= 1u << (c & 1);
                 }
-                if (c == 4) WS_STAMP(0, 15);
                 unsigned char* a2hi = smem + sm.a2 + (size_t)(c & 1) * (2u * 128u * CH * 2u);
                 unsigned char* a2lo = a2hi + 128u * CH * 2u;
 #pragma unroll
@@ -291,7 +264,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                     *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
                     *reinterpret_cast<uint4*>(a2lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
                 }
-                if (c == 4) WS_STAMP(0, 16);
                 // this warp's 32 rows of the chunk are written (and its T columns read): tell the issue warp
                 proxy_fence();
                 tc_fence_before();
@@ -299,7 +271,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 if (lane == 0 && !bad) mbar_arrive(&bars[kBarA2Rdy + (c & 1)]);
                 ++gc;
                 if (++stage == NS) { stage = 0; phF ^= 1u; }
-                WS_STAMP(0, 2 + c);
             }
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 3);
@@ -545,7 +516,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             unsigned char* sA1lo = sA1hi + OPB;
             unsigned char* sB1 = sA1lo + OPB;
 
-            WS_STAMP(512, 0);
             // gates of the current token (one warp per head needs them for the weight scan): requested early
             float tok_beta = 0.f, tok_a = 1.f;
             if (fwarp < NH && p.has_token) {
@@ -616,7 +586,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                     break;
                 }
             }
-            WS_STAMP(512, 1);
             if (p.q != nullptr) {       // query columns of this tile's group (bf16-exact: lo = 0)
                 for (int idx = gt; idx < K * NH; idx += kGroup) {
                     const int i = idx % K, hd = idx / K, g = QA + 8 * b + hd;
@@ -650,7 +619,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             }
             proxy_fence();         // W is read by MMA 2 (async proxy)
             group_sync(2);
-            WS_STAMP(512, 2);
 
             // ---- MMA 1 over blocks of kTokBlock tokens per head ----
             for (int blk = 0; blk < n_blocks; ++blk) {
@@ -757,7 +725,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
                 }
                 stage_next();
             }
-            WS_STAMP(512, 3);
 
             // ---- sketch rows and exact output of the previous tile, once the stream group has finished it ----
             if (prev_tile >= 0) {
@@ -768,7 +735,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             }
             prev_tile = tile;
             last_b = b;
-            WS_STAMP(512, 4);
         }
         if (!dead && prev_tile >= 0) {
             // the last tile used buffer (number of tiles - 1) & 1; phU tells which buffer has an odd number of stores
@@ -786,14 +752,6 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 
     tc_fence_before();
     __syncthreads();
-#ifdef SKETCHSSM_PHASE_TIMING
-    if (tid == 0) {
-        unsigned long long t_ns;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
-        long long* rec = reinterpret_cast<long long*>(p.work) + 2048 + 4 * blockIdx.x;
-        rec[1] = (long long)t_ns; rec[3] = clock64() - rec[3];
-    }
-#endif
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }

@@ -42,16 +42,6 @@ namespace {
 
 using namespace tc;
 
-// Optional phase stamps of the first CTA into the work buffer; compiled out by default.
-#ifdef SKETCHSSM_PHASE_TIMING
-#define G_STAMP(base, k, i)                                                                              \
-    do {                                                                                                 \
-        if ((tid & 127) == 0 && blockIdx.x == 0 && (k) >= 8 && (k) < 16)                                   \
-            reinterpret_cast<long long*>(p.work)[(base) + ((k) - 8) * 16 + (i)] = clock64();             \
-    } while (0)
-#else
-#define G_STAMP(base, k, i) do { } while (0)
-#endif
 
 constexpr int kGThreads = 448;       // pass-A group (4 warps), front group (4 warps), MMA issue warp, state-load warp, pass-B group (4 warps)
 constexpr int kGrp = 128;
@@ -322,17 +312,12 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const int raw = seq_get(k + 1);
                 if (raw < -1) { bad = true; break; }
                 if (raw < 0) break;
-                G_STAMP(0, k, 0);
                 wait_pro(b ^ 1);
-                G_STAMP(0, k, 1);
                 pass_a(b ^ 1, true);
-                G_STAMP(0, k, 2);
                 // the E' operand buffer is read by K^T E' of tile k: that must be complete before it is rewritten
                 bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);
                 phT ^= 1u << b;
-                G_STAMP(0, k, 3);
                 do_e(b ^ 1);
-                G_STAMP(0, k, 5);
             }
         } else if (cur < -1) {
             bad = true;
@@ -351,10 +336,8 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bh = (size_t)bb * H + h;
             float* So = p.state + bh * (size_t)K * V + j;
-            G_STAMP(128, k, 0);
             bad |= !mbar_wait_bounded(&bars[gTfull + b], (phT >> b) & 1u);      // K^T E' and the sketch correction are complete
             phT ^= 1u << b;
-            G_STAMP(128, k, 1);
             tc_fence_after();
             const float dtot = sDt[b];
 #pragma unroll 2
@@ -371,7 +354,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = t[ii];
                 }
             }
-            G_STAMP(128, k, 2);
             // this warp has read its lanes of K^T E': the accumulator may be overwritten
             tc_fence_before();
             bad = __any_sync(0xffffffffu, bad);
@@ -398,7 +380,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 __syncwarp();
                 if (lane == 0) g_arrive(&bars[gBufFree + b]);       // the slot is free for pass A of tile k + 2
             }
-            G_STAMP(128, k, 3);
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 11);
     } else if (warp == 8) {
@@ -423,7 +404,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 const uint32_t tmem_win = slot + (b ? 0u : 16u);
                 const uint32_t tmem_u0 = slot + (b ? 0u : 32u);
                 const uint32_t win = sW + (b ? 2u : 0u) * SBO;
-                G_STAMP(384, k, 0);
 #pragma unroll 2
                 for (int c = 0; c < NCH; ++c) {
                     const int ab = c & (kA2 - 1);
@@ -441,14 +421,11 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                     tc_commit(&bars[gA2free + ab]);
                     if (c == NCH - 1) tc_commit(&bars[gPfull + b]);
                 }
-                G_STAMP(384, k, 1);
             };
             auto step_e = [&](int k) {          // T = K^T E' (128 columns) and the sketch correction E'^T (K W) over the spent P
                 const int b = k & 1;
-                G_STAMP(384, k, 2);
                 if (!mbar_wait_bounded(&bars[gErdy], phE)) { bad = true; where = 43; return; }
                 phE ^= 1u;
-                G_STAMP(384, k, 3);
                 if (k >= 1) {                   // the pass-B group must have read K^T E' of the tile before
                     if (!mbar_wait_bounded(&bars[gBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 44; return; }
                 }
@@ -468,7 +445,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 tc_mma_bf16(tmem_c, elo, bchi, idescU, 1u);
                 tc_mma_bf16(tmem_c, ehi, bclo, idescU, 1u);
                 tc_commit(&bars[gTfull + b]);
-                G_STAMP(384, k, 4);
             };
             int cur = seq_get(0);
             if (cur >= 0) {
@@ -634,7 +610,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             const size_t bh = (size_t)bb * H + h;
             unsigned char* set = set_ptr(b);
 
-            G_STAMP(256, k, 0);
             // gates of the current token: requested early
             float tok_beta = 0.f, tok_a = 1.f;
             if (gt < kNTok && p.has_token) {
@@ -656,7 +631,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 break;
             }
             phS ^= 1;
-            G_STAMP(256, k, 1);
 
             // ---- key layouts, value rows, query column, gates ----
 #pragma unroll
@@ -726,7 +700,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 sGm[(r0 + 8) * kGS + c0 + 1] = acc[3];
             }
             g_sync(2);
-            G_STAMP(256, k, 2);
             // beta_s A_sj in place of the Gram entries (strictly lower triangle)
             if (gt < n_tot) {
                 const int s = gt;
@@ -734,7 +707,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 for (int jj = 0; jj < s; ++jj) sGm[s * kGS + jj] *= bs * sPm[s * kGS + jj];
             }
             g_sync(2);
-            G_STAMP(256, k, 3);
             // ---- T = (I + Bd A)^{-1} Bd by forward substitution: one column per thread, held in registers ----
             if (gt < kNTok) {
                 const int c = gt;
@@ -757,7 +729,6 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
                 for (int s = 0; s < kNTok; ++s) sTm[s * kGS + c] = tcol[s] * bc;
             }
             g_sync(2);
-            G_STAMP(256, k, 4);
             // ---- T1 = Dn T (rows and columns beyond the tokens are zero), C diagonal, total decay ----
             {
                 float* sT1 = reinterpret_cast<float*>(set + sm.set_t1);
@@ -841,9 +812,7 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             g_sync(2);
             if (gt == 0) g_arrive(&bars[gPro + b]);
             next_tile(k + 1);      // the staging buffer has been read: the next tile's rows may come in
-            G_STAMP(256, k, 5);
 
-            G_STAMP(256, k, 6);
         }
         if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
             __threadfence();

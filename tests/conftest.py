@@ -10,8 +10,3 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: test needs a CUDA device (run with -m gpu on a B200)")
-
-
-def pytest_collection_modifyitems(config, items):
-    """GPU tests fail loudly instead of silently skipping when selected on a box without CUDA."""
-    return

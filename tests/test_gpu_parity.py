@@ -37,27 +37,40 @@ def make_layer(w, layer=0, out="f32"):
     return m, S0, Om, C, dev
 
 
-def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32"):
-    """Algorithm 1 on GPU and oracle; returns the worst per-step relative error and the final-state errors."""
+def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", input_batch=None, per_element=None):
+    """Algorithm 1 on GPU and oracle; returns the worst per-step relative error and the final-state errors.
+
+    input_batch: generate the token inputs for this many batch entries and repeat them over the batch (the initial
+    states stay distinct per entry, so every entry still follows its own trajectory); keeps the host-side input
+    generation of the largest batches short.  per_element: optional callable(got, ref) run on every step's outputs.
+    errs["windows"] lists the worst output error of each window, so drift across flushes is visible."""
     m, S0, Om, C, dev = make_layer(w, out=out)
     for key, val in (tune or {}).items():
         m.tune(key, val)
     bs, hs = harness.select_heads(w, max_heads)
+    wi = w if not input_batch or input_batch >= w.batch else w.replace(batch=input_batch)
+    reps = w.batch // wi.batch
+    assert reps * wi.batch == w.batch
+    bsi = bs % wi.batch
     m.state_update(0)                                   # initial sketch from the prefilled state
     S = S0[bs, hs].astype(np.float64)
     Om_s, C_s = Om[hs].astype(np.float64), C[hs].astype(np.float64)
     U = orc.sketch_of(S, Om_s)
     errs = {"u0": harness.rel_err(m.sketch.cpu().numpy()[bs, hs].transpose(0, 2, 1), U)}
     worst = 0.0
+    windows = []
     ring = []
     o_dev = m.new_output()
     L = w.buf_len
+    bs_t, hs_t = torch.from_numpy(bs).to(dev), torch.from_numpy(hs).to(dev)
     for t in range(steps):
-        x = synth.step_inputs(w, 0, t)
-        tt = harness.token_tensors(w, x, dev)
+        x = synth.step_inputs(wi, 0, t)
+        tt = harness.token_tensors(wi, x, dev)
+        if reps > 1:
+            tt = {k: v.repeat(reps, *([1] * (v.dim() - 1))).contiguous() for k, v in tt.items()}
         n = t % L
-        ring.append(harness.oracle_token(x, bs, hs))
-        q = x["q"][bs, hs].astype(np.float64)
+        ring.append(harness.oracle_token(x, bsi, hs))
+        q = x["q"][bsi, hs].astype(np.float64)
         if n < L - 1:
             if mode == "sketch":
                 m.decode_step(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
@@ -71,18 +84,27 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32"):
             ring = []
         # the two-kernel decode launches twice; a GDN flush of more than 16 tokens is one launch per block of 16
         assert 1 <= m.last_launch_count() <= max(2, (w.buf_len + 15) // 16)
-        got = o_dev.float().cpu().numpy()[bs, hs]
+        got = o_dev[bs_t, hs_t].float().cpu().numpy()
         assert np.all(np.isfinite(got))
-        worst = max(worst, harness.rel_err(got, ref))
+        if per_element is not None:
+            per_element(got, ref)
+        e = harness.rel_err(got, ref)
+        worst = max(worst, e)
+        if n == 0:
+            windows.append(0.0)
+        windows[-1] = max(windows[-1], e)
     m.check_status()
     errs["out"] = worst
-    errs["S"] = harness.rel_err(m.state.cpu().numpy()[bs, hs], S)
-    errs["U"] = harness.rel_err(m.sketch.cpu().numpy()[bs, hs].transpose(0, 2, 1), U)
+    errs["S"] = harness.rel_err(m.state[bs_t, hs_t].cpu().numpy(), S)
+    errs["U"] = harness.rel_err(m.sketch[bs_t, hs_t].cpu().numpy().transpose(0, 2, 1), U)
+    errs["windows"] = windows
     return errs
 
 
 def check(errs, io, guard=FP32_GUARD):
     for key, e in errs.items():
+        if key == "windows":
+            continue
         assert e <= TOL[io], (key, e, errs)
         assert e <= guard, (key, e, errs)
 
@@ -132,12 +154,9 @@ def test_ranks_and_window_lengths(kind, rank, buf_len):
 @pytest.mark.parametrize("kind", synth.KINDS)
 @pytest.mark.parametrize("tune", [{"decode_impl": 1, "decode_stages": 1, "decode_batches_per_cta": 1},
                                   {"decode_impl": 1, "decode_stages": 2, "decode_batches_per_cta": 7},
-                                  {"decode_impl": 2, "decode_stages": 1, "decode_warps_per_cta": 1},
-                                  {"decode_impl": 2, "decode_stages": 2, "decode_warps_per_cta": 3},
-                                  {"decode_impl": 2, "decode_l2_prefetch": 0},
                                   {"decode_impl": 0, "decode_stages": 2, "decode_warps_per_cta": 2},
                                   {"decode_impl": 0, "decode_stages": 1, "decode_max_warps_per_sm": 4},
-                                  {"decode_impl": 1, "decode_mma": 1}, {"update_impl": 1}])
+                                  {"update_impl": 1}])
 def test_launch_tunings_and_ragged_batches(kind, tune):
     w = synth.Workload("t", kind, 37, 3, 128, 128, 16, 16, 0, "bf16", 7, basis="qr")
     check(run_schedule(w, 20, max_heads=10**9, tune=tune), "bf16")
@@ -146,9 +165,8 @@ def test_launch_tunings_and_ragged_batches(kind, tune):
 
 @pytest.mark.parametrize("dv,rank,buf_len", [(64, 16, 16), (128, 40, 48), (64, 5, 64)])
 def test_mamba2_tensor_core_variants(dv, rank, buf_len):
-    """Mamba-2 decode with mma.sync dot products, and the tcgen05 update against the CUDA-core update."""
+    """The Mamba-2 flush on CUDA cores and as the single-group tcgen05 kernel (ranks above 32 use it by default)."""
     w = synth.Workload("t", "mamba2", 6, 3, 128, dv, rank, buf_len, 0, "bf16", 77, basis="qr")
-    check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"decode_mma": 1}), "bf16")
     check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"update_impl": 1}), "bf16")
     check(run_schedule(w, buf_len + 5, max_heads=10**9, tune={"update_impl": 3}), "bf16")     # single-group tcgen05 kernel
 
@@ -161,13 +179,6 @@ def test_mamba2_update_several_tiles_per_cta(tune, dv, batch, heads, buf_len, ra
     sets and W buffers; head index changes inside a CTA's range), over two windows."""
     w = synth.Workload("t", "mamba2", batch, heads, 128, dv, rank, buf_len, 0, "bf16", 79, basis="qr")
     check(run_schedule(w, 2 * buf_len + 2, max_heads=96, tune=tune), "bf16")
-
-
-@pytest.mark.parametrize("rank,buf_len,steps", [(16, 16, 37), (8, 32, 70), (40, 12, 30)])
-def test_gdn_tensor_core_update(rank, buf_len, steps):
-    """The gated delta rule flush as tcgen05 contractions (WY form) against the oracle's token-by-token replay."""
-    w = synth.Workload("t", "gdn", 5, 3, 128, 128, rank, buf_len, 0, "bf16", 91, basis="qr")
-    check(run_schedule(w, steps, max_heads=10**9, tune={"update_impl": 2}), "bf16")
 
 
 @pytest.mark.parametrize("tune", [{}, {"decode_max_warps_per_sm": 10}, {"pdl": 0}])
@@ -221,10 +232,15 @@ def test_flush_at_any_ring_fill(kind, dv, buf_len, fills):
 
 
 def test_bf16_output_mode():
+    """A bf16-stored output carries its own rounding on top of the arithmetic error; checked element by element:
+    |o_gpu - o_ref| <= 2e-3 * max|o_ref| + 2^-8 |o_ref_i| for every output element of every step."""
     w = synth.Workload("t", "gdn", 4, 2, 128, 128, 16, 8, 0, "bf16", 5, basis="qr")
-    errs = run_schedule(w, 12, max_heads=10**9, out="bf16")
-    # a bf16-stored output carries its own rounding of 2^-8 relative on top of the arithmetic error
-    assert errs["out"] <= 2e-3 + 2.0 ** -8, errs
+
+    def per_element(got, ref):
+        bound = 2e-3 * np.abs(ref).max() + 2.0 ** -8 * np.abs(ref)
+        assert np.all(np.abs(got.astype(np.float64) - ref) <= bound)
+
+    errs = run_schedule(w, 12, max_heads=10**9, out="bf16", per_element=per_element)
     assert errs["S"] <= FP32_GUARD and errs["U"] <= FP32_GUARD
 
 

@@ -15,7 +15,7 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2609_33051_b200 import binding, synth
+from paper_2609_33051_b200 import binding, build, synth
 from tests import harness
 
 TOL = 2e-5      # same fp32 arithmetic on the same bits; only the summation order differs between the two paths
@@ -43,6 +43,10 @@ def test_static_decode_matches_regular_decode_on_two_calls_in_a_row(kind):
     ref, got = m.new_output(), m.new_output()
     for t in range(3):                                   # three buffered tokens through the regular path
         m.decode_step(t, *args(t), ref)
+    # the caller's scratch must never be touched by the static call: fill it with a sentinel and compare afterwards
+    # (the regular decode step runs as one kernel and leaves it alone too)
+    sentinel = torch.arange(m.work.numel(), dtype=torch.float32, device=dev) * 0.5 - 7.0
+    m.work.copy_(sentinel)
     # call 1: token 3 at ring fill 3, not appended by the reference, appended by the static call
     m.decode_step(3, *args(3), ref, flags=binding.NO_APPEND)
     m.decode_step_static(3, *args(3), got)
@@ -56,11 +60,22 @@ def test_static_decode_matches_regular_decode_on_two_calls_in_a_row(kind):
     rk, rv, rb, rd = m.ring_views()
     assert torch.equal(rk[:, :, 3], toks[3]["k"]) and torch.equal(rv[:, :, 3], toks[3]["v"])
     assert torch.equal(rb[:, :, 3], toks[3]["beta"]) and torch.equal(rd[:, :, 3], toks[3]["decay"])
+    assert torch.equal(m.work, sentinel), "sketchssm_decode_step_static wrote to the caller's work buffer"
+    # and against the oracle directly: the step at ring fill 4 over the five tokens now known to the ring
+    from oracle import sketchssm_oracle as orc
+    Om, C = harness.basis_for(w)
+    S0 = synth.initial_state(w).astype(np.float64)
+    U = orc.sketch_of(S0, Om.astype(np.float64)[None])
+    xs = [synth.step_inputs(w, 0, t) for t in range(5)]
+    ring = [tuple(x[n].astype(np.float64) for n in ("k", "v", "beta", "decay")) for x in xs]
+    want = orc.decode_step(kind, U, C.astype(np.float64)[None], ring, xs[4]["q"].astype(np.float64))
+    assert harness.rel_err(got.cpu().numpy(), want) <= 5e-5
     m.check_status()
 
 
 def test_static_decode_rejects_what_does_not_fit_its_array():
     """Host-side check, no GPU needed: batch * heads * (dk + buf_len) floats must fit in 4 MiB."""
+    build.build()
     lib = binding.load_library()
     cfg = binding.Config(kind=0, batch=256, heads=64, dk=128, dv=64, rank=16, buf_len=16, io_dtype=1, out_dtype=0, device=0)
     ctx = ctypes.c_void_p()
