@@ -81,3 +81,20 @@ def test_rank_sharding_and_max_over_ranks_timing_with_gloo(tmp_path):
     assert r0["ms"] == 15.0                       # max over ranks
     assert abs(r0["value"] - 2 * 1000 / 15e-3) < 1e-6
     assert r0["shard"] == [0, 4] and r1["shard"] == [4, 9]     # disjoint cover of the batch, no exchange needed
+
+
+def test_logical_layers_map_onto_the_physical_slots_that_fit():
+    """The 48-layer stack of the large-batch sweep does not fit at batch 2048: the benchmark maps the logical layers
+    round-robin onto as many physical slots as its memory budget holds."""
+    import bench
+    w = synth.sweep_point(2048, 16, 16)
+    per = bench.layer_bytes(w)
+    assert per > 2048 * 64 * 128 * 64 * 4                       # at least the state: 4 GiB per layer
+    assert 48 * per > 180e9                                     # 48 distinct layers exceed the GPU's memory
+    n = bench.physical_layers(per, int(100e9), 48)
+    assert 1 <= n < 48 and n * per <= 100e9 < (n + 1) * per
+    assert bench.physical_layers(bench.layer_bytes(synth.sweep_point(64, 4, 8)), int(40e9), 48) == 48
+    assert bench.physical_layers(10**12, 10**9, 48) == 1        # never fewer than one slot
+    assert [l % n for l in range(48)].count(0) == -(-48 // n)   # slot 0 serves ceil(48 / n) logical layers
+    assert bench.update_kernel_name(w) == "update_tc_ws_mamba2_kernel"
+    assert bench.update_kernel_name(synth.CONFIGS["c4_kda"]) == "update_kernel"
