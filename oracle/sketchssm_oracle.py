@@ -25,8 +25,12 @@ the scalar alpha_t (GDN) or the vector g_t in (0,1)^K (KDA).
 Pinned by tests/test_oracle_pins.py against: the exact decomposition of the
 read (Eq. 4), explicit dense transition matrices built with Python loops, the
 identity-basis special case, replay == repeated single updates, the empty-buffer
-case, the WY identities (Eq. 41-45), the PCA closed forms of Appendix A.1 and
-the traffic-reduction values printed in Tables 4-7.  Absolute output values on
+case, the WY identities (Eq. 41-45), the PCA closed forms of Appendix A.1, the
+traffic-reduction values printed in Tables 4-7, and for the state-dependent
+coefficient maps of Appendix A.2: a library least-squares solve of the ridge
+problem, the range projection in the limit of no ridge, independence of the
+orthogonal completion, the Woodbury step against a dense inverse, exactness of
+the pivot approximation when P >= G, and a hand-rolled brute force on tiny heads.  Absolute output values on
 the benchmark workloads have no printed counterpart in the paper: for those,
 parity is pinned only through the identities above ("parity unpinned" by a
 worked numeric example).
@@ -293,6 +297,120 @@ def state_dependent_coefficient_map(S0, U):
     """C = (U^T U)^+ U^T S_0^T (Eq. 9), the least-squares map for the current state."""
     S0, U = _f64(S0), _f64(U)
     return np.linalg.pinv(U.T @ U) @ U.T @ S0.T
+
+
+def _orthogonal_completion(Omega):
+    """R in R^{K x K} with R^T R = I whose first G rows are Omega^T (Appendix A.2.2, Step 1: the orthonormal
+    sketching matrix completed to an orthogonal matrix R^T = [Omega | Omega_perp], so that Omega = R^T J)."""
+    Omega = _f64(Omega)
+    K, G = Omega.shape
+    assert np.allclose(Omega.T @ Omega, np.eye(G), atol=1e-5), "Appendix A.2.2 assumes an orthonormal sketching matrix"
+    Uf, _s, _vt = np.linalg.svd(Omega, full_matrices=True)        # columns G.. of Uf span the complement of range(Omega)
+    return np.concatenate([Omega, Uf[:, G:]], axis=1).T
+
+
+def _rotated_metric(S0, Omega):
+    """S'_0 = R S_0, x-coordinates R, the normalisation mu = ||S'_0||_F^2 / K (mu = 1 for a zero state) and the
+    normalised state metric H = S'_0 S'_0^T / mu (Eq. 26-27)."""
+    S0 = _f64(S0)
+    K = S0.shape[0]
+    R = _orthogonal_completion(Omega)
+    Sp = R @ S0
+    mu = float(np.sum(Sp * Sp)) / K
+    if mu == 0.0:
+        mu = 1.0
+    return R, Sp, mu, Sp @ Sp.T / mu
+
+
+def ridge_coefficient_map(S0, Omega, lam=0.1):
+    """Exact regularised state-dependent coefficient map of one head (Appendix A.2.2, Step 1, Eq. 28-29).
+
+    In the basis-aligned coordinates x_t = R q~_t the coefficient vector minimises
+    (x_t - J c)^T H (x_t - J c) + lam ||c||^2, so c = (J^T H J + lam I_G)^{-1} J^T H x_t with J the first G
+    coordinate vectors.  Returned as the map C [G, K] acting on the effective query itself: c = C q~_t.
+    S0 [K, V], Omega [K, G] orthonormal.
+    """
+    Omega = _f64(Omega)
+    K, G = Omega.shape
+    R, _Sp, _mu, H = _rotated_metric(S0, Omega)
+    J = np.eye(K)[:, :G]
+    return np.linalg.solve(J.T @ H @ J + lam * np.eye(G), J.T @ H) @ R
+
+
+def pivot_metric_factors(S0, Omega, P=4):
+    """The low-rank-plus-diagonal factors of Appendix A.2.2, Step 2 (Eq. 30-33), for one head.
+
+    p = min(G, P); Q [V, p] is an orthonormal basis of the first p columns of the sketch U = S'_0^T J, built by
+    Gram-Schmidt in column order (a column that lies in the span of its predecessors contributes a zero column);
+    L = S'_0 Q / sqrt(mu) [K, p]; d_i = max(H_ii - ||L_i||^2, 0).  Returns (R, mu, Q, L, d).
+    """
+    Omega = _f64(Omega)
+    K, G = Omega.shape
+    R, Sp, mu, H = _rotated_metric(S0, Omega)
+    p = min(G, P)
+    J = np.eye(K)[:, :G]
+    U = Sp.T @ J                                                   # the current sketch, V x G
+    Q = np.zeros((U.shape[0], p))
+    for j in range(p):
+        u = U[:, j].copy()
+        for i in range(j):
+            u -= Q[:, i] * (Q[:, i] @ U[:, j])
+        for i in range(j):                                         # second sweep: re-orthogonalise
+            u -= Q[:, i] * (Q[:, i] @ u)
+        nrm, ref = np.linalg.norm(u), np.linalg.norm(U[:, j])
+        Q[:, j] = u / nrm if nrm > 1e-10 * max(ref, 1e-300) and ref > 0 else 0.0
+    L = Sp @ Q / np.sqrt(mu)
+    d = np.maximum(np.diag(H) - np.sum(L * L, axis=1), 0.0)
+    return R, mu, Q, L, d
+
+
+def pivot_coefficient_map(S0, Omega, lam=0.1, P=4):
+    """State-dependent coefficient map with the approximated state metric H^ = L L^T + Diag(d)
+    (Appendix A.2.2, Steps 2-4, Eq. 30-37), for one head; returns C [G, K] with c_t = C q~_t.
+
+    With L_G = J^T L, D_G = Diag(J^T d) + lam I:  c = (D_G + L_G L_G^T)^{-1} [L_G (L^T x_t) + J^T Diag(d) x_t],
+    the inverse taken through the Woodbury identity with the p x p system T_P = I_p + L_G^T D_G^{-1} L_G.
+    """
+    Omega = _f64(Omega)
+    K, G = Omega.shape
+    R, _mu, _Q, L, d = pivot_metric_factors(S0, Omega, P)
+    p = L.shape[1]
+    J = np.eye(K)[:, :G]
+    LG = J.T @ L                                                   # G x p
+    DG = J.T @ d + lam                                             # diagonal of D_G
+    rhs = LG @ L.T + J.T @ np.diag(d)                              # G x K: maps x_t to J^T H^ x_t
+    TP = np.eye(p) + LG.T @ (LG / DG[:, None])
+    Dinv_rhs = rhs / DG[:, None]
+    A_inv_rhs = Dinv_rhs - (LG / DG[:, None]) @ np.linalg.solve(TP, LG.T @ Dinv_rhs)
+    return A_inv_rhs @ R
+
+
+def coefficient_maps(S, Omega, mode, lam=0.1, P=4):
+    """Per-head state-dependent maps for a batch of heads: S [N, K, V], Omega [N, K, G] -> C [N, G, K].
+    mode "ridge": ridge_coefficient_map; mode "pivot": pivot_coefficient_map."""
+    S, Omega = _f64(S), _f64(Omega)
+    fn = {"ridge": lambda s, o: ridge_coefficient_map(s, o, lam), "pivot": lambda s, o: pivot_coefficient_map(s, o, lam, P)}[mode]
+    return np.stack([fn(S[i], Omega[i]) for i in range(S.shape[0])])
+
+
+def run_schedule_state_dependent(kind, S_init, Omega, step_tokens, step_queries, L, mode, lam=0.1, P=4):
+    """Algorithm 1 with the coefficient map rebuilt from the state at every flush (and from the initial state):
+    "construct the initial U, C from S_0", then per window L-1 sketch reads and one exact flush followed by U, C.
+    Heads on the leading axis: S_init [N, K, V], Omega [N, K, G].  Returns (outputs, S, U, C)."""
+    S = _f64(S_init)
+    U = sketch_of(S, Omega)
+    C = coefficient_maps(S, Omega, mode, lam, P)
+    ring, outs = [], []
+    for tok, q in zip(step_tokens, step_queries):
+        ring.append(tok)
+        if len(ring) < L:
+            outs.append(decode_step(kind, U, C, ring, q))
+        else:
+            S, U, o = state_update(kind, S, ring, Omega, q)
+            C = coefficient_maps(S, Omega, mode, lam, P)
+            outs.append(o)
+            ring = []
+    return outs, S, U, C
 
 
 # ----------------------------------------------------------------------------

@@ -436,3 +436,181 @@ def test_schedule_flush_outputs_are_exact_and_state_matches_recurrence(kind):
     for t in range(T):
         S = orc.transition(kind, S, *toks[t])
         np.testing.assert_allclose(outs_id[t], S.T @ qs[t], atol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# State-dependent coefficient maps (Appendix A.2.2, Eq. 26-37)
+# ---------------------------------------------------------------------------
+
+def _head(rng, K, V, G):
+    S = rng.standard_normal((K, V)) * rng.uniform(0.2, 2.0, (K, 1))
+    Om = np.linalg.qr(rng.standard_normal((K, G)))[0]
+    return S, Om
+
+
+def test_ridge_map_is_the_regularised_least_squares_solution():
+    """c = C q~ minimises ||S^T (q~ - Omega c)||^2 / mu + lam ||c||^2 (Eq. 28-29 carried back to the original
+    coordinates, which the orthogonal change of basis preserves): a library least-squares solve of the stacked
+    system [S^T Omega / sqrt(mu); sqrt(lam) I] c = [S^T q~ / sqrt(mu); 0] gives the same vector."""
+    rng = np.random.default_rng(11)
+    for (K, V, G, lam) in [(16, 12, 5, 0.1), (24, 8, 8, 0.1), (10, 10, 3, 2.5)]:
+        S, Om = _head(rng, K, V, G)
+        C = orc.ridge_coefficient_map(S, Om, lam)
+        mu = float((S * S).sum()) / K
+        for _ in range(3):
+            q = rng.standard_normal(K)
+            A = np.concatenate([S.T @ Om / np.sqrt(mu), np.sqrt(lam) * np.eye(G)])
+            b = np.concatenate([S.T @ q / np.sqrt(mu), np.zeros(G)])
+            c_ls = np.linalg.lstsq(A, b, rcond=None)[0]
+            np.testing.assert_allclose(C @ q, c_ls, atol=1e-10)
+
+
+def test_ridge_map_tends_to_the_range_projection_without_ridge():
+    """lam -> 0 with a full-column-rank sketch: the map of Eq. 9, and U c is the orthogonal projection of the
+    exact read onto range(U) (Eq. 25)."""
+    rng = np.random.default_rng(12)
+    S, Om = _head(rng, 20, 14, 6)
+    U = S.T @ Om
+    C0 = orc.ridge_coefficient_map(S, Om, 1e-13)
+    np.testing.assert_allclose(C0, orc.state_dependent_coefficient_map(S, U), atol=1e-7)
+    q = rng.standard_normal(20)
+    resid = S.T @ q - U @ (C0 @ q)
+    np.testing.assert_allclose(U.T @ resid, 0.0, atol=1e-7)
+
+
+def test_state_dependent_maps_do_not_depend_on_the_orthogonal_completion():
+    """R completes Omega to an orthogonal matrix; any completion must give the same map.  A second completion is
+    obtained by rotating the complement, and the maps are rebuilt from scratch in those coordinates."""
+    rng = np.random.default_rng(13)
+    K, V, G = 14, 9, 5
+    S, Om = _head(rng, K, V, G)
+    R1 = orc._orthogonal_completion(Om)
+    W = np.linalg.qr(rng.standard_normal((K - G, K - G)))[0]
+    R2 = np.concatenate([R1[:G], W @ R1[G:]])
+    np.testing.assert_allclose(R2 @ R2.T, np.eye(K), atol=1e-12)
+    lam = 0.1
+    mu = float((S * S).sum()) / K
+    J = np.eye(K)[:, :G]
+    for name, C in (("ridge", orc.ridge_coefficient_map(S, Om, lam)), ("pivot", orc.pivot_coefficient_map(S, Om, lam, 3))):
+        Sp = R2 @ S
+        H = Sp @ Sp.T / mu
+        if name == "ridge":
+            C2 = np.linalg.solve(J.T @ H @ J + lam * np.eye(G), J.T @ H) @ R2
+        else:
+            Uq = np.linalg.qr((Sp.T @ J)[:, :3])[0]
+            L = Sp @ Uq / np.sqrt(mu)
+            d = np.maximum(np.diag(H) - (L * L).sum(1), 0.0)
+            Hh = L @ L.T + np.diag(d)
+            C2 = np.linalg.solve(J.T @ Hh @ J + lam * np.eye(G), J.T @ Hh) @ R2
+        np.testing.assert_allclose(C, C2, atol=1e-10, err_msg=name)
+
+
+def test_pivot_map_woodbury_step_equals_a_dense_solve_and_keeps_the_diagonal():
+    """(D_G + L_G L_G^T)^{-1} through the p x p Woodbury system equals a dense G x G solve with H^ = L L^T + Diag(d)
+    (Eq. 34-37), and H^ keeps the diagonal of H (Eq. 33)."""
+    rng = np.random.default_rng(14)
+    for (K, V, G, P) in [(16, 12, 7, 4), (12, 20, 5, 2), (18, 6, 6, 4)]:
+        S, Om = _head(rng, K, V, G)
+        lam = 0.1
+        R, mu, Q, L, d = orc.pivot_metric_factors(S, Om, P)
+        Sp = R @ S
+        H = Sp @ Sp.T / mu
+        np.testing.assert_allclose(Q.T @ Q, np.eye(min(G, P)), atol=1e-12)
+        # Q spans the first p sketch columns
+        Up = (S.T @ Om)[:, :min(G, P)]
+        np.testing.assert_allclose(Q @ (Q.T @ Up), Up, atol=1e-10)
+        Hh = L @ L.T + np.diag(d)
+        np.testing.assert_allclose(np.diag(Hh), np.diag(H), atol=1e-12)
+        J = np.eye(K)[:, :G]
+        dense = np.linalg.solve(J.T @ Hh @ J + lam * np.eye(G), J.T @ Hh) @ R
+        np.testing.assert_allclose(orc.pivot_coefficient_map(S, Om, lam, P), dense, atol=1e-10)
+
+
+def test_pivot_map_with_all_sketch_columns_as_pivots_is_the_ridge_map():
+    """P >= G: Q spans range(U), so L L^T reproduces every block of H the solve uses and the residual diagonal on the
+    retained coordinates vanishes: the approximation is exact."""
+    rng = np.random.default_rng(15)
+    S, Om = _head(rng, 16, 11, 4)
+    for P in (4, 6):
+        np.testing.assert_allclose(orc.pivot_coefficient_map(S, Om, 0.1, P), orc.ridge_coefficient_map(S, Om, 0.1), atol=1e-10)
+    assert np.abs(orc.pivot_coefficient_map(S, Om, 0.1, 2) - orc.ridge_coefficient_map(S, Om, 0.1)).max() > 1e-3
+
+
+def test_pivot_map_handles_dependent_pivot_columns_and_the_zero_state():
+    rng = np.random.default_rng(16)
+    K, V, G = 10, 8, 4
+    S, Om = _head(rng, K, V, G)
+    # make the second sketch column a multiple of the first: S^T (omega_2 - 3 omega_1) = 0
+    w = Om[:, 1] - 3.0 * Om[:, 0]
+    S = S - np.outer(w, w @ S) / (w @ w)
+    R, mu, Q, L, d = orc.pivot_metric_factors(S, Om, 4)
+    assert np.allclose(Q[:, 1], 0.0) and np.linalg.matrix_rank(Q) == 3
+    assert np.all(np.isfinite(orc.pivot_coefficient_map(S, Om)))
+    Z = np.zeros((K, V))
+    assert np.allclose(orc.pivot_coefficient_map(Z, Om), 0.0) and np.allclose(orc.ridge_coefficient_map(Z, Om), 0.0)
+
+
+def test_pivot_map_brute_force_on_tiny_heads():
+    """K, V <= 4 with Python loops only: rotate the state, build mu, H, the Gram-Schmidt basis of the first p sketch
+    columns, L, d and H^ entry by entry, and solve the G x G normal equations by hand-written elimination."""
+    rng = np.random.default_rng(17)
+    K, V, G, P, lam = 4, 3, 3, 2, 0.1
+    S, Om = _head(rng, K, V, G)
+    R = orc._orthogonal_completion(Om)
+    Sp = [[sum(R[i][l] * S[l][j] for l in range(K)) for j in range(V)] for i in range(K)]
+    mu = sum(Sp[i][j] ** 2 for i in range(K) for j in range(V)) / K
+    Hd = [sum(Sp[i][j] ** 2 for j in range(V)) / mu for i in range(K)]
+    # Gram-Schmidt on the first two sketch columns (column g of the sketch is row g of S')
+    u1 = Sp[0][:]
+    n1 = sum(x * x for x in u1) ** 0.5
+    q1 = [x / n1 for x in u1]
+    r12 = sum(a * b for a, b in zip(q1, Sp[1]))
+    u2 = [b - r12 * a for a, b in zip(q1, Sp[1])]
+    n2 = sum(x * x for x in u2) ** 0.5
+    q2 = [x / n2 for x in u2]
+    Lm = [[sum(Sp[i][j] * q[j] for j in range(V)) / mu ** 0.5 for q in (q1, q2)] for i in range(K)]
+    dd = [max(Hd[i] - Lm[i][0] ** 2 - Lm[i][1] ** 2, 0.0) for i in range(K)]
+    Hh = [[Lm[i][0] * Lm[j][0] + Lm[i][1] * Lm[j][1] + (dd[i] if i == j else 0.0) for j in range(K)] for i in range(K)]
+    q = list(rng.standard_normal(K))
+    x = [sum(R[i][l] * q[l] for l in range(K)) for i in range(K)]
+    A = [[Hh[i][j] + (lam if i == j else 0.0) for j in range(G)] for i in range(G)]
+    b = [sum(Hh[i][j] * x[j] for j in range(K)) for i in range(G)]
+    for col in range(G):                                   # Gaussian elimination, no pivoting needed (SPD)
+        for row in range(col + 1, G):
+            f = A[row][col] / A[col][col]
+            for j in range(col, G):
+                A[row][j] -= f * A[col][j]
+            b[row] -= f * b[col]
+    c = [0.0] * G
+    for i in range(G - 1, -1, -1):
+        c[i] = (b[i] - sum(A[i][j] * c[j] for j in range(i + 1, G))) / A[i][i]
+    np.testing.assert_allclose(orc.pivot_coefficient_map(S, Om, lam, P) @ np.array(q), c, atol=1e-10)
+
+
+@pytest.mark.parametrize("kind", KINDS)
+def test_schedule_with_state_dependent_map_rebuilds_it_at_every_flush(kind):
+    """run_schedule_state_dependent: the map in force during a window is the one of the state at the window's start;
+    flush outputs are exact; with all sketch columns as pivots and no ridge the sketch read is the projection of the
+    exact read onto range(U)."""
+    rng = np.random.default_rng(18)
+    N, K, V, G, L = 3, 8, 6, 3, 4
+    S0 = rng.standard_normal((N, K, V))
+    Om = np.stack([np.linalg.qr(rng.standard_normal((K, G)))[0] for _ in range(N)])
+    toks = rand_tokens(rng, kind, 2 * L + 1, K, V, lead=(N,))
+    qs = [rng.standard_normal((N, K)) for _ in toks]
+    outs, S, U, C = orc.run_schedule_state_dependent(kind, S0, Om, toks, qs, L, "pivot", lam=0.1, P=2)
+    # replay by hand
+    St = S0.copy()
+    Sw = S0.copy()
+    for t, (tok, q) in enumerate(zip(toks, qs)):
+        St = orc.transition(kind, St, *tok)
+        exact = orc.exact_read(St, q)
+        if t % L == L - 1:
+            np.testing.assert_allclose(outs[t], exact, atol=1e-10)
+            Sw = St.copy()
+        else:
+            ring = toks[(t // L) * L: t + 1]
+            Cw = np.stack([orc.pivot_coefficient_map(Sw[i], Om[i], 0.1, 2) for i in range(N)])
+            want = orc.decode_step(kind, orc.sketch_of(Sw, Om), Cw, ring, q)
+            np.testing.assert_allclose(outs[t], want, atol=1e-10)
+    np.testing.assert_allclose(C, np.stack([orc.pivot_coefficient_map(Sw[i], Om[i], 0.1, 2) for i in range(N)]), atol=1e-12)
