@@ -39,7 +39,8 @@
  *   state  S      [B][H][K][V]  fp32
  *   sketch U      [B][H][r][V]  fp32   (U^T of the paper's V x r matrix: row g is S^T omega_g)
  *   omega  Omega  [H][K][r]     fp32   (fixed offline, shared by the batch)
- *   coef   C      [H][r][K]     fp32   (fixed offline coefficient map, Eq. 10)
+ *   coef   C      [H][r][K]     fp32   (fixed offline coefficient map, Eq. 10), or with config.coef_per_seq
+ *                 [B][H][r][K]  fp32   (state-dependent map, written by sketchssm_state_update)
  *   ring          [B][H] blocks of sketchssm_sizes.ring_head_bytes, each
  *                   k     [L][K] io
  *                   v     [L][V] io
@@ -87,6 +88,14 @@ typedef struct sketchssm_config {
     int32_t io_dtype;   /* sketchssm_dtype of q, k, v, KDA g and of the ring's k, v, g */
     int32_t out_dtype;  /* sketchssm_dtype of o */
     int32_t device;     /* CUDA device ordinal */
+    int32_t coef_per_seq;   /* 0: C is the fixed offline map [H][r][K], an input shared by the batch (Eq. 10).
+                               1: C is the state-dependent map (Eq. 9 with the ridge of Appendix A.2.2), one per
+                                  (batch, head), [B][H][r][K]; every sketchssm_state_update that writes the sketch
+                                  rebuilds it from the updated state, and the decode step reads it beside U.
+                                  Omega must then have orthonormal columns (the appendix's assumption). */
+    int32_t coef_pivots;    /* coef_per_seq = 1: pivot count P of the low-rank-plus-diagonal state metric
+                               (Eq. 30-37; the paper uses 4; 1..8), or 0 for the exact ridge solve (Eq. 29) */
+    float ridge_lambda;     /* coef_per_seq = 1: ridge lambda > 0 (the paper uses 0.1) */
 } sketchssm_config;
 
 typedef struct sketchssm_sizes {
@@ -150,6 +159,12 @@ int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* bufs);
  *   flags    : SKETCHSSM_NO_SKETCH leaves U untouched.
  * With n_before = 0 and no token, S is left untouched and only U (and out) are produced:
  * this builds the initial sketch from a prefilled state.
+ * With config.coef_per_seq = 1 every call that writes U also rebuilds the coefficient maps C of all (batch, head)
+ * pairs from S_new and U (a second kernel of the same call: the map needs the complete sketch before it can be
+ * contracted with the state, so S_new is read once more): mu = ||S_new||_F^2 / K, then either the exact ridge form
+ * C = (U^T U + lambda mu I)^{-1} U^T S_new^T or, with P = config.coef_pivots > 0, the approximation of Appendix A.2.2
+ * (Gram-Schmidt basis Q of the first min(r, P) sketch columns, L = S Q / sqrt(mu), residual diagonal d, Woodbury
+ * solve of the P x P system).
  * After the call the caller's ring count is 0. */
 int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
                            const void* v, const void* beta, const void* decay, void* out,
@@ -158,7 +173,10 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
 /* Non-flush decode step of Algorithm 1: store the token in ring slot n_before, form q~_t and
  * the buffer weights from the n_before+1 buffered tokens (Eq. 4), c_t = C q~_t, and write
  * o = U c_t + sum_s a_s v_s.  S is not touched.  n_before in 0..L-1; all pointers required.
- * After the call the caller's ring count is n_before + 1 (unless SKETCHSSM_NO_APPEND). */
+ * After the call the caller's ring count is n_before + 1 (unless SKETCHSSM_NO_APPEND).
+ * With config.coef_per_seq = 1 the head's own map C[b][h] is read (r * K * 4 more bytes per head and step); only the
+ * default one-kernel decode supports this ("decode_impl" = 0 and sketchssm_decode_step_static return
+ * SKETCHSSM_UNSUPPORTED_SHAPE). */
 int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
                           const void* v, const void* beta, const void* decay, void* out,
                           uint32_t flags, void* stream);

@@ -33,7 +33,8 @@ OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
-                ("kind", "batch", "heads", "dk", "dv", "rank", "buf_len", "io_dtype", "out_dtype", "device")]
+                ("kind", "batch", "heads", "dk", "dv", "rank", "buf_len", "io_dtype", "out_dtype", "device",
+                 "coef_per_seq", "coef_pivots")] + [("ridge_lambda", ctypes.c_float)]
 
 
 class Sizes(ctypes.Structure):
@@ -103,17 +104,21 @@ class SketchSSM:
     """One layer's decode state on one GPU: owns the torch buffers, forwards to the C ABI.
 
     Tensors (all on `device`): state [B,H,K,V] f32, sketch [B,H,r,V] f32, ring (bytes),
-    omega [H,K,r] f32, coef [H,r,K] f32.  Token arguments follow the C header:
+    omega [H,K,r] f32, coef [H,r,K] f32 (or [B,H,r,K] with coef_per_seq: the state-dependent map that every
+    state update rebuilds).  Token arguments follow the C header:
     q,k [B,H,K] io; v [B,H,V] io; beta [B,H] f32; decay [B,H] f32 or [B,H,K] io (KDA).
     """
 
     def __init__(self, kind: str, batch: int, heads: int, dk: int, dv: int, rank: int, buf_len: int,
-                 io: str = "bf16", out: str = "f32", device: int = 0, allocate: bool = True):
+                 io: str = "bf16", out: str = "f32", device: int = 0, allocate: bool = True,
+                 coef_per_seq: bool = False, coef_pivots: int = 4, ridge_lambda: float = 0.1):
         self.lib = load_library()
         self.kind, self.io, self.out = kind, io, out
         self.B, self.H, self.K, self.V, self.R, self.L = batch, heads, dk, dv, rank, buf_len
         self.device = torch.device("cuda", device)
-        self.cfg = Config(KIND[kind], batch, heads, dk, dv, rank, buf_len, DTYPE[io], DTYPE[out], device)
+        self.coef_per_seq = bool(coef_per_seq)
+        self.cfg = Config(KIND[kind], batch, heads, dk, dv, rank, buf_len, DTYPE[io], DTYPE[out], device,
+                          int(self.coef_per_seq), coef_pivots, ridge_lambda)
         self._ctx = ctypes.c_void_p()
         self._check("sketchssm_create", self.lib.sketchssm_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.sizes = Sizes()
@@ -129,7 +134,7 @@ class SketchSSM:
         self.sketch = torch.zeros(self.B, self.H, self.R, self.V, dtype=torch.float32, device=d)
         self.ring = torch.zeros(self.sizes.ring_bytes, dtype=torch.uint8, device=d)
         self.omega = torch.zeros(self.H, self.K, self.R, dtype=torch.float32, device=d)
-        self.coef = torch.zeros(self.H, self.R, self.K, dtype=torch.float32, device=d)
+        self.coef = torch.zeros(*((self.B,) if self.coef_per_seq else ()), self.H, self.R, self.K, dtype=torch.float32, device=d)
         self.status = torch.zeros(self.sizes.status_bytes // 4, dtype=torch.int32, device=d)
         self.work = torch.zeros(self.sizes.work_bytes // 4, dtype=torch.float32, device=d)
         self.bind()

@@ -57,6 +57,9 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.max_warps_per_sm = ctx->tune_max_warps;
     p.update_impl = ctx->tune_update_impl;
     p.pdl = ctx->tune_pdl;
+    p.coef_per_seq = ctx->cfg.coef_per_seq;
+    p.pivots = ctx->cfg.coef_pivots;
+    p.ridge_lambda = ctx->cfg.ridge_lambda;
     return p;
 }
 
@@ -87,6 +90,26 @@ int decode_params(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     return SKETCHSSM_OK;
 }
 
+// The flush kernel for this configuration: the warp-specialised tensor-core kernels where their shape limits allow,
+// the single-group tensor-core kernel for Mamba-2 ranks above 32, CUDA cores otherwise.
+int dispatch_update(sketchssm_ctx* ctx, const Params& p, cudaStream_t cs) {
+    if (p.update_impl != 1) {
+        int rc;
+        if (p.update_impl != 3) {
+            rc = launch_update_tc_ws(ctx, p, cs);
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        }
+        rc = launch_update_tc(ctx, p, cs);
+        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        // gated delta rule: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 16, rank <= 16)
+        if (p.update_impl == 0) {
+            rc = launch_update_tc_ws_gdn(ctx, p, cs);
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+        }
+    }
+    return launch_update(ctx, p, cs);
+}
+
 int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q, const void* k, const void* v,
                   const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
     Params p;
@@ -107,6 +130,7 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     }
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
     if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
+    if (p.coef_per_seq && !full_read) return SKETCHSSM_UNSUPPORTED_SHAPE;   // the two-kernel decode stages one map per head index
     switch (ctx->cfg.kind) {
         case SKETCHSSM_MAMBA2:
             return bf ? launch_decode_split_mamba2_bf16(ctx, p, cs) : launch_decode_split_mamba2_f32(ctx, p, cs);
@@ -133,6 +157,11 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     if (cfg->rank > kMaxRank) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if (cfg->buf_len < 4 || cfg->buf_len > kMaxBufLen || (cfg->buf_len & 3)) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if ((size_t)cfg->batch * cfg->heads > (size_t)1 << 24) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (cfg->coef_per_seq != 0 && cfg->coef_per_seq != 1) return SKETCHSSM_INVALID_ARG;
+    if (cfg->coef_per_seq) {
+        if (!(cfg->ridge_lambda > 0.f) || cfg->coef_pivots < 0) return SKETCHSSM_INVALID_ARG;
+        if (cfg->coef_pivots > 8) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    }
     sketchssm_ctx* c = new (std::nothrow) sketchssm_ctx();
     if (c == nullptr) return SKETCHSSM_INVALID_ARG;
     c->cfg = *cfg;
@@ -168,7 +197,7 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
     out->sketch_bytes = bh * c.rank * c.dv * 4;
     out->ring_bytes = bh * ctx->ring.head_bytes;
     out->omega_bytes = (size_t)c.heads * c.dk * c.rank * 4;
-    out->coef_bytes = (size_t)c.heads * c.rank * c.dk * 4;
+    out->coef_bytes = (c.coef_per_seq ? bh : (size_t)c.heads) * c.rank * c.dk * 4;
     out->status_bytes = (((size_t)(kStatusInts + 4 + c.heads) * sizeof(int32_t)) + 15) & ~(size_t)15;   // status word + tile scheduler counters
     out->work_bytes = bh * (size_t)(c.dk + c.buf_len) * 4;
     out->ring_head_bytes = ctx->ring.head_bytes;
@@ -219,21 +248,15 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     p.write_state = n_tot > 0 ? 1 : 0;
     ctx->sketch_fresh = true;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (p.update_impl != 1) {
-        // Mamba-2: warp-specialised tensor-core kernel, then the single-group one (ranks above 32); 3 skips the former
-        if (p.update_impl != 3) {
-            rc = launch_update_tc_ws(ctx, p, cs);
-            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        }
-        rc = launch_update_tc(ctx, p, cs);
-        if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        // gated delta rule: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 16, rank <= 16)
-        if (p.update_impl == 0) {
-            rc = launch_update_tc_ws_gdn(ctx, p, cs);
-            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        }
+    rc = dispatch_update(ctx, p, cs);
+    if (rc != SKETCHSSM_OK) return rc;
+    if (p.coef_per_seq && sketch) {
+        const int launched = ctx->last_launches;
+        rc = launch_coef_map(ctx, p, cs);         // C from S_new and U, after the flush kernel has completed
+        if (rc != SKETCHSSM_OK) return rc;
+        ctx->last_launches = launched + 1;
     }
-    return launch_update(ctx, p, cs);
+    return SKETCHSSM_OK;
 }
 
 int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
@@ -251,6 +274,7 @@ int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q
     Params p;
     int rc = decode_params(ctx, 0, n_before, q, k, v, beta, decay, out, flags, &p);
     if (rc != SKETCHSSM_OK) return rc;
+    if (ctx->cfg.coef_per_seq) return SKETCHSSM_UNSUPPORTED_SHAPE;    // runs the two-kernel decode (one map per head index)
     // the size limit of the library's static array is checked (on the host, before any CUDA call) by the launcher
     const sketchssm_config& c = ctx->cfg;
     if ((size_t)c.batch * c.heads * (size_t)(c.dk + c.buf_len) * sizeof(float) > (size_t)SKETCHSSM_STATIC_WORK_BYTES)

@@ -29,6 +29,7 @@ namespace {
 
 struct StageLayout {
     uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
+    uint32_t c_off, c_bytes;        // the head's own coefficient map (sketch mode with a per-sequence map only)
     uint32_t k_off, k_bytes;        // n buffered keys
     uint32_t v_off, v_bytes;        // n buffered values
     uint32_t gate_off, gate_bytes;  // beta[L] (+ decay[L] for scalar kinds)
@@ -38,10 +39,13 @@ struct StageLayout {
 };
 
 __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K, int V, int R, int L, int n,
-                                                         int full_read) {
+                                                         int full_read, int coef_per_seq) {
     StageLayout s;
     uint32_t off = 0;
     s.u_off = off; s.u_bytes = full_read ? 0u : (uint32_t)(R * V * 4); off += s.u_bytes;
+    // rows padded to the reduction width are read (their sums are never used), so they get room but are not copied
+    s.c_off = off; s.c_bytes = (!full_read && coef_per_seq) ? (uint32_t)(R * K * 4) : 0u;
+    off += (!full_read && coef_per_seq) ? (uint32_t)(((R + 7) & ~7) * K * 4) : 0u;
     s.k_off = off; s.k_bytes = (uint32_t)(n * K * io); off += s.k_bytes;
     s.v_off = off; s.v_bytes = (uint32_t)(n * V * io); off += s.v_bytes;
     s.gate_off = off;
@@ -62,10 +66,11 @@ struct DecodeSmem {
     uint32_t coef_slot_bytes, bar_off, scratch_off, scratch_stride, stage_off, total;
 };
 
-__host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps, int full_read, uint32_t stage_bytes) {
+__host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps, int full_read, int coef_per_seq,
+                                                       uint32_t stage_bytes) {
     DecodeSmem d;
     const int RP = (R + 7) & ~7;                       // coefficient rows padded to the reduction width
-    d.coef_slot_bytes = full_read ? 0u : (uint32_t)(RP * K * 4);
+    d.coef_slot_bytes = (full_read || coef_per_seq) ? 0u : (uint32_t)(RP * K * 4);
     d.bar_off = 2u * d.coef_slot_bytes;
     uint32_t off = d.bar_off + (((uint32_t)(nwarps * 2 * 8 + 16) + 127u) & ~127u);    // two mbarriers per warp, the head counter
     d.scratch_stride = (uint32_t)((K + 80) * 4);       // per warp: q~ (full read) or c (K floats), then 64+ dot products
@@ -92,8 +97,8 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     const int L = p.L, H = p.H, B = p.B, n = p.n_before;
     const int RP = (R + 7) & ~7;
 
-    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n, p.full_read);
-    const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, sl.total);
+    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n, p.full_read, p.coef_per_seq);
+    const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, p.coef_per_seq, sl.total);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * 2;
     float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
     float* sP = sX + K;                                                                               // dot products
@@ -113,7 +118,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     }
     // coefficient maps of the (at most two) head indices of this range, rows padded with zeros.  C is a constant of
     // the layer (never written by these kernels), so it may be staged before the predecessor in the stream is done.
-    if (!p.full_read && item1 > item0) {
+    if (!p.full_read && !p.coef_per_seq && item1 > item0) {
         const int nslots = h_last > h_first ? 2 : 1;
         for (int s = 0; s < nslots; ++s) {
             const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
@@ -130,7 +135,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     // used, so the next head's loads overlap the rest of the current head's arithmetic without a second stage.
     // Every copy is issued by its own lane from per-lane constants set up once (base pointer, bytes per head, target).
     const uint32_t txA = sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes + 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
-    const uint32_t txB = sl.u_bytes;
+    const uint32_t txB = sl.u_bytes + sl.c_bytes;
     const unsigned char* cp_base = nullptr;
     size_t cp_stride = 0;
     uint32_t cp_dst = 0, cp_bytes = 0;
@@ -144,6 +149,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_bytes = sl.v_bytes; break;
         case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_bytes = sl.g_bytes; break;
         case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * 4; cp_dst = sl.u_off; cp_bytes = sl.u_bytes; break;
+        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_bytes = sl.c_bytes; break;
         default: break;
     }
     uint64_t* barA = &bars[0];
@@ -154,10 +160,9 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         if (lane < 8 && cp_bytes) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barA);
     };
     auto issue_b = [&](size_t bh) {      // whole warp
-        if (lane == 8 && cp_bytes) {
-            mbar_expect_tx(barB, txB);
-            bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barB);
-        }
+        if (lane == 8 && txB) mbar_expect_tx(barB, txB);
+        __syncwarp();
+        if ((lane == 8 || lane == 9) && cp_bytes) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barB);
     };
 
     // The CTA's heads are handed to its warps at run time (a counter in shared memory): a warp claims its next head
@@ -341,8 +346,17 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         if (has_next) issue_a(bh_next);
         if (!p.full_read) {
             // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
-            const float* sC = reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
+            const float* sC = p.coef_per_seq ? reinterpret_cast<const float*>(sb + sl.c_off)
+                                             : reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
             __syncwarp();
+            if (p.coef_per_seq) {        // the head's own map arrives with its sketch rows
+                if (__any_sync(0xffffffffu, !DEC_WAIT(barB, parity))) {
+                    if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
+                    pendB = (int)parity;
+                    pendA = has_next ? (int)(parity ^ 1u) : -1;
+                    break;
+                }
+            }
 #pragma unroll
             for (int g0 = 0; g0 < (RT ? ((RT + 7) & ~7) : RP); g0 += NB) {
                 float part[NB];
@@ -415,7 +429,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 template <int KIND, typename IO, int K, int V>
 static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     const int io = (int)sizeof(IO);
-    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read);
+    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq);
     const uint32_t smem_budget = 227u * 1024u;
     if (ctx->sm_count == 0) {
         int dev = 0, sms = 0;
@@ -440,7 +454,7 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     int best_nw = 0, best_ctas = 1, best_warps = 0;
     for (int nw = 8; nw >= 1; --nw) {
         if (p.warps_per_cta && nw != p.warps_per_cta) continue;
-        const DecodeSmem d = make_decode_smem(K, p.R, nw, p.full_read, sl.total);
+        const DecodeSmem d = make_decode_smem(K, p.R, nw, p.full_read, p.coef_per_seq, sl.total);
         if (d.total > smem_budget) continue;
         int ctas = (int)((228u * 1024u) / (d.total + 1024u));
         if (ctas * nw > cap) ctas = cap / nw;
@@ -449,7 +463,7 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
         if (ctas * nw > best_warps) { best_warps = ctas * nw; best_nw = nw; best_ctas = ctas; }
     }
     if (best_nw == 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
-    const DecodeSmem d = make_decode_smem(K, p.R, best_nw, p.full_read, sl.total);
+    const DecodeSmem d = make_decode_smem(K, p.R, best_nw, p.full_read, p.coef_per_seq, sl.total);
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)d.total)) != cudaSuccess)
         return SKETCHSSM_CUDA_ERROR;

@@ -72,6 +72,9 @@ struct Params {
     int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
     int early_sketch;     // decode: the first head's sketch rows may be requested before the predecessor in the stream is
                           // waited for (no kernel that may still be running writes the sketch)
+    int coef_per_seq;     // the coefficient map is per (batch, head) [B][H][r][K] and rebuilt by every state update
+    int pivots;           // coefficient-map construction: pivot count P of the approximated state metric; 0 = exact ridge form
+    float ridge_lambda;   // ridge of the state-dependent coefficient map
     int tok_base;         // update (GDN tensor-core kernel): first ring row of this pass when a flush is replayed in blocks of 16 tokens
 };
 
@@ -86,6 +89,7 @@ int launch_decode_split_gdn_bf16(Ctx* ctx, const Params& p, cudaStream_t stream)
 int launch_decode_split_kda_f32(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_decode_split_kda_bf16(Ctx* ctx, const Params& p, cudaStream_t stream);
 int launch_update(Ctx* ctx, const Params& p, cudaStream_t stream);       // CUDA cores, every configuration
+int launch_coef_map(Ctx* ctx, const Params& p, cudaStream_t stream);     // state-dependent coefficient maps from S_new and U (after a flush)
 int launch_wait_probe(Ctx* ctx, int poll_limit, int where, cudaStream_t stream);   // self-test: a bounded wait that runs out
 int launch_update_tc(Ctx* ctx, const Params& p, cudaStream_t stream);    // tcgen05 tensor cores, Mamba-2; UNSUPPORTED_SHAPE outside its domain
 int launch_update_tc_ws(Ctx* ctx, const Params& p, cudaStream_t stream); // same, two warp groups per CTA (operand building overlaps the state stream)

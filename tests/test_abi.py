@@ -55,6 +55,18 @@ def test_create_validates_configuration(lib):
     assert make(lib, buf_len=68)[0] == -2
     assert lib.sketchssm_create(None, None) == -1
     assert lib.sketchssm_destroy(None) == -1
+    # state-dependent coefficient map: needs a positive ridge, at most 8 pivots (0 = exact ridge solve)
+    assert make(lib, coef_per_seq=1, coef_pivots=4, ridge_lambda=0.1)[0] == 0
+    assert make(lib, coef_per_seq=1, coef_pivots=0, ridge_lambda=0.1)[0] == 0
+    assert make(lib, coef_per_seq=1, coef_pivots=4, ridge_lambda=0.0)[0] == -1
+    assert make(lib, coef_per_seq=1, coef_pivots=-1, ridge_lambda=0.1)[0] == -1
+    assert make(lib, coef_per_seq=1, coef_pivots=9, ridge_lambda=0.1)[0] == -2
+    assert make(lib, coef_per_seq=2)[0] == -1
+    rc, ctx = make(lib, coef_per_seq=1, coef_pivots=4, ridge_lambda=0.1, batch=3, heads=5, rank=8)
+    s = binding.Sizes()
+    assert rc == 0 and lib.sketchssm_query_sizes(ctx, ctypes.byref(s)) == 0
+    assert s.coef_bytes == 3 * 5 * 8 * 128 * 4                  # one map per (batch, head)
+    lib.sketchssm_destroy(ctx)
 
 
 @pytest.mark.parametrize("kind,io,K,V,L,expect_head", [

@@ -1,0 +1,71 @@
+"""The state-dependent coefficient map on the GPU (rebuilt by every state update, read per head by the decode step)
+against the oracle's statement of Appendix A.2.2: the exact ridge form and the pivot approximation, all three
+recurrences, over several windows so that the maps in force change with the state."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_33051_b200 import binding, synth
+from tests.test_gpu_parity import FP32_GUARD, check, make_layer, run_schedule
+
+pytestmark = pytest.mark.gpu
+
+COEF_GUARD = 2e-4       # max |C_gpu - C_oracle| / max |C|: fp32 solves against fp64 ones
+
+
+def check_coef(errs, io):
+    assert errs["c0"] <= COEF_GUARD and errs["C"] <= COEF_GUARD, errs
+    check({k: v for k, v in errs.items() if k not in ("c0", "C")}, io, guard=2e-4)
+
+
+@pytest.mark.parametrize("kind,dv", [("mamba2", 64), ("mamba2", 128), ("gdn", 128), ("kda", 128), ("gdn", 64)])
+@pytest.mark.parametrize("coef,pivots", [("pivot", 4), ("pivot", 1), ("pivot", 8), ("ridge", 0)])
+def test_state_dependent_map_matches_the_oracle(kind, dv, coef, pivots):
+    w = synth.Workload("t", kind, 5, 3, 128, dv, 16, 8, 0, "bf16", 101, basis="qr")
+    check_coef(run_schedule(w, 2 * w.buf_len + 3, max_heads=10**9, coef=coef, pivots=pivots), "bf16")
+
+
+@pytest.mark.parametrize("rank,dk,dv", [(3, 64, 64), (5, 128, 64), (32, 128, 128), (64, 64, 128)])
+@pytest.mark.parametrize("coef", ["pivot", "ridge"])
+def test_state_dependent_map_ranks_and_shapes(rank, dk, dv, coef):
+    w = synth.Workload("t", "gdn", 3, 2, dk, dv, rank, 8, 0, "f32", 103, basis="qr")
+    check_coef(run_schedule(w, w.buf_len + 3, max_heads=10**9, coef=coef), "f32")
+
+
+@pytest.mark.parametrize("name", ["c2_mamba2", "c3_gdn"])
+def test_state_dependent_map_full_batch_sampled_heads(name):
+    w = synth.CONFIGS[name]
+    check_coef(run_schedule(w, 2 * w.buf_len + 3, max_heads=32, coef="pivot"), w.io)
+
+
+def test_pivot_map_with_all_columns_as_pivots_equals_the_ridge_map():
+    """P >= r: the approximation is exact, so the two constructions must agree (two different kernels paths)."""
+    w = synth.Workload("t", "kda", 4, 2, 128, 128, 4, 8, 0, "bf16", 107, basis="qr")
+    ma, *_ = make_layer(w, coef="pivot", pivots=4)
+    mb, *_ = make_layer(w, coef="ridge")
+    ma.state_update(0); mb.state_update(0)
+    ca, cb = ma.coef.cpu().numpy(), mb.coef.cpu().numpy()
+    assert np.abs(ca - cb).max() <= 1e-4 * np.abs(cb).max()
+
+
+def test_zero_state_gives_a_zero_map_and_unsupported_paths_say_so():
+    w = synth.Workload("t", "gdn", 2, 2, 128, 128, 8, 8, 0, "bf16", 109, basis="qr")
+    m, S0, Om, C, dev = make_layer(w, coef="pivot")
+    m.state.zero_()
+    m.coef.fill_(7.0)
+    m.state_update(0)
+    assert torch.count_nonzero(m.coef).item() == 0 and torch.count_nonzero(m.sketch).item() == 0
+    # NO_SKETCH leaves both the sketch and the maps alone
+    m.coef.fill_(3.0)
+    m.state_update(0, flags=binding.NO_SKETCH)
+    assert bool((m.coef == 3.0).all().item())
+    from tests import harness
+    tt = harness.token_tensors(w, synth.step_inputs(w, 0, 0), dev)
+    o = m.new_output()
+    m.tune("decode_impl", 0)
+    with pytest.raises(binding.SketchSSMError):
+        m.decode_step(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+    with pytest.raises(binding.SketchSSMError):
+        m.decode_step_static(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
+    m.full_read_decode(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)      # unaffected by the map
+    m.check_status()

@@ -25,26 +25,32 @@ def _device():
     return torch.device("cuda", 0)
 
 
-def make_layer(w, layer=0, out="f32"):
+def make_layer(w, layer=0, out="f32", coef=None, lam=0.1, pivots=4):
+    """coef: None (fixed offline map, an input), "pivot" or "ridge" (state-dependent map, rebuilt by every flush)."""
     from paper_2609_33051_b200.binding import SketchSSM
     dev = _device()
     Om, C = harness.basis_for(w, layer)
-    m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out=out, device=0)
+    m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out=out, device=0,
+                  coef_per_seq=coef is not None, coef_pivots=pivots if coef == "pivot" else 0, ridge_lambda=lam)
     S0 = synth.initial_state(w, layer)
     m.state.copy_(torch.from_numpy(S0))
     m.omega.copy_(torch.from_numpy(Om))
-    m.coef.copy_(torch.from_numpy(C))
+    if coef is None:
+        m.coef.copy_(torch.from_numpy(C))
     return m, S0, Om, C, dev
 
 
-def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", input_batch=None, per_element=None):
+def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", input_batch=None, per_element=None,
+                 coef=None, lam=0.1, pivots=4):
     """Algorithm 1 on GPU and oracle; returns the worst per-step relative error and the final-state errors.
 
     input_batch: generate the token inputs for this many batch entries and repeat them over the batch (the initial
     states stay distinct per entry, so every entry still follows its own trajectory); keeps the host-side input
     generation of the largest batches short.  per_element: optional callable(got, ref) run on every step's outputs.
-    errs["windows"] lists the worst output error of each window, so drift across flushes is visible."""
-    m, S0, Om, C, dev = make_layer(w, out=out)
+    errs["windows"] lists the worst output error of each window, so drift across flushes is visible.
+    coef: None, or "pivot" / "ridge": the state-dependent coefficient map, which both sides rebuild from the state at
+    the initial sketch construction and at every flush (errs["C"]: the final maps)."""
+    m, S0, Om, C, dev = make_layer(w, out=out, coef=coef, lam=lam, pivots=pivots)
     for key, val in (tune or {}).items():
         m.tune(key, val)
     bs, hs = harness.select_heads(w, max_heads)
@@ -57,6 +63,9 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
     Om_s, C_s = Om[hs].astype(np.float64), C[hs].astype(np.float64)
     U = orc.sketch_of(S, Om_s)
     errs = {"u0": harness.rel_err(m.sketch.cpu().numpy()[bs, hs].transpose(0, 2, 1), U)}
+    if coef is not None:
+        C_s = orc.coefficient_maps(S, Om_s, coef, lam, pivots)
+        errs["c0"] = harness.rel_err(m.coef.cpu().numpy()[bs, hs], C_s)
     worst = 0.0
     windows = []
     ring = []
@@ -81,9 +90,11 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
         else:
             m.state_update(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
             S, U, ref = orc.state_update(w.kind, S, ring, Om_s, q)
+            if coef is not None:
+                C_s = orc.coefficient_maps(S, Om_s, coef, lam, pivots)
             ring = []
         # the two-kernel decode launches twice; a GDN flush of more than 16 tokens is one launch per block of 16
-        assert 1 <= m.last_launch_count() <= max(2, (w.buf_len + 15) // 16)
+        assert 1 <= m.last_launch_count() <= max(2, (w.buf_len + 15) // 16) + (1 if coef else 0)
         got = o_dev[bs_t, hs_t].float().cpu().numpy()
         assert np.all(np.isfinite(got))
         if per_element is not None:
@@ -97,6 +108,8 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
     errs["out"] = worst
     errs["S"] = harness.rel_err(m.state[bs_t, hs_t].cpu().numpy(), S)
     errs["U"] = harness.rel_err(m.sketch[bs_t, hs_t].cpu().numpy().transpose(0, 2, 1), U)
+    if coef is not None:
+        errs["C"] = harness.rel_err(m.coef[bs_t, hs_t].cpu().numpy(), C_s)
     errs["windows"] = windows
     return errs
 
