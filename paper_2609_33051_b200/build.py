@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsketchssm.so")
 # (source, object suffix, extra defines); the two-kernel decode is compiled once per (recurrence kind, I/O type)
 UNITS = [("api.cu", "", []), ("decode.cu", "", []), ("update.cu", "", []), ("update_tc.cu", "", []),
-         ("update_tc_ws.cu", "", []), ("update_tc_ws_gdn.cu", "", []), ("decode_static.cu", "", []), ("selftest.cu", "", []), ("coef_map.cu", "", []),
+         ("update_tc_ws.cu", "", []), ("update_tc_ws_gdn.cu", "", []), ("update_tc_ws_kda.cu", "", []), ("decode_static.cu", "", []), ("selftest.cu", "", []), ("coef_map.cu", "", []),
          *[("decode_split.cu", f"_k{k}_io{io}", [f"-DSKETCHSSM_GROUP_KIND={k}", f"-DSKETCHSSM_GROUP_IO={io}"])
            for k in range(3) for io in range(2)]]
 HEADERS = [os.path.join(CSRC, "internal.cuh"), os.path.join(CSRC, "lanegroup.cuh"), os.path.join(CSRC, "tc_common.cuh"),

@@ -105,6 +105,9 @@ int dispatch_update(sketchssm_ctx* ctx, const Params& p, cudaStream_t cs) {
         if (p.update_impl == 0) {
             rc = launch_update_tc_ws_gdn(ctx, p, cs);
             if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
+            // delta rule with per-channel decay: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 32, rank <= 16)
+            rc = launch_update_tc_ws_kda(ctx, p, cs);
+            if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
         }
     }
     return launch_update(ctx, p, cs);

@@ -93,7 +93,8 @@ int launch_coef_map(Ctx* ctx, const Params& p, cudaStream_t stream);     // stat
 int launch_wait_probe(Ctx* ctx, int poll_limit, int where, cudaStream_t stream);   // self-test: a bounded wait that runs out
 int launch_update_tc(Ctx* ctx, const Params& p, cudaStream_t stream);    // tcgen05 tensor cores, Mamba-2; UNSUPPORTED_SHAPE outside its domain
 int launch_update_tc_ws(Ctx* ctx, const Params& p, cudaStream_t stream); // same, two warp groups per CTA (operand building overlaps the state stream)
-int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p, cudaStream_t stream); // gated delta rule, warp-specialised, two passes over the state
+int launch_update_tc_ws_gdn(Ctx* ctx, const Params& p, cudaStream_t stream); // gated delta rule, warp-specialised, the state read once
+int launch_update_tc_ws_kda(Ctx* ctx, const Params& p, cudaStream_t stream); // delta rule with per-channel decay, warp-specialised, up to 32 tokens per pass
 
 // ---------------------------------------------------------------------------------------------
 // device helpers

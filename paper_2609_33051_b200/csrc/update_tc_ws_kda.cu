@@ -1,0 +1,871 @@
+// Warp-specialised state-update (flush) kernel for the delta rule with per-channel decay (KDA) on tcgen05 + TMEM, sm_100a.
+//
+// Replaying n tokens of S_s = (I - beta_s k_s k_s^T) Diag(g_s) S_{s-1} + beta_s k_s v_s^T (Eq. 1, 3) unrolled over the
+// window -- the WY form of Appendix C (Eq. 38-42) applied to the state, with the diagonal decays kept as vectors:
+//     G_s   = prod_{m<=s} g_m (per channel),   Dn_s = prod_{m>s} g_m
+//     Khat_s = G_s * k_s,   Ktil_s = Dn_s * k_s                  n x K     decayed keys (fp32 values: bf16 hi + lo)
+//     A_sj  = sum_i k_s[i] k_j[i] prod_{j<m<=s} g_m[i]  (j < s)  n x n     every product of decays formed by multiplication
+//     P     = Khat S_0                                           n x V
+//     E     = T (V - P),   T = (I + Bd A)^{-1} Bd                n x V
+//     S_new = Diag(G_n) S_0 + Ktil^T E                           K x V
+//     [U | o] = S_0^T (G_n * [Omega | q]) + E^T (Ktil [Omega | q])         (Eq. 7 and the exact output of the flush step)
+// No quotient of cumulative decays is ever formed (they underflow within a window on real gates).
+//
+// Same schedule as the gated-delta-rule kernel: tile = one head (K = V = 128), TMEM lane = value column; the state is
+// read once by bulk copies into a ring of shared-memory stages; the pass-A group splits the S_0 chunks into bf16 hi + lo,
+// leaves G_n * S_0 in the accumulator of Ktil^T E (tcgen05.st) and later forms E; one thread issues every MMA; the pass-B
+// group writes the accumulator (S_new) back and stores the sketch rows; the front group builds the ring-only operands two
+// tiles ahead.  What differs: up to 32 tokens per pass (the MMAs over tokens take two k-steps), both key operands and the
+// basis operand are per tile and carry hi + lo halves, so the B operand of pass A is a double-buffered per-tile window
+// [Khat (32 rows) | G_n * [Omega | q] (32 rows)], and the kernel runs one CTA per SM.
+//
+// Front group, thread = channel i: reads column i of the staged key and decay rows into registers, forms the running
+// products, writes Khat / Ktil / G_n * W in the operand layouts, and the 496 pair sums of A as per-channel products
+// reduced over the 128 channels by transposing butterflies (per-warp partials summed in a fixed order: results are
+// bitwise reproducible).  T by forward substitution (one column per thread of warp 0) while warps 1-3 form Ktil [Omega | q].
+//
+// Domain: KDA, bf16 I/O, K = V = 128, rank <= 16; 1..32 tokens per pass, up to 64 tokens per flush in blocks of 32.
+#include "internal.cuh"
+#include "lanegroup.cuh"
+#include "tc_common.cuh"
+
+namespace sketchssm {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kKThreads = 448;       // pass-A group (4 warps), front group (4 warps), MMA issue warp, state-load warp, pass-B group (4 warps)
+constexpr int kKGrp = 128;
+constexpr int kNT = 32;              // tokens per pass
+constexpr int kKStages = 8;          // upper bound on the shared-memory stages of state rows
+constexpr int kAS = 36;              // row stride (floats) of the 32 x 32 matrix A
+constexpr int kKA2 = 2;              // chunk buffers between the pass-A group and the MMA issue warp
+constexpr int kNPk = 32;             // columns of [Omega | q]: Omega in 0..R-1, q at column QA = round_up(R, 8) <= 16
+
+struct KSmem {
+    uint32_t a2, e, w, w_stride, w_lo, set, set_stride, set_bt, set_bt_lo, set_vv, set_t1, set_bc, set_gn, stg, stg_g, stg_v,
+        stg_beta, stg_q, mats, bars, misc, sst, sst_bytes, total;
+};
+
+__host__ __device__ inline KSmem make_ksmem(int stages) {
+    KSmem s;
+    uint32_t off = 0;
+    s.a2 = off; off += (uint32_t)kKA2 * 2u * 128u * 16u * 2u;     // 16-row chunk buffers, hi + lo
+    s.e = off; off += 2u * 128u * (uint32_t)kNT * 2u;             // E hi + lo: A operand of Ktil^T E (128 x 32 tokens each)
+    // B operand of pass A, per tile and double-buffered: 64 rows [Khat (32) | G_n * [Omega | q] (32)] x 128 channels, hi then lo
+    s.w = off; s.w_lo = 64u * kK * 2u; s.w_stride = 2u * s.w_lo; off += 2u * s.w_stride;
+    // per-tile operand set, double-buffered: Ktil as B operand of Ktil^T E (MN-major, hi | lo), raw value rows, T,
+    // Ktil [Omega | q] hi | lo (B operand of the sketch correction), G_n
+    s.set = off;
+    s.set_bt = 0u; s.set_bt_lo = 8192u; s.set_vv = 16384u; s.set_t1 = 24576u; s.set_bc = 28672u; s.set_gn = 32768u;
+    s.set_stride = 33280u;
+    off += 2u * s.set_stride;
+    // staging of the next tile's raw rows: keys [32][256 B], decays [32][256 B], values [32][256 B], beta [L] floats, query row.
+    // Once a tile's rows are in registers the key / decay area is re-used (A partials, then Ktil in fp32).
+    s.stg_g = 8192u; s.stg_v = 16384u; s.stg_beta = 24576u; s.stg_q = 24832u;
+    s.stg = off; off += 25088u;
+    s.mats = off; off += (uint32_t)kNT * kAS * 4u + 256u;         // A (beta_s A_sj), beta
+    s.bars = off; off += 512u;
+    s.misc = off; off += 128u;
+    off = (off + 127u) & ~127u;
+    s.sst_bytes = 16u * 128u * 4u;
+    s.sst = off; off += (uint32_t)stages * s.sst_bytes;
+    s.total = off;
+    return s;
+}
+
+enum { kPro = 0, kPfull = 2, kTfull = 4, kBdone = 6, kBufFree = 8, kA2free = 10, kA2rdy = 10 + kKA2, kErdy = 10 + 2 * kKA2,
+       kStg = 11 + 2 * kKA2, kFull = 14 + 2 * kKA2, kEmpty = 14 + 2 * kKA2 + kKStages,
+       kTfree = 14 + 2 * kKA2 + 2 * kKStages, kNumBars = 16 + 2 * kKA2 + 2 * kKStages };
+
+__device__ __forceinline__ void k_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void k_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ bool k_or(int id, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %2, 0;\n\t"
+        "bar.red.or.pred p, %1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(flag ? 1u : 0u)
+        : "memory");
+    return r != 0;
+}
+// group-wide bounded wait: one warp polls, the others sleep in the named barrier
+__device__ __forceinline__ bool k_wait(int id, int gt, uint64_t* bar, uint32_t phase) {
+    bool bad = false;
+    if (gt < 32) bad = !mbar_wait_bounded(bar, phase);
+    return !k_or(id, bad);
+}
+
+__device__ __forceinline__ float bf16_at(const unsigned char* base, uint32_t elem) {
+    return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[elem]);
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Params p) {
+    constexpr int K = kK, V = 128, CH = 16, NCH = K / CH, NP = kNPk;
+    extern __shared__ __align__(1024) unsigned char smem[];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gt = tid & 127;
+    const int R = p.R, H = p.H, B = p.B;
+    const int QA = (R + 7) & ~7;                          // column of the query
+    const int NS = p.stages;
+    const int n_ring = p.n_before, n_tot = n_ring + (p.has_token ? 1 : 0);     // 1..32 per pass (the launcher sees to it)
+    const int ksteps = n_tot > 16 ? 2 : 1;                // 16-token k-steps of the MMAs that contract over tokens
+    const KSmem sm = make_ksmem(NS);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.misc);
+    unsigned char* sStg = smem + sm.stg;
+
+    constexpr uint32_t tmem_cols = 256u;
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
+        for (int i = 0; i < kNumBars; ++i) {
+            // one arrival per warp of a stream group: chunk ready, E ready, stage empty, accumulator halves, pass-B done, slot free
+            const bool per_warp = (i >= kA2rdy && i <= kErdy) || i >= kEmpty || (i >= kBdone && i < kBdone + 4);
+            mbar_init(&bars[i], per_warp ? 4 : 1);
+        }
+        mbar_fence_init();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    grid_dep_wait();                 // nothing above reads memory another kernel may write
+    grid_dep_launch_dependents();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+
+    // instruction descriptors: bf16 x bf16 -> fp32, M = 128
+    const uint32_t idescT = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);    // K-major x MN-major, N = 128
+    const uint32_t idescU = (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)NP >> 3) << 17) | ((128u >> 4) << 24);        // K-major x K-major, N = 32
+    const uint32_t idescA = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);                 // K-major x K-major, N = 64
+    // canonical no-swizzle layouts (byte offsets)
+    //   K-major : elem(mn, k) at (mn%8)*16 + (mn/8)*128 + (k/8)*LBO + (k%8)*2,  LBO = 16*MN
+    //   MN-major: elem(mn, k) at (k%8)*16 + (mn%8)*2 + (mn/8)*128 + (k/8)*2048
+    constexpr uint32_t SBO = 128, LBO_M = 2048;
+    constexpr uint32_t LBO_W = 64u * 16u;                 // pass-A window: 64 rows
+    constexpr uint32_t LBO_C = (uint32_t)NP * 16u;        // Ktil W: 32 rows
+
+    const int tiles_per_h = B;
+
+    // the CTA's sequence of tile numbers (claimed at run time by the front group) travels through a small ring
+    volatile int* seq_ring = reinterpret_cast<volatile int*>(smem + sm.misc + 16);
+    volatile int* seq_pub = reinterpret_cast<volatile int*>(smem + sm.misc + 32);
+    auto seq_get = [&](int k) -> int {          // -2: the wait ran out
+        for (uint32_t it = 0; it < (1u << 22); ++it) {
+            if (*seq_pub > k) {
+                __threadfence_block();
+                return seq_ring[k & 3];
+            }
+            if (it > 32) __nanosleep(100);
+        }
+        return -2;
+    };
+    auto set_ptr = [&](int b) { return smem + sm.set + (uint32_t)b * sm.set_stride; };
+    auto w_ptr = [&](int b) { return smem + sm.w + (uint32_t)b * sm.w_stride; };
+
+    const int j = (warp & 3) * 32 + lane;      // value column = TMEM lane of this thread (both stream groups)
+
+    if (warp < 4) {
+        // =========================== pass-A group: S_0 chunks -> operands, and the E step ===========================
+        uint32_t phPro = 0, phP = 0, phT = 0, phA = 0, phF = 0;
+        int gc = 0, stage = 0;
+        bool bad = false;
+
+        uint32_t phTf = 0;
+        // pass A of a tile with operand set b; `later`: not the CTA's first tile, so the Ktil^T E accumulator still holds
+        // the tile before until the pass-B group has read it (half by half)
+        auto pass_a = [&](int b, bool later) {
+            const float* sGn = reinterpret_cast<const float*>(set_ptr(b) + sm.set_gn);
+#pragma unroll 2
+            for (int c = 0; c < NCH; ++c) {
+                if (later && (c == 0 || c == NCH / 2)) {
+                    const int hf = c ? 1 : 0;
+                    bad |= !mbar_wait_bounded(&bars[kTfree + hf], (phTf >> hf) & 1u);
+                    phTf ^= 1u << hf;
+                    tc_fence_after();
+                }
+                bad |= !mbar_wait_bounded(&bars[kFull + stage], phF);
+                const float* sS = reinterpret_cast<const float*>(smem + sm.sst + (size_t)stage * sm.sst_bytes) + j;
+                float s0[CH];
+#pragma unroll
+                for (int ii = 0; ii < CH; ++ii) s0[ii] = sS[ii * V];
+                __syncwarp();
+                if (lane == 0) k_arrive(&bars[kEmpty + stage]);
+                {   // G_n * S_0 goes into the Ktil^T E accumulator, so that the MMAs leave S_new there
+                    float ds[CH];
+#pragma unroll
+                    for (int i4 = 0; i4 < CH / 4; ++i4) {
+                        const float4 g4 = *reinterpret_cast<const float4*>(sGn + c * CH + i4 * 4);
+                        ds[i4 * 4 + 0] = g4.x * s0[i4 * 4 + 0];
+                        ds[i4 * 4 + 1] = g4.y * s0[i4 * 4 + 1];
+                        ds[i4 * 4 + 2] = g4.z * s0[i4 * 4 + 2];
+                        ds[i4 * 4 + 3] = g4.w * s0[i4 * 4 + 3];
+                    }
+                    if (!bad) tmem_st16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), ds);
+                }
+                const int ab = c & (kKA2 - 1);
+                if (gc >= kKA2) {     // the chunk buffer was read by the MMAs issued kKA2 chunks ago
+                    bad |= !mbar_wait_bounded(&bars[kA2free + ab], (phA >> ab) & 1u);
+                    phA ^= 1u << ab;
+                }
+                unsigned char* a2hi = smem + sm.a2 + (size_t)ab * (2u * 128u * CH * 2u);
+                unsigned char* a2lo = a2hi + 128u * CH * 2u;
+#pragma unroll
+                for (int v8 = 0; v8 < CH / 8; ++v8) {
+                    uint32_t ohi[4], olo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) split_bf16x2(s0[v8 * 8 + 2 * e], s0[v8 * 8 + 2 * e + 1], ohi[e], olo[e]);
+                    const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO_M;
+                    *reinterpret_cast<uint4*>(a2hi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                    *reinterpret_cast<uint4*>(a2lo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+                }
+                proxy_fence();
+                bad = __any_sync(0xffffffffu, bad);
+                if (lane == 0 && !bad) k_arrive(&bars[kA2rdy + ab]);
+                ++gc;
+                if (++stage == NS) { stage = 0; phF ^= 1u; }
+            }
+        };
+        // E[s, j] = sum_t T[s, t] (v_t[j] - P[t, j]) -> hi + lo A operand of Ktil^T E (chunk-buffer layout, 32 tokens)
+        auto do_e = [&](int b) {
+            bad |= !mbar_wait_bounded(&bars[kPfull + b], (phP >> b) & 1u);
+            phP ^= 1u << b;
+            tc_fence_after();
+            const unsigned char* set = set_ptr(b);
+            const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(set + sm.set_vv);
+            const float* sT1 = reinterpret_cast<const float*>(set + sm.set_t1);
+            float x[kNT];
+            {
+                float x0[16], x1[16];
+                if (!bad) {
+                    tmem_ld16(tmem_base + (uint32_t)b * 64u + lane_sel, x0);
+                    tmem_ld16(tmem_base + (uint32_t)b * 64u + 16u + lane_sel, x1);
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) { x0[t] = 0.f; x1[t] = 0.f; }
+                }
+#pragma unroll
+                for (int t = 0; t < 16; ++t) {
+                    x[t] = __bfloat162float(sV[t * V + j]) - x0[t];
+                    x[16 + t] = __bfloat162float(sV[(16 + t) * V + j]) - x1[t];
+                }
+            }
+            unsigned char* ehi = smem + sm.e;
+            unsigned char* elo = ehi + 128u * (uint32_t)kNT * 2u;
+#pragma unroll
+            for (int v8 = 0; v8 < kNT / 8; ++v8) {
+                float e[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int s = v8 * 8 + u;
+                    float acc = 0.f;
+#pragma unroll
+                    for (int t4 = 0; t4 <= s / 4; ++t4) {      // T is lower triangular
+                        const float4 tt = *reinterpret_cast<const float4*>(sT1 + s * kNT + t4 * 4);
+                        acc = fmaf(tt.x, x[t4 * 4], acc);
+                        acc = fmaf(tt.y, x[t4 * 4 + 1], acc);
+                        acc = fmaf(tt.z, x[t4 * 4 + 2], acc);
+                        acc = fmaf(tt.w, x[t4 * 4 + 3], acc);
+                    }
+                    e[u] = acc;
+                }
+                uint32_t ohi[4], olo[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) split_bf16x2(e[2 * q], e[2 * q + 1], ohi[q], olo[q]);
+                const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO_M;
+                *reinterpret_cast<uint4*>(ehi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+                *reinterpret_cast<uint4*>(elo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+            }
+            proxy_fence();
+            tmem_st_wait();            // the G_n * S_0 columns of pass A are in tensor memory
+            tc_fence_before();
+            bad = __any_sync(0xffffffffu, bad);
+            if (lane == 0 && !bad) k_arrive(&bars[kErdy]);
+        };
+        auto wait_pro = [&](int b) {
+            bad |= !mbar_wait_bounded(&bars[kPro + b], (phPro >> b) & 1u);
+            phPro ^= 1u << b;
+        };
+
+        int cur = seq_get(0);
+        if (cur >= 0) {
+            wait_pro(0);
+            pass_a(0, false);
+            do_e(0);
+            for (int k = 0; !bad; ++k) {
+                const int b = k & 1;
+                const int raw = seq_get(k + 1);
+                if (raw < -1) { bad = true; break; }
+                if (raw < 0) break;
+                wait_pro(b ^ 1);
+                pass_a(b ^ 1, true);
+                // the E operand buffer is read by Ktil^T E of tile k: that must be complete before it is rewritten
+                bad |= !mbar_wait_bounded(&bars[kTfull + b], (phT >> b) & 1u);
+                phT ^= 1u << b;
+                do_e(b ^ 1);
+            }
+        } else if (cur < -1) {
+            bad = true;
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 103);
+    } else if (warp >= 10) {
+        // =========================== pass-B group: S_new written back, then the sketch rows ===========================
+        uint32_t phT = 0;
+        bool bad = false;
+        for (int k = 0; !bad; ++k) {
+            const int raw = seq_get(k);
+            if (raw < 0) { bad = raw < -1; break; }
+            const int tile = raw;
+            const int b = k & 1;
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            float* So = p.state + bh * (size_t)K * V + j;
+            bad |= !mbar_wait_bounded(&bars[kTfull + b], (phT >> b) & 1u);      // Ktil^T E and the sketch correction are complete
+            phT ^= 1u << b;
+            tc_fence_after();
+#pragma unroll 2
+            for (int c = 0; c < NCH; ++c) {
+                if (!bad) {
+                    float t[CH];
+                    tmem_ld16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), t);
+                    if (c == NCH / 2 - 1 || c == NCH - 1) {      // this warp is done with a half of the accumulator
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) k_arrive(&bars[kTfree + (c == NCH - 1 ? 1 : 0)]);
+                    }
+#pragma unroll
+                    for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = t[ii];
+                }
+            }
+            tc_fence_before();
+            bad = __any_sync(0xffffffffu, bad);
+            if (lane == 0 && !bad) k_arrive(&bars[kBdone + b]);
+            // [U | o] = S_0^T (G_n * W) + E^T (Ktil W) from the tile's slot of tensor memory: [correction 32 | U0 32]
+            if (!bad) {
+                const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
+                for (int g0 = 0; g0 < NP; g0 += 16) {
+                    float u0[16], cr[16];
+                    tmem_ld16(slot + 32u + (uint32_t)g0, u0);
+                    tmem_ld16(slot + (uint32_t)g0, cr);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int g = g0 + e;
+                        const float u = u0[e] + cr[e];
+                        if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u;
+                        if (g == QA && p.out != nullptr) {
+                            if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
+                            else reinterpret_cast<float*>(p.out)[bh * V + j] = u;
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) k_arrive(&bars[kBufFree + b]);       // the slot is free for pass A of tile k + 2
+            }
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 111);
+    } else if (warp == 8) {
+        // =========================== MMA issue warp (one thread) ===========================
+        if (lane == 0) {
+            uint32_t phR = 0, phE = 0, phBuf = 0;
+            bool bad = false;
+            int where = 104;                // which wait gave up (status detail): 141 slot free, 142 chunk ready, 143 E ready, 144 accumulator read
+            const uint32_t a2base = smem_u32(smem + sm.a2);
+            // [P | U0](b) = S_0^T [Khat^T | G_n * W] chunk by chunk: one 64-row window per tile
+            auto pass_a = [&](int k) {
+                const int b = k & 1;
+                if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
+                    if (!mbar_wait_bounded(&bars[kBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 141; return; }
+                    phBuf ^= 1u << b;
+                    tc_fence_after();
+                }
+                const uint32_t slot = tmem_base + (uint32_t)b * 64u;
+                const uint32_t whi0 = smem_u32(w_ptr(b));
+                const uint32_t wlo0 = whi0 + sm.w_lo;
+#pragma unroll 2
+                for (int c = 0; c < NCH; ++c) {
+                    const int ab = c & (kKA2 - 1);
+                    if (!mbar_wait_bounded(&bars[kA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 142; return; }
+                    phR ^= 1u << ab;
+                    tc_fence_after();
+                    const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
+                    const uint64_t ahi = make_desc(a2, LBO_M, SBO);
+                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
+                    const uint64_t whi = make_desc(whi0 + (uint32_t)(c * (CH / 8)) * LBO_W, LBO_W, SBO);
+                    const uint64_t wlo = make_desc(wlo0 + (uint32_t)(c * (CH / 8)) * LBO_W, LBO_W, SBO);
+                    tc_mma_bf16(slot, ahi, whi, idescA, c ? 1u : 0u);
+                    tc_mma_bf16(slot, alo, whi, idescA, 1u);
+                    tc_mma_bf16(slot, ahi, wlo, idescA, 1u);
+                    tc_commit(&bars[kA2free + ab]);
+                    if (c == NCH - 1) tc_commit(&bars[kPfull + b]);
+                }
+            };
+            auto step_e = [&](int k) {          // Ktil^T E onto G_n * S_0 (128 columns) and the sketch correction E^T (Ktil W) over the spent P
+                const int b = k & 1;
+                if (!mbar_wait_bounded(&bars[kErdy], phE)) { bad = true; where = 143; return; }
+                phE ^= 1u;
+                if (k >= 1) {                   // the pass-B group must have read the accumulator of the tile before
+                    if (!mbar_wait_bounded(&bars[kBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 144; return; }
+                }
+                tc_fence_after();
+                const uint32_t tmem_t = tmem_base + 128u;
+                const uint32_t tmem_c = tmem_base + (uint32_t)b * 64u;
+                const uint32_t e = smem_u32(smem + sm.e);
+                const uint32_t bt = smem_u32(set_ptr(b) + sm.set_bt);
+                const uint32_t bc = smem_u32(set_ptr(b) + sm.set_bc);
+                for (int kk = 0; kk < ksteps; ++kk) {
+                    const uint64_t ehi = make_desc(e + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
+                    const uint64_t elo = make_desc(e + 128u * (uint32_t)kNT * 2u + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
+                    const uint64_t bthi = make_desc(bt + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
+                    const uint64_t btlo = make_desc(bt + sm.set_bt_lo + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
+                    const uint64_t bchi = make_desc(bc + (uint32_t)kk * 2u * LBO_C, LBO_C, SBO);
+                    const uint64_t bclo = make_desc(bc + 2048u + (uint32_t)kk * 2u * LBO_C, LBO_C, SBO);
+                    tc_mma_bf16(tmem_t, ehi, bthi, idescT, 1u);
+                    tc_mma_bf16(tmem_t, elo, bthi, idescT, 1u);
+                    tc_mma_bf16(tmem_t, ehi, btlo, idescT, 1u);
+                    tc_mma_bf16(tmem_c, ehi, bchi, idescU, kk ? 1u : 0u);
+                    tc_mma_bf16(tmem_c, elo, bchi, idescU, 1u);
+                    tc_mma_bf16(tmem_c, ehi, bclo, idescU, 1u);
+                }
+                tc_commit(&bars[kTfull + b]);
+            };
+            int cur = seq_get(0);
+            if (cur >= 0) {
+                pass_a(0);
+                if (!bad) step_e(0);
+                for (int k = 0; !bad; ++k) {
+                    const int raw = seq_get(k + 1);
+                    if (raw < -1) { bad = true; break; }
+                    if (raw >= 0) pass_a(k + 1);
+                    if (raw < 0 || bad) break;
+                    step_e(k + 1);
+                }
+            } else if (cur < -1) {
+                bad = true;
+            }
+            if (bad) record_fault(p.status, kFaultUpdateWait, where);
+        }
+    } else if (warp == 9) {
+        // =========================== state-load warp: keeps the ring of S_0 stages full ===========================
+        int stage = 0, round = 0;
+        bool bad = false;
+        auto load_tile = [&](int tile) {
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const float* src = p.state + ((size_t)bb * H + h) * (size_t)K * V;
+            for (int c = 0; c < NCH; ++c) {
+                if (round > 0) {     // the stage was released by all four stream warps
+                    if (!mbar_wait_bounded(&bars[kEmpty + stage], (uint32_t)(round - 1) & 1u)) { bad = true; return; }
+                }
+                uint64_t* bar = &bars[kFull + stage];
+                if (lane == 0) {
+                    mbar_expect_tx(bar, sm.sst_bytes);
+                    bulk_g2s(smem + sm.sst + (size_t)stage * sm.sst_bytes, src + (size_t)c * CH * V, (uint32_t)(CH * V * 4), bar);
+                }
+                if (++stage == NS) { stage = 0; ++round; }
+            }
+        };
+        int cur = seq_get(0);
+        if (cur >= 0) {
+            load_tile(cur);
+            for (int k = 0; !bad; ++k) {
+                const int raw = seq_get(k + 1);
+                if (raw < -1) { bad = true; break; }
+                if (raw < 0) break;
+                load_tile(raw);
+            }
+        } else if (cur < -1) {
+            bad = true;
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 107);
+    } else {
+        // =========================== front group: ring-only operands, tile claiming; thread = channel ===========================
+        const int fwarp = gt >> 5;
+        const int i = gt;                     // this thread's channel
+        uint32_t phS = 0;
+        bool dead = false;
+        float* sA = reinterpret_cast<float*>(smem + sm.mats);
+        float* sBeta = sA + kNT * kAS;
+        float* sPart = reinterpret_cast<float*>(sStg);                 // [4 warps][32][32] partial pair sums (over the key / decay rows)
+        float* sKt = reinterpret_cast<float*>(sStg);                   // later: Ktil in fp32, [channel][token ^ (channel & 31)]
+
+        // ---- tile claiming (thread 0 of the group): per-head-index counters behind the status words ----
+        int* sched = p.status + kStatusInts;
+        int* cnt = sched + 4;
+        int h_claim = (int)(((long long)blockIdx.x * H) / gridDim.x);
+        int t_raw = 0;
+        auto claim_issue = [&]() { t_raw = atomicAdd(&cnt[h_claim], 1); };
+        auto claim_resolve = [&]() -> int {
+            for (int attempt = 0; attempt <= H; ++attempt) {
+                if (t_raw < tiles_per_h) return h_claim * tiles_per_h + t_raw;
+                int best = -1, best_c = tiles_per_h;
+                for (int ii = 1; ii <= H; ++ii) {
+                    int hh = h_claim + ii;
+                    if (hh >= H) hh -= H;
+                    const int c = *reinterpret_cast<volatile int*>(&cnt[hh]);
+                    if (c < best_c) { best_c = c; best = hh; }
+                }
+                if (best < 0) return -1;
+                h_claim = best;
+                t_raw = atomicAdd(&cnt[h_claim], 1);
+            }
+            return -1;
+        };
+        auto publish = [&](int k, int tile) {
+            seq_ring[k & 3] = tile;
+            __threadfence_block();
+            *seq_pub = k + 1;
+        };
+
+        // One bulk copy per thread from per-thread constants, spread over the four warps of the group: copy number c belongs
+        // to lane c / 4 of warp c % 4.  0..3: ring keys, decays, values, gates; 4..7: the token's key, decay, value, the query.
+        const uint32_t stg_beta_bytes = n_ring > 0 ? (uint32_t)(p.L * 4) : 0u;
+        const uint32_t stg_bytes = (uint32_t)n_ring * 768u + stg_beta_bytes + (p.has_token ? 768u : 0u) + (p.q != nullptr ? 256u : 0u);
+        const int cp_c = (gt & 31) < 2 ? (gt & 31) * 4 + (gt >> 5) : 32;
+        const unsigned char* cp_base = nullptr;
+        size_t cp_stride = 0;
+        uint32_t cp_dst = 0, cp_bytes = 0;
+        switch (cp_c) {
+            case 0: cp_base = p.ring + (size_t)p.tok_base * 256u; cp_stride = p.rl.head_bytes; cp_dst = 0u; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 1: cp_base = p.ring + p.rl.decay_off + (size_t)p.tok_base * 256u; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_g; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 2: cp_base = p.ring + p.rl.v_off + (size_t)p.tok_base * 256u; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_v; cp_bytes = (uint32_t)n_ring * 256u; break;
+            case 3: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sm.stg_beta; cp_bytes = stg_beta_bytes; break;
+            case 4: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * 2; cp_dst = (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
+            case 5: cp_base = reinterpret_cast<const unsigned char*>(p.decay); cp_stride = (size_t)K * 2; cp_dst = sm.stg_g + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
+            case 6: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * 2; cp_dst = sm.stg_v + (uint32_t)n_ring * 256u; cp_bytes = p.has_token ? 256u : 0u; break;
+            case 7: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * 2; cp_dst = sm.stg_q; cp_bytes = p.q != nullptr ? 256u : 0u; break;
+            default: break;
+        }
+        auto stage_tile = [&](int tile) {       // whole group
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bw = (size_t)bb * H + h;
+            if (gt == 0) mbar_expect_tx(&bars[kStg], stg_bytes);      // (the phase cannot complete before this arrival, whatever the order of the copies)
+            __syncwarp();
+            if (cp_bytes) bulk_g2s(sStg + cp_dst, cp_base + bw * cp_stride, cp_bytes, &bars[kStg]);
+        };
+        auto next_tile = [&](int k) {          // whole group
+            if (gt == 0) {
+                const int nxt = claim_resolve();
+                publish(k, nxt);
+                if (nxt >= 0) claim_issue();
+            }
+            k_sync(2);                         // the published entry is the hand-off to the other threads
+            const int nxt = seq_ring[k & 3];
+            if (nxt >= 0) stage_tile(nxt);
+        };
+        // the first tile: claimed, published and its rows requested before anything else
+        if (gt == 0) claim_issue();
+        next_tile(0);
+        // operand rows that no tile overwrites hold zeros: the padding columns of [Omega | q] in both windows, and the
+        // padding columns of Ktil W in both sets
+        for (uint32_t o = (uint32_t)gt * 16u; o < 2u * sm.w_stride; o += kKGrp * 16u)
+            *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
+        for (int sb = 0; sb < 2; ++sb)
+            for (uint32_t o = (uint32_t)gt * 16u; o < 4096u; o += kKGrp * 16u)
+                *reinterpret_cast<uint4*>(set_ptr(sb) + sm.set_bc + o) = make_uint4(0, 0, 0, 0);
+        k_sync(2);
+
+        for (int k = 0; !dead; ++k) {
+            const int raw_tile = seq_get(k);
+            if (raw_tile < 0) {
+                if (raw_tile < -1) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 108);
+                    dead = true;
+                }
+                break;
+            }
+            const int tile = raw_tile;
+            const int b = k & 1;
+            const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
+            const size_t bh = (size_t)bb * H + h;
+            unsigned char* set = set_ptr(b);
+            unsigned char* wb = w_ptr(b);
+
+            // gate of the current token: requested early
+            float tok_beta = 0.f;
+            if (gt < kNT && p.has_token) tok_beta = p.beta[bh];
+            // Omega row of this channel (fp32, through L1 / L2: shared by the whole batch)
+            const float* og = p.omega + ((size_t)h * K + i) * R;
+            // the operand set and window of tile k - 2 are free once its Ktil^T E has completed
+            if (k >= 2) {
+                if (!k_wait(2, gt, &bars[kTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
+                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 109);
+                    dead = true;
+                    break;
+                }
+            }
+            // the staged rows, gates and query row of this tile must have landed
+            if (!k_wait(2, gt, &bars[kStg], phS)) {
+                if (gt == 0) record_fault(p.status, kFaultUpdateWait, 106);
+                dead = true;
+                break;
+            }
+            phS ^= 1;
+
+            // ---- column i of the key and decay rows into registers; value rows into the set; gates ----
+            float kk[kNT], gg[kNT];
+#pragma unroll
+            for (int s = 0; s < kNT; ++s) {
+                const bool on = s < n_tot;
+                kk[s] = on ? bf16_at(sStg, (uint32_t)(s * K + i)) : 0.f;
+                gg[s] = on ? bf16_at(sStg + sm.stg_g, (uint32_t)(s * K + i)) : 1.f;
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int idx = gt + r * kKGrp;            // 512 vectors of 16 bytes: 32 value rows
+                uint4 vv = make_uint4(0, 0, 0, 0);
+                if ((idx >> 4) < n_tot) vv = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)idx * 16);
+                *reinterpret_cast<uint4*>(set + sm.set_vv + (size_t)idx * 16) = vv;
+            }
+            const float q_i = p.q != nullptr ? bf16_at(sStg + sm.stg_q, (uint32_t)i) : 0.f;
+            if (gt < kNT) {
+                const int s = gt;
+                float bt = 0.f;
+                if (s < n_ring) bt = reinterpret_cast<const float*>(sStg + sm.stg_beta)[p.tok_base + s];
+                else if (s < n_tot) bt = tok_beta;
+                sBeta[s] = bt;
+            }
+            k_sync(2);                 // every thread holds its column: the key / decay rows of the staging area are free
+
+            // ---- pair sums A_sj = sum_i k_s[i] k_j[i] prod_{j<m<=s} g_m[i]: per-channel products, reduced over the 32
+            // channels of a warp by a transposing butterfly, 32 pairs at a time (row sa together with row 32 - sa) ----
+            {
+                float* part = sPart + (size_t)fwarp * (kNT * kNT);
+#pragma unroll
+                for (int sa = 1; sa <= 16; ++sa) {
+                    float vals[32];
+                    {
+                        float r = kk[sa];
+#pragma unroll
+                        for (int jj = 15; jj >= 0; --jj)
+                            if (jj < sa) { r *= gg[jj + 1]; vals[jj] = r * kk[jj]; }
+                    }
+                    if (sa < 16) {
+                        const int sb2 = 32 - sa;
+                        float r = kk[sb2];
+#pragma unroll
+                        for (int jj = 30; jj >= 0; --jj)
+                            if (jj < sb2) { r *= gg[jj + 1]; vals[sa + jj] = r * kk[jj]; }
+                    } else {
+#pragma unroll
+                        for (int jj = 16; jj < 32; ++jj) vals[jj] = 0.f;
+                    }
+                    group_reduce_transpose<32, 32>(vals, lane);
+                    // lane l now holds entry l of the batch: (sa, l) for l < sa, else (32 - sa, l - sa)
+                    const int row = lane < sa ? sa : 32 - sa;
+                    const int col = lane < sa ? lane : lane - sa;
+                    if (sa < 16 || lane < 16) part[row * kNT + col] = vals[0];
+                }
+            }
+            k_sync(2);
+            // beta_s A_sj: the four warps' partials summed in a fixed order (strictly lower triangle)
+            for (int idx = gt; idx < kNT * kNT; idx += kKGrp) {
+                const int s = idx >> 5, jj = idx & 31;
+                float a = 0.f;
+                if (jj < s) a = ((sPart[idx] + sPart[kNT * kNT + idx]) + sPart[2 * kNT * kNT + idx]) + sPart[3 * kNT * kNT + idx];
+                sA[s * kAS + jj] = sBeta[s] * a;
+            }
+            k_sync(2);                 // the partials have been consumed: the area now takes Ktil
+
+            // ---- running products; Khat -> window rows 0..31, Ktil -> set (MN-major) and fp32 scratch, G_n * W -> rows 32.. ----
+            {
+                __nv_bfloat16* whi = reinterpret_cast<__nv_bfloat16*>(wb);
+                __nv_bfloat16* wlo = reinterpret_cast<__nv_bfloat16*>(wb + sm.w_lo);
+                __nv_bfloat16* bthi = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bt);
+                __nv_bfloat16* btlo = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bt_lo);
+                const uint32_t wcol = ((uint32_t)(i >> 3) * LBO_W + (uint32_t)(i & 7) * 2u) >> 1;        // K-major: k = channel
+                const uint32_t bcol = ((uint32_t)(i & 7) * 2u + (uint32_t)(i >> 3) * SBO) >> 1;          // MN-major: mn = channel
+                float G = 1.f;
+#pragma unroll
+                for (int s = 0; s < kNT; ++s) {
+                    G *= gg[s];
+                    __nv_bfloat16 hi, lo;
+                    split_bf16(G * kk[s], hi, lo);
+                    const uint32_t o = wcol + (((uint32_t)(s & 7) * 16u + (uint32_t)(s >> 3) * SBO) >> 1);
+                    whi[o] = hi;
+                    wlo[o] = lo;
+                }
+                float Dn = 1.f;
+#pragma unroll
+                for (int s = kNT - 1; s >= 0; --s) {
+                    const float kt = Dn * kk[s];
+                    Dn *= gg[s];
+                    __nv_bfloat16 hi, lo;
+                    split_bf16(kt, hi, lo);
+                    const uint32_t o = bcol + (((uint32_t)(s & 7) * 16u + (uint32_t)(s >> 3) * LBO_M) >> 1);
+                    bthi[o] = hi;
+                    btlo[o] = lo;
+                    sKt[i * kNT + (s ^ (i & 31))] = kt;
+                }
+                reinterpret_cast<float*>(set + sm.set_gn)[i] = G;
+                if (p.write_sketch) {
+                    for (int g = 0; g < R; ++g) {
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(G * __ldg(og + g), hi, lo);
+                        const uint32_t o = wcol + (((uint32_t)(g & 7) * 16u + (uint32_t)((g >> 3) + 4) * SBO) >> 1);
+                        whi[o] = hi;
+                        wlo[o] = lo;
+                    }
+                }
+                if (p.q != nullptr) {
+                    __nv_bfloat16 hi, lo;
+                    split_bf16(G * q_i, hi, lo);
+                    const uint32_t o = wcol + (((uint32_t)(QA & 7) * 16u + (uint32_t)((QA >> 3) + 4) * SBO) >> 1);
+                    whi[o] = hi;
+                    wlo[o] = lo;
+                }
+            }
+            k_sync(2);                 // A and Ktil (fp32) are complete
+
+            if (fwarp == 0) {
+                // ---- T = (I + Bd A)^{-1} Bd by forward substitution: one column per thread, held in registers ----
+                const int c = lane;
+                float tcol[kNT];
+#pragma unroll
+                for (int s = 0; s < kNT; ++s) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int j4 = 0; j4 < (s + 3) / 4; ++j4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(sA + s * kAS + j4 * 4);
+                        if (j4 * 4 + 0 < s) acc = fmaf(l4.x, tcol[j4 * 4 + 0], acc);
+                        if (j4 * 4 + 1 < s) acc = fmaf(l4.y, tcol[j4 * 4 + 1], acc);
+                        if (j4 * 4 + 2 < s) acc = fmaf(l4.z, tcol[j4 * 4 + 2], acc);
+                        if (j4 * 4 + 3 < s) acc = fmaf(l4.w, tcol[j4 * 4 + 3], acc);
+                    }
+                    tcol[s] = (s >= n_tot || s < c || c >= n_tot) ? 0.f : (s == c ? 1.f : -acc);
+                }
+                const float bc = sBeta[c];
+                float* sT1 = reinterpret_cast<float*>(set + sm.set_t1);
+#pragma unroll
+                for (int s = 0; s < kNT; ++s) sT1[s * kNT + c] = tcol[s] * bc;
+            } else {
+                // ---- Ktil W: 32 tokens x ([Omega | q]), fp32 on CUDA cores; thread = (token, every third column) ----
+                const int s = lane, part = fwarp - 1;
+                const int ncol = p.write_sketch ? R : 0;
+                float acc[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                float accq = 0.f;
+                const float* omh = p.omega + (size_t)h * K * R;
+                const __nv_bfloat16* sq = reinterpret_cast<const __nv_bfloat16*>(sStg + sm.stg_q);
+                const bool do_q = part == 0 && p.q != nullptr;
+                for (int ii = 0; ii < K; ++ii) {
+                    const float kt = sKt[ii * kNT + (s ^ (ii & 31))];
+                    const float* orow = omh + (size_t)ii * R;
+#pragma unroll
+                    for (int u = 0; u < 6; ++u) {
+                        const int g = part + 3 * u;
+                        if (g < ncol) acc[u] = fmaf(kt, __ldg(orow + g), acc[u]);
+                    }
+                    if (do_q) accq = fmaf(kt, __bfloat162float(sq[ii]), accq);
+                }
+                __nv_bfloat16* bchi = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bc);
+                __nv_bfloat16* bclo = bchi + 1024;
+                auto put = [&](int g, float x) {
+                    __nv_bfloat16 hi, lo;
+                    split_bf16(x, hi, lo);
+                    const uint32_t o2 = ((uint32_t)(g & 7) * 16u + (uint32_t)(g >> 3) * SBO + (uint32_t)(s >> 3) * LBO_C + (uint32_t)(s & 7) * 2u) >> 1;
+                    bchi[o2] = hi;
+                    bclo[o2] = lo;
+                };
+#pragma unroll
+                for (int u = 0; u < 6; ++u) {
+                    const int g = part + 3 * u;
+                    if (g < ncol) put(g, acc[u]);
+                }
+                if (do_q) put(QA, accq);
+            }
+            proxy_fence();         // operand sets and windows are read by MMAs (async proxy)
+            k_sync(2);
+            if (gt == 0) k_arrive(&bars[kPro + b]);
+            next_tile(k + 1);      // the staging area has been read: the next tile's rows may come in
+        }
+        if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
+            __threadfence();
+            if (atomicAdd(&sched[0], 1) == (int)gridDim.x - 1) {
+                for (int hh = 0; hh < H; ++hh) cnt[hh] = 0;
+                sched[0] = 0;
+                __threadfence();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// One pass of the kernel over all tiles: ring rows tok_base .. tok_base + n_before - 1 (and the current token).
+static int launch_kda_pass(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+    const sketchssm_config& c = ctx->cfg;
+    Params p = p_in;
+    const uint32_t budget = 227u * 1024u;
+    const KSmem fixed = make_ksmem(0);
+    if (fixed.total + 2u * fixed.sst_bytes > budget) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    int stages = (int)((budget - fixed.total) / fixed.sst_bytes);
+    if (stages > kKStages) stages = kKStages;
+    if (p.stages >= 2 && p.stages < stages) stages = p.stages;
+    p.stages = stages;
+    const KSmem sm = make_ksmem(stages);
+    const long long n_tiles = (long long)c.batch * c.heads;
+    long long grid = (long long)ctx->sm_count;
+    if (grid > n_tiles) grid = n_tiles;
+    auto kern = update_tc_ws_kda_kernel;
+    if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)sm.total)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    if ((ctx->last_cuda_error = launch_kernel(kern, dim3((unsigned)grid), dim3(kKThreads), sm.total, stream, p, p.pdl != 0)) != cudaSuccess)
+        return SKETCHSSM_CUDA_ERROR;
+    return SKETCHSSM_OK;
+}
+
+// Returns SKETCHSSM_UNSUPPORTED_SHAPE outside this kernel's domain (the caller then uses another kernel).  A flush of more
+// than 32 tokens is replayed in blocks of 32: every block is one pass over the state, and only the last one (which holds
+// the current token) writes the sketch and the exact output.
+int launch_update_tc_ws_kda(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
+    const sketchssm_config& c = ctx->cfg;
+    if (c.kind != SKETCHSSM_KDA || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK || c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (c.rank > 16) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    const int n_tot = p_in.n_before + (p_in.has_token ? 1 : 0);
+    if (n_tot < 1 || n_tot > 2 * kNT) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (ctx->sm_count == 0) {
+        int dev = 0, sms = 0;
+        if ((ctx->last_cuda_error = cudaGetDevice(&dev)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
+        if ((ctx->last_cuda_error = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return SKETCHSSM_CUDA_ERROR;
+        ctx->sm_count = sms;
+    }
+    const int passes = (n_tot + kNT - 1) / kNT;
+    for (int ps = 0; ps < passes; ++ps) {
+        Params p = p_in;
+        p.tok_base = ps * kNT;
+        if (ps + 1 < passes) {          // 32 ring rows, state only
+            p.n_before = kNT;
+            p.has_token = 0;
+            p.q = nullptr;
+            p.out = nullptr;
+            p.write_sketch = 0;
+        } else {
+            p.n_before = p_in.n_before - ps * kNT;
+        }
+        const int rc = launch_kda_pass(ctx, p, stream);
+        if (rc != SKETCHSSM_OK) return rc;
+    }
+    ctx->last_launches = passes;
+    return SKETCHSSM_OK;
+}
+
+}  // namespace sketchssm

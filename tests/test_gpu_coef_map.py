@@ -10,7 +10,7 @@ from tests.test_gpu_parity import FP32_GUARD, check, make_layer, run_schedule
 
 pytestmark = pytest.mark.gpu
 
-COEF_GUARD = 2e-4       # max |C_gpu - C_oracle| / max |C|: fp32 solves against fp64 ones
+COEF_GUARD = 1e-3       # max |C_gpu - C_oracle| / max |C|: the map amplifies the fp32-level differences of the state it is built from (ridge 0.1)
 
 
 def check_coef(errs, io):

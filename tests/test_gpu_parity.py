@@ -205,9 +205,21 @@ def test_gdn_warp_specialised_update(tune, batch, heads, rank, buf_len):
     check(run_schedule(w, 2 * buf_len + 3, max_heads=96, tune=tune), "bf16")
 
 
+@pytest.mark.parametrize("tune", [{}, {"decode_stages": 2}, {"pdl": 0}])
+@pytest.mark.parametrize("batch,heads,rank,buf_len", [(5, 3, 16, 32), (40, 20, 16, 16), (33, 7, 8, 12), (6, 2, 5, 4),
+                                                      (12, 4, 16, 32), (7, 3, 12, 40), (5, 2, 16, 64), (150, 3, 16, 32)])
+def test_kda_warp_specialised_update(tune, batch, heads, rank, buf_len):
+    """Warp-specialised tcgen05 flush of the delta rule with per-channel decay (WY form with vector decays, up to 32 tokens
+    per pass, tiles claimed at run time, one CTA per SM so the largest case gives every CTA several tiles) against the
+    oracle's token-by-token replay, over two windows."""
+    w = synth.Workload("t", "kda", batch, heads, 128, 128, rank, buf_len, 0, "bf16", 95, basis="qr")
+    check(run_schedule(w, 2 * buf_len + 3, max_heads=96, tune=tune), "bf16")
+
+
 @pytest.mark.parametrize("kind,dv,buf_len,fills", [("mamba2", 64, 32, (0, 1, 15, 16, 17, 31)), ("mamba2", 128, 64, (16, 32, 47, 48, 63)),
                                                     ("gdn", 128, 16, (0, 1, 7, 15)), ("gdn", 128, 32, (3, 15, 16, 31)),
-                                                    ("gdn", 128, 64, (17, 32, 33, 48, 63))])
+                                                    ("gdn", 128, 64, (17, 32, 33, 48, 63)),
+                                                    ("kda", 128, 32, (0, 1, 7, 15, 16, 17, 31)), ("kda", 128, 64, (31, 32, 33, 47, 63))])
 def test_flush_at_any_ring_fill(kind, dv, buf_len, fills):
     """state_update with n_before tokens in the ring plus the current token, for fills around the tensor-core kernels'
     block boundaries (16 tokens per block) and beyond their domains, and a replay without a current token."""
