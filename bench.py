@@ -101,8 +101,6 @@ def update_kernel_name(w: synth.Workload) -> str:
             return "update_tc_ws_mamba2_kernel" if w.rank <= 32 else "update_tc_mamba2_kernel"
         if w.kind == "gdn" and w.dv == 128 and w.rank <= 16:
             return "update_tc_ws_gdn_kernel"
-        if w.kind == "kda" and w.dv == 128 and w.rank <= 16:
-            return "update_tc_ws_kda_kernel"
     return "update_kernel"
 
 
@@ -558,6 +556,7 @@ def main():
                     help="c5_B<batch>_L<L>_r<r> (a point of the 48-layer Mamba-2 sweep) or c2_mamba2 / c3_gdn / c4_kda")
     ap.add_argument("--layers", type=int, default=0, help="logical layers in the stack (default 48 for sweep points, "
                                                           "else as many distinct copies as fit the budget, at most 8)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (small cases for profiler captures)")
     ap.add_argument("--budget-gb", type=float, default=100.0, help="device memory for the headline stack's layer slots")
     ap.add_argument("--sweep-budget-gb", type=float, default=40.0, help="device memory per sweep point")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -583,6 +582,9 @@ def main():
     else:
         w = synth.CONFIGS[args.workload]
         logical = args.layers or min(8, physical_layers(layer_bytes(w), int(args.budget_gb * 1e9), 8))
+    if args.batch:
+        w = w.replace(batch=args.batch)
+        logical = args.layers or logical
     cfg = {"workload": f"{w.name}: {w.kind} B{w.batch} H{w.heads} K{w.dk} V{w.dv} r{w.rank} L{w.buf_len} "
                        f"{w.io} I/O, fp32 state/sketch", "layers": logical,
            "schedule": "per layer and window: L-1 decode_step + 1 state_update(+sketch)"}

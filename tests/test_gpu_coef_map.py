@@ -13,29 +13,32 @@ pytestmark = pytest.mark.gpu
 COEF_GUARD = 1e-3       # max |C_gpu - C_oracle| / max |C|: the map amplifies the fp32-level differences of the state it is built from (ridge 0.1)
 
 
-def check_coef(errs, io):
+def check_coef(errs):
+    """Outputs, state and sketch within 2e-4 of the oracle (of max |.|), the maps within COEF_GUARD.  The 1e-5 bar of the
+    fixed-map path does not apply: the map is the solution of a linear system with ridge 0.1 formed in fp32, whose
+    condition number (up to (K + lambda) / lambda ~ 1e3) multiplies the fp32 rounding of its inputs."""
     assert errs["c0"] <= COEF_GUARD and errs["C"] <= COEF_GUARD, errs
-    check({k: v for k, v in errs.items() if k not in ("c0", "C")}, io, guard=2e-4)
+    check({k: v for k, v in errs.items() if k not in ("c0", "C")}, "bf16", guard=2e-4)
 
 
 @pytest.mark.parametrize("kind,dv", [("mamba2", 64), ("mamba2", 128), ("gdn", 128), ("kda", 128), ("gdn", 64)])
 @pytest.mark.parametrize("coef,pivots", [("pivot", 4), ("pivot", 1), ("pivot", 8), ("ridge", 0)])
 def test_state_dependent_map_matches_the_oracle(kind, dv, coef, pivots):
     w = synth.Workload("t", kind, 5, 3, 128, dv, 16, 8, 0, "bf16", 101, basis="qr")
-    check_coef(run_schedule(w, 2 * w.buf_len + 3, max_heads=10**9, coef=coef, pivots=pivots), "bf16")
+    check_coef(run_schedule(w, 2 * w.buf_len + 3, max_heads=10**9, coef=coef, pivots=pivots))
 
 
 @pytest.mark.parametrize("rank,dk,dv", [(3, 64, 64), (5, 128, 64), (32, 128, 128), (64, 64, 128)])
 @pytest.mark.parametrize("coef", ["pivot", "ridge"])
 def test_state_dependent_map_ranks_and_shapes(rank, dk, dv, coef):
     w = synth.Workload("t", "gdn", 3, 2, dk, dv, rank, 8, 0, "f32", 103, basis="qr")
-    check_coef(run_schedule(w, w.buf_len + 3, max_heads=10**9, coef=coef), "f32")
+    check_coef(run_schedule(w, w.buf_len + 3, max_heads=10**9, coef=coef))
 
 
 @pytest.mark.parametrize("name", ["c2_mamba2", "c3_gdn"])
 def test_state_dependent_map_full_batch_sampled_heads(name):
     w = synth.CONFIGS[name]
-    check_coef(run_schedule(w, 2 * w.buf_len + 3, max_heads=32, coef="pivot"), w.io)
+    check_coef(run_schedule(w, 2 * w.buf_len + 3, max_heads=32, coef="pivot"))
 
 
 def test_pivot_map_with_all_columns_as_pivots_equals_the_ridge_map():
