@@ -82,7 +82,7 @@ typedef struct sketchssm_config {
     int32_t batch;      /* B >= 1 */
     int32_t heads;      /* H >= 1 */
     int32_t dk;         /* K: 64 or 128 */
-    int32_t dv;         /* V: 64 or 128 */
+    int32_t dv;         /* V: 64, 80 (with dk = 128) or 128 */
     int32_t rank;       /* r: 1..64 */
     int32_t buf_len;    /* L: 4..64, multiple of 4 */
     int32_t io_dtype;   /* sketchssm_dtype of q, k, v, KDA g and of the ring's k, v, g */
@@ -124,6 +124,12 @@ typedef struct sketchssm_buffers {
     void* work;    /* work_bytes of scratch for the decode calls (contents are transient: written and
                       consumed inside one call; calls that overlap on the GPU need separate contexts
                       with separate work buffers) */
+    void* head_rank; /* optional (may be NULL): int32[H], the sketch rank of every head index of this layer, as an
+                      offline rank allocation assigns it (Appendix E): 1..rank = the head uses that many columns
+                      of Omega (its sketch rows and coefficient rows beyond them are ignored and its decode step
+                      fetches only that many); 0 = a dense-fallback head whose decode step reads the full state
+                      exactly, inside the same launch.  Layouts keep the configured `rank` as their row stride.
+                      Only the default one-kernel decode supports the table. */
 } sketchssm_buffers;
 
 typedef struct sketchssm_ctx sketchssm_ctx; /* host-only metadata; owns no device memory */
@@ -137,7 +143,7 @@ int sketchssm_destroy(sketchssm_ctx* ctx);
 /* Byte sizes and ring sub-offsets for this configuration.  Host-only. */
 int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out);
 
-/* Record the caller's device buffers (all seven required, 16-byte aligned).  The context
+/* Record the caller's device buffers (the first seven required, 16-byte aligned; head_rank optional, 4-byte aligned).  The context
  * stores the pointers only; the caller keeps ownership and must keep them alive.
  * Between calls on a context its sketch is written by sketchssm_state_update only.  The library's kernels
  * are launched with programmatic dependent launch, and a decode step that does not directly follow a state
@@ -180,6 +186,21 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
 int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k,
                           const void* v, const void* beta, const void* decay, void* out,
                           uint32_t flags, void* stream);
+
+/* One step of Algorithm 1 for a batch whose sequences are at different window phases (continuous batching: sequences
+ * join and flush at different times).  `phase` is a DEVICE array int32[B], one entry per batch entry b:
+ *     phase[b] = n >= 0       the sequence takes a non-flush decode step with n tokens already buffered (0..L-1):
+ *                             exactly sketchssm_decode_step for its heads;
+ *     phase[b] = -(n + 1) < 0 the sequence takes the flush step with n tokens buffered (0..L-1) plus the current one:
+ *                             exactly sketchssm_state_update with the token, q and out for its heads (the flush may
+ *                             come before the ring is full).
+ * The call enqueues the decode kernel (which skips the flushing sequences) and the flush kernel (which skips the
+ * others; with per-sequence phases the CUDA-core flush kernel is used), then, with config.coef_per_seq, the
+ * coefficient-map kernel for the flushed sequences.  All token pointers are required; `out` receives every
+ * sequence's output.  The caller keeps the counts: after the call a sequence with phase n >= 0 holds n + 1 tokens,
+ * a flushed one none.  `phase` is read by the kernels, so it must not change until they have run. */
+int sketchssm_step_mixed(sketchssm_ctx* ctx, const int32_t* phase, const void* q, const void* k, const void* v,
+                         const void* beta, const void* decay, void* out, uint32_t flags, void* stream);
 
 /* Exact decode step that reads the whole state: o = S_0^T q~_t + sum_s a_s v_s (Eq. 4).
  * Same arguments and ring behaviour as sketchssm_decode_step; U and C are not read.

@@ -26,7 +26,7 @@ EXPORTED = (
     "sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode",
     "sketchssm_read_status", "sketchssm_last_launch_count", "sketchssm_tune",
     "sketchssm_status_string", "sketchssm_version", "sketchssm_last_cuda_error", "sketchssm_step_host",
-    "sketchssm_decode_step_static", "sketchssm_selftest_wait_timeout",
+    "sketchssm_decode_step_static", "sketchssm_selftest_wait_timeout", "sketchssm_step_mixed",
 )
 OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 
@@ -44,7 +44,7 @@ class Sizes(ctypes.Structure):
 
 
 class Buffers(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status", "work")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status", "work", "head_rank")]
 
 
 class Staging(ctypes.Structure):
@@ -78,6 +78,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     for name in ("sketchssm_state_update", "sketchssm_decode_step", "sketchssm_full_read_decode",
                  "sketchssm_decode_step_static"):
         getattr(lib, name).argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, u32, vp]
+    lib.sketchssm_step_mixed.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, u32, vp]
     lib.sketchssm_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, ctypes.POINTER(Staging), u32, vp]
     lib.sketchssm_selftest_wait_timeout.argtypes = [vp, i32, i32, vp]
     lib.sketchssm_read_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32 * 4), vp]
@@ -124,6 +125,7 @@ class SketchSSM:
         self.sizes = Sizes()
         self._check("sketchssm_query_sizes", self.lib.sketchssm_query_sizes(self._ctx, ctypes.byref(self.sizes)))
         self.state = self.sketch = self.ring = self.omega = self.coef = self.status = self.work = None
+        self.head_rank = None        # optional int32 [H] device tensor: per-head sketch rank (0 = full-state read); set, then bind()
         if allocate:
             self.allocate()
 
@@ -144,7 +146,8 @@ class SketchSSM:
         assert self.sketch.numel() * 4 == self.sizes.sketch_bytes
         assert self.ring.numel() == self.sizes.ring_bytes
         b = Buffers(self.state.data_ptr(), self.sketch.data_ptr(), self.ring.data_ptr(),
-                    self.omega.data_ptr(), self.coef.data_ptr(), self.status.data_ptr(), self.work.data_ptr())
+                    self.omega.data_ptr(), self.coef.data_ptr(), self.status.data_ptr(), self.work.data_ptr(),
+                    self.head_rank.data_ptr() if self.head_rank is not None else None)
         self._check("sketchssm_bind", self.lib.sketchssm_bind(self._ctx, ctypes.byref(b)))
 
     def close(self):
@@ -206,6 +209,15 @@ class SketchSSM:
         rc = self.lib.sketchssm_decode_step_static(self._ctx, n_before, _ptr(q), _ptr(k), _ptr(v), _ptr(beta),
                                                    _ptr(decay), _ptr(out), flags, self._stream(stream))
         self._check("sketchssm_decode_step_static", rc)
+        return out
+
+    def step_mixed(self, phase: torch.Tensor, q, k, v, beta, decay, out, stream=None):
+        """sketchssm_step_mixed: one step for sequences at different window phases; phase is an int32 [B] device tensor
+        (n >= 0: decode step at ring fill n; -(n + 1): flush with n buffered tokens plus the current one)."""
+        assert phase.dtype == torch.int32 and phase.is_cuda and phase.numel() == self.B
+        rc = self.lib.sketchssm_step_mixed(self._ctx, _ptr(phase), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(decay),
+                                           _ptr(out), 0, self._stream(stream))
+        self._check("sketchssm_step_mixed", rc)
         return out
 
     def full_read_decode(self, n_before: int, q, k, v, beta, decay, out, flags: int = 0, stream=None):

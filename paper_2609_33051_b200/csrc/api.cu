@@ -46,6 +46,9 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.coef = static_cast<const float*>(ctx->bufs.coef);
     p.status = static_cast<int*>(ctx->bufs.status);
     p.work = static_cast<float*>(ctx->bufs.work);
+    p.head_rank = static_cast<const int*>(ctx->bufs.head_rank);
+    p.n_dev = nullptr;
+    p.n_cap = 0;
     p.wstride = ctx->cfg.dk + ctx->cfg.buf_len;
     p.rl = ctx->ring;
     p.B = ctx->cfg.batch; p.H = ctx->cfg.heads; p.R = ctx->cfg.rank; p.L = ctx->cfg.buf_len;
@@ -136,7 +139,8 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     }
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
     if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
-    if (p.coef_per_seq && !full_read) return SKETCHSSM_UNSUPPORTED_SHAPE;   // the two-kernel decode stages one map per head index
+    // the two-kernel decode stages one map per head index, knows one rank and the value widths 64 and 128
+    if ((p.coef_per_seq && !full_read) || p.head_rank != nullptr || ctx->cfg.dv == 80) return SKETCHSSM_UNSUPPORTED_SHAPE;
     switch (ctx->cfg.kind) {
         case SKETCHSSM_MAMBA2:
             return bf ? launch_decode_split_mamba2_bf16(ctx, p, cs) : launch_decode_split_mamba2_f32(ctx, p, cs);
@@ -159,7 +163,8 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     if (cfg->out_dtype != SKETCHSSM_F32 && cfg->out_dtype != SKETCHSSM_BF16) return SKETCHSSM_INVALID_ARG;
     if (cfg->batch < 1 || cfg->heads < 1 || cfg->device < 0) return SKETCHSSM_INVALID_ARG;
     if (cfg->rank < 1 || cfg->buf_len < 1) return SKETCHSSM_INVALID_ARG;
-    if ((cfg->dk != 64 && cfg->dk != 128) || (cfg->dv != 64 && cfg->dv != 128)) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if ((cfg->dk != 64 && cfg->dk != 128) || (cfg->dv != 64 && cfg->dv != 128 && !(cfg->dv == 80 && cfg->dk == 128)))
+        return SKETCHSSM_UNSUPPORTED_SHAPE;
     if (cfg->rank > kMaxRank) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if (cfg->buf_len < 4 || cfg->buf_len > kMaxBufLen || (cfg->buf_len & 3)) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if ((size_t)cfg->batch * cfg->heads > (size_t)1 << 24) return SKETCHSSM_UNSUPPORTED_SHAPE;
@@ -220,6 +225,7 @@ int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* b) {
     for (const void* p : ps) {
         if (p == nullptr || !aligned16(p)) return SKETCHSSM_INVALID_ARG;
     }
+    if (b->head_rank != nullptr && (reinterpret_cast<uintptr_t>(b->head_rank) & 3u)) return SKETCHSSM_INVALID_ARG;
     ctx->bufs = *b;
     ctx->bound = true;
     ctx->sketch_fresh = true;       // whatever filled the buffers may still be running
@@ -265,6 +271,46 @@ int sketchssm_state_update(sketchssm_ctx* ctx, int n_before, const void* q, cons
     return SKETCHSSM_OK;
 }
 
+int sketchssm_step_mixed(sketchssm_ctx* ctx, const int32_t* phase, const void* q, const void* k, const void* v,
+                         const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
+    if (ctx == nullptr) return SKETCHSSM_INVALID_ARG;
+    ctx->last_launches = 0;
+    if (!ctx->bound) return SKETCHSSM_NOT_BOUND;
+    if (phase == nullptr || (reinterpret_cast<uintptr_t>(phase) & 3u) || flags != 0) return SKETCHSSM_INVALID_ARG;
+    const int L = ctx->cfg.buf_len;
+    // decode part: the stage has room for the largest fill a decoding sequence may have (L - 1 buffered tokens)
+    Params pd;
+    int rc = decode_params(ctx, 0, L - 1, q, k, v, beta, decay, out, 0u, &pd);
+    if (rc != SKETCHSSM_OK) return rc;
+    rc = set_device(ctx);
+    if (rc != SKETCHSSM_OK) return rc;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    pd.n_dev = phase;
+    pd.early_sketch = 0;
+    rc = launch_decode(ctx, pd, cs);
+    if (rc != SKETCHSSM_OK) return rc;
+    int launched = ctx->last_launches;
+    // flush part: every flushing sequence replays its own count of buffered tokens plus the current one
+    Params pu = base_params(ctx);
+    pu.q = q; pu.k = k; pu.v = v; pu.beta = static_cast<const float*>(beta); pu.decay = decay; pu.out = out;
+    pu.n_before = L - 1;
+    pu.has_token = 1;
+    pu.write_sketch = 1;
+    pu.write_state = 1;
+    pu.n_dev = phase;
+    rc = launch_update(ctx, pu, cs);
+    if (rc != SKETCHSSM_OK) return rc;
+    launched += ctx->last_launches;
+    if (pu.coef_per_seq) {
+        rc = launch_coef_map(ctx, pu, cs);
+        if (rc != SKETCHSSM_OK) return rc;
+        launched += 1;
+    }
+    ctx->last_launches = launched;
+    ctx->sketch_fresh = true;
+    return SKETCHSSM_OK;
+}
+
 int sketchssm_decode_step(sketchssm_ctx* ctx, int n_before, const void* q, const void* k, const void* v,
                           const void* beta, const void* decay, void* out, uint32_t flags, void* stream) {
     return decode_common(ctx, 0, n_before, q, k, v, beta, decay, out, flags, stream);
@@ -280,7 +326,8 @@ int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q
     Params p;
     int rc = decode_params(ctx, 0, n_before, q, k, v, beta, decay, out, flags, &p);
     if (rc != SKETCHSSM_OK) return rc;
-    if (ctx->cfg.coef_per_seq) return SKETCHSSM_UNSUPPORTED_SHAPE;    // runs the two-kernel decode (one map per head index)
+    // runs the two-kernel decode (one map per head index, one rank, value widths 64 and 128)
+    if (ctx->cfg.coef_per_seq || ctx->bufs.head_rank != nullptr || ctx->cfg.dv == 80) return SKETCHSSM_UNSUPPORTED_SHAPE;
     // the size limit of the library's static array is checked (on the host, before any CUDA call) by the launcher
     const sketchssm_config& c = ctx->cfg;
     if ((size_t)c.batch * c.heads * (size_t)(c.dk + c.buf_len) * sizeof(float) > (size_t)SKETCHSSM_STATIC_WORK_BYTES)

@@ -63,9 +63,19 @@ template <int K, int V, int EXACT>
 __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int G = p.R;
+    const size_t bh = blockIdx.x;
+    const int h = (int)(bh % (size_t)p.H);
+    // sketch rank of this head: the configured rank or the caller's per-head table (0: the head reads the full state and has
+    // no map); with per-sequence phases only the sequences that were just flushed get a new map
+    int G = p.R;
+    if (p.head_rank != nullptr) {
+        const int r = p.head_rank[h];
+        G = r < 0 ? 0 : (r > p.R ? p.R : r);
+    }
+    if (G == 0) return;
+    if (p.n_dev != nullptr && p.n_dev[bh / (size_t)p.H] >= 0) return;
     const int m = EXACT ? G : min(G, p.pivots);
-    const CoefSmem sm = make_coef_smem(K, V, G, m);
+    const CoefSmem sm = make_coef_smem(K, V, p.R, EXACT ? p.R : min(p.R, p.pivots));
     float* sU = reinterpret_cast<float*>(smem + sm.probe);
     float* sY = reinterpret_cast<float*>(smem + sm.y);
     float* sRU = reinterpret_cast<float*>(smem + sm.ru);
@@ -76,12 +86,11 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
     float* sRed = sSm + 2 * G + m * m; // block reduction scratch
     const int PT = sm.pitch, MP = m + 1;
 
-    const size_t bh = blockIdx.x;
-    const int h = (int)(bh % (size_t)p.H);
-    const float* Ug = p.sketch + bh * (size_t)G * V;
+    const int RS = p.R;                // row strides of U, C and Omega follow the configured rank
+    const float* Ug = p.sketch + bh * (size_t)RS * V;
     const float* Sg = p.state + bh * (size_t)K * V;
-    float* Cg = const_cast<float*>(p.coef) + bh * (size_t)G * K;
-    const float* Om = p.omega + (size_t)h * K * G;
+    float* Cg = const_cast<float*>(p.coef) + bh * (size_t)RS * K;
+    const float* Om = p.omega + (size_t)h * K * RS;
 
     // ---- sketch rows into shared memory ----
     for (int i = tid; i < G * V / 4; i += kCoefThreads) {
@@ -99,20 +108,21 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
         // ---- Gram-Schmidt on the first m sketch rows, in place, by warp 0 (two sweeps; a row that lies in the span of
         // its predecessors becomes zero) ----
         if (warp == 0) {
-            constexpr int EV = V / 32;
+            constexpr int EV = (V + 31) / 32;          // elements per lane; beyond V (V = 80) they are zero and never stored
+            auto on = [&](int e) { return V % 32 == 0 || lane + 32 * e < V; };
             for (int j = 0; j < m; ++j) {
                 float u[EV], ref = 0.f;
 #pragma unroll
-                for (int e = 0; e < EV; ++e) { u[e] = sU[j * PT + lane + 32 * e]; ref = fmaf(u[e], u[e], ref); }
+                for (int e = 0; e < EV; ++e) { u[e] = on(e) ? sU[j * PT + lane + 32 * e] : 0.f; ref = fmaf(u[e], u[e], ref); }
                 ref = warp_sum(ref);
                 for (int sweep = 0; sweep < 2; ++sweep) {
                     for (int i = 0; i < j; ++i) {
                         float d = 0.f;
 #pragma unroll
-                        for (int e = 0; e < EV; ++e) d = fmaf(sU[i * PT + lane + 32 * e], u[e], d);
+                        for (int e = 0; e < EV; ++e) d = fmaf(on(e) ? sU[i * PT + lane + 32 * e] : 0.f, u[e], d);
                         d = warp_sum(d);
 #pragma unroll
-                        for (int e = 0; e < EV; ++e) u[e] = fmaf(-d, sU[i * PT + lane + 32 * e], u[e]);
+                        for (int e = 0; e < EV; ++e) u[e] = fmaf(-d, on(e) ? sU[i * PT + lane + 32 * e] : 0.f, u[e]);
                     }
                 }
                 float nn = 0.f;
@@ -123,10 +133,10 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
                 __syncwarp();
                 // the raw row is still needed for <U_j, Q_i> below: park it in the (not yet used) Y area
 #pragma unroll
-                for (int e = 0; e < EV; ++e) sY[j * V + lane + 32 * e] = sU[j * PT + lane + 32 * e];
+                for (int e = 0; e < EV; ++e) if (on(e)) sY[j * V + lane + 32 * e] = sU[j * PT + lane + 32 * e];
                 __syncwarp();
 #pragma unroll
-                for (int e = 0; e < EV; ++e) sU[j * PT + lane + 32 * e] = u[e] * inv;
+                for (int e = 0; e < EV; ++e) if (on(e)) sU[j * PT + lane + 32 * e] = u[e] * inv;
                 __syncwarp();
             }
         }
@@ -227,7 +237,7 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
             for (int g = 0; g < G; ++g) {
                 float Mg = 0.f;
                 for (int j = 0; j < m; ++j) Mg = fmaf(sRU[g * MP + j], y[j], Mg);
-                Mg = fmaf(Mg, inv_mu, sUU[g] * Om[(size_t)k * G + g]);
+                Mg = fmaf(Mg, inv_mu, sUU[g] * Om[(size_t)k * RS + g]);
                 const float t = Mg / sD[g];
                 for (int j = 0; j < m; ++j) z[j] = fmaf(sRU[g * MP + j], t, z[j]);
             }
@@ -240,7 +250,7 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
             for (int g = 0; g < G; ++g) {
                 float Mg = 0.f, corr = 0.f;
                 for (int j = 0; j < m; ++j) { Mg = fmaf(sRU[g * MP + j], y[j], Mg); corr = fmaf(sRU[g * MP + j], wv[j], corr); }
-                Mg = fmaf(Mg, inv_mu, sUU[g] * Om[(size_t)k * G + g]);
+                Mg = fmaf(Mg, inv_mu, sUU[g] * Om[(size_t)k * RS + g]);
                 Cg[(size_t)g * K + k] = (Mg - corr) / sD[g];
             }
         }
@@ -303,6 +313,7 @@ int launch_coef_map(Ctx* ctx, const Params& p, cudaStream_t stream) {
     const int K = ctx->cfg.dk, V = ctx->cfg.dv;
     if (K == 128 && V == 128) return launch_coef_kv<128, 128>(ctx, p, stream);
     if (K == 128 && V == 64) return launch_coef_kv<128, 64>(ctx, p, stream);
+    if (K == 128 && V == 80) return launch_coef_kv<128, 80>(ctx, p, stream);
     if (K == 64 && V == 64) return launch_coef_kv<64, 64>(ctx, p, stream);
     if (K == 64 && V == 128) return launch_coef_kv<64, 128>(ctx, p, stream);
     return SKETCHSSM_UNSUPPORTED_SHAPE;

@@ -26,6 +26,9 @@ namespace {
 
 
 #define DEC_WAIT(bar, parity) mbar_wait_bounded(bar, parity)
+// parity of the sketch barrier's phase for the current head: with one rank for all heads both barriers advance together
+// (the ring barrier's parity has already been flipped when the sketch is waited for)
+#define PARB (GEN ? parB : (parA ^ 1u))
 
 struct StageLayout {
     uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
@@ -83,10 +86,13 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
 }  // namespace
 
 // RT: the sketch rank as a compile-time constant (loops over ranks unroll fully), or 0 for any rank.
-template <int KIND, typename IO, int K, int V, int RT>
+// GEN: 0 = one ring fill and one rank for every head of the launch (copy sizes are per-lane constants);
+//      1 = per-sequence phases and / or a per-head rank table (sizes follow the head).
+template <int KIND, typename IO, int K, int V, int RT, int GEN>
 __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
-    constexpr int EV = V / 32;
+    constexpr int EV = V % 32 == 0 ? V / 32 : 4;        // value elements per lane ...
+    constexpr int VL = V / EV;                          // ... on the first VL lanes (all 32, or 20 for V = 80)
     constexpr int NB = 8;                               // dot products per transposing reduction
     extern __shared__ __align__(128) unsigned char smem[];
 
@@ -94,10 +100,12 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
     const int R = RT ? RT : p.R;
-    const int L = p.L, H = p.H, B = p.B, n = p.n_before;
+    const int L = p.L, H = p.H, B = p.B;
+    const int n_cap = p.n_before;                       // ring rows the stage has room for (per-sequence phases: the largest fill)
+    const bool vlane = VL == 32 || lane < VL;           // this lane holds value elements
     const int RP = (R + 7) & ~7;
 
-    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n, p.full_read, p.coef_per_seq);
+    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, p.coef_per_seq);
     const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, p.coef_per_seq, sl.total);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * 2;
     float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
@@ -130,39 +138,64 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     __syncthreads();
 
     // A warp's stage is filled by two groups of bulk copies, each completing on its own mbarrier: group A holds what
-    // the ring sweep reads (the token's rows and the buffered keys / values / gates), group B the sketch U.  Group A of
-    // the warp's next head is issued as soon as the sweep of the current head is over and group B as soon as U has been
-    // used, so the next head's loads overlap the rest of the current head's arithmetic without a second stage.
-    // Every copy is issued by its own lane from per-lane constants set up once (base pointer, bytes per head, target).
-    const uint32_t txA = sl.k_bytes + sl.v_bytes + sl.gate_bytes + sl.g_bytes + 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
-    const uint32_t txB = sl.u_bytes + sl.c_bytes;
+    // the ring sweep reads (the token's rows and the buffered keys / values / gates), group B the sketch U (and, with a
+    // per-sequence coefficient map, the head's own C).  Group A of the warp's next head is issued as soon as the sweep of
+    // the current head is over and group B as soon as U has been used, so the next head's loads overlap the rest of the
+    // current head's arithmetic without a second stage.  Every copy is issued by its own lane from per-lane constants set
+    // up once (base pointer, bytes per head, target); its size is fixed, or a multiple of the head's ring fill (the fill
+    // is per sequence when the caller passes per-sequence phases) or of the head's sketch rank (per-head rank table).
     const unsigned char* cp_base = nullptr;
     size_t cp_stride = 0;
-    uint32_t cp_dst = 0, cp_bytes = 0;
+    uint32_t cp_dst = 0, cp_unit = 0;
+    int cp_mode = 0;            // bytes of the copy: 0 cp_unit; 1 cp_unit * ring fill; 2 cp_unit if the ring is not empty; 3 cp_unit * rank
     switch (lane) {
-        case 0: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tq_off; cp_bytes = sl.tqk_bytes; break;
-        case 1: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tk_off; cp_bytes = sl.tqk_bytes; break;
-        case 2: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * sizeof(IO); cp_dst = sl.tv_off; cp_bytes = sl.tv_bytes; break;
-        case 3: cp_base = reinterpret_cast<const unsigned char*>(p.decay); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tg_off; cp_bytes = sl.tg_bytes; break;
-        case 4: cp_base = p.ring; cp_stride = p.rl.head_bytes; cp_dst = sl.k_off; cp_bytes = sl.k_bytes; break;
-        case 5: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sl.gate_off; cp_bytes = sl.gate_bytes; break;
-        case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_bytes = sl.v_bytes; break;
-        case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_bytes = sl.g_bytes; break;
-        case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * 4; cp_dst = sl.u_off; cp_bytes = sl.u_bytes; break;
-        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_bytes = sl.c_bytes; break;
+        case 0: cp_base = reinterpret_cast<const unsigned char*>(p.q); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tq_off; cp_unit = sl.tqk_bytes; break;
+        case 1: cp_base = reinterpret_cast<const unsigned char*>(p.k); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tk_off; cp_unit = sl.tqk_bytes; break;
+        case 2: cp_base = reinterpret_cast<const unsigned char*>(p.v); cp_stride = (size_t)V * sizeof(IO); cp_dst = sl.tv_off; cp_unit = sl.tv_bytes; break;
+        case 3: cp_base = reinterpret_cast<const unsigned char*>(p.decay); cp_stride = (size_t)K * sizeof(IO); cp_dst = sl.tg_off; cp_unit = sl.tg_bytes; break;
+        case 4: cp_base = p.ring; cp_stride = p.rl.head_bytes; cp_dst = sl.k_off; cp_unit = (uint32_t)(K * sizeof(IO)); cp_mode = 1; break;
+        case 5: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sl.gate_off; cp_unit = (uint32_t)((KIND == SKETCHSSM_KDA ? 1 : 2) * L * 4); cp_mode = 2; break;
+        case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_unit = (uint32_t)(V * sizeof(IO)); cp_mode = 1; break;
+        case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_unit = KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u; cp_mode = 1; break;
+        case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * 4; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * 4); cp_mode = 3; break;
+        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_unit = p.coef_per_seq ? (uint32_t)(K * 4) : 0u; cp_mode = 3; break;
         default: break;
     }
+    const uint32_t tokA = 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
+    const uint32_t rowA = (uint32_t)((K + V) * sizeof(IO)) + (KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u);
+    const uint32_t gateA = (uint32_t)((KIND == SKETCHSSM_KDA ? 1 : 2) * L * 4);
+    const uint32_t rowB = (uint32_t)(V * 4) + (p.coef_per_seq ? (uint32_t)(K * 4) : 0u);
+    const int r_uni = p.full_read ? 0 : R;          // GEN = 0: the rank of every head
+    // GEN = 0: the size of this lane's copy and the two transaction totals are constants of the launch
+    const uint32_t cp_fixed = cp_mode == 0 ? cp_unit : cp_mode == 1 ? cp_unit * (uint32_t)n_cap
+                            : cp_mode == 2 ? (n_cap > 0 ? cp_unit : 0u) : cp_unit * (uint32_t)r_uni;
+    const uint32_t txA_fixed = tokA + (uint32_t)n_cap * rowA + (n_cap > 0 ? gateA : 0u);
+    const uint32_t txB_fixed = (uint32_t)r_uni * rowB;
     uint64_t* barA = &bars[0];
     uint64_t* barB = &bars[1];
-    auto issue_a = [&](size_t bh) {      // whole warp
-        if (lane == 0) mbar_expect_tx(barA, txA);
-        __syncwarp();
-        if (lane < 8 && cp_bytes) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barA);
+    auto issue_a = [&](size_t bh, int n_it) {      // whole warp; n_it: ring fill of the head
+        if constexpr (GEN) {
+            if (lane == 0) mbar_expect_tx(barA, tokA + (uint32_t)n_it * rowA + (n_it > 0 ? gateA : 0u));
+            __syncwarp();
+            const uint32_t bytes = cp_mode == 0 ? cp_unit : cp_mode == 1 ? cp_unit * (uint32_t)n_it : (n_it > 0 ? cp_unit : 0u);
+            if (lane < 8 && bytes) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, bytes, barA);
+        } else {
+            if (lane == 0) mbar_expect_tx(barA, txA_fixed);
+            __syncwarp();
+            if (lane < 8 && cp_fixed) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_fixed, barA);
+        }
     };
-    auto issue_b = [&](size_t bh) {      // whole warp
-        if (lane == 8 && txB) mbar_expect_tx(barB, txB);
-        __syncwarp();
-        if ((lane == 8 || lane == 9) && cp_bytes) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_bytes, barB);
+    auto issue_b = [&](size_t bh, int r_it) {      // whole warp; r_it: sketch rank of the head (0: nothing to fetch)
+        if constexpr (GEN) {
+            if (lane == 8 && r_it > 0) mbar_expect_tx(barB, (uint32_t)r_it * rowB);
+            __syncwarp();
+            if ((lane == 8 || lane == 9) && cp_unit && r_it > 0)
+                bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_unit * (uint32_t)r_it, barB);
+        } else {
+            if (lane == 8 && txB_fixed) mbar_expect_tx(barB, txB_fixed);
+            __syncwarp();
+            if ((lane == 8 || lane == 9) && cp_fixed) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_fixed, barB);
+        }
     };
 
     // The CTA's heads are handed to its warps at run time (a counter in shared memory): a warp claims its next head
@@ -181,9 +214,27 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         hh = item >= second_h_start ? h_first + 1 : h_first;
         bb = item - hh * B;
     };
+    // Per-head sketch rank: the configured rank, or the caller's table (0 = this head reads the full state instead).
+    // The table is a layer constant like C, so it may be read before the predecessor in the stream is done.
+    auto rank_of = [&](int hh) -> int {
+        if constexpr (!GEN) return r_uni;
+        if (p.full_read) return 0;
+        if (p.head_rank == nullptr) return R;
+        const int r = p.head_rank[hh];
+        return r < 0 ? 0 : (r > R ? R : r);
+    };
+    // Per-sequence ring fill: the call's n_before, or the caller's per-sequence phase (negative: the sequence takes the
+    // flush step in this call and is skipped here).
+    auto fill_of = [&](int bb) -> int {
+        if constexpr (!GEN) return n_cap;
+        return p.n_dev == nullptr ? n_cap : p.n_dev[bb];
+    };
+
     int item = warp < n_items ? item0 + warp : item1;      // the first head of every warp is fixed (the counter starts at nwarps)
     int h = 0, b = 0, hn = 0, bn = 0;
     if (item < item1) head_of(item, h, b);
+    int rk = item < item1 ? rank_of(h) : 0, rk_next = 0;
+    int n = 0, n_next = 0;
 
     // the token's scalar gates travel in registers, fetched one head ahead
     auto scalar_gates = [&](size_t bh, float& bt, float& dsc) {
@@ -194,38 +245,56 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     float bt_next = 0.f, dsc_next = 1.f;
     // Only a state update writes the sketch; unless one may still be running (the caller of the launcher knows), the first
     // head's sketch rows are requested before the predecessor in the stream is waited for, so they travel during its tail.
-    const bool early_u = p.early_sketch != 0;
-    if (item < item1 && early_u) issue_b((size_t)b * H + h);
+    // (Not with per-sequence phases: whether the head takes part at all is only known after the wait.)
+    const bool early_u = p.early_sketch != 0 && p.n_dev == nullptr;
+    if (item < item1 && early_u) issue_b((size_t)b * H + h, rk);
     grid_dep_wait();                 // from here on the ring and the token tensors (and otherwise the sketch) are read
     // Dependents are released only now: a successor that reads its sketch early must not start before this kernel has
     // seen its own predecessor (possibly a state update) complete.
     grid_dep_launch_dependents();
     if (item < item1) {
         const size_t bh0 = (size_t)b * H + h;
-        issue_a(bh0);
-        if (!early_u) issue_b(bh0);
-        scalar_gates(bh0, bt_next, dsc_next);
+        n = fill_of(b);
+        if (n >= 0) {
+            issue_a(bh0, n);
+            if (!early_u) issue_b(bh0, rk);
+            scalar_gates(bh0, bt_next, dsc_next);
+        }
     }
     // A wait that runs out ends the warp's loop; the decision is taken by vote so that all lanes leave together.
     // pendA / pendB: parity of a phase whose copies may still be in flight when the loop is left that way (-1: none).
     int pendA = -1, pendB = -1;
+    uint32_t parA = 0, parB = 0;     // phase parities of the two barriers (a phase passes only for heads that issued copies)
 
-    for (int it = 0; item < item1; ++it) {
-        const uint32_t parity = it & 1;
+    while (item < item1) {
+        if constexpr (!GEN) { n = n_cap; n_next = n_cap; rk = r_uni; rk_next = r_uni; }      // launch constants
         const size_t bh = (size_t)b * H + h;
         const int item_next = claim();
         const bool has_next = item_next < item1;
-        if (has_next) head_of(item_next, hn, bn);
+        if (has_next) {
+            head_of(item_next, hn, bn);
+            rk_next = rank_of(hn);
+            n_next = fill_of(bn);
+        }
+        const bool go_next = has_next && n_next >= 0;          // the next head takes a decode step in this call
         const size_t bh_next = (size_t)bn * H + hn;
         const float bt = bt_next, dsc = dsc_next;
-        if (has_next) scalar_gates(bh_next, bt_next, dsc_next);
+        if (go_next) scalar_gates(bh_next, bt_next, dsc_next);
 
-        if (__any_sync(0xffffffffu, !DEC_WAIT(barA, parity))) {
+        if (n < 0) {                 // this sequence takes the flush step in this call: nothing to do here
+            if (go_next) { issue_a(bh_next, n_next); issue_b(bh_next, rk_next); }
+            item = item_next; h = hn; b = bn; n = n_next; rk = rk_next;
+            continue;
+        }
+        const bool full = rk == 0;   // exact read of the whole state for this head
+
+        if (__any_sync(0xffffffffu, !DEC_WAIT(barA, parA))) {
             if (lane == 0) record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
-            pendA = (int)parity;
-            pendB = p.full_read ? -1 : (int)parity;
+            pendA = (int)parA;
+            pendB = full ? -1 : (int)(GEN ? parB : parA);
             break;
         }
+        parA ^= 1u;
         const unsigned char* sb = my_stage;
         const IO* sK = reinterpret_cast<const IO*>(sb + sl.k_off);
         const IO* sV = reinterpret_cast<const IO*>(sb + sl.v_off);
@@ -236,13 +305,15 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         float q0[EK], x[EK], kk[EK], gg[EK], vv[EV], o[EV];
         load_io<EK>(reinterpret_cast<const IO*>(sb + sl.tq_off), lane * EK, q0);
         load_io<EK>(reinterpret_cast<const IO*>(sb + sl.tk_off), lane * EK, kk);
-        load_io<EV>(reinterpret_cast<const IO*>(sb + sl.tv_off), lane * EV, vv);
+#pragma unroll
+        for (int e = 0; e < EV; ++e) vv[e] = 0.f;
+        if (vlane) load_io<EV>(reinterpret_cast<const IO*>(sb + sl.tv_off), lane * EV, vv);
         if constexpr (KIND == SKETCHSSM_KDA) load_io<EK>(reinterpret_cast<const IO*>(sb + sl.tg_off), lane * EK, gg);
 
         if (p.append) {
             unsigned char* rh = p.ring + bh * p.rl.head_bytes;
             store_io<EK>(reinterpret_cast<IO*>(rh) + (size_t)n * K, lane * EK, kk);
-            store_io<EV>(reinterpret_cast<IO*>(rh + p.rl.v_off) + (size_t)n * V, lane * EV, vv);
+            if (vlane) store_io<EV>(reinterpret_cast<IO*>(rh + p.rl.v_off) + (size_t)n * V, lane * EV, vv);
             if constexpr (KIND == SKETCHSSM_KDA) {
                 store_io<EK>(reinterpret_cast<IO*>(rh + p.rl.decay_off) + (size_t)n * K, lane * EK, gg);
                 if (lane == 0) reinterpret_cast<float*>(rh + p.rl.beta_off)[n] = bt;
@@ -309,10 +380,12 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
             for (int s = n - 1; s >= 0; --s) {
                 const float a = sBeta[s] * dsuf * sP[s];
                 dsuf *= sDec[s];
-                float vr[EV];
-                load_io<EV>(sV, s * V + lane * EV, vr);
+                if (vlane) {
+                    float vr[EV];
+                    load_io<EV>(sV, s * V + lane * EV, vr);
 #pragma unroll
-                for (int e = 0; e < EV; ++e) o[e] = fmaf(a, vr[e], o[e]);
+                    for (int e = 0; e < EV; ++e) o[e] = fmaf(a, vr[e], o[e]);
+                }
             }
 #pragma unroll
             for (int e = 0; e < EK; ++e) x[e] = dsuf * q0[e];
@@ -321,7 +394,9 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
             for (int s = n - 1; s >= 0; --s) {
                 float kr[EK], vr[EV];
                 load_io<EK>(sK, s * K + lane * EK, kr);
-                load_io<EV>(sV, s * V + lane * EV, vr);
+#pragma unroll
+                for (int e = 0; e < EV; ++e) vr[e] = 0.f;
+                if (vlane) load_io<EV>(sV, s * V + lane * EV, vr);
                 float part = 0.f;
 #pragma unroll
                 for (int e = 0; e < EK; ++e) part = fmaf(kr[e], x[e], part);
@@ -343,22 +418,23 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 
         // the sweep is done with the ring part of the stage: the next head's group A may come in
         __syncwarp();
-        if (has_next) issue_a(bh_next);
-        if (!p.full_read) {
+        if (go_next) issue_a(bh_next, n_next);
+        if (!full) {
             // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
             const float* sC = p.coef_per_seq ? reinterpret_cast<const float*>(sb + sl.c_off)
                                              : reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
             __syncwarp();
             if (p.coef_per_seq) {        // the head's own map arrives with its sketch rows
-                if (__any_sync(0xffffffffu, !DEC_WAIT(barB, parity))) {
+                if (__any_sync(0xffffffffu, !DEC_WAIT(barB, PARB))) {
                     if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
-                    pendB = (int)parity;
-                    pendA = has_next ? (int)(parity ^ 1u) : -1;
+                    pendB = (int)PARB;
+                    pendA = go_next ? (int)parA : -1;
                     break;
                 }
             }
+            const int rp_it = RT ? ((RT + 7) & ~7) : ((rk + 7) & ~7);
 #pragma unroll
-            for (int g0 = 0; g0 < (RT ? ((RT + 7) & ~7) : RP); g0 += NB) {
+            for (int g0 = 0; g0 < (RT ? ((RT + 7) & ~7) : rp_it); g0 += NB) {
                 float part[NB];
 #pragma unroll
                 for (int i = 0; i < NB; ++i) {
@@ -373,52 +449,65 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
             __syncwarp();
-            if (__any_sync(0xffffffffu, !DEC_WAIT(barB, parity))) {
-                if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
-                pendB = (int)parity;
-                pendA = has_next ? (int)(parity ^ 1u) : -1;
-                break;
+            if (!p.coef_per_seq) {
+                if (__any_sync(0xffffffffu, !DEC_WAIT(barB, PARB))) {
+                    if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
+                    pendB = (int)PARB;
+                    pendA = go_next ? (int)parA : -1;
+                    break;
+                }
             }
+            if constexpr (GEN) parB ^= 1u;
             const float* sU = reinterpret_cast<const float*>(sb + sl.u_off);
+            if (vlane) {
 #pragma unroll (RT ? RT : 4)
-            for (int g = 0; g < R; ++g) {
-                const float cg = sX[g];
-                float uu[EV];
-                load_io<EV>(sU, g * V + lane * EV, uu);
+                for (int g = 0; g < (RT ? RT : rk); ++g) {
+                    const float cg = sX[g];
+                    float uu[EV];
+                    load_io<EV>(sU, g * V + lane * EV, uu);
 #pragma unroll
-                for (int e = 0; e < EV; ++e) o[e] = fmaf(cg, uu[e], o[e]);
+                    for (int e = 0; e < EV; ++e) o[e] = fmaf(cg, uu[e], o[e]);
+                }
             }
             __syncwarp();
-            if (has_next) issue_b(bh_next);
+            if (go_next) issue_b(bh_next, rk_next);
         } else {
             __syncwarp();
             store_io<EK>(sX, lane * EK, x);
             __syncwarp();
-            const float* Sg = p.state + bh * (size_t)K * V + lane * EV;
-            constexpr int RB = 8;
-            for (int i0 = 0; i0 < K; i0 += RB) {
-                float rows[RB][EV];
+            if (vlane) {
+                const float* Sg = p.state + bh * (size_t)K * V + lane * EV;
+                constexpr int RB = 8;
+                for (int i0 = 0; i0 < K; i0 += RB) {
+                    float rows[RB][EV];
 #pragma unroll
-                for (int r = 0; r < RB; ++r) load_io<EV>(Sg, (i0 + r) * V, rows[r]);
+                    for (int r = 0; r < RB; ++r) load_io<EV>(Sg, (i0 + r) * V, rows[r]);
 #pragma unroll
-                for (int r = 0; r < RB; ++r) {
-                    const float xi = sX[i0 + r];
+                    for (int r = 0; r < RB; ++r) {
+                        const float xi = sX[i0 + r];
 #pragma unroll
-                    for (int e = 0; e < EV; ++e) o[e] = fmaf(rows[r][e], xi, o[e]);
+                        for (int e = 0; e < EV; ++e) o[e] = fmaf(rows[r][e], xi, o[e]);
+                    }
                 }
             }
+            // a head that reads the full state fetched no sketch rows; the next head's are requested here
+            if (go_next) issue_b(bh_next, rk_next);
         }
 
-        if (p.out_bf16) {
-            store_io<EV>(reinterpret_cast<__nv_bfloat16*>(p.out) + bh * V, lane * EV, o);
-        } else {
-            store_io<EV>(reinterpret_cast<float*>(p.out) + bh * V, lane * EV, o);
+        if (vlane) {
+            if (p.out_bf16) {
+                store_io<EV>(reinterpret_cast<__nv_bfloat16*>(p.out) + bh * V, lane * EV, o);
+            } else {
+                store_io<EV>(reinterpret_cast<float*>(p.out) + bh * V, lane * EV, o);
+            }
         }
 
         __syncwarp();  // every lane is done with the scratch before it is reused
         item = item_next;
         h = hn;
         b = bn;
+        n = n_next;
+        rk = rk_next;
     }
     // Left on a timeout: bulk copies already issued into this warp's stage get a short, bounded grace period, so that
     // they do not land in shared memory that has meanwhile been handed to another CTA.
@@ -441,10 +530,12 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
     // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
-    auto kern = p.R == 16 ? decode_kernel<KIND, IO, K, V, 16> : decode_kernel<KIND, IO, K, V, 0>;
+    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr;
+    const bool fixed16 = p.R == 16 && !gen;     // the unrolled rank-16 instantiation needs one rank for all heads
+    auto kern = gen ? decode_kernel<KIND, IO, K, V, 0, 1> : fixed16 ? decode_kernel<KIND, IO, K, V, 16, 0> : decode_kernel<KIND, IO, K, V, 0, 0>;
     // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does
-    static int regs_per_thread[2] = {0, 0};
-    int& regs = regs_per_thread[p.R == 16 ? 1 : 0];
+    static int regs_per_thread[3] = {0, 0, 0};
+    int& regs = regs_per_thread[gen ? 2 : fixed16 ? 1 : 0];
     if (regs == 0) {
         cudaFuncAttributes fa;
         if ((ctx->last_cuda_error = cudaFuncGetAttributes(&fa, kern)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
@@ -484,6 +575,7 @@ static int launch_decode_shape(Ctx* ctx, const Params& p, cudaStream_t stream) {
     const int K = ctx->cfg.dk, V = ctx->cfg.dv;
     if (K == 128 && V == 128) return launch_decode_t<KIND, IO, 128, 128>(ctx, p, stream);
     if (K == 128 && V == 64) return launch_decode_t<KIND, IO, 128, 64>(ctx, p, stream);
+    if (K == 128 && V == 80) return launch_decode_t<KIND, IO, 128, 80>(ctx, p, stream);
     if (K == 64 && V == 64) return launch_decode_t<KIND, IO, 64, 64>(ctx, p, stream);
     if (K == 64 && V == 128) return launch_decode_t<KIND, IO, 64, 128>(ctx, p, stream);
     return SKETCHSSM_UNSUPPORTED_SHAPE;

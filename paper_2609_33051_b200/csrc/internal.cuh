@@ -76,6 +76,10 @@ struct Params {
     int coef_per_seq;     // the coefficient map is per (batch, head) [B][H][r][K] and rebuilt by every state update
     int pivots;           // coefficient-map construction: pivot count P of the approximated state metric; 0 = exact ridge form
     float ridge_lambda;   // ridge of the state-dependent coefficient map
+    const int* head_rank; // optional [H]: sketch rank per head index (0: the head reads the full state); nullptr: R for every head
+    const int* n_dev;     // optional [B]: per-sequence phase of a mixed step (>= 0: decode step at that ring fill; < 0: flush with
+                          // -v - 1 buffered tokens); nullptr: n_before for every sequence
+    int n_cap;            // update (CUDA cores) with per-sequence phases: ring rows the shared-memory layout has room for
     int tok_base;         // update (GDN tensor-core kernel): first ring row of this pass when a flush is replayed in blocks of 16 tokens
 };
 

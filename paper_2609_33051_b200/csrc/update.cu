@@ -12,9 +12,7 @@
 
 namespace sketchssm {
 
-constexpr int kVT = 64;                 // columns per CTA
-constexpr int kParts = 4;               // threads per column
-constexpr int kUpdThreads = kVT * kParts;
+constexpr int kParts = 4;               // threads per column; a CTA owns VT = 64 columns (80 when V = 80) of one head
 
 // shared-memory row of K floats split into kParts parts, each padded by 4 floats so that the four
 // parts of a warp read from different banks with 128-bit loads
@@ -50,7 +48,7 @@ struct UpdateSmem {
 };
 
 template <int K>
-__host__ __device__ inline UpdateSmem make_update_smem(int kind, int n_tot, int R4) {
+__host__ __device__ inline UpdateSmem make_update_smem(int kind, int n_tot, int R4, int kVT) {
     UpdateSmem u;
     const int ntok = n_tot > 0 ? n_tot : 1;
     uint32_t off = 0;
@@ -65,8 +63,9 @@ __host__ __device__ inline UpdateSmem make_update_smem(int kind, int n_tot, int 
     return u;
 }
 
-template <int KIND, typename IO, int K>
-__global__ void __launch_bounds__(kUpdThreads) update_kernel(const Params p) {
+template <int KIND, typename IO, int K, int kVT>
+__global__ void __launch_bounds__(kVT * kParts) update_kernel(const Params p) {
+    constexpr int kUpdThreads = kVT * kParts;
     using PR = PaddedRow<K>;
     constexpr int RP = PR::RP;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -78,11 +77,17 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const Params p) {
     const int bh = blockIdx.x / vtiles;
     const int v0 = (blockIdx.x % vtiles) * kVT;
     const int b = bh / H, h = bh % H;
-    (void)b;
-    const int n_ring = p.n_before;
+    // ring fill: the call's n_before, or with per-sequence phases the sequence's own (a sequence whose phase says
+    // "decode step" is left alone by this kernel)
+    int n_ring = p.n_before;
+    if (p.n_dev != nullptr) {
+        const int ph = p.n_dev[b];
+        if (ph >= 0) return;
+        n_ring = -ph - 1;
+    }
     const int n_tot = n_ring + (p.has_token ? 1 : 0);
 
-    const UpdateSmem us = make_update_smem<K>(KIND, n_tot, R4);
+    const UpdateSmem us = make_update_smem<K>(KIND, p.n_dev != nullptr ? p.n_cap : n_tot, R4, kVT);
     float* sK = reinterpret_cast<float*>(smem + us.k_off);
     float* sG = reinterpret_cast<float*>(smem + us.g_off);
     float* sV = reinterpret_cast<float*>(smem + us.v_off);
@@ -282,13 +287,15 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const Params p) {
     }
 }
 
-template <int KIND, typename IO, int K>
+template <int KIND, typename IO, int K, int kVT>
 static int launch_update_t(Ctx* ctx, Params p, cudaStream_t stream) {
+    constexpr int kUpdThreads = kVT * kParts;
     const int V = ctx->cfg.dv;
     const int n_tot = p.n_before + (p.has_token ? 1 : 0);
     const int R4 = (p.R + 3) & ~3;
-    const UpdateSmem us = make_update_smem<K>(KIND, n_tot, R4);
-    auto kern = update_kernel<KIND, IO, K>;
+    if (p.n_dev != nullptr) p.n_cap = n_tot;        // per-sequence phases: n_before is the largest fill any sequence may have
+    const UpdateSmem us = make_update_smem<K>(KIND, n_tot, R4, kVT);
+    auto kern = update_kernel<KIND, IO, K, kVT>;
     if (us.total > 226u * 1024u) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      (int)us.total)) != cudaSuccess)
@@ -303,8 +310,10 @@ static int launch_update_t(Ctx* ctx, Params p, cudaStream_t stream) {
 
 template <int KIND, typename IO>
 static int launch_update_shape(Ctx* ctx, const Params& p, cudaStream_t stream) {
-    if (ctx->cfg.dk == 128) return launch_update_t<KIND, IO, 128>(ctx, p, stream);
-    if (ctx->cfg.dk == 64) return launch_update_t<KIND, IO, 64>(ctx, p, stream);
+    if (ctx->cfg.dk == 128 && ctx->cfg.dv == 80) return launch_update_t<KIND, IO, 128, 80>(ctx, p, stream);
+    if (ctx->cfg.dv % 64 != 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (ctx->cfg.dk == 128) return launch_update_t<KIND, IO, 128, 64>(ctx, p, stream);
+    if (ctx->cfg.dk == 64) return launch_update_t<KIND, IO, 64, 64>(ctx, p, stream);
     return SKETCHSSM_UNSUPPORTED_SHAPE;
 }
 

@@ -48,7 +48,9 @@ def test_create_validates_configuration(lib):
     assert make(lib, batch=0)[0] == -1
     assert make(lib, io_dtype=2)[0] == -1
     assert make(lib, dk=96)[0] == -2
-    assert make(lib, dv=80)[0] == -2
+    assert make(lib, dv=96)[0] == -2
+    assert make(lib, dv=80)[0] == 0              # K = 128, V = 80: the second Mamba-2 head shape
+    assert make(lib, dk=64, dv=80)[0] == -2
     assert make(lib, rank=65)[0] == -2
     assert make(lib, rank=0)[0] == -1
     assert make(lib, buf_len=6)[0] == -2
