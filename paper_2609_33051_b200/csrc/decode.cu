@@ -103,10 +103,11 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     const int L = p.L, H = p.H, B = p.B;
     const int n_cap = p.n_before;                       // ring rows the stage has room for (per-sequence phases: the largest fill)
     const bool vlane = VL == 32 || lane < VL;           // this lane holds value elements
+    const bool per_seq = GEN && p.coef_per_seq;         // the head's own coefficient map travels with its sketch rows
     const int RP = (R + 7) & ~7;
 
-    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, p.coef_per_seq);
-    const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, p.coef_per_seq, sl.total);
+    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, per_seq);
+    const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, per_seq, sl.total);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * 2;
     float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
     float* sP = sX + K;                                                                               // dot products
@@ -126,7 +127,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     }
     // coefficient maps of the (at most two) head indices of this range, rows padded with zeros.  C is a constant of
     // the layer (never written by these kernels), so it may be staged before the predecessor in the stream is done.
-    if (!p.full_read && !p.coef_per_seq && item1 > item0) {
+    if (!p.full_read && !per_seq && item1 > item0) {
         const int nslots = h_last > h_first ? 2 : 1;
         for (int s = 0; s < nslots; ++s) {
             const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
@@ -158,13 +159,13 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_unit = (uint32_t)(V * sizeof(IO)); cp_mode = 1; break;
         case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_unit = KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u; cp_mode = 1; break;
         case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * 4; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * 4); cp_mode = 3; break;
-        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_unit = p.coef_per_seq ? (uint32_t)(K * 4) : 0u; cp_mode = 3; break;
+        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_unit = per_seq ? (uint32_t)(K * 4) : 0u; cp_mode = 3; break;
         default: break;
     }
     const uint32_t tokA = 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
     const uint32_t rowA = (uint32_t)((K + V) * sizeof(IO)) + (KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u);
     const uint32_t gateA = (uint32_t)((KIND == SKETCHSSM_KDA ? 1 : 2) * L * 4);
-    const uint32_t rowB = (uint32_t)(V * 4) + (p.coef_per_seq ? (uint32_t)(K * 4) : 0u);
+    const uint32_t rowB = (uint32_t)(V * 4) + (per_seq ? (uint32_t)(K * 4) : 0u);
     const int r_uni = p.full_read ? 0 : R;          // GEN = 0: the rank of every head
     // GEN = 0: the size of this lane's copy and the two transaction totals are constants of the launch
     const uint32_t cp_fixed = cp_mode == 0 ? cp_unit : cp_mode == 1 ? cp_unit * (uint32_t)n_cap
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     if (item < item1) {
         const size_t bh0 = (size_t)b * H + h;
         n = fill_of(b);
-        if (n >= 0) {
+        if (!GEN || n >= 0) {
             issue_a(bh0, n);
             if (!early_u) issue_b(bh0, rk);
             scalar_gates(bh0, bt_next, dsc_next);
@@ -276,15 +277,17 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
             rk_next = rank_of(hn);
             n_next = fill_of(bn);
         }
-        const bool go_next = has_next && n_next >= 0;          // the next head takes a decode step in this call
+        const bool go_next = has_next && (!GEN || n_next >= 0);          // the next head takes a decode step in this call
         const size_t bh_next = (size_t)bn * H + hn;
         const float bt = bt_next, dsc = dsc_next;
         if (go_next) scalar_gates(bh_next, bt_next, dsc_next);
 
-        if (n < 0) {                 // this sequence takes the flush step in this call: nothing to do here
-            if (go_next) { issue_a(bh_next, n_next); issue_b(bh_next, rk_next); }
-            item = item_next; h = hn; b = bn; n = n_next; rk = rk_next;
-            continue;
+        if constexpr (GEN) {
+            if (n < 0) {             // this sequence takes the flush step in this call: nothing to do here
+                if (go_next) { issue_a(bh_next, n_next); issue_b(bh_next, rk_next); }
+                item = item_next; h = hn; b = bn; n = n_next; rk = rk_next;
+                continue;
+            }
         }
         const bool full = rk == 0;   // exact read of the whole state for this head
 
@@ -421,10 +424,10 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         if (go_next) issue_a(bh_next, n_next);
         if (!full) {
             // c = C x, eight coefficients per transposing reduction, handed to all lanes through the scratch
-            const float* sC = p.coef_per_seq ? reinterpret_cast<const float*>(sb + sl.c_off)
+            const float* sC = per_seq ? reinterpret_cast<const float*>(sb + sl.c_off)
                                              : reinterpret_cast<const float*>(smem + (size_t)(h - h_first) * ds.coef_slot_bytes);
             __syncwarp();
-            if (p.coef_per_seq) {        // the head's own map arrives with its sketch rows
+            if (per_seq) {        // the head's own map arrives with its sketch rows
                 if (__any_sync(0xffffffffu, !DEC_WAIT(barB, PARB))) {
                     if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
                     pendB = (int)PARB;
@@ -449,7 +452,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
             __syncwarp();
-            if (!p.coef_per_seq) {
+            if (!per_seq) {
                 if (__any_sync(0xffffffffu, !DEC_WAIT(barB, PARB))) {
                     if (lane == 0) record_fault(p.status, kFaultDecodeWait, (int)blockIdx.x);
                     pendB = (int)PARB;
@@ -518,7 +521,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 template <int KIND, typename IO, int K, int V>
 static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     const int io = (int)sizeof(IO);
-    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq);
+    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq);   // (the general instantiation runs whenever coef_per_seq is set)
     const uint32_t smem_budget = 227u * 1024u;
     if (ctx->sm_count == 0) {
         int dev = 0, sms = 0;
@@ -530,7 +533,7 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
     // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
-    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr;
+    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq;
     const bool fixed16 = p.R == 16 && !gen;     // the unrolled rank-16 instantiation needs one rank for all heads
     auto kern = gen ? decode_kernel<KIND, IO, K, V, 0, 1> : fixed16 ? decode_kernel<KIND, IO, K, V, 16, 0> : decode_kernel<KIND, IO, K, V, 0, 0>;
     // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does

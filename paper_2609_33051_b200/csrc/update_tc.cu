@@ -394,6 +394,8 @@ __global__ void __launch_bounds__(kTcThreads) update_tc_mamba2_kernel(const Para
 int launch_update_tc(Ctx* ctx, const Params& p_in, cudaStream_t stream) {
     const sketchssm_config& c = ctx->cfg;
     if (c.kind != SKETCHSSM_MAMBA2 || c.io_dtype != SKETCHSSM_BF16 || c.dk != kK) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (c.dv != 64 && c.dv != 128) return SKETCHSSM_UNSUPPORTED_SHAPE;       // a tile is 128 value columns: two heads of 64 or one of 128
+    if (p_in.n_dev != nullptr) return SKETCHSSM_UNSUPPORTED_SHAPE;            // per-sequence phases: CUDA-core kernel
     const int NH = 128 / c.dv;
     if (c.batch % NH != 0) return SKETCHSSM_UNSUPPORTED_SHAPE;
     const int NP = (c.rank + NH + 15) & ~15;
