@@ -225,9 +225,12 @@ class Stack:
     """`logical` layers of one workload on one GPU, mapped round-robin onto `n_phys` physical layer slots, with one
     window of device-resident inputs per slot."""
 
-    def __init__(self, w: synth.Workload, n_phys: int, logical: int, device: int):
+    def __init__(self, w: synth.Workload, n_phys: int, logical: int, device: int, coef=None, sketch="f32"):
+        """coef: None (fixed offline map) or "pivot" / "ridge" (state-dependent map rebuilt by every flush);
+        sketch: storage type of U and C."""
         from paper_2609_33051_b200.binding import SketchSSM
         self.w, self.n_phys, self.logical, self.device = w, n_phys, logical, device
+        self.coef, self.sketch = coef, sketch
         dev = torch.device("cuda", device)
         Om, C = fitted_basis(w)
         wi = input_workload(w)
@@ -247,11 +250,13 @@ class Stack:
         gen = torch.Generator(device=dev)
         Om_t, C_t = torch.from_numpy(Om), torch.from_numpy(C)
         for li in range(n_phys):
-            m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out="f32", device=device)
+            m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out="f32", device=device,
+                          coef_per_seq=coef is not None, coef_pivots=4 if coef == "pivot" else 0, sketch=sketch)
             gen.manual_seed(w.seed * 1000 + li)
             m.state.normal_(0.0, w.state_std, generator=gen)          # S_init ~ N(0, 0.02^2), drawn on the device
             m.omega.copy_(Om_t)
-            m.coef.copy_(C_t)
+            if coef is None:
+                m.coef.copy_(C_t)
             m.state_update(0)
             self.layers.append(m)
             # every slot gets its own copy of the window so that no input is served from L2 across layers
@@ -367,9 +372,10 @@ class Stack:
         return h2d, d2h
 
 
-def make_stack(w: synth.Workload, budget_gb: float, logical: int, device: int) -> Stack:
-    n_phys = physical_layers(layer_bytes(w), int(budget_gb * 1e9), logical)
-    return Stack(w, n_phys, logical, device)
+def make_stack(w: synth.Workload, budget_gb: float, logical: int, device: int, coef=None, sketch="f32") -> Stack:
+    per = layer_bytes(w) + (w.batch * w.heads * w.rank * w.dk * 4 if coef else 0)
+    n_phys = physical_layers(per, int(budget_gb * 1e9), logical)
+    return Stack(w, n_phys, logical, device, coef=coef, sketch=sketch)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -442,13 +448,14 @@ def kernel_figures(w, stack, timer, ms_window, reps, peak):
     and the bandwidth fractions.  `ms_window` is the time of one window over all logical layers."""
     L, B, H = w.buf_len, w.batch, w.heads
     n_log = stack.logical
+    tkw = dict(sketch_bytes=2 if stack.sketch == "bf16" else 4, coef_per_seq=stack.coef is not None)
     ms_d, _, _ = timer.region(stack.run_decode_only, reps, 1)
     us_dec_b2b = 1e3 * ms_d / ((L - 1) * n_log)
     ms_u, _, _ = timer.region(stack.run_update_only, reps, 1)
     us_upd = 1e3 * ms_u / n_log
     stack.run_window("sketch", None)     # leave every layer at the start of a window again
-    by_d = sum(traffic.decode_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io) for t in range(L - 1)) / (L - 1)
-    by_u = traffic.update_bytes(w.kind, B, H, w.dk, w.dv, w.rank, L - 1, w.io)
+    by_d = sum(traffic.decode_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io, **tkw) for t in range(L - 1)) / (L - 1)
+    by_u = traffic.update_bytes(w.kind, B, H, w.dk, w.dv, w.rank, L - 1, w.io, **tkw)
     # what a decode launch costs inside the window: the window minus the flush, over its L-1 decode launches
     us_dec_win = max((1e3 * ms_window / n_log - us_upd) / (L - 1), 1e-3)
     gbs = lambda by, us: by / (us * 1e-6) / 1e9
@@ -465,9 +472,9 @@ def kernel_figures(w, stack, timer, ms_window, reps, peak):
     }
 
 
-def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25):
+def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25, coef=None, sketch="f32"):
     """One sweep record: the sketch window, the full-read window, per-kernel figures, byte accounting, clocks."""
-    stack = make_stack(w, budget_gb, logical, device)
+    stack = make_stack(w, budget_gb, logical, device, coef=coef, sketch=sketch)
     try:
         L, B, H = w.buf_len, w.batch, w.heads
         tokens = B * L * logical
@@ -485,11 +492,22 @@ def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25):
         for m in stack.layers:
             m.check_status()
         mean_n = (L - 2) / 2.0
-        dec_b = traffic.decode_bytes(w.kind, 1, 1, w.dk, w.dv, w.rank, 0, w.io) - w.rank * w.dk * 4
+        tkw = dict(sketch_bytes=2 if sketch == "bf16" else 4, coef_per_seq=coef is not None)
+        dec_b = traffic.decode_bytes(w.kind, 1, 1, w.dk, w.dv, w.rank, 0, w.io, **tkw)
+        if coef is None:
+            dec_b -= w.rank * w.dk * tkw["sketch_bytes"]          # the shared map is read once per launch, not per head
+        from paper_2609_33051_b200.binding import NO_SKETCH
+        ms_u0, _, _ = timer.region(lambda: stack.run_update_only(NO_SKETCH), max(2, steps // 2), 1)
+        stack.run_window("sketch", None)
         full_b = traffic.decode_bytes(w.kind, 1, 1, w.dk, w.dv, w.rank, 0, w.io, full_read=True)
         slot = traffic.slot_bytes(w.kind, w.dk, w.dv, w.io)
         return {
             "workload": f"{w.name}: {w.kind} B{B} H{H} K{w.dk} V{w.dv} r{w.rank} L{L}", "logical_layers": logical,
+            "coefficient_map": {None: "fixed offline map [H][r][K]", "pivot": "state-dependent, P = 4 approximation, lambda 0.1, "
+                                "rebuilt by every flush [B][H][r][K]", "ridge": "state-dependent, exact ridge solve, lambda 0.1"}[coef],
+            "sketch_storage": sketch,
+            "flush_without_sketch_us": 1e3 * ms_u0 / logical,
+            "sketch_and_map_overhead_on_flush": figs["update"]["back_to_back_us"] / (1e3 * ms_u0 / logical) - 1.0,
             "n_phys": stack.n_phys, "device_bytes": stack.device_bytes(), "steps": steps,
             "value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_window_all_layers": ms,
             "decode_in_window_us": figs["decode"]["in_window_us"],
@@ -568,6 +586,8 @@ def main():
     ap.add_argument("--skip-full-read", action="store_true")
     ap.add_argument("--skip-graph", action="store_true")
     ap.add_argument("--tune", default="", help="comma list key=value passed to sketchssm_tune")
+    ap.add_argument("--coef", default="fixed", choices=["fixed", "pivot", "ridge"], help="coefficient map of the headline stack")
+    ap.add_argument("--sketch", default="f32", choices=["f32", "bf16"], help="storage type of U and C of the headline stack")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -630,7 +650,7 @@ def main():
     timer = Timer(dist, local_rank)
     peak, peak_kind = measured_peaks()
 
-    stack = make_stack(w, args.budget_gb, logical, local_rank)
+    stack = make_stack(w, args.budget_gb, logical, local_rank, coef=None if args.coef == "fixed" else args.coef, sketch=args.sketch)
     for kv in filter(None, args.tune.split(",")):
         k, v = kv.split("=")
         for m in stack.layers:
@@ -766,6 +786,14 @@ def main():
                         continue
                     sweep.append(measure_point(ww, args.sweep_budget_gb, LOGICAL_LAYERS, local_rank, timer, peak))
 
+    # ---- the headline workload in the paper's own configuration of the method: state-dependent coefficient map (P = 4),
+    # and bfloat16 storage of the sketch; and the KDA layer with the tensor-core flush ----
+    variants = None
+    if not args.no_sweep and world == 1:
+        variants = [measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, coef="pivot"),
+                    measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, sketch="bf16"),
+                    measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, coef="pivot")]
+
     # ---- CPU oracle on a bounded sample (rank 0, N = 1) ----
     cpu = None
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
@@ -782,7 +810,7 @@ def main():
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step[0] * args.steps, "roofline": roofline,
                 "kernels": kern, "ms_per_step_with_launch_events": ms_step_instrumented, "full_read_baseline": full,
                 "graph_replay": graph, "sustained": sustained, "cpu_baseline": cpu, "per_gpu_heads": B * H,
-                "sweep": sweep}
+                "sweep": sweep, "variants": variants}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

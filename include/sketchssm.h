@@ -37,7 +37,8 @@
  * Layouts (B = batch, H = heads, K = dk, V = dv, r = rank, L = buf_len; "io" is
  * float or bfloat16 as configured):
  *   state  S      [B][H][K][V]  fp32
- *   sketch U      [B][H][r][V]  fp32   (U^T of the paper's V x r matrix: row g is S^T omega_g)
+ *   sketch U      [B][H][r][V]  fp32   (U^T of the paper's V x r matrix: row g is S^T omega_g); bfloat16 with
+ *                                      config.sketch_dtype = SKETCHSSM_BF16 (then C is bfloat16 too)
  *   omega  Omega  [H][K][r]     fp32   (fixed offline, shared by the batch)
  *   coef   C      [H][r][K]     fp32   (fixed offline coefficient map, Eq. 10), or with config.coef_per_seq
  *                 [B][H][r][K]  fp32   (state-dependent map, written by sketchssm_state_update)
@@ -96,6 +97,11 @@ typedef struct sketchssm_config {
     int32_t coef_pivots;    /* coef_per_seq = 1: pivot count P of the low-rank-plus-diagonal state metric
                                (Eq. 30-37; the paper uses 4; 1..8), or 0 for the exact ridge solve (Eq. 29) */
     float ridge_lambda;     /* coef_per_seq = 1: ridge lambda > 0 (the paper uses 0.1) */
+    int32_t sketch_dtype;   /* sketchssm_dtype of the stored sketch U and coefficient map C: SKETCHSSM_F32 (default) or
+                               SKETCHSSM_BF16, the storage the paper's traffic model assumes (T_G = 2 G (V + K) bytes per
+                               non-flush read, Appendix D).  U is rounded to bfloat16 once, when the flush stores it; all
+                               arithmetic stays fp32.  With bfloat16 storage C is the fixed offline map (coef_per_seq = 0),
+                               handed over as bfloat16 [H][r][K], and only the default one-kernel decode is available. */
 } sketchssm_config;
 
 typedef struct sketchssm_sizes {

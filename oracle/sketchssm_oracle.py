@@ -92,6 +92,15 @@ def sketch_of(S, Omega):
     return np.einsum("...kv,...kg->...vg", _f64(S), _f64(Omega))
 
 
+def round_bf16(x):
+    """Round to the nearest bfloat16 (ties to even), returned as float64: the storage precision the paper uses for the
+    sketch, the coefficient map and the erase vectors (Appendix D, Appendix F setup).  The value is first rounded to
+    float32, the precision the sketch is formed in before it is stored."""
+    bits = np.ascontiguousarray(_f64(x).astype(np.float32)).view(np.uint32).astype(np.uint64)
+    rounded = ((bits + 0x7FFF + ((bits >> 16) & 1)) >> 16) << 16
+    return rounded.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
 # ----------------------------------------------------------------------------
 # Read decomposition (Section 3.1, Eq. 4)
 # ----------------------------------------------------------------------------

@@ -34,7 +34,7 @@ OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("kind", "batch", "heads", "dk", "dv", "rank", "buf_len", "io_dtype", "out_dtype", "device",
-                 "coef_per_seq", "coef_pivots")] + [("ridge_lambda", ctypes.c_float)]
+                 "coef_per_seq", "coef_pivots")] + [("ridge_lambda", ctypes.c_float), ("sketch_dtype", ctypes.c_int32)]
 
 
 class Sizes(ctypes.Structure):
@@ -112,14 +112,15 @@ class SketchSSM:
 
     def __init__(self, kind: str, batch: int, heads: int, dk: int, dv: int, rank: int, buf_len: int,
                  io: str = "bf16", out: str = "f32", device: int = 0, allocate: bool = True,
-                 coef_per_seq: bool = False, coef_pivots: int = 4, ridge_lambda: float = 0.1):
+                 coef_per_seq: bool = False, coef_pivots: int = 4, ridge_lambda: float = 0.1, sketch: str = "f32"):
         self.lib = load_library()
         self.kind, self.io, self.out = kind, io, out
         self.B, self.H, self.K, self.V, self.R, self.L = batch, heads, dk, dv, rank, buf_len
         self.device = torch.device("cuda", device)
         self.coef_per_seq = bool(coef_per_seq)
         self.cfg = Config(KIND[kind], batch, heads, dk, dv, rank, buf_len, DTYPE[io], DTYPE[out], device,
-                          int(self.coef_per_seq), coef_pivots, ridge_lambda)
+                          int(self.coef_per_seq), coef_pivots, ridge_lambda, DTYPE[sketch])
+        self.sketch_dtype = sketch
         self._ctx = ctypes.c_void_p()
         self._check("sketchssm_create", self.lib.sketchssm_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.sizes = Sizes()
@@ -133,17 +134,18 @@ class SketchSSM:
     def allocate(self):
         d = self.device
         self.state = torch.zeros(self.B, self.H, self.K, self.V, dtype=torch.float32, device=d)
-        self.sketch = torch.zeros(self.B, self.H, self.R, self.V, dtype=torch.float32, device=d)
+        self.sketch = torch.zeros(self.B, self.H, self.R, self.V, dtype=TORCH_DTYPE[self.sketch_dtype], device=d)
         self.ring = torch.zeros(self.sizes.ring_bytes, dtype=torch.uint8, device=d)
         self.omega = torch.zeros(self.H, self.K, self.R, dtype=torch.float32, device=d)
-        self.coef = torch.zeros(*((self.B,) if self.coef_per_seq else ()), self.H, self.R, self.K, dtype=torch.float32, device=d)
+        self.coef = torch.zeros(*((self.B,) if self.coef_per_seq else ()), self.H, self.R, self.K,
+                                dtype=TORCH_DTYPE[self.sketch_dtype], device=d)
         self.status = torch.zeros(self.sizes.status_bytes // 4, dtype=torch.int32, device=d)
         self.work = torch.zeros(self.sizes.work_bytes // 4, dtype=torch.float32, device=d)
         self.bind()
 
     def bind(self):
         assert self.state.numel() * 4 == self.sizes.state_bytes
-        assert self.sketch.numel() * 4 == self.sizes.sketch_bytes
+        assert self.sketch.numel() * self.sketch.element_size() == self.sizes.sketch_bytes
         assert self.ring.numel() == self.sizes.ring_bytes
         b = Buffers(self.state.data_ptr(), self.sketch.data_ptr(), self.ring.data_ptr(),
                     self.omega.data_ptr(), self.coef.data_ptr(), self.status.data_ptr(), self.work.data_ptr(),

@@ -63,6 +63,7 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.coef_per_seq = ctx->cfg.coef_per_seq;
     p.pivots = ctx->cfg.coef_pivots;
     p.ridge_lambda = ctx->cfg.ridge_lambda;
+    p.sketch_bf16 = ctx->cfg.sketch_dtype == SKETCHSSM_BF16;
     return p;
 }
 
@@ -140,7 +141,8 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
     if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
     // the two-kernel decode stages one map per head index, knows one rank and the value widths 64 and 128
-    if ((p.coef_per_seq && !full_read) || p.head_rank != nullptr || ctx->cfg.dv == 80) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if ((p.coef_per_seq && !full_read) || p.head_rank != nullptr || ctx->cfg.dv == 80 || (p.sketch_bf16 && !full_read))
+        return SKETCHSSM_UNSUPPORTED_SHAPE;
     switch (ctx->cfg.kind) {
         case SKETCHSSM_MAMBA2:
             return bf ? launch_decode_split_mamba2_bf16(ctx, p, cs) : launch_decode_split_mamba2_f32(ctx, p, cs);
@@ -169,6 +171,8 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     if (cfg->buf_len < 4 || cfg->buf_len > kMaxBufLen || (cfg->buf_len & 3)) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if ((size_t)cfg->batch * cfg->heads > (size_t)1 << 24) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if (cfg->coef_per_seq != 0 && cfg->coef_per_seq != 1) return SKETCHSSM_INVALID_ARG;
+    if (cfg->sketch_dtype != SKETCHSSM_F32 && cfg->sketch_dtype != SKETCHSSM_BF16) return SKETCHSSM_INVALID_ARG;
+    if (cfg->sketch_dtype == SKETCHSSM_BF16 && cfg->coef_per_seq) return SKETCHSSM_UNSUPPORTED_SHAPE;   // bfloat16 storage: fixed offline map
     if (cfg->coef_per_seq) {
         if (!(cfg->ridge_lambda > 0.f) || cfg->coef_pivots < 0) return SKETCHSSM_INVALID_ARG;
         if (cfg->coef_pivots > 8) return SKETCHSSM_UNSUPPORTED_SHAPE;
@@ -205,10 +209,11 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
     const sketchssm_config& c = ctx->cfg;
     const size_t bh = (size_t)c.batch * c.heads;
     out->state_bytes = bh * c.dk * c.dv * 4;
-    out->sketch_bytes = bh * c.rank * c.dv * 4;
+    const size_t su = c.sketch_dtype == SKETCHSSM_BF16 ? 2 : 4;
+    out->sketch_bytes = bh * c.rank * c.dv * su;
     out->ring_bytes = bh * ctx->ring.head_bytes;
     out->omega_bytes = (size_t)c.heads * c.dk * c.rank * 4;
-    out->coef_bytes = (c.coef_per_seq ? bh : (size_t)c.heads) * c.rank * c.dk * 4;
+    out->coef_bytes = (c.coef_per_seq ? bh : (size_t)c.heads) * c.rank * c.dk * su;
     out->status_bytes = (((size_t)(kStatusInts + 4 + c.heads) * sizeof(int32_t)) + 15) & ~(size_t)15;   // status word + tile scheduler counters
     out->work_bytes = bh * (size_t)(c.dk + c.buf_len) * 4;
     out->ring_head_bytes = ctx->ring.head_bytes;
@@ -327,7 +332,8 @@ int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q
     int rc = decode_params(ctx, 0, n_before, q, k, v, beta, decay, out, flags, &p);
     if (rc != SKETCHSSM_OK) return rc;
     // runs the two-kernel decode (one map per head index, one rank, value widths 64 and 128)
-    if (ctx->cfg.coef_per_seq || ctx->bufs.head_rank != nullptr || ctx->cfg.dv == 80) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    if (ctx->cfg.coef_per_seq || ctx->bufs.head_rank != nullptr || ctx->cfg.dv == 80 || ctx->cfg.sketch_dtype == SKETCHSSM_BF16)
+        return SKETCHSSM_UNSUPPORTED_SHAPE;
     // the size limit of the library's static array is checked (on the host, before any CUDA call) by the launcher
     const sketchssm_config& c = ctx->cfg;
     if ((size_t)c.batch * c.heads * (size_t)(c.dk + c.buf_len) * sizeof(float) > (size_t)SKETCHSSM_STATIC_WORK_BYTES)

@@ -42,10 +42,10 @@ struct StageLayout {
 };
 
 __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K, int V, int R, int L, int n,
-                                                         int full_read, int coef_per_seq) {
+                                                         int full_read, int coef_per_seq, int sketch_bytes = 4) {
     StageLayout s;
     uint32_t off = 0;
-    s.u_off = off; s.u_bytes = full_read ? 0u : (uint32_t)(R * V * 4); off += s.u_bytes;
+    s.u_off = off; s.u_bytes = full_read ? 0u : (uint32_t)(R * V * sketch_bytes); off += (s.u_bytes + 15u) & ~15u;
     // rows padded to the reduction width are read (their sums are never used), so they get room but are not copied
     s.c_off = off; s.c_bytes = (!full_read && coef_per_seq) ? (uint32_t)(R * K * 4) : 0u;
     off += (!full_read && coef_per_seq) ? (uint32_t)(((R + 7) & ~7) * K * 4) : 0u;
@@ -104,9 +104,11 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     const int n_cap = p.n_before;                       // ring rows the stage has room for (per-sequence phases: the largest fill)
     const bool vlane = VL == 32 || lane < VL;           // this lane holds value elements
     const bool per_seq = GEN && p.coef_per_seq;         // the head's own coefficient map travels with its sketch rows
+    const bool u_bf16 = GEN && p.sketch_bf16;           // sketch rows (and the fixed coefficient map) stored as bfloat16
+    const int su = u_bf16 ? 2 : 4;
     const int RP = (R + 7) & ~7;
 
-    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, per_seq);
+    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, per_seq, su);
     const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, per_seq, sl.total);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * 2;
     float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
@@ -130,10 +132,23 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     if (!p.full_read && !per_seq && item1 > item0) {
         const int nslots = h_last > h_first ? 2 : 1;
         for (int s = 0; s < nslots; ++s) {
-            const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
             float4* dst = reinterpret_cast<float4*>(smem + (size_t)s * ds.coef_slot_bytes);
-            for (int i = threadIdx.x; i < RP * K / 4; i += blockDim.x)
-                dst[i] = i < R * K / 4 ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (u_bf16) {        // the map is stored as bfloat16: widened while it is staged
+                const uint2* src = reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(p.coef) + (size_t)(h_first + s) * R * K);
+                for (int i = threadIdx.x; i < RP * K / 4; i += blockDim.x) {
+                    float4 c4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (i < R * K / 4) {
+                        const uint2 t = src[i];
+                        c4 = make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
+                                         __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+                    }
+                    dst[i] = c4;
+                }
+            } else {
+                const float4* src = reinterpret_cast<const float4*>(p.coef + (size_t)(h_first + s) * R * K);
+                for (int i = threadIdx.x; i < RP * K / 4; i += blockDim.x)
+                    dst[i] = i < R * K / 4 ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
     }
     __syncthreads();
@@ -158,14 +173,14 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         case 5: cp_base = p.ring + p.rl.beta_off; cp_stride = p.rl.head_bytes; cp_dst = sl.gate_off; cp_unit = (uint32_t)((KIND == SKETCHSSM_KDA ? 1 : 2) * L * 4); cp_mode = 2; break;
         case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_unit = (uint32_t)(V * sizeof(IO)); cp_mode = 1; break;
         case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_unit = KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u; cp_mode = 1; break;
-        case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * 4; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * 4); cp_mode = 3; break;
+        case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * su; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * su); cp_mode = 3; break;
         case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_unit = per_seq ? (uint32_t)(K * 4) : 0u; cp_mode = 3; break;
         default: break;
     }
     const uint32_t tokA = 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
     const uint32_t rowA = (uint32_t)((K + V) * sizeof(IO)) + (KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u);
     const uint32_t gateA = (uint32_t)((KIND == SKETCHSSM_KDA ? 1 : 2) * L * 4);
-    const uint32_t rowB = (uint32_t)(V * 4) + (per_seq ? (uint32_t)(K * 4) : 0u);
+    const uint32_t rowB = (uint32_t)(V * su) + (per_seq ? (uint32_t)(K * 4) : 0u);
     const int r_uni = p.full_read ? 0 : R;          // GEN = 0: the rank of every head
     // GEN = 0: the size of this lane's copy and the two transaction totals are constants of the launch
     const uint32_t cp_fixed = cp_mode == 0 ? cp_unit : cp_mode == 1 ? cp_unit * (uint32_t)n_cap
@@ -467,7 +482,8 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 for (int g = 0; g < (RT ? RT : rk); ++g) {
                     const float cg = sX[g];
                     float uu[EV];
-                    load_io<EV>(sU, g * V + lane * EV, uu);
+                    if (u_bf16) load_io<EV>(reinterpret_cast<const __nv_bfloat16*>(sU), g * V + lane * EV, uu);
+                    else load_io<EV>(sU, g * V + lane * EV, uu);
 #pragma unroll
                     for (int e = 0; e < EV; ++e) o[e] = fmaf(cg, uu[e], o[e]);
                 }
@@ -521,7 +537,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 template <int KIND, typename IO, int K, int V>
 static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     const int io = (int)sizeof(IO);
-    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq);   // (the general instantiation runs whenever coef_per_seq is set)
+    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq, p.sketch_bf16 ? 2 : 4);   // (the general instantiation runs whenever coef_per_seq or sketch_bf16 is set)
     const uint32_t smem_budget = 227u * 1024u;
     if (ctx->sm_count == 0) {
         int dev = 0, sms = 0;
@@ -533,7 +549,7 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
     // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
-    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq;
+    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq || p.sketch_bf16;
     const bool fixed16 = p.R == 16 && !gen;     // the unrolled rank-16 instantiation needs one rank for all heads
     auto kern = gen ? decode_kernel<KIND, IO, K, V, 0, 1> : fixed16 ? decode_kernel<KIND, IO, K, V, 16, 0> : decode_kernel<KIND, IO, K, V, 0, 0>;
     // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does

@@ -80,6 +80,7 @@ struct Params {
     const int* n_dev;     // optional [B]: per-sequence phase of a mixed step (>= 0: decode step at that ring fill; < 0: flush with
                           // -v - 1 buffered tokens); nullptr: n_before for every sequence
     int n_cap;            // update (CUDA cores) with per-sequence phases: ring rows the shared-memory layout has room for
+    int sketch_bf16;      // U (and the fixed C) are stored as bfloat16
     int tok_base;         // update (GDN tensor-core kernel): first ring row of this pass when a flush is replayed in blocks of 16 tokens
 };
 
@@ -183,6 +184,12 @@ __device__ __forceinline__ void record_fault(int* status, int code, int where) {
     if (status != nullptr) {
         if (atomicCAS(status, 0, code) == 0) status[1] = where;
     }
+}
+
+// One element of the sketch, in the configured storage type (index in elements).
+__device__ __forceinline__ void store_sketch(const Params& p, size_t idx, float u) {
+    if (p.sketch_bf16) reinterpret_cast<__nv_bfloat16*>(p.sketch)[idx] = __float2bfloat16_rn(u);
+    else p.sketch[idx] = u;
 }
 
 __device__ __forceinline__ float warp_sum(float x) {

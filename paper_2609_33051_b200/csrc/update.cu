@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(kVT * kParts) update_kernel(const Params p) {
 
     // ---- sketch rows U[g, j] = <S_new[:, j], omega_g>, 4 ranks at a time ----
     if (p.write_sketch) {
-        float* Ug = p.sketch + (size_t)bh * R * V + j;
+        const size_t ug = (size_t)bh * R * V + j;
         for (int g0 = 0; g0 < R4; g0 += 4) {
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
             const float* op = sOm + (size_t)part * (RP * R4 + 4) + g0;
@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(kVT * kParts) update_kernel(const Params p) {
             a3 += __shfl_xor_sync(0xffffffffu, a3, 8);  a3 += __shfl_xor_sync(0xffffffffu, a3, 16);
             // part p stores rank g0 + p
             const float mine = part == 0 ? a0 : part == 1 ? a1 : part == 2 ? a2 : a3;
-            if (g0 + part < R) Ug[(size_t)(g0 + part) * V] = mine;
+            if (g0 + part < R) store_sketch(p, ug + (size_t)(g0 + part) * V, mine);
         }
     }
 }

@@ -475,7 +475,7 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
                     const int g = g0 + e;
-                    if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u[e];
+                    if (g < R && p.write_sketch) store_sketch(p, (bh * R + g) * (size_t)V + j, u[e]);
                     if (g == QA + 8 * b + my_head && p.out != nullptr) {
                         if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u[e]);
                         else reinterpret_cast<float*>(p.out)[bh * V + j] = u[e];

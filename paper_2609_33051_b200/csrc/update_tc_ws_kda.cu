@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     for (int e = 0; e < 16; ++e) {
                         const int g = g0 + e;
                         const float u = u0[e] + cr[e];
-                        if (g < R && p.write_sketch) p.sketch[(bh * R + g) * (size_t)V + j] = u;
+                        if (g < R && p.write_sketch) store_sketch(p, (bh * R + g) * (size_t)V + j, u);
                         if (g == QA && p.out != nullptr) {
                             if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
                             else reinterpret_cast<float*>(p.out)[bh * V + j] = u;

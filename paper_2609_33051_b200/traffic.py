@@ -21,25 +21,35 @@ def token_bytes(kind: str, K: int, V: int, io: str) -> int:
     return K * _io(io) + slot_bytes(kind, K, V, io)
 
 
-def decode_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, full_read=False, append=True) -> int:
-    """decode_step / full_read_decode launch at ring fill n_before."""
-    per_head = (K * V * 4 if full_read else r * V * 4)            # S or U
+def decode_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, full_read=False, append=True,
+                 sketch_bytes=4, coef_per_seq=False) -> int:
+    """decode_step / full_read_decode launch at ring fill n_before.  sketch_bytes: storage of U and C (4 or 2);
+    coef_per_seq: every head reads its own coefficient map instead of the one shared by the batch."""
+    per_head = (K * V * 4 if full_read else r * V * sketch_bytes)   # S or U
     per_head += n_before * slot_bytes(kind, K, V, io)               # ring read
     per_head += token_bytes(kind, K, V, io)                         # q, k, v, gates of the token
     per_head += slot_bytes(kind, K, V, io) if append else 0         # append write
     per_head += V * out_bytes                                       # o
-    shared = 0 if full_read else H * r * K * 4                      # C
+    shared = 0
+    if not full_read:
+        if coef_per_seq:
+            per_head += r * K * 4                                   # the head's own C (fp32)
+        else:
+            shared = H * r * K * sketch_bytes                       # C, once per launch
     return B * H * per_head + shared
 
 
 def update_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, has_token=True, sketch=True,
-                 with_output=True) -> int:
-    """state_update launch replaying n_before buffered tokens (+ the current one)."""
+                 with_output=True, sketch_bytes=4, coef_per_seq=False) -> int:
+    """state_update launch replaying n_before buffered tokens (+ the current one).  With coef_per_seq the write of the
+    per-head coefficient map is counted (what the method must move); the second read of the state that this
+    implementation's separate coefficient kernel performs is not algorithmic and shows up as a lower fraction."""
     n_tot = n_before + (1 if has_token else 0)
     per_head = K * V * 4 * (2 if n_tot > 0 else 1)                  # S read (+ write)
     per_head += n_before * slot_bytes(kind, K, V, io)
     per_head += slot_bytes(kind, K, V, io) if has_token else 0
     per_head += (K * _io(io) + V * out_bytes) if with_output else 0  # q in, o out
-    per_head += r * V * 4 if sketch else 0                          # U write
+    per_head += r * V * sketch_bytes if sketch else 0               # U write
+    per_head += r * K * 4 if (sketch and coef_per_seq) else 0       # C write
     shared = H * K * r * 4 if sketch else 0                         # Omega
     return B * H * per_head + shared

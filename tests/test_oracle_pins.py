@@ -614,3 +614,16 @@ def test_schedule_with_state_dependent_map_rebuilds_it_at_every_flush(kind):
             want = orc.decode_step(kind, orc.sketch_of(Sw, Om), Cw, ring, q)
             np.testing.assert_allclose(outs[t], want, atol=1e-10)
     np.testing.assert_allclose(C, np.stack([orc.pivot_coefficient_map(Sw[i], Om[i], 0.1, 2) for i in range(N)]), atol=1e-12)
+
+
+def test_round_bf16_is_round_to_nearest_even_on_the_top_16_bits():
+    """Pinned against hand-picked values: bfloat16 keeps 8 significand bits (spacing 2^-7 in [1, 2))."""
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -0.3, 0.0, 3.0e38])
+    want = np.array([1.0, 1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7, -0.30078125, 0.0, 226.0 / 128.0 * 2.0 ** 127])
+    got = orc.round_bf16(x)
+    np.testing.assert_allclose(got, want, rtol=1e-7)
+    # idempotent, and within half a spacing of the input
+    np.testing.assert_array_equal(orc.round_bf16(got), got)
+    rng = np.random.default_rng(21)
+    y = rng.standard_normal(1000)
+    assert np.all(np.abs(orc.round_bf16(y) - y) <= np.abs(y) * 2.0 ** -8)
