@@ -20,6 +20,7 @@
 // column k of C (coalesced across the CTA).  The kernel runs after the flush kernel of the same call and re-reads
 // S_new and U from memory: the map needs the complete sketch before it can contract the state with it.
 #include "internal.cuh"
+#include "lanegroup.cuh"
 
 namespace sketchssm {
 
@@ -29,8 +30,8 @@ constexpr int kCoefThreads = 128;
 constexpr int kMaxPivots = 8;
 
 struct CoefSmem {
-    uint32_t probe, y, ru, small, total;   // byte offsets
-    int pitch;                             // floats per probe row
+    uint32_t probe, y, ru, small, om, total;   // byte offsets
+    int pitch;                                 // floats per probe row
 };
 
 __host__ __device__ inline CoefSmem make_coef_smem(int K, int V, int G, int m) {
@@ -40,8 +41,9 @@ __host__ __device__ inline CoefSmem make_coef_smem(int K, int V, int G, int m) {
     s.probe = off; off += (uint32_t)(G * s.pitch * 4);        // the G sketch rows; the first m become the probe rows
     const int yf = K * (m + 1) > m * V ? K * (m + 1) : m * V;
     s.y = off; off += (uint32_t)(yf * 4);                     // Y[k][0..m) (pitch m + 1); before that, the m raw pivot rows
-    s.ru = off; off += (uint32_t)(G * (m + 1) * 4);           // RU[g][j] = <U_g, probe_j> (pitch m + 1)
-    s.small = off; off += (uint32_t)((4 * G + m * m + 2 * m + 64) * 4);
+    s.ru = off; off += (uint32_t)(G * (m + 1 > 8 ? m + 1 : 8) * 4);   // RU[g][j] = <U_g, probe_j> (pitch m + 1 for the exact form, else the padded pivot count)
+    s.small = off; off += (uint32_t)((4 * G + 2 * 8 * 8 + 64) * 4);
+    s.om = off; off += (uint32_t)(K * (G | 1) * 4);           // Omega of the head index, odd pitch (a thread reads its own row)
     s.total = (off + 15u) & ~15u;
     return s;
 }
@@ -58,8 +60,9 @@ __device__ __forceinline__ float block_sum(float x, float* scratch) {
 
 }  // namespace
 
-// EXACT = 0: pivot approximation with m = min(G, P) probe rows;  EXACT = 1: ridge form with m = G.
-template <int K, int V, int EXACT>
+// EXACT = 0: pivot approximation with m = min(G, P) <= PM probe rows (PM = 4 or 8: loops over pivots unroll and stay in
+// registers);  EXACT = 1: ridge form with m = G.
+template <int K, int V, int EXACT, int PM>
 __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -80,11 +83,12 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
     float* sY = reinterpret_cast<float*>(smem + sm.y);
     float* sRU = reinterpret_cast<float*>(smem + sm.ru);
     float* sSm = reinterpret_cast<float*>(smem + sm.small);
-    float* sUU = sSm;                  // [G] ||U_g||^2
-    float* sD = sSm + G;               // [G] d_g, then D_G
-    float* sT = sSm + 2 * G;           // [m][m] T_P^{-1} (pivot) -- the exact form keeps its Cholesky factor in sRU
-    float* sRed = sSm + 2 * G + m * m; // block reduction scratch
-    const int PT = sm.pitch, MP = m + 1;
+    float* sUU = sSm;                  // [G] ||U_g||^2, then d_g
+    float* sD = sSm + G;               // [G] 1 / D_G
+    float* sT = sSm + 2 * G;           // [PM][2 PM] T_P next to the identity, inverted in place (pivot) -- the exact form keeps its Cholesky factor in sRU
+    float* sRed = sSm + 2 * G + 2 * 8 * 8; // block reduction scratch
+    const int PT = sm.pitch, MP = m + 1;   // MP: pitch of Y (odd or small: the per-row accesses of a warp spread over the banks)
+    constexpr int RUP = PM;                // pitch of RU in the pivot form (16- or 32-byte rows, zero beyond m)
 
     const int RS = p.R;                // row strides of U, C and Omega follow the configured rank
     const float* Ug = p.sketch + bh * (size_t)RS * V;
@@ -142,12 +146,14 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
         }
         __syncthreads();
         // RU[g][j] = <U_g, Q_j>; the raw rows g < m were parked in the Y area
-        for (int i = tid; i < G * m; i += kCoefThreads) {
-            const int g = i / m, j = i - g * m;
-            const float* ur = g < m ? sY + g * V : sU + g * PT;
+        for (int i = tid; i < G * RUP; i += kCoefThreads) {
+            const int g = i / RUP, j = i - g * RUP;
             float a = 0.f;
-            for (int v = 0; v < V; ++v) a = fmaf(ur[v], sU[j * PT + v], a);
-            sRU[g * MP + j] = a;
+            if (j < m) {
+                const float* ur = g < m ? sY + g * V : sU + g * PT;
+                for (int v = 0; v < V; ++v) a = fmaf(ur[v], sU[j * PT + v], a);
+            }
+            sRU[g * RUP + j] = a;
         }
         __syncthreads();
     } else {
@@ -165,93 +171,159 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
 
     // ---- stream the state: Y[k][j] = <S[k,:], probe_j>, ||S||_F^2 ----
     float ss = 0.f;
-    for (int k = tid; k < K; k += kCoefThreads) {
-        const float* row = Sg + (size_t)k * V;
-        constexpr int JB = 8;                                     // probe rows per pass over the (cached) state row
-        for (int j0 = 0; j0 < m; j0 += JB) {
-            float acc[JB];
+    if constexpr (!EXACT) {
+        // A warp reads whole rows (lanes along the value index: every fetched sector is used once); the 32 partial dot
+        // products of a block of rows (32 / PM rows x PM probes) are reduced over the lanes by one transposing butterfly.
+        constexpr int EV = V % 32 == 0 ? V / 32 : 4;
+        constexpr int VL = V / EV;
+        constexpr int RB = 32 / PM;                 // rows per block
+        const bool vlane = VL == 32 || lane < VL;
+        float qf[PM][EV];
 #pragma unroll
-            for (int j = 0; j < JB; ++j) acc[j] = 0.f;
-#pragma unroll 4
-            for (int c = 0; c < V / 4; ++c) {
-                const float4 s4 = *reinterpret_cast<const float4*>(row + 4 * c);
-                if (j0 == 0) ss = fmaf(s4.x, s4.x, fmaf(s4.y, s4.y, fmaf(s4.z, s4.z, fmaf(s4.w, s4.w, ss))));
+        for (int j = 0; j < PM; ++j)
 #pragma unroll
-                for (int j = 0; j < JB; ++j) {
-                    if (j0 + j < m) {
-                        const float4 q4 = *reinterpret_cast<const float4*>(sU + (j0 + j) * PT + 4 * c);
-                        acc[j] = fmaf(s4.x, q4.x, fmaf(s4.y, q4.y, fmaf(s4.z, q4.z, fmaf(s4.w, q4.w, acc[j]))));
-                    }
+            for (int e = 0; e < EV; ++e) qf[j][e] = (j < m && vlane) ? sU[j * PT + lane * EV + e] : 0.f;
+        constexpr int RPW = K / (kCoefThreads / 32);        // rows per warp
+        for (int k0 = warp * RPW; k0 < (warp + 1) * RPW; k0 += RB) {
+            float part[32];
+#pragma unroll
+            for (int r = 0; r < RB; ++r) {
+                float sv[EV];
+#pragma unroll
+                for (int e = 0; e < EV; ++e) sv[e] = 0.f;
+                if (vlane) load_io<EV>(Sg, (k0 + r) * V + lane * EV, sv);
+#pragma unroll
+                for (int e = 0; e < EV; ++e) ss = fmaf(sv[e], sv[e], ss);
+#pragma unroll
+                for (int j = 0; j < PM; ++j) {
+                    float a = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EV; ++e) a = fmaf(sv[e], qf[j][e], a);
+                    part[r * PM + j] = a;
                 }
             }
+            group_reduce_transpose<32, 32>(part, lane);
+            const int r = lane / PM, j = lane - r * PM;      // lane l holds the complete sum of entry l
+            if (j < m) sY[(k0 + r) * MP + j] = part[0];
+        }
+        // Omega of this head index into shared memory (coalesced), for the last step
+        {
+            float* sOm = reinterpret_cast<float*>(smem + sm.om);
+            const int OP = p.R | 1;
+            for (int i = tid; i < K * RS; i += kCoefThreads) {
+                const int kk = i / RS, g = i - kk * RS;
+                if (g < G) sOm[kk * OP + g] = Om[i];
+            }
+        }
+    } else {
+        for (int k = tid; k < K; k += kCoefThreads) {
+            const float* row = Sg + (size_t)k * V;
+            constexpr int JB = 8;                                     // probe rows per pass over the (cached) state row
+            for (int j0 = 0; j0 < m; j0 += JB) {
+                float acc[JB];
 #pragma unroll
-            for (int j = 0; j < JB; ++j)
-                if (j0 + j < m) sY[k * MP + j0 + j] = acc[j];
+                for (int j = 0; j < JB; ++j) acc[j] = 0.f;
+#pragma unroll 4
+                for (int c = 0; c < V / 4; ++c) {
+                    const float4 s4 = *reinterpret_cast<const float4*>(row + 4 * c);
+                    if (j0 == 0) ss = fmaf(s4.x, s4.x, fmaf(s4.y, s4.y, fmaf(s4.z, s4.z, fmaf(s4.w, s4.w, ss))));
+#pragma unroll
+                    for (int j = 0; j < JB; ++j) {
+                        if (j0 + j < m) {
+                            const float4 q4 = *reinterpret_cast<const float4*>(sU + (j0 + j) * PT + 4 * c);
+                            acc[j] = fmaf(s4.x, q4.x, fmaf(s4.y, q4.y, fmaf(s4.z, q4.z, fmaf(s4.w, q4.w, acc[j]))));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < JB; ++j)
+                    if (j0 + j < m) sY[k * MP + j0 + j] = acc[j];
+            }
         }
     }
     ss = block_sum(ss, sRed);
     const float mu = ss > 0.f ? ss / (float)K : 1.f;
     const float lam = p.ridge_lambda;
 
-    if (!EXACT) {
+    if constexpr (!EXACT) {
         const float inv_mu = 1.f / mu;
-        // d_g and D_G
+        // d_g and 1 / D_G
         for (int g = tid; g < G; g += kCoefThreads) {
             float r2 = 0.f;
-            for (int j = 0; j < m; ++j) r2 = fmaf(sRU[g * MP + j], sRU[g * MP + j], r2);
+#pragma unroll
+            for (int j = 0; j < PM; ++j) r2 = fmaf(sRU[g * RUP + j], sRU[g * RUP + j], r2);
             const float d = fmaxf((sUU[g] - r2) * inv_mu, 0.f);
-            sUU[g] = d;                 // d_g
-            sD[g] = d + lam;            // D_G
+            sUU[g] = d;
+            sD[g] = 1.f / (d + lam);
         }
         __syncthreads();
-        // T_P = I + L_G^T D_G^{-1} L_G = I + RU^T D_G^{-1} RU / mu, inverted by Gauss-Jordan (symmetric positive definite,
-        // eigenvalues >= 1: no pivoting needed); one thread, p <= 8
-        if (tid == 0) {
-            float T[kMaxPivots][kMaxPivots], Ti[kMaxPivots][kMaxPivots];
-            for (int a = 0; a < m; ++a)
-                for (int b = 0; b < m; ++b) {
-                    float t = 0.f;
-                    for (int g = 0; g < G; ++g) t = fmaf(sRU[g * MP + a] / sD[g], sRU[g * MP + b], t);
-                    T[a][b] = t * inv_mu + (a == b ? 1.f : 0.f);
-                    Ti[a][b] = a == b ? 1.f : 0.f;
-                }
-            for (int c = 0; c < m; ++c) {
-                const float piv = 1.f / T[c][c];
-                for (int b = 0; b < m; ++b) { T[c][b] *= piv; Ti[c][b] *= piv; }
-                for (int a = 0; a < m; ++a) {
+        // T_P = I + L_G^T D_G^{-1} L_G = I + RU^T D_G^{-1} RU / mu (one entry per thread), next to the identity
+        if (tid < PM * PM) {
+            const int a = tid / PM, b = tid - a * PM;
+            float t = 0.f;
+            for (int g = 0; g < G; ++g) t = fmaf(sRU[g * RUP + a] * sD[g], sRU[g * RUP + b], t);
+            sT[a * 2 * PM + b] = t * inv_mu + (a == b ? 1.f : 0.f);       // (rows / columns beyond m: identity)
+            sT[a * 2 * PM + PM + b] = a == b ? 1.f : 0.f;
+        }
+        __syncthreads();
+        // Gauss-Jordan on [T_P | I] by one warp, lane = column (symmetric positive definite, eigenvalues >= 1: no pivoting)
+        if (warp == 0) {
+            for (int c = 0; c < PM; ++c) {
+                const float piv = 1.f / sT[c * 2 * PM + c];
+                __syncwarp();
+                if (lane < 2 * PM) sT[c * 2 * PM + lane] *= piv;
+                __syncwarp();
+                for (int a = 0; a < PM; ++a) {
                     if (a == c) continue;
-                    const float f = T[a][c];
-                    for (int b = 0; b < m; ++b) { T[a][b] = fmaf(-f, T[c][b], T[a][b]); Ti[a][b] = fmaf(-f, Ti[c][b], Ti[a][b]); }
+                    const float f = sT[a * 2 * PM + c];
+                    __syncwarp();
+                    if (lane < 2 * PM) sT[a * 2 * PM + lane] = fmaf(-f, sT[c * 2 * PM + lane], sT[a * 2 * PM + lane]);
+                    __syncwarp();
                 }
             }
-            for (int a = 0; a < m; ++a)
-                for (int b = 0; b < m; ++b) sT[a * m + b] = Ti[a][b];
         }
         __syncthreads();
-        // column k of C:  M_g = sum_j RU[g][j] Y[k][j] / mu + d_g Omega[k][g];  z = RU^T D^{-1} M / sqrt(mu) ... all factors
-        // of 1 / sqrt(mu) are collected: L_G = RU / sqrt(mu), L^T x -> Y / sqrt(mu).
+        // column k of C:  M_g = sum_j RU[g][j] Y[k][j] / mu + d_g Omega[k][g];  z = RU^T D^{-1} M;  w = T_P^{-1} z / mu;
+        // C[g][k] = (M_g - sum_j RU[g][j] w_j) / D_g   (L_G = RU / sqrt(mu): the two factors 1 / sqrt(mu) are collected in w)
         for (int k = tid; k < K; k += kCoefThreads) {
-            float y[kMaxPivots], z[kMaxPivots], wv[kMaxPivots];
-            for (int j = 0; j < m; ++j) { y[j] = sY[k * MP + j]; z[j] = 0.f; }
-            // first pass: z = L_G^T D_G^{-1} M
+            float y[PM], z[PM], wv[PM];
+#pragma unroll
+            for (int j = 0; j < PM; ++j) { y[j] = j < m ? sY[k * MP + j] : 0.f; z[j] = 0.f; }
+            const float* omk = reinterpret_cast<const float*>(smem + sm.om) + k * (p.R | 1);
             for (int g = 0; g < G; ++g) {
+                float ru[PM];
+#pragma unroll
+                for (int j4 = 0; j4 < PM / 4; ++j4) {
+                    const float4 r4 = *reinterpret_cast<const float4*>(sRU + g * RUP + 4 * j4);
+                    ru[4 * j4] = r4.x; ru[4 * j4 + 1] = r4.y; ru[4 * j4 + 2] = r4.z; ru[4 * j4 + 3] = r4.w;
+                }
                 float Mg = 0.f;
-                for (int j = 0; j < m; ++j) Mg = fmaf(sRU[g * MP + j], y[j], Mg);
-                Mg = fmaf(Mg, inv_mu, sUU[g] * Om[(size_t)k * RS + g]);
-                const float t = Mg / sD[g];
-                for (int j = 0; j < m; ++j) z[j] = fmaf(sRU[g * MP + j], t, z[j]);
+#pragma unroll
+                for (int j = 0; j < PM; ++j) Mg = fmaf(ru[j], y[j], Mg);
+                Mg = fmaf(Mg, inv_mu, sUU[g] * omk[g]);
+                const float t = Mg * sD[g];
+#pragma unroll
+                for (int j = 0; j < PM; ++j) z[j] = fmaf(ru[j], t, z[j]);
             }
-            const float rs = rsqrtf(mu);
-            for (int a = 0; a < m; ++a) {
+#pragma unroll
+            for (int a = 0; a < PM; ++a) {
                 float t = 0.f;
-                for (int b = 0; b < m; ++b) t = fmaf(sT[a * m + b], z[b] * rs, t);
-                wv[a] = t * rs;                      // (T_P^{-1} L_G^T D^{-1} M), pre-scaled for L_G = RU / sqrt(mu)
+#pragma unroll
+                for (int b = 0; b < PM; ++b) t = fmaf(sT[a * 2 * PM + PM + b], z[b], t);
+                wv[a] = t * inv_mu;
             }
             for (int g = 0; g < G; ++g) {
+                float ru[PM];
+#pragma unroll
+                for (int j4 = 0; j4 < PM / 4; ++j4) {
+                    const float4 r4 = *reinterpret_cast<const float4*>(sRU + g * RUP + 4 * j4);
+                    ru[4 * j4] = r4.x; ru[4 * j4 + 1] = r4.y; ru[4 * j4 + 2] = r4.z; ru[4 * j4 + 3] = r4.w;
+                }
                 float Mg = 0.f, corr = 0.f;
-                for (int j = 0; j < m; ++j) { Mg = fmaf(sRU[g * MP + j], y[j], Mg); corr = fmaf(sRU[g * MP + j], wv[j], corr); }
-                Mg = fmaf(Mg, inv_mu, sUU[g] * Om[(size_t)k * RS + g]);
-                Cg[(size_t)g * K + k] = (Mg - corr) / sD[g];
+#pragma unroll
+                for (int j = 0; j < PM; ++j) { Mg = fmaf(ru[j], y[j], Mg); corr = fmaf(ru[j], wv[j], corr); }
+                Mg = fmaf(Mg, inv_mu, sUU[g] * omk[g]);
+                Cg[(size_t)g * K + k] = (Mg - corr) * sD[g];
             }
         }
     } else {
@@ -295,7 +367,7 @@ static int launch_coef_kv(Ctx* ctx, const Params& p, cudaStream_t stream) {
     const bool exact = p.pivots <= 0;
     const int m = exact ? p.R : (p.R < p.pivots ? p.R : p.pivots);
     const CoefSmem sm = make_coef_smem(K, V, p.R, m);
-    auto kern = exact ? coef_map_kernel<K, V, 1> : coef_map_kernel<K, V, 0>;
+    auto kern = exact ? coef_map_kernel<K, V, 1, 4> : (m <= 4 ? coef_map_kernel<K, V, 0, 4> : coef_map_kernel<K, V, 0, 8>);
     if (sm.total > 48u * 1024u) {
         if ((ctx->last_cuda_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm.total)) != cudaSuccess)
             return SKETCHSSM_CUDA_ERROR;
