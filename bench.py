@@ -100,6 +100,8 @@ def update_kernel_name(w: synth.Workload) -> str:
             return "update_tc_ws_mamba2_kernel" if w.rank <= 32 else "update_tc_mamba2_kernel"
         if w.kind == "gdn" and w.dv == 128 and w.rank <= 16:
             return "update_tc_ws_gdn_kernel"
+        if w.kind == "kda" and w.dv == 128 and w.rank <= 16:
+            return "update_tc_ws_kda_kernel"
     return "update_kernel"
 
 

@@ -284,8 +284,7 @@ int sketchssm_last_launch_count(const sketchssm_ctx* ctx);
  * bound >= 2 on their shared-memory stages of state rows; 0 = library default), "decode_warps_per_cta",
  * "decode_max_warps_per_sm" (also caps the update kernels' CTAs per SM), "update_impl" (0 = warp-specialised
  * tensor-core kernels where their shape limits allow and CUDA cores otherwise, the default; 1 = CUDA cores
- * only; 3 = as 0 but the single-group tensor-core kernel for Mamba-2 and CUDA cores for the delta-rule kinds;
- * 4 = as 0 plus the warp-specialised tensor-core kernel for KDA),
+ * only; 3 = as 0 but the single-group tensor-core kernel for Mamba-2 and CUDA cores for the delta-rule kinds),
  * "decode_impl" (0 = two kernels; 1 = one fused kernel with a warp per head, the default), "pdl"
  * (1 = programmatic dependent launch, the default).
  * Results depend on these only through floating-point summation order. */

@@ -106,13 +106,10 @@ int dispatch_update(sketchssm_ctx* ctx, const Params& p, cudaStream_t cs) {
         rc = launch_update_tc(ctx, p, cs);
         if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
         // gated delta rule: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 16, rank <= 16)
-        if (p.update_impl == 0 || p.update_impl == 4) {
+        if (p.update_impl == 0) {
             rc = launch_update_tc_ws_gdn(ctx, p, cs);
             if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
-        }
-        // delta rule with per-channel decay: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 32, rank <= 16);
-        // selectable only: its ring-only operand construction is instruction-bound and the CUDA-core kernel is still faster
-        if (p.update_impl == 4) {
+            // delta rule with per-channel decay: warp-specialised tensor-core kernel (up to 64 tokens in blocks of 32, rank <= 16)
             rc = launch_update_tc_ws_kda(ctx, p, cs);
             if (rc != SKETCHSSM_UNSUPPORTED_SHAPE) return rc;
         }

@@ -14,11 +14,13 @@
 // (J^T R = Omega^T, J^T H R = U^T S^T / mu, J^T H J = U^T U / mu); R itself is never needed.
 //
 // One CTA of 128 threads per (batch, head).  The probe rows (Q_j, or the U_g themselves for the exact form) sit in
-// shared memory; thread k streams row k of S with 128-bit loads (a row is read in full by one thread, so every
-// fetched sector is used) and forms Y[k][j] = <S[k,:], probe_j> and its share of ||S||_F^2 without any cross-lane
-// reduction; the small G x G / p x p systems are solved redundantly per thread or by one warp; thread k then writes
-// column k of C (coalesced across the CTA).  The kernel runs after the flush kernel of the same call and re-reads
-// S_new and U from memory: the map needs the complete sketch before it can contract the state with it.
+// shared memory.  Pivot form: a warp reads whole rows of S (lanes along the value index, every fetched sector used
+// once) and the 32 partial products of a block of rows x probes are reduced by one transposing butterfly, giving
+// Y[k][j] = <S[k,:], Q_j> and ||S||_F^2; the p x p system is built one entry per thread and inverted by one warp;
+// thread k then forms column k of C with the pivot loops unrolled in registers and Omega staged in shared memory
+// (stores coalesced across the CTA).  Exact form: thread k streams row k of S against all G sketch rows, Cholesky by
+// one warp, one pair of triangular solves per thread.  The kernel runs after the flush kernel of the same call and
+// re-reads S_new and U from memory: the map needs the complete sketch before it can contract the state with it.
 #include "internal.cuh"
 #include "lanegroup.cuh"
 

@@ -68,8 +68,7 @@ struct Params {
     int warps_per_cta;   // decode: 0 = library default
     int max_warps_per_sm; // decode weights kernel: cap on resident warps per SM (0 = default)
     int update_impl;      // 0: warp-specialised tensor-core kernels where their shape limits allow, CUDA cores otherwise;
-                          // 1: CUDA cores only; 3: single-group tensor-core kernel for Mamba-2, CUDA cores otherwise;
-                          // 4: as 0 plus the warp-specialised tensor-core kernel for KDA
+                          // 1: CUDA cores only; 3: single-group tensor-core kernel for Mamba-2, CUDA cores otherwise
     int pdl;              // launch the default decode and the tensor-core update with programmatic dependent launch
     int early_sketch;     // decode: the first head's sketch rows may be requested before the predecessor in the stream is
                           // waited for (no kernel that may still be running writes the sketch)

@@ -20,9 +20,12 @@
 // [Khat (32 rows) | G_n * [Omega | q] (32 rows)], and the kernel runs one CTA per SM.
 //
 // Front group, thread = channel i: reads column i of the staged key and decay rows into registers, forms the running
-// products, writes Khat / Ktil / G_n * W in the operand layouts, and the 496 pair sums of A as per-channel products
-// reduced over the 128 channels by transposing butterflies (per-warp partials summed in a fixed order: results are
-// bitwise reproducible).  T by forward substitution (one column per thread of warp 0) while warps 1-3 form Ktil [Omega | q].
+// products and writes Khat / Ktil / G_n * W in the operand layouts.  The 32 x 32 system is handled as two blocks of 16
+// tokens: the 2 x 120 pair sums inside the blocks are per-channel products reduced over the 128 channels by transposing
+// butterflies (per-warp partials summed in a fixed order: results are bitwise reproducible); the 16 x 16 block that
+// couples the two blocks is an mma.sync product of rescaled keys (the decay product splits at the block boundary without
+// a quotient); T_11 and T_22 by forward substitution (one column per thread, two warps) while two warps form
+// Ktil [Omega | q] with mma.sync; the pass-A group then solves E_1 = T_11 x_1, E_2 = T_22 (x_2 - A_21 E_1).
 //
 // Domain: KDA, bf16 I/O, K = V = 128, rank <= 16; 1..32 tokens per pass, up to 64 tokens per flush in blocks of 32.
 #include "internal.cuh"
@@ -39,7 +42,10 @@ constexpr int kKThreads = 448;       // pass-A group (4 warps), front group (4 w
 constexpr int kKGrp = 128;
 constexpr int kNT = 32;              // tokens per pass
 constexpr int kKStages = 8;          // upper bound on the shared-memory stages of state rows
-constexpr int kAS = 36;              // row stride (floats) of the 32 x 32 matrix A
+constexpr int kAS = 36;              // (sizes the work area of A: 32 rows of 36 floats)
+constexpr int kAS2 = 20;             // row stride (floats) of the two 16 x 16 triangles of A
+constexpr uint32_t kZPitch = 272u;   // bytes between the rows of the rescaled keys Z[token][channel]: 256 + 16, so that the 8 rows of an ldmatrix fall in different banks
+constexpr uint32_t kZHalf = 32u * kZPitch;   // hi rows, then lo rows
 constexpr int kKA2 = 2;              // chunk buffers between the pass-A group and the MMA issue warp
 constexpr int kNPk = 32;             // columns of [Omega | q]: Omega in 0..R-1, q at column QA = round_up(R, 8) <= 16
 
@@ -100,6 +106,19 @@ __device__ __forceinline__ bool k_wait(int id, int gt, uint64_t* bar, uint32_t p
     bool bad = false;
     if (gt < 32) bad = !mbar_wait_bounded(bar, phase);
     return !k_or(id, bad);
+}
+
+__device__ __forceinline__ void k_ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void k_ldmatrix_x2(uint32_t addr, uint32_t (&r)[2]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void k_mma_16816(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
 __device__ __forceinline__ float bf16_at(const unsigned char* base, uint32_t elem) {
@@ -240,7 +259,8 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 if (++stage == NS) { stage = 0; phF ^= 1u; }
             }
         };
-        // E[s, j] = sum_t T[s, t] (v_t[j] - P[t, j]) -> hi + lo A operand of Ktil^T E (chunk-buffer layout, 32 tokens)
+        // E = T (V - P) with T = (I + Bd A)^{-1} Bd solved in two blocks of 16 tokens -> hi + lo A operand of Ktil^T E
+        // (chunk-buffer layout, 32 tokens)
         auto do_e = [&](int b) {
             bad |= !mbar_wait_bounded(&bars[kPfull + b], (phP >> b) & 1u);
             phP ^= 1u << b;
@@ -264,28 +284,61 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     x[16 + t] = __bfloat162float(sV[(16 + t) * V + j]) - x1[t];
                 }
             }
+            // The 32 x 32 system in two blocks of 16 tokens:  E_1 = T_11 x_1,  E_2 = T_22 (x_2 - A_21 E_1)
+            const float* sT11 = sT1;
+            const float* sT22 = sT1 + 256;
+            const float* sA21 = sT1 + 512;
+            float e1[16], e2[16];
+#pragma unroll
+            for (int s = 0; s < 16; ++s) {
+                float acc = 0.f;
+#pragma unroll
+                for (int t4 = 0; t4 <= s / 4; ++t4) {      // T_11 is lower triangular
+                    const float4 tt = *reinterpret_cast<const float4*>(sT11 + s * 16 + t4 * 4);
+                    acc = fmaf(tt.x, x[t4 * 4], acc);
+                    acc = fmaf(tt.y, x[t4 * 4 + 1], acc);
+                    acc = fmaf(tt.z, x[t4 * 4 + 2], acc);
+                    acc = fmaf(tt.w, x[t4 * 4 + 3], acc);
+                }
+                e1[s] = acc;
+            }
+#pragma unroll
+            for (int s = 0; s < 16; ++s) {
+                float acc = x[16 + s];
+#pragma unroll
+                for (int t4 = 0; t4 < 4; ++t4) {
+                    const float4 aa = *reinterpret_cast<const float4*>(sA21 + s * 16 + t4 * 4);
+                    acc = fmaf(-aa.x, e1[t4 * 4], acc);
+                    acc = fmaf(-aa.y, e1[t4 * 4 + 1], acc);
+                    acc = fmaf(-aa.z, e1[t4 * 4 + 2], acc);
+                    acc = fmaf(-aa.w, e1[t4 * 4 + 3], acc);
+                }
+                x[16 + s] = acc;
+            }
+#pragma unroll
+            for (int s = 0; s < 16; ++s) {
+                float acc = 0.f;
+#pragma unroll
+                for (int t4 = 0; t4 <= s / 4; ++t4) {      // T_22 is lower triangular
+                    const float4 tt = *reinterpret_cast<const float4*>(sT22 + s * 16 + t4 * 4);
+                    acc = fmaf(tt.x, x[16 + t4 * 4], acc);
+                    acc = fmaf(tt.y, x[16 + t4 * 4 + 1], acc);
+                    acc = fmaf(tt.z, x[16 + t4 * 4 + 2], acc);
+                    acc = fmaf(tt.w, x[16 + t4 * 4 + 3], acc);
+                }
+                e2[s] = acc;
+            }
             unsigned char* ehi = smem + sm.e;
             unsigned char* elo = ehi + 128u * (uint32_t)kNT * 2u;
 #pragma unroll
             for (int v8 = 0; v8 < kNT / 8; ++v8) {
-                float e[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int s = v8 * 8 + u;
-                    float acc = 0.f;
-#pragma unroll
-                    for (int t4 = 0; t4 <= s / 4; ++t4) {      // T is lower triangular
-                        const float4 tt = *reinterpret_cast<const float4*>(sT1 + s * kNT + t4 * 4);
-                        acc = fmaf(tt.x, x[t4 * 4], acc);
-                        acc = fmaf(tt.y, x[t4 * 4 + 1], acc);
-                        acc = fmaf(tt.z, x[t4 * 4 + 2], acc);
-                        acc = fmaf(tt.w, x[t4 * 4 + 3], acc);
-                    }
-                    e[u] = acc;
-                }
                 uint32_t ohi[4], olo[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) split_bf16x2(e[2 * q], e[2 * q + 1], ohi[q], olo[q]);
+                for (int q = 0; q < 4; ++q) {
+                    const float ea = v8 < 2 ? e1[(v8 & 1) * 8 + 2 * q] : e2[(v8 & 1) * 8 + 2 * q];
+                    const float eb = v8 < 2 ? e1[(v8 & 1) * 8 + 2 * q + 1] : e2[(v8 & 1) * 8 + 2 * q + 1];
+                    split_bf16x2(ea, eb, ohi[q], olo[q]);
+                }
                 const uint32_t off = (gt & 7) * 16 + (gt >> 3) * SBO + v8 * LBO_M;
                 *reinterpret_cast<uint4*>(ehi + off) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
                 *reinterpret_cast<uint4*>(elo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
@@ -499,8 +552,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         bool dead = false;
         float* sA = reinterpret_cast<float*>(smem + sm.mats);
         float* sBeta = sA + kNT * kAS;
-        float* sPart = reinterpret_cast<float*>(sStg);                 // [4 warps][32][32] partial pair sums (over the key / decay rows)
-        float* sKt = reinterpret_cast<float*>(sStg);                   // later: Ktil in fp32, [channel][token ^ (channel & 31)]
+        float* sPart = reinterpret_cast<float*>(sStg + 2u * kZHalf);   // [4 warps][8 batches][32] partial pair sums (over the value rows, copied out by then)
 
         // ---- tile claiming (thread 0 of the group): per-head-index counters behind the status words ----
         int* sched = p.status + kStatusInts;
@@ -640,55 +692,54 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             }
             k_sync(2);                 // every thread holds its column: the key / decay rows of the staging area are free
 
-            // ---- pair sums A_sj = sum_i k_s[i] k_j[i] prod_{j<m<=s} g_m[i]: per-channel products, reduced over the 32
-            // channels of a warp by a transposing butterfly, 32 pairs at a time (row sa together with row 32 - sa) ----
+            // ---- pair sums inside each block of 16 tokens (the two triangles of A): A_sj = sum_i k_s[i] k_j[i]
+            // prod_{j<m<=s} g_m[i] as per-channel products, reduced over the 32 channels of a warp by a transposing
+            // butterfly, 32 pairs at a time: rows sa and 16 - sa of block 0 in entries 0..15, of block 1 in 16..31 ----
             {
-                float* part = sPart + (size_t)fwarp * (kNT * kNT);
+                float* part = sPart + (size_t)fwarp * (8 * 32);
 #pragma unroll
-                for (int sa = 1; sa <= 16; ++sa) {
+                for (int sa = 1; sa <= 8; ++sa) {
                     float vals[32];
-                    {
-                        float r = kk[sa];
 #pragma unroll
-                        for (int jj = 15; jj >= 0; --jj)
-                            if (jj < sa) { r *= gg[jj + 1]; vals[jj] = r * kk[jj]; }
+                    for (int blk = 0; blk < 2; ++blk) {
+                        const int b0 = 16 * blk;
+                        {
+                            float r = kk[b0 + sa];
+#pragma unroll
+                            for (int jj = 7; jj >= 0; --jj)
+                                if (jj < sa) { r *= gg[b0 + jj + 1]; vals[b0 + jj] = r * kk[b0 + jj]; }
+                        }
+                        if (sa < 8) {
+                            const int sb2 = 16 - sa;
+                            float r = kk[b0 + sb2];
+#pragma unroll
+                            for (int jj = 14; jj >= 0; --jj)
+                                if (jj < sb2) { r *= gg[b0 + jj + 1]; vals[b0 + sa + jj] = r * kk[b0 + jj]; }
+                        } else {
+#pragma unroll
+                            for (int jj = 8; jj < 16; ++jj) vals[b0 + jj] = 0.f;
+                        }
                     }
-                    if (sa < 16) {
-                        const int sb2 = 32 - sa;
-                        float r = kk[sb2];
-#pragma unroll
-                        for (int jj = 30; jj >= 0; --jj)
-                            if (jj < sb2) { r *= gg[jj + 1]; vals[sa + jj] = r * kk[jj]; }
-                    } else {
-#pragma unroll
-                        for (int jj = 16; jj < 32; ++jj) vals[jj] = 0.f;
-                    }
-                    group_reduce_transpose<32, 32>(vals, lane);
-                    // lane l now holds entry l of the batch: (sa, l) for l < sa, else (32 - sa, l - sa)
-                    const int row = lane < sa ? sa : 32 - sa;
-                    const int col = lane < sa ? lane : lane - sa;
-                    if (sa < 16 || lane < 16) part[row * kNT + col] = vals[0];
+                    group_reduce_transpose<32, 32>(vals, lane);      // lane l now holds entry l of the batch
+                    part[(sa - 1) * 32 + lane] = vals[0];
                 }
             }
-            k_sync(2);
-            // beta_s A_sj: the four warps' partials summed in a fixed order (strictly lower triangle)
-            for (int idx = gt; idx < kNT * kNT; idx += kKGrp) {
-                const int s = idx >> 5, jj = idx & 31;
-                float a = 0.f;
-                if (jj < s) a = ((sPart[idx] + sPart[kNT * kNT + idx]) + sPart[2 * kNT * kNT + idx]) + sPart[3 * kNT * kNT + idx];
-                sA[s * kAS + jj] = sBeta[s] * a;
-            }
-            k_sync(2);                 // the partials have been consumed: the area now takes Ktil
 
-            // ---- running products; Khat -> window rows 0..31, Ktil -> set (MN-major) and fp32 scratch, G_n * W -> rows 32.. ----
+            // ---- running products.  Khat -> window rows 0..31; Ktil -> set (MN-major); G_n * W -> window rows 32..;
+            // and for the 16 x 16 block of A that couples the two token blocks, whose decay product splits at the block
+            // boundary without a quotient (prod_{j<m<=s} = prod_{16<=m<=s} * prod_{j<m<=15}), the rescaled keys
+            // X_s = k_s prod_{16<=m<=s} g_m (s >= 16) and Y_j = k_j prod_{j<m<=15} g_m (j < 16) as bf16 hi + lo rows
+            // Z[token][channel] over the (now free) key / decay rows of the staging area ----
             {
                 __nv_bfloat16* whi = reinterpret_cast<__nv_bfloat16*>(wb);
                 __nv_bfloat16* wlo = reinterpret_cast<__nv_bfloat16*>(wb + sm.w_lo);
                 __nv_bfloat16* bthi = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bt);
                 __nv_bfloat16* btlo = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bt_lo);
+                __nv_bfloat16* zhi = reinterpret_cast<__nv_bfloat16*>(sStg);
+                __nv_bfloat16* zlo = reinterpret_cast<__nv_bfloat16*>(sStg + kZHalf);
                 const uint32_t wcol = ((uint32_t)(i >> 3) * LBO_W + (uint32_t)(i & 7) * 2u) >> 1;        // K-major: k = channel
                 const uint32_t bcol = ((uint32_t)(i & 7) * 2u + (uint32_t)(i >> 3) * SBO) >> 1;          // MN-major: mn = channel
-                float G = 1.f;
+                float G = 1.f, X = 1.f;
 #pragma unroll
                 for (int s = 0; s < kNT; ++s) {
                     G *= gg[s];
@@ -697,8 +748,14 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     const uint32_t o = wcol + (((uint32_t)(s & 7) * 16u + (uint32_t)(s >> 3) * SBO) >> 1);
                     whi[o] = hi;
                     wlo[o] = lo;
+                    if (s >= 16) {
+                        X *= gg[s];
+                        split_bf16(X * kk[s], hi, lo);
+                        zhi[s * (kZPitch / 2) + i] = hi;
+                        zlo[s * (kZPitch / 2) + i] = lo;
+                    }
                 }
-                float Dn = 1.f;
+                float Dn = 1.f, Yd = 1.f;
 #pragma unroll
                 for (int s = kNT - 1; s >= 0; --s) {
                     const float kt = Dn * kk[s];
@@ -708,7 +765,12 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     const uint32_t o = bcol + (((uint32_t)(s & 7) * 16u + (uint32_t)(s >> 3) * LBO_M) >> 1);
                     bthi[o] = hi;
                     btlo[o] = lo;
-                    sKt[i * kNT + (s ^ (i & 31))] = kt;
+                    if (s < 16) {
+                        split_bf16(Yd * kk[s], hi, lo);
+                        zhi[s * (kZPitch / 2) + i] = hi;
+                        zlo[s * (kZPitch / 2) + i] = lo;
+                        Yd *= gg[s];
+                    }
                 }
                 reinterpret_cast<float*>(set + sm.set_gn)[i] = G;
                 if (p.write_sketch) {
@@ -728,51 +790,126 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     wlo[o] = lo;
                 }
             }
-            k_sync(2);                 // A and Ktil (fp32) are complete
+            k_sync(2);                 // partial pair sums, Z rows and Ktil are complete
 
-            if (fwarp == 0) {
-                // ---- T = (I + Bd A)^{-1} Bd by forward substitution: one column per thread, held in registers ----
-                const int c = lane;
-                float tcol[kNT];
+            if (fwarp == 3) {
+                // ---- A_21 = X Y^T (16 x 16, tokens 16..31 against tokens 0..15) as mma.sync products of the Z rows,
+                // hi * hi + lo * hi + hi * lo ----
+                float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                const uint32_t zb = smem_u32(sStg);
+                const uint32_t abase = zb + (uint32_t)(16 + (lane & 15)) * kZPitch + (uint32_t)(lane >> 4) * 16u;
+                const uint32_t bbase = zb + (uint32_t)(lane & 7) * kZPitch + (uint32_t)((lane >> 3) & 1) * 16u;
 #pragma unroll
-                for (int s = 0; s < kNT; ++s) {
-                    float acc = 0.f;
+                for (int ks = 0; ks < K / 16; ++ks) {
+                    uint32_t ahi[4], alo[4];
+                    k_ldmatrix_x4(abase + ks * 32, ahi);
+                    k_ldmatrix_x4(abase + kZHalf + ks * 32, alo);
 #pragma unroll
-                    for (int j4 = 0; j4 < (s + 3) / 4; ++j4) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(sA + s * kAS + j4 * 4);
-                        if (j4 * 4 + 0 < s) acc = fmaf(l4.x, tcol[j4 * 4 + 0], acc);
-                        if (j4 * 4 + 1 < s) acc = fmaf(l4.y, tcol[j4 * 4 + 1], acc);
-                        if (j4 * 4 + 2 < s) acc = fmaf(l4.z, tcol[j4 * 4 + 2], acc);
-                        if (j4 * 4 + 3 < s) acc = fmaf(l4.w, tcol[j4 * 4 + 3], acc);
+                    for (int nt = 0; nt < 2; ++nt) {
+                        uint32_t bhi[2], blo[2];
+                        k_ldmatrix_x2(bbase + (uint32_t)(nt * 8) * kZPitch + ks * 32, bhi);
+                        k_ldmatrix_x2(bbase + (uint32_t)(nt * 8) * kZPitch + kZHalf + ks * 32, blo);
+                        k_mma_16816(acc[nt], ahi, bhi);
+                        k_mma_16816(acc[nt], alo, bhi);
+                        k_mma_16816(acc[nt], ahi, blo);
                     }
-                    tcol[s] = (s >= n_tot || s < c || c >= n_tot) ? 0.f : (s == c ? 1.f : -acc);
                 }
-                const float bc = sBeta[c];
-                float* sT1 = reinterpret_cast<float*>(set + sm.set_t1);
+                float* sA21 = reinterpret_cast<float*>(set + sm.set_t1) + 512;
 #pragma unroll
-                for (int s = 0; s < kNT; ++s) sT1[s * kNT + c] = tcol[s] * bc;
+                for (int nt = 0; nt < 2; ++nt) {
+                    const int r0 = lane >> 2, c0 = nt * 8 + (lane & 3) * 2;
+                    sA21[r0 * 16 + c0] = acc[nt][0];
+                    sA21[r0 * 16 + c0 + 1] = acc[nt][1];
+                    sA21[(r0 + 8) * 16 + c0] = acc[nt][2];
+                    sA21[(r0 + 8) * 16 + c0 + 1] = acc[nt][3];
+                }
             } else {
-                // ---- Ktil W: 32 tokens x ([Omega | q]), fp32 on CUDA cores; thread = (token, every third column) ----
-                const int s = lane, part = fwarp - 1;
-                const int ncol = p.write_sketch ? R : 0;
-                float acc[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                float accq = 0.f;
+                // ---- beta_s A_sj of the two triangles: the four warps' partials summed in a fixed order ----
+                for (int idx = gt; idx < 2 * 16 * 16; idx += 96) {
+                    const int blk = idx >> 8, s = (idx >> 4) & 15, jj = idx & 15;
+                    float a = 0.f;
+                    if (jj < s) {
+                        const int sa = s <= 8 ? s : 16 - s;
+                        const int e = (sa - 1) * 32 + blk * 16 + (s <= 8 ? jj : sa + jj);
+                        a = ((sPart[e] + sPart[256 + e]) + sPart[512 + e]) + sPart[768 + e];
+                    }
+                    sA[blk * (16 * kAS2) + s * kAS2 + jj] = sBeta[16 * blk + s] * a;
+                }
+            }
+            k_sync(2);                 // A is complete
+
+            if (fwarp < 2) {
+                // ---- T_bb = (I + Bd A_bb)^{-1} Bd of block fwarp by forward substitution: one column per thread, in registers ----
+                if (lane < 16) {
+                    const int c = lane;
+                    const int nb = min(max(n_tot - 16 * fwarp, 0), 16);      // tokens of this block
+                    const float* sAb = sA + fwarp * (16 * kAS2);
+                    float tcol[16];
+#pragma unroll
+                    for (int s = 0; s < 16; ++s) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int j4 = 0; j4 < (s + 3) / 4; ++j4) {
+                            const float4 l4 = *reinterpret_cast<const float4*>(sAb + s * kAS2 + j4 * 4);
+                            if (j4 * 4 + 0 < s) acc = fmaf(l4.x, tcol[j4 * 4 + 0], acc);
+                            if (j4 * 4 + 1 < s) acc = fmaf(l4.y, tcol[j4 * 4 + 1], acc);
+                            if (j4 * 4 + 2 < s) acc = fmaf(l4.z, tcol[j4 * 4 + 2], acc);
+                            if (j4 * 4 + 3 < s) acc = fmaf(l4.w, tcol[j4 * 4 + 3], acc);
+                        }
+                        tcol[s] = (s >= nb || s < c || c >= nb) ? 0.f : (s == c ? 1.f : -acc);
+                    }
+                    const float bc = sBeta[16 * fwarp + c];
+                    float* sT = reinterpret_cast<float*>(set + sm.set_t1) + fwarp * 256;
+#pragma unroll
+                    for (int s = 0; s < 16; ++s) sT[s * 16 + c] = tcol[s] * bc;
+                }
+            } else {
+                // ---- Ktil W: 16 tokens (block fwarp - 2) x 24 columns of [Omega | q] as mma.sync products.  A: the Ktil
+                // operand just written (its 8 x 8 core matrices are the row-major fragments ldmatrix wants), hi + lo;
+                // B: Omega and q straight from memory into fragments, split into hi + lo in registers ----
+                const int mt = fwarp - 2;
+                float acc[3][4];
+#pragma unroll
+                for (int nt = 0; nt < 3; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+                const uint32_t btb = smem_u32(set + sm.set_bt);
+                const uint32_t a_row = btb + (uint32_t)(2 * mt + ((lane >> 3) & 1)) * LBO_M + (uint32_t)(lane >> 4) * SBO + (uint32_t)(lane & 7) * 16u;
                 const float* omh = p.omega + (size_t)h * K * R;
                 const __nv_bfloat16* sq = reinterpret_cast<const __nv_bfloat16*>(sStg + sm.stg_q);
-                const bool do_q = part == 0 && p.q != nullptr;
-                for (int ii = 0; ii < K; ++ii) {
-                    const float kt = sKt[ii * kNT + (s ^ (ii & 31))];
-                    const float* orow = omh + (size_t)ii * R;
+                const int ncol = p.write_sketch ? R : 0;
+                const bool has_q = p.q != nullptr;
+                for (int ks = 0; ks < K / 16; ++ks) {
+                    uint32_t ahi[4], alo[4];
+                    k_ldmatrix_x4(a_row + (uint32_t)(2 * ks) * SBO, ahi);
+                    k_ldmatrix_x4(a_row + sm.set_bt_lo + (uint32_t)(2 * ks) * SBO, alo);
+                    const int i0 = ks * 16 + (lane & 3) * 2;
 #pragma unroll
-                    for (int u = 0; u < 6; ++u) {
-                        const int g = part + 3 * u;
-                        if (g < ncol) acc[u] = fmaf(kt, __ldg(orow + g), acc[u]);
+                    for (int nt = 0; nt < 3; ++nt) {
+                        const int g = nt * 8 + (lane >> 2);
+                        float w[4] = {0.f, 0.f, 0.f, 0.f};
+                        if (g < ncol) {
+                            w[0] = __ldg(omh + (size_t)i0 * R + g);
+                            w[1] = __ldg(omh + (size_t)(i0 + 1) * R + g);
+                            w[2] = __ldg(omh + (size_t)(i0 + 8) * R + g);
+                            w[3] = __ldg(omh + (size_t)(i0 + 9) * R + g);
+                        } else if (g == QA && has_q) {
+                            w[0] = __bfloat162float(sq[i0]);
+                            w[1] = __bfloat162float(sq[i0 + 1]);
+                            w[2] = __bfloat162float(sq[i0 + 8]);
+                            w[3] = __bfloat162float(sq[i0 + 9]);
+                        }
+                        uint32_t bhi[2], blo[2];
+                        split_bf16x2(w[0], w[1], bhi[0], blo[0]);
+                        split_bf16x2(w[2], w[3], bhi[1], blo[1]);
+                        k_mma_16816(acc[nt], ahi, bhi);
+                        k_mma_16816(acc[nt], alo, bhi);
+                        k_mma_16816(acc[nt], ahi, blo);
                     }
-                    if (do_q) accq = fmaf(kt, __bfloat162float(sq[ii]), accq);
                 }
                 __nv_bfloat16* bchi = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bc);
                 __nv_bfloat16* bclo = bchi + 1024;
-                auto put = [&](int g, float x) {
+                auto put = [&](int s, int g, float x) {
                     __nv_bfloat16 hi, lo;
                     split_bf16(x, hi, lo);
                     const uint32_t o2 = ((uint32_t)(g & 7) * 16u + (uint32_t)(g >> 3) * SBO + (uint32_t)(s >> 3) * LBO_C + (uint32_t)(s & 7) * 2u) >> 1;
@@ -780,11 +917,13 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     bclo[o2] = lo;
                 };
 #pragma unroll
-                for (int u = 0; u < 6; ++u) {
-                    const int g = part + 3 * u;
-                    if (g < ncol) put(g, acc[u]);
+                for (int nt = 0; nt < 3; ++nt) {
+                    const int s0 = 16 * mt + (lane >> 2), g0 = nt * 8 + (lane & 3) * 2;
+                    put(s0, g0, acc[nt][0]);
+                    put(s0, g0 + 1, acc[nt][1]);
+                    put(s0 + 8, g0, acc[nt][2]);
+                    put(s0 + 8, g0 + 1, acc[nt][3]);
                 }
-                if (do_q) put(QA, accq);
             }
             proxy_fence();         // operand sets and windows are read by MMAs (async proxy)
             k_sync(2);

@@ -213,7 +213,7 @@ def test_gdn_warp_specialised_update(tune, batch, heads, rank, buf_len):
     check(run_schedule(w, 2 * buf_len + 3, max_heads=96, tune=tune), "bf16")
 
 
-@pytest.mark.parametrize("tune", [{"update_impl": 4}, {"update_impl": 4, "decode_stages": 2}, {"update_impl": 4, "pdl": 0}])
+@pytest.mark.parametrize("tune", [{}, {"decode_stages": 2}, {"pdl": 0}])
 @pytest.mark.parametrize("batch,heads,rank,buf_len", [(5, 3, 16, 32), (40, 20, 16, 16), (33, 7, 8, 12), (6, 2, 5, 4),
                                                       (12, 4, 16, 32), (7, 3, 12, 40), (5, 2, 16, 64), (150, 3, 16, 32)])
 def test_kda_warp_specialised_update(tune, batch, heads, rank, buf_len):

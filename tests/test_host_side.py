@@ -97,5 +97,5 @@ def test_logical_layers_map_onto_the_physical_slots_that_fit():
     assert bench.physical_layers(10**12, 10**9, 48) == 1        # never fewer than one slot
     assert [l % n for l in range(48)].count(0) == -(-48 // n)   # slot 0 serves ceil(48 / n) logical layers
     assert bench.update_kernel_name(w) == "update_tc_ws_mamba2_kernel"
-    assert bench.update_kernel_name(synth.CONFIGS["c4_kda"]) == "update_kernel"
+    assert bench.update_kernel_name(synth.CONFIGS["c4_kda"]) == "update_tc_ws_kda_kernel"
     assert bench.update_kernel_name(synth.CONFIGS["c1_gdn_tiny"]) == "update_kernel"
