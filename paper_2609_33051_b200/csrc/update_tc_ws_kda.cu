@@ -13,8 +13,8 @@
 //
 // Same schedule as the gated-delta-rule kernel: tile = one head (K = V = 128), TMEM lane = value column; the state is
 // read once by bulk copies into a ring of shared-memory stages; the pass-A group splits the S_0 chunks into bf16 hi + lo,
-// leaves G_n * S_0 in the accumulator of Ktil^T E (tcgen05.st) and later forms E; one thread issues every MMA; the pass-B
-// group writes the accumulator (S_new) back and stores the sketch rows; the front group builds the ring-only operands two
+// leaves G_n * S_0 in the accumulator of Ktil^T E (tcgen05.st); one thread issues every MMA; the pass-B
+// group forms E, writes the accumulator (S_new) back and stores the sketch rows; the front group builds the ring-only operands two
 // tiles ahead.  What differs: up to 32 tokens per pass (the MMAs over tokens take two k-steps), both key operands and the
 // basis operand are per tile and carry hi + lo halves, so the B operand of pass A is a double-buffered per-tile window
 // [Khat (32 rows) | G_n * [Omega | q] (32 rows)], and the kernel runs one CTA per SM.
@@ -25,7 +25,8 @@
 // butterflies (per-warp partials summed in a fixed order: results are bitwise reproducible); the 16 x 16 block that
 // couples the two blocks is an mma.sync product of rescaled keys (the decay product splits at the block boundary without
 // a quotient); T_11 and T_22 by forward substitution (one column per thread, two warps) while two warps form
-// Ktil [Omega | q] with mma.sync; the pass-A group then solves E_1 = T_11 x_1, E_2 = T_22 (x_2 - A_21 E_1).
+// Ktil [Omega | q] with mma.sync.  The E step (E_1 = T_11 x_1, E_2 = T_22 (x_2 - A_21 E_1), 528 multiply-adds per lane) runs
+// on the pass-B group, between the write-back of one tile and the next, so that the pass-A group only streams.
 //
 // Domain: KDA, bf16 I/O, K = V = 128, rank <= 16; 1..32 tokens per pass, up to 64 tokens per flush in blocks of 32.
 #include "internal.cuh"
@@ -82,7 +83,7 @@ __host__ __device__ inline KSmem make_ksmem(int stages) {
 }
 
 enum { kPro = 0, kPfull = 2, kTfull = 4, kBdone = 6, kBufFree = 8, kA2free = 10, kA2rdy = 10 + kKA2, kErdy = 10 + 2 * kKA2,
-       kStg = 11 + 2 * kKA2, kFull = 14 + 2 * kKA2, kEmpty = 14 + 2 * kKA2 + kKStages,
+       kStg = 11 + 2 * kKA2, kStDone = 12 + 2 * kKA2, kFull = 14 + 2 * kKA2, kEmpty = 14 + 2 * kKA2 + kKStages,
        kTfree = 14 + 2 * kKA2 + 2 * kKStages, kNumBars = 16 + 2 * kKA2 + 2 * kKStages };
 
 __device__ __forceinline__ void k_arrive(uint64_t* bar) {
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
         for (int i = 0; i < kNumBars; ++i) {
             // one arrival per warp of a stream group: chunk ready, E ready, stage empty, accumulator halves, pass-B done, slot free
-            const bool per_warp = (i >= kA2rdy && i <= kErdy) || i >= kEmpty || (i >= kBdone && i < kBdone + 4);
+            const bool per_warp = (i >= kA2rdy && i <= kErdy) || i == kStDone || i >= kEmpty || (i >= kBdone && i < kBdone + 4);
             mbar_init(&bars[i], per_warp ? 4 : 1);
         }
         mbar_fence_init();
@@ -200,7 +201,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
 
     if (warp < 4) {
         // =========================== pass-A group: S_0 chunks -> operands, and the E step ===========================
-        uint32_t phPro = 0, phP = 0, phT = 0, phA = 0, phF = 0;
+        uint32_t phPro = 0, phA = 0, phF = 0;
         int gc = 0, stage = 0;
         bool bad = false;
 
@@ -258,7 +259,36 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 ++gc;
                 if (++stage == NS) { stage = 0; phF ^= 1u; }
             }
+            tmem_st_wait();            // this warp's G_n * S_0 columns are in tensor memory
+            tc_fence_before();
+            bad = __any_sync(0xffffffffu, bad);
+            if (lane == 0 && !bad) k_arrive(&bars[kStDone]);
         };
+        auto wait_pro = [&](int b) {
+            bad |= !mbar_wait_bounded(&bars[kPro + b], (phPro >> b) & 1u);
+            phPro ^= 1u << b;
+        };
+
+        int cur = seq_get(0);
+        if (cur >= 0) {
+            wait_pro(0);
+            pass_a(0, false);
+            for (int k = 0; !bad; ++k) {
+                const int b = k & 1;
+                const int raw = seq_get(k + 1);
+                if (raw < -1) { bad = true; break; }
+                if (raw < 0) break;
+                wait_pro(b ^ 1);
+                pass_a(b ^ 1, true);
+            }
+        } else if (cur < -1) {
+            bad = true;
+        }
+        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 103);
+    } else if (warp >= 10) {
+        // =========================== pass-B group: S_new written back, then the sketch rows ===========================
+        uint32_t phT = 0, phP = 0;
+        bool bad = false;
         // E = T (V - P) with T = (I + Bd A)^{-1} Bd solved in two blocks of 16 tokens -> hi + lo A operand of Ktil^T E
         // (chunk-buffer layout, 32 tokens)
         auto do_e = [&](int b) {
@@ -344,44 +374,14 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 *reinterpret_cast<uint4*>(elo + off) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
             }
             proxy_fence();
-            tmem_st_wait();            // the G_n * S_0 columns of pass A are in tensor memory
             tc_fence_before();
             bad = __any_sync(0xffffffffu, bad);
             if (lane == 0 && !bad) k_arrive(&bars[kErdy]);
         };
-        auto wait_pro = [&](int b) {
-            bad |= !mbar_wait_bounded(&bars[kPro + b], (phPro >> b) & 1u);
-            phPro ^= 1u << b;
-        };
-
-        int cur = seq_get(0);
-        if (cur >= 0) {
-            wait_pro(0);
-            pass_a(0, false);
-            do_e(0);
-            for (int k = 0; !bad; ++k) {
-                const int b = k & 1;
-                const int raw = seq_get(k + 1);
-                if (raw < -1) { bad = true; break; }
-                if (raw < 0) break;
-                wait_pro(b ^ 1);
-                pass_a(b ^ 1, true);
-                // the E operand buffer is read by Ktil^T E of tile k: that must be complete before it is rewritten
-                bad |= !mbar_wait_bounded(&bars[kTfull + b], (phT >> b) & 1u);
-                phT ^= 1u << b;
-                do_e(b ^ 1);
-            }
-        } else if (cur < -1) {
-            bad = true;
-        }
-        if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 103);
-    } else if (warp >= 10) {
-        // =========================== pass-B group: S_new written back, then the sketch rows ===========================
-        uint32_t phT = 0;
-        bool bad = false;
-        for (int k = 0; !bad; ++k) {
-            const int raw = seq_get(k);
-            if (raw < 0) { bad = raw < -1; break; }
+        int raw = seq_get(0);
+        if (raw >= 0) do_e(0);
+        else bad = raw < -1;
+        for (int k = 0; !bad && raw >= 0; ++k) {
             const int tile = raw;
             const int b = k & 1;
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
@@ -429,12 +429,17 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 __syncwarp();
                 if (lane == 0) k_arrive(&bars[kBufFree + b]);       // the slot is free for pass A of tile k + 2
             }
+            // the E step of the next tile: its P is complete once pass A of that tile is, and the E operand buffer is free
+            // because Ktil^T E of this tile has completed (waited for above)
+            raw = seq_get(k + 1);
+            if (raw < 0) { bad |= raw < -1; break; }
+            if (!bad) do_e(b ^ 1);
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 111);
     } else if (warp == 8) {
         // =========================== MMA issue warp (one thread) ===========================
         if (lane == 0) {
-            uint32_t phR = 0, phE = 0, phBuf = 0;
+            uint32_t phR = 0, phE = 0, phBuf = 0, phSt = 0;
             bool bad = false;
             int where = 104;                // which wait gave up (status detail): 141 slot free, 142 chunk ready, 143 E ready, 144 accumulator read
             const uint32_t a2base = smem_u32(smem + sm.a2);
@@ -471,6 +476,8 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 const int b = k & 1;
                 if (!mbar_wait_bounded(&bars[kErdy], phE)) { bad = true; where = 143; return; }
                 phE ^= 1u;
+                if (!mbar_wait_bounded(&bars[kStDone], phSt)) { bad = true; where = 145; return; }       // G_n * S_0 is in the accumulator
+                phSt ^= 1u;
                 if (k >= 1) {                   // the pass-B group must have read the accumulator of the tile before
                     if (!mbar_wait_bounded(&bars[kBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 144; return; }
                 }
