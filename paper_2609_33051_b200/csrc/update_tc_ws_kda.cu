@@ -52,7 +52,7 @@ constexpr int kNPk = 32;             // columns of [Omega | q]: Omega in 0..R-1,
 
 struct KSmem {
     uint32_t a2, e, w, w_stride, w_lo, set, set_stride, set_bt, set_bt_lo, set_vv, set_t1, set_bc, set_gn, stg, stg_g, stg_v,
-        stg_beta, stg_q, mats, bars, misc, sst, sst_bytes, total;
+        stg_beta, stg_q, mats, om, bars, misc, sst, sst_bytes, total;
 };
 
 __host__ __device__ inline KSmem make_ksmem(int stages) {
@@ -73,6 +73,7 @@ __host__ __device__ inline KSmem make_ksmem(int stages) {
     s.stg_g = 8192u; s.stg_v = 16384u; s.stg_beta = 24576u; s.stg_q = 24832u;
     s.stg = off; off += 25088u;
     s.mats = off; off += (uint32_t)kNT * kAS * 4u + 256u;         // A (beta_s A_sj), beta
+    s.om = off; off += (uint32_t)kK * 16u * 4u;                   // Omega of the current head index, fp32 [K][16] (zero beyond the rank)
     s.bars = off; off += 512u;
     s.misc = off; off += 128u;
     off = (off + 127u) & ~127u;
@@ -559,6 +560,8 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         bool dead = false;
         float* sA = reinterpret_cast<float*>(smem + sm.mats);
         float* sBeta = sA + kNT * kAS;
+        float* sOm = reinterpret_cast<float*>(smem + sm.om);
+        int cur_h = -1;
         float* sPart = reinterpret_cast<float*>(sStg + 2u * kZHalf);   // [4 warps][8 batches][32] partial pair sums (over the value rows, copied out by then)
 
         // ---- tile claiming (thread 0 of the group): per-head-index counters behind the status words ----
@@ -656,8 +659,16 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             // gate of the current token: requested early
             float tok_beta = 0.f;
             if (gt < kNT && p.has_token) tok_beta = p.beta[bh];
-            // Omega row of this channel (fp32, through L1 / L2: shared by the whole batch)
-            const float* og = p.omega + ((size_t)h * K + i) * R;
+            // Omega of this head index in shared memory (global loads here would sit on the group's critical path)
+            if (h != cur_h) {
+                const float* omg = p.omega + (size_t)h * K * R;
+                for (int idx = gt; idx < K * 16; idx += kKGrp) {
+                    const int kk2 = idx >> 4, g = idx & 15;
+                    sOm[idx] = (g < R && p.write_sketch) ? __ldg(omg + (size_t)kk2 * R + g) : 0.f;
+                }
+                cur_h = h;            // (visible to the group after the barrier below)
+            }
+            const float* og = sOm + i * 16;
             // the operand set and window of tile k - 2 are free once its Ktil^T E has completed
             if (k >= 2) {
                 if (!k_wait(2, gt, &bars[kTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
@@ -783,7 +794,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 if (p.write_sketch) {
                     for (int g = 0; g < R; ++g) {
                         __nv_bfloat16 hi, lo;
-                        split_bf16(G * __ldg(og + g), hi, lo);
+                        split_bf16(G * og[g], hi, lo);
                         const uint32_t o = wcol + (((uint32_t)(g & 7) * 16u + (uint32_t)((g >> 3) + 4) * SBO) >> 1);
                         whi[o] = hi;
                         wlo[o] = lo;
@@ -882,7 +893,6 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
                 const uint32_t btb = smem_u32(set + sm.set_bt);
                 const uint32_t a_row = btb + (uint32_t)(2 * mt + ((lane >> 3) & 1)) * LBO_M + (uint32_t)(lane >> 4) * SBO + (uint32_t)(lane & 7) * 16u;
-                const float* omh = p.omega + (size_t)h * K * R;
                 const __nv_bfloat16* sq = reinterpret_cast<const __nv_bfloat16*>(sStg + sm.stg_q);
                 const int ncol = p.write_sketch ? R : 0;
                 const bool has_q = p.q != nullptr;
@@ -896,10 +906,10 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                         const int g = nt * 8 + (lane >> 2);
                         float w[4] = {0.f, 0.f, 0.f, 0.f};
                         if (g < ncol) {
-                            w[0] = __ldg(omh + (size_t)i0 * R + g);
-                            w[1] = __ldg(omh + (size_t)(i0 + 1) * R + g);
-                            w[2] = __ldg(omh + (size_t)(i0 + 8) * R + g);
-                            w[3] = __ldg(omh + (size_t)(i0 + 9) * R + g);
+                            w[0] = sOm[i0 * 16 + g];
+                            w[1] = sOm[(i0 + 1) * 16 + g];
+                            w[2] = sOm[(i0 + 8) * 16 + g];
+                            w[3] = sOm[(i0 + 9) * 16 + g];
                         } else if (g == QA && has_q) {
                             w[0] = __bfloat162float(sq[i0]);
                             w[1] = __bfloat162float(sq[i0 + 1]);
