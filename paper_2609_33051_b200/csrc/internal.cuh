@@ -191,6 +191,13 @@ __device__ __forceinline__ void store_sketch(const Params& p, size_t idx, float 
     else p.sketch[idx] = u;
 }
 
+// The same with the storage type fixed at compile time (for loops that branch once on p.sketch_bf16 outside).
+template <bool BF>
+__device__ __forceinline__ void store_sketch_as(const Params& p, size_t idx, float u) {
+    if (BF) reinterpret_cast<__nv_bfloat16*>(p.sketch)[idx] = __float2bfloat16_rn(u);
+    else p.sketch[idx] = u;
+}
+
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);

@@ -74,6 +74,24 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16]) {
     for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(u[i]);
 }
 
+// one column of this thread's TMEM lane
+__device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
+    uint32_t u;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(u) : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    return __uint_as_float(u);
+}
+
+// one column at each of two addresses of this thread's TMEM lane, both loads in flight together
+__device__ __forceinline__ void tmem_ld1x2(uint32_t ta, uint32_t tb, float& a, float& b) {
+    uint32_t ua, ub;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(ua) : "r"(ta) : "memory");
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(ub) : "r"(tb) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    a = __uint_as_float(ua);
+    b = __uint_as_float(ub);
+}
+
 // 16 columns of this thread's TMEM lane from registers; completion is awaited separately (tmem_st_wait)
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&r)[16]) {
     asm volatile(

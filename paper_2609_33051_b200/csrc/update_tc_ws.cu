@@ -24,6 +24,7 @@
 // W = [Omega | q-group A | q-group B]: consecutive tiles alternate between the two query groups, so the front group
 // can write the next tile's query columns while MMA 2 of the current tile still reads the buffer (it then also reads
 // half-written columns of the other group, whose outputs nobody uses).
+#include <type_traits>
 #include "internal.cuh"
 #include "tc_common.cuh"
 
@@ -469,18 +470,31 @@ __global__ void __launch_bounds__(kWsThreads, 2) update_tc_ws_mamba2_kernel(cons
             if (!group_wait(2, gt, &bars[kBarU + b], (phU >> b) & 1u)) return false;
             phU ^= 1u << b;
             tc_fence_after();
-            for (int g0 = 0; g0 < NP; g0 += 16) {
-                float u[16];
-                tmem_ld16(tmem_base + (uint32_t)b * 128u + lane_sel + (uint32_t)g0, u);
+            // sketch rows: column g of the accumulator is U[g][j]; full groups of 16 ranks take the unpredicated stores
+            const uint32_t trow = tmem_base + (uint32_t)b * 128u + lane_sel;
+            auto rows = [&](auto bf) {
+                constexpr bool BF = decltype(bf)::value;
+                const size_t base = (bh * R) * (size_t)V + j;
+                for (int g0 = 0; g0 < R; g0 += 16) {
+                    float u[16];
+                    tmem_ld16(trow + (uint32_t)g0, u);
+                    if (g0 + 16 <= R) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int g = g0 + e;
-                    if (g < R && p.write_sketch) store_sketch(p, (bh * R + g) * (size_t)V + j, u[e]);
-                    if (g == QA + 8 * b + my_head && p.out != nullptr) {
-                        if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u[e]);
-                        else reinterpret_cast<float*>(p.out)[bh * V + j] = u[e];
+                        for (int e = 0; e < 16; ++e) store_sketch_as<BF>(p, base + (size_t)(g0 + e) * V, u[e]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (g0 + e < R) store_sketch_as<BF>(p, base + (size_t)(g0 + e) * V, u[e]);
                     }
                 }
+            };
+            if (p.write_sketch) {
+                if (p.sketch_bf16) rows(std::true_type{}); else rows(std::false_type{});
+            }
+            if (p.out != nullptr) {       // exact output: the query column of this head
+                const float o = tmem_ld1(trow + (uint32_t)(QA + 8 * b + my_head));
+                if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(o);
+                else reinterpret_cast<float*>(p.out)[bh * V + j] = o;
             }
             tc_fence_before();     // ordered before the next MMA 1 into this accumulator by the group barriers that follow
             return true;

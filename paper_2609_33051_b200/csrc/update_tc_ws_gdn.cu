@@ -33,6 +33,7 @@
 //
 // Domain: GDN, bf16 I/O, K = V = 128, rank <= 16; 1..16 tokens per pass, up to 64 tokens per flush in blocks of 16
 // (one pass over the state per block).
+#include <type_traits>
 #include "internal.cuh"
 #include "tc_common.cuh"
 
@@ -361,20 +362,35 @@ __global__ void __launch_bounds__(kGThreads, 2) update_tc_ws_gdn_kernel(const Pa
             // [U | o] = d S_0^T W + E'^T (K W) from the tile's slot of tensor memory
             if (!bad) {
                 const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
-                for (int g0 = 0; g0 < NP; g0 += 16) {
-                    float u0[16], cr[16];
-                    tmem_ld16(slot + (b ? 0u : 32u) + (uint32_t)g0, u0);
-                    tmem_ld16(slot + (b ? 32u : 0u) + (uint32_t)g0, cr);
+                const uint32_t s_u0 = slot + (b ? 0u : 32u), s_cr = slot + (b ? 32u : 0u);
+                auto rows = [&](auto bf) {
+                    constexpr bool BF = decltype(bf)::value;
+                    const size_t base = (bh * R) * (size_t)V + j;
+                    for (int g0 = 0; g0 < R; g0 += 16) {
+                        float u0[16], cr[16];
+                        tmem_ld16(s_u0 + (uint32_t)g0, u0);
+                        tmem_ld16(s_cr + (uint32_t)g0, cr);
+                        if (g0 + 16 <= R) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int g = g0 + e;
-                        const float u = fmaf(dtot, u0[e], cr[e]);
-                        if (g < R && p.write_sketch) store_sketch(p, (bh * R + g) * (size_t)V + j, u);
-                        if (g == QA + 8 * b && p.out != nullptr) {
-                            if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
-                            else reinterpret_cast<float*>(p.out)[bh * V + j] = u;
+                            for (int e = 0; e < 16; ++e)
+                                store_sketch_as<BF>(p, base + (size_t)(g0 + e) * V, fmaf(dtot, u0[e], cr[e]));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e)
+                                if (g0 + e < R) store_sketch_as<BF>(p, base + (size_t)(g0 + e) * V, fmaf(dtot, u0[e], cr[e]));
                         }
                     }
+                };
+                if (p.write_sketch) {
+                    if (p.sketch_bf16) rows(std::true_type{}); else rows(std::false_type{});
+                }
+                if (p.out != nullptr) {       // exact output: the query column of this tile's group
+                    const uint32_t qc = (uint32_t)(QA + 8 * b);
+                    float ou, oc;
+                    tmem_ld1x2(s_u0 + qc, s_cr + qc, ou, oc);
+                    const float o = fmaf(dtot, ou, oc);
+                    if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(o);
+                    else reinterpret_cast<float*>(p.out)[bh * V + j] = o;
                 }
                 tc_fence_before();
                 __syncwarp();

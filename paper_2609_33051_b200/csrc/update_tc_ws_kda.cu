@@ -29,6 +29,7 @@
 // on the pass-B group, between the write-back of one tile and the next, so that the pass-A group only streams.
 //
 // Domain: KDA, bf16 I/O, K = V = 128, rank <= 16; 1..32 tokens per pass, up to 64 tokens per flush in blocks of 32.
+#include <type_traits>
 #include "internal.cuh"
 #include "lanegroup.cuh"
 #include "tc_common.cuh"
@@ -411,20 +412,32 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             // [U | o] = S_0^T (G_n * W) + E^T (Ktil W) from the tile's slot of tensor memory: [correction 32 | U0 32]
             if (!bad) {
                 const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
-                for (int g0 = 0; g0 < NP; g0 += 16) {
-                    float u0[16], cr[16];
-                    tmem_ld16(slot + 32u + (uint32_t)g0, u0);
-                    tmem_ld16(slot + (uint32_t)g0, cr);
+                auto rows = [&](auto bf) {
+                    constexpr bool BF = decltype(bf)::value;
+                    const size_t base = (bh * R) * (size_t)V + j;
+                    for (int g0 = 0; g0 < R; g0 += 16) {
+                        float u0[16], cr[16];
+                        tmem_ld16(slot + 32u + (uint32_t)g0, u0);
+                        tmem_ld16(slot + (uint32_t)g0, cr);
+                        if (g0 + 16 <= R) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int g = g0 + e;
-                        const float u = u0[e] + cr[e];
-                        if (g < R && p.write_sketch) store_sketch(p, (bh * R + g) * (size_t)V + j, u);
-                        if (g == QA && p.out != nullptr) {
-                            if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(u);
-                            else reinterpret_cast<float*>(p.out)[bh * V + j] = u;
+                            for (int e = 0; e < 16; ++e) store_sketch_as<BF>(p, base + (size_t)(g0 + e) * V, u0[e] + cr[e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e)
+                                if (g0 + e < R) store_sketch_as<BF>(p, base + (size_t)(g0 + e) * V, u0[e] + cr[e]);
                         }
                     }
+                };
+                if (p.write_sketch) {
+                    if (p.sketch_bf16) rows(std::true_type{}); else rows(std::false_type{});
+                }
+                if (p.out != nullptr) {       // exact output: the query column
+                    float ou, oc;
+                    tmem_ld1x2(slot + 32u + (uint32_t)QA, slot + (uint32_t)QA, ou, oc);
+                    const float o = ou + oc;
+                    if (p.out_bf16) reinterpret_cast<__nv_bfloat16*>(p.out)[bh * V + j] = __float2bfloat16_rn(o);
+                    else reinterpret_cast<float*>(p.out)[bh * V + j] = o;
                 }
                 tc_fence_before();
                 __syncwarp();
