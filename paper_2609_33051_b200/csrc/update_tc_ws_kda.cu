@@ -40,8 +40,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kKThreads = 448;       // pass-A group (4 warps), front group (4 warps), MMA issue warp, state-load warp, pass-B group (4 warps)
-constexpr int kKGrp = 128;
+constexpr int kKThreads = 576;       // pass-A group (4 warps), front group part 1 (4 warps), MMA issue warp, state-load warp, pass-B group (4 warps), front group part 2 (4 warps)
+constexpr int kKFront = 256;         // threads of the front group
 constexpr int kNT = 32;              // tokens per pass
 constexpr int kKStages = 8;          // upper bound on the shared-memory stages of state rows
 constexpr int kAS = 36;              // (sizes the work area of A: 32 rows of 36 floats)
@@ -91,7 +91,6 @@ enum { kPro = 0, kPfull = 2, kTfull = 4, kBdone = 6, kBufFree = 8, kA2free = 10,
 __device__ __forceinline__ void k_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void k_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 __device__ __forceinline__ bool k_or(int id, bool flag) {
     uint32_t r;
     asm volatile(
@@ -104,13 +103,22 @@ __device__ __forceinline__ bool k_or(int id, bool flag) {
         : "memory");
     return r != 0;
 }
-// group-wide bounded wait: one warp polls, the others sleep in the named barrier
-__device__ __forceinline__ bool k_wait(int id, int gt, uint64_t* bar, uint32_t phase) {
+// the same for the 256 threads of the front group (named barrier 2)
+__device__ __forceinline__ void f_sync() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
+__device__ __forceinline__ bool f_wait(int ft, uint64_t* bar, uint32_t phase) {
     bool bad = false;
-    if (gt < 32) bad = !mbar_wait_bounded(bar, phase);
-    return !k_or(id, bad);
+    if (ft < 32) bad = !mbar_wait_bounded(bar, phase);
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 2, 256, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(bad ? 1u : 0u)
+        : "memory");
+    return r == 0;
 }
-
 __device__ __forceinline__ void k_ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -287,7 +295,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             bad = true;
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 103);
-    } else if (warp >= 10) {
+    } else if (warp >= 10 && warp < 14) {
         // =========================== pass-B group: S_new written back, then the sketch rows ===========================
         uint32_t phT = 0, phP = 0;
         bool bad = false;
@@ -566,16 +574,21 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         }
         if (bad && lane == 0) record_fault(p.status, kFaultUpdateWait, 107);
     } else {
-        // =========================== front group: ring-only operands, tile claiming; thread = channel ===========================
-        const int fwarp = gt >> 5;
-        const int i = gt;                     // this thread's channel
+        // =========================== front group: ring-only operands, tile claiming ===========================
+        // 256 threads: thread = (token block fg, channel i).  Block fg holds tokens 16 fg .. 16 fg + 15 of the pass: its
+        // threads build that block's triangle of A, its rows of Khat / Ktil and its rescaled keys, so that the two
+        // halves of a tile's ring-only work run side by side.
+        const int ft = warp < 8 ? tid - 128 : tid - (kKThreads - 128) + 128;      // 0..255 (warps 4-7, then the last four warps)
+        const int fg = ft >> 7;               // token block
+        const int i = ft & 127;               // this thread's channel
+        const int fw = ft >> 5;               // warp of the group, 0..7
         uint32_t phS = 0;
         bool dead = false;
         float* sA = reinterpret_cast<float*>(smem + sm.mats);
         float* sBeta = sA + kNT * kAS;
         float* sOm = reinterpret_cast<float*>(smem + sm.om);
         int cur_h = -1;
-        float* sPart = reinterpret_cast<float*>(sStg + 2u * kZHalf);   // [4 warps][8 batches][32] partial pair sums (over the value rows, copied out by then)
+        float* sPart = reinterpret_cast<float*>(sStg + 2u * kZHalf);   // [8 warps][4 batches][32] partial pair sums (over the value rows, copied out by then)
 
         // ---- tile claiming (thread 0 of the group): per-head-index counters behind the status words ----
         int* sched = p.status + kStatusInts;
@@ -605,11 +618,11 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             *seq_pub = k + 1;
         };
 
-        // One bulk copy per thread from per-thread constants, spread over the four warps of the group: copy number c belongs
-        // to lane c / 4 of warp c % 4.  0..3: ring keys, decays, values, gates; 4..7: the token's key, decay, value, the query.
+        // One bulk copy per thread from per-thread constants, spread over the first four warps of the group: copy number c
+        // belongs to lane c / 4 of warp c % 4.  0..3: ring keys, decays, values, gates; 4..7: the token's key, decay, value, the query.
         const uint32_t stg_beta_bytes = n_ring > 0 ? (uint32_t)(p.L * 4) : 0u;
         const uint32_t stg_bytes = (uint32_t)n_ring * 768u + stg_beta_bytes + (p.has_token ? 768u : 0u) + (p.q != nullptr ? 256u : 0u);
-        const int cp_c = (gt & 31) < 2 ? (gt & 31) * 4 + (gt >> 5) : 32;
+        const int cp_c = (ft < 128 && (ft & 31) < 2) ? (ft & 31) * 4 + (ft >> 5) : 32;
         const unsigned char* cp_base = nullptr;
         size_t cp_stride = 0;
         uint32_t cp_dst = 0, cp_bytes = 0;
@@ -627,37 +640,37 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         auto stage_tile = [&](int tile) {       // whole group
             const int h = tile / tiles_per_h, bb = tile - h * tiles_per_h;
             const size_t bw = (size_t)bb * H + h;
-            if (gt == 0) mbar_expect_tx(&bars[kStg], stg_bytes);      // (the phase cannot complete before this arrival, whatever the order of the copies)
+            if (ft == 0) mbar_expect_tx(&bars[kStg], stg_bytes);      // (the phase cannot complete before this arrival, whatever the order of the copies)
             __syncwarp();
             if (cp_bytes) bulk_g2s(sStg + cp_dst, cp_base + bw * cp_stride, cp_bytes, &bars[kStg]);
         };
         auto next_tile = [&](int k) {          // whole group
-            if (gt == 0) {
+            if (ft == 0) {
                 const int nxt = claim_resolve();
                 publish(k, nxt);
                 if (nxt >= 0) claim_issue();
             }
-            k_sync(2);                         // the published entry is the hand-off to the other threads
+            f_sync();                          // the published entry is the hand-off to the other threads
             const int nxt = seq_ring[k & 3];
             if (nxt >= 0) stage_tile(nxt);
         };
         // the first tile: claimed, published and its rows requested before anything else
-        if (gt == 0) claim_issue();
+        if (ft == 0) claim_issue();
         next_tile(0);
         // operand rows that no tile overwrites hold zeros: the padding columns of [Omega | q] in both windows, and the
         // padding columns of Ktil W in both sets
-        for (uint32_t o = (uint32_t)gt * 16u; o < 2u * sm.w_stride; o += kKGrp * 16u)
+        for (uint32_t o = (uint32_t)ft * 16u; o < 2u * sm.w_stride; o += kKFront * 16u)
             *reinterpret_cast<uint4*>(smem + sm.w + o) = make_uint4(0, 0, 0, 0);
         for (int sb = 0; sb < 2; ++sb)
-            for (uint32_t o = (uint32_t)gt * 16u; o < 4096u; o += kKGrp * 16u)
+            for (uint32_t o = (uint32_t)ft * 16u; o < 4096u; o += kKFront * 16u)
                 *reinterpret_cast<uint4*>(set_ptr(sb) + sm.set_bc + o) = make_uint4(0, 0, 0, 0);
-        k_sync(2);
+        f_sync();
 
         for (int k = 0; !dead; ++k) {
             const int raw_tile = seq_get(k);
             if (raw_tile < 0) {
                 if (raw_tile < -1) {
-                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 108);
+                    if (ft == 0) record_fault(p.status, kFaultUpdateWait, 108);
                     dead = true;
                 }
                 break;
@@ -671,11 +684,11 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
 
             // gate of the current token: requested early
             float tok_beta = 0.f;
-            if (gt < kNT && p.has_token) tok_beta = p.beta[bh];
+            if (ft < kNT && p.has_token) tok_beta = p.beta[bh];
             // Omega of this head index in shared memory (global loads here would sit on the group's critical path)
             if (h != cur_h) {
                 const float* omg = p.omega + (size_t)h * K * R;
-                for (int idx = gt; idx < K * 16; idx += kKGrp) {
+                for (int idx = ft; idx < K * 16; idx += kKFront) {
                     const int kk2 = idx >> 4, g = idx & 15;
                     sOm[idx] = (g < R && p.write_sketch) ? __ldg(omg + (size_t)kk2 * R + g) : 0.f;
                 }
@@ -684,83 +697,91 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             const float* og = sOm + i * 16;
             // the operand set and window of tile k - 2 are free once its Ktil^T E has completed
             if (k >= 2) {
-                if (!k_wait(2, gt, &bars[kTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
-                    if (gt == 0) record_fault(p.status, kFaultUpdateWait, 109);
+                if (!f_wait(ft, &bars[kTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
+                    if (ft == 0) record_fault(p.status, kFaultUpdateWait, 109);
                     dead = true;
                     break;
                 }
             }
             // the staged rows, gates and query row of this tile must have landed
-            if (!k_wait(2, gt, &bars[kStg], phS)) {
-                if (gt == 0) record_fault(p.status, kFaultUpdateWait, 106);
+            if (!f_wait(ft, &bars[kStg], phS)) {
+                if (ft == 0) record_fault(p.status, kFaultUpdateWait, 106);
                 dead = true;
                 break;
             }
             phS ^= 1;
 
-            // ---- column i of the key and decay rows into registers; value rows into the set; gates ----
-            float kk[kNT], gg[kNT];
+            // ---- column i of this block's key and decay rows into registers, the product of the other block's decays;
+            // value rows into the set; gates ----
+            const int t0 = 16 * fg;
+            float kk[16], gg[16];
 #pragma unroll
-            for (int s = 0; s < kNT; ++s) {
-                const bool on = s < n_tot;
-                kk[s] = on ? bf16_at(sStg, (uint32_t)(s * K + i)) : 0.f;
-                gg[s] = on ? bf16_at(sStg + sm.stg_g, (uint32_t)(s * K + i)) : 1.f;
+            for (int s = 0; s < 16; ++s) {
+                const bool on = t0 + s < n_tot;
+                kk[s] = on ? bf16_at(sStg, (uint32_t)((t0 + s) * K + i)) : 0.f;
+                gg[s] = on ? bf16_at(sStg + sm.stg_g, (uint32_t)((t0 + s) * K + i)) : 1.f;
+            }
+            float gother = 1.f;
+#pragma unroll
+            for (int s = 0; s < 16; ++s) {
+                const int t = 16 * (1 - fg) + s;
+                if (t < n_tot) gother *= bf16_at(sStg + sm.stg_g, (uint32_t)(t * K + i));
             }
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const int idx = gt + r * kKGrp;            // 512 vectors of 16 bytes: 32 value rows
+            for (int r = 0; r < 2; ++r) {
+                const int idx = ft + r * kKFront;          // 512 vectors of 16 bytes: 32 value rows
                 uint4 vv = make_uint4(0, 0, 0, 0);
                 if ((idx >> 4) < n_tot) vv = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)idx * 16);
                 *reinterpret_cast<uint4*>(set + sm.set_vv + (size_t)idx * 16) = vv;
             }
             const float q_i = p.q != nullptr ? bf16_at(sStg + sm.stg_q, (uint32_t)i) : 0.f;
-            if (gt < kNT) {
-                const int s = gt;
+            if (ft < kNT) {
+                const int s = ft;
                 float bt = 0.f;
                 if (s < n_ring) bt = reinterpret_cast<const float*>(sStg + sm.stg_beta)[p.tok_base + s];
                 else if (s < n_tot) bt = tok_beta;
                 sBeta[s] = bt;
             }
-            k_sync(2);                 // every thread holds its column: the key / decay rows of the staging area are free
+            f_sync();                  // every thread holds its column: the key / decay rows of the staging area are free
 
-            // ---- pair sums inside each block of 16 tokens (the two triangles of A): A_sj = sum_i k_s[i] k_j[i]
+            // ---- pair sums inside this block of 16 tokens (its triangle of A): A_sj = sum_i k_s[i] k_j[i]
             // prod_{j<m<=s} g_m[i] as per-channel products, reduced over the 32 channels of a warp by a transposing
-            // butterfly, 32 pairs at a time: rows sa and 16 - sa of block 0 in entries 0..15, of block 1 in 16..31 ----
+            // butterfly, 32 pairs at a time: rows sa and 16 - sa in entries 0..15, rows sa + 1 and 15 - sa in 16..31 ----
             {
-                float* part = sPart + (size_t)fwarp * (8 * 32);
+                float* part = sPart + (size_t)fw * 128;
 #pragma unroll
-                for (int sa = 1; sa <= 8; ++sa) {
+                for (int bi = 0; bi < 4; ++bi) {
                     float vals[32];
 #pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
-                        const int b0 = 16 * blk;
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int sa = 2 * bi + 1 + hh, o = 16 * hh;
                         {
-                            float r = kk[b0 + sa];
+                            float r = kk[sa];
 #pragma unroll
                             for (int jj = 7; jj >= 0; --jj)
-                                if (jj < sa) { r *= gg[b0 + jj + 1]; vals[b0 + jj] = r * kk[b0 + jj]; }
+                                if (jj < sa) { r *= gg[jj + 1]; vals[o + jj] = r * kk[jj]; }
                         }
                         if (sa < 8) {
                             const int sb2 = 16 - sa;
-                            float r = kk[b0 + sb2];
+                            float r = kk[sb2];
 #pragma unroll
                             for (int jj = 14; jj >= 0; --jj)
-                                if (jj < sb2) { r *= gg[b0 + jj + 1]; vals[b0 + sa + jj] = r * kk[b0 + jj]; }
+                                if (jj < sb2) { r *= gg[jj + 1]; vals[o + sa + jj] = r * kk[jj]; }
                         } else {
 #pragma unroll
-                            for (int jj = 8; jj < 16; ++jj) vals[b0 + jj] = 0.f;
+                            for (int jj = 8; jj < 16; ++jj) vals[o + jj] = 0.f;
                         }
                     }
                     group_reduce_transpose<32, 32>(vals, lane);      // lane l now holds entry l of the batch
-                    part[(sa - 1) * 32 + lane] = vals[0];
+                    part[bi * 32 + lane] = vals[0];
                 }
             }
 
-            // ---- running products.  Khat -> window rows 0..31; Ktil -> set (MN-major); G_n * W -> window rows 32..;
-            // and for the 16 x 16 block of A that couples the two token blocks, whose decay product splits at the block
-            // boundary without a quotient (prod_{j<m<=s} = prod_{16<=m<=s} * prod_{j<m<=15}), the rescaled keys
-            // X_s = k_s prod_{16<=m<=s} g_m (s >= 16) and Y_j = k_j prod_{j<m<=15} g_m (j < 16) as bf16 hi + lo rows
-            // Z[token][channel] over the (now free) key / decay rows of the staging area ----
+            // ---- running products of this block.  Khat -> window rows 0..31; Ktil -> set (MN-major); G_n * W -> window
+            // rows 32..; and for the 16 x 16 block of A that couples the two token blocks, whose decay product splits at
+            // the block boundary without a quotient (prod_{j<m<=s} = prod_{16<=m<=s} * prod_{j<m<=15}), the rescaled keys
+            // X_s = k_s prod_{16<=m<=s} g_m (s >= 16, by block 1) and Y_j = k_j prod_{j<m<=15} g_m (j < 16, by block 0)
+            // as bf16 hi + lo rows Z[token][channel] over the (now free) key / decay rows of the staging area ----
             {
                 __nv_bfloat16* whi = reinterpret_cast<__nv_bfloat16*>(wb);
                 __nv_bfloat16* wlo = reinterpret_cast<__nv_bfloat16*>(wb + sm.w_lo);
@@ -770,60 +791,64 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 __nv_bfloat16* zlo = reinterpret_cast<__nv_bfloat16*>(sStg + kZHalf);
                 const uint32_t wcol = ((uint32_t)(i >> 3) * LBO_W + (uint32_t)(i & 7) * 2u) >> 1;        // K-major: k = channel
                 const uint32_t bcol = ((uint32_t)(i & 7) * 2u + (uint32_t)(i >> 3) * SBO) >> 1;          // MN-major: mn = channel
-                float G = 1.f, X = 1.f;
+                float G = fg ? gother : 1.f, X = 1.f;
 #pragma unroll
-                for (int s = 0; s < kNT; ++s) {
+                for (int s = 0; s < 16; ++s) {
                     G *= gg[s];
                     __nv_bfloat16 hi, lo;
                     split_bf16(G * kk[s], hi, lo);
-                    const uint32_t o = wcol + (((uint32_t)(s & 7) * 16u + (uint32_t)(s >> 3) * SBO) >> 1);
+                    const uint32_t o = wcol + (((uint32_t)(s & 7) * 16u + (uint32_t)((s >> 3) + 2 * fg) * SBO) >> 1);
                     whi[o] = hi;
                     wlo[o] = lo;
-                    if (s >= 16) {
+                    if (fg) {
                         X *= gg[s];
                         split_bf16(X * kk[s], hi, lo);
-                        zhi[s * (kZPitch / 2) + i] = hi;
-                        zlo[s * (kZPitch / 2) + i] = lo;
+                        zhi[(16 + s) * (kZPitch / 2) + i] = hi;
+                        zlo[(16 + s) * (kZPitch / 2) + i] = lo;
                     }
                 }
-                float Dn = 1.f, Yd = 1.f;
+                const float Gn = fg ? G : G * gother;       // decay of the whole pass
+                float Dn = fg ? 1.f : gother, Yd = 1.f;
 #pragma unroll
-                for (int s = kNT - 1; s >= 0; --s) {
+                for (int s = 15; s >= 0; --s) {
                     const float kt = Dn * kk[s];
                     Dn *= gg[s];
                     __nv_bfloat16 hi, lo;
                     split_bf16(kt, hi, lo);
-                    const uint32_t o = bcol + (((uint32_t)(s & 7) * 16u + (uint32_t)(s >> 3) * LBO_M) >> 1);
+                    const uint32_t o = bcol + (((uint32_t)(s & 7) * 16u + (uint32_t)((s >> 3) + 2 * fg) * LBO_M) >> 1);
                     bthi[o] = hi;
                     btlo[o] = lo;
-                    if (s < 16) {
+                    if (!fg) {
                         split_bf16(Yd * kk[s], hi, lo);
                         zhi[s * (kZPitch / 2) + i] = hi;
                         zlo[s * (kZPitch / 2) + i] = lo;
                         Yd *= gg[s];
                     }
                 }
-                reinterpret_cast<float*>(set + sm.set_gn)[i] = G;
+                if (!fg) reinterpret_cast<float*>(set + sm.set_gn)[i] = Gn;
+                // G_n * [Omega | q]: block 0 takes the first half of the sketch columns, block 1 the rest and the query
+                const int Rh = (R + 1) >> 1;
                 if (p.write_sketch) {
-                    for (int g = 0; g < R; ++g) {
+                    const int g_lo = fg ? Rh : 0, g_hi = fg ? R : Rh;
+                    for (int g = g_lo; g < g_hi; ++g) {
                         __nv_bfloat16 hi, lo;
-                        split_bf16(G * og[g], hi, lo);
+                        split_bf16(Gn * og[g], hi, lo);
                         const uint32_t o = wcol + (((uint32_t)(g & 7) * 16u + (uint32_t)((g >> 3) + 4) * SBO) >> 1);
                         whi[o] = hi;
                         wlo[o] = lo;
                     }
                 }
-                if (p.q != nullptr) {
+                if (fg && p.q != nullptr) {
                     __nv_bfloat16 hi, lo;
-                    split_bf16(G * q_i, hi, lo);
+                    split_bf16(Gn * q_i, hi, lo);
                     const uint32_t o = wcol + (((uint32_t)(QA & 7) * 16u + (uint32_t)((QA >> 3) + 4) * SBO) >> 1);
                     whi[o] = hi;
                     wlo[o] = lo;
                 }
             }
-            k_sync(2);                 // partial pair sums, Z rows and Ktil are complete
+            f_sync();                  // partial pair sums, Z rows and Ktil are complete
 
-            if (fwarp == 3) {
+            if (fw == 7) {
                 // ---- A_21 = X Y^T (16 x 16, tokens 16..31 against tokens 0..15) as mma.sync products of the Z rows,
                 // hi * hi + lo * hi + hi * lo ----
                 float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -855,26 +880,28 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     sA21[(r0 + 8) * 16 + c0 + 1] = acc[nt][3];
                 }
             } else {
-                // ---- beta_s A_sj of the two triangles: the four warps' partials summed in a fixed order ----
-                for (int idx = gt; idx < 2 * 16 * 16; idx += 96) {
+                // ---- beta_s A_sj of the two triangles: the partials of a block's four warps summed in a fixed order ----
+                for (int idx = ft; idx < 2 * 16 * 16; idx += 224) {
                     const int blk = idx >> 8, s = (idx >> 4) & 15, jj = idx & 15;
                     float a = 0.f;
                     if (jj < s) {
                         const int sa = s <= 8 ? s : 16 - s;
-                        const int e = (sa - 1) * 32 + blk * 16 + (s <= 8 ? jj : sa + jj);
-                        a = ((sPart[e] + sPart[256 + e]) + sPart[512 + e]) + sPart[768 + e];
+                        const int e = ((sa - 1) >> 1) * 32 + ((sa - 1) & 1) * 16 + (s <= 8 ? jj : sa + jj);
+                        const float* pp = sPart + blk * 512 + e;
+                        a = ((pp[0] + pp[128]) + pp[256]) + pp[384];
                     }
                     sA[blk * (16 * kAS2) + s * kAS2 + jj] = sBeta[16 * blk + s] * a;
                 }
             }
-            k_sync(2);                 // A is complete
+            f_sync();                  // A is complete
 
-            if (fwarp < 2) {
-                // ---- T_bb = (I + Bd A_bb)^{-1} Bd of block fwarp by forward substitution: one column per thread, in registers ----
+            if ((fw & 3) == 0) {
+                // ---- T_bb = (I + Bd A_bb)^{-1} Bd of block fw / 4 by forward substitution: one column per thread, in registers ----
+                const int blk = fw >> 2;
                 if (lane < 16) {
                     const int c = lane;
-                    const int nb = min(max(n_tot - 16 * fwarp, 0), 16);      // tokens of this block
-                    const float* sAb = sA + fwarp * (16 * kAS2);
+                    const int nb = min(max(n_tot - 16 * blk, 0), 16);      // tokens of this block
+                    const float* sAb = sA + blk * (16 * kAS2);
                     float tcol[16];
 #pragma unroll
                     for (int s = 0; s < 16; ++s) {
@@ -889,78 +916,70 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                         }
                         tcol[s] = (s >= nb || s < c || c >= nb) ? 0.f : (s == c ? 1.f : -acc);
                     }
-                    const float bc = sBeta[16 * fwarp + c];
-                    float* sT = reinterpret_cast<float*>(set + sm.set_t1) + fwarp * 256;
+                    const float bc = sBeta[16 * blk + c];
+                    float* sT = reinterpret_cast<float*>(set + sm.set_t1) + blk * 256;
 #pragma unroll
                     for (int s = 0; s < 16; ++s) sT[s * 16 + c] = tcol[s] * bc;
                 }
             } else {
-                // ---- Ktil W: 16 tokens (block fwarp - 2) x 24 columns of [Omega | q] as mma.sync products.  A: the Ktil
-                // operand just written (its 8 x 8 core matrices are the row-major fragments ldmatrix wants), hi + lo;
-                // B: Omega and q straight from memory into fragments, split into hi + lo in registers ----
-                const int mt = fwarp - 2;
-                float acc[3][4];
-#pragma unroll
-                for (int nt = 0; nt < 3; ++nt)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+                // ---- Ktil W: 16 tokens (block fw / 4) x 8 columns of [Omega | q] (columns 8 nt .., nt = fw % 4 - 1) as
+                // mma.sync products.  A: the Ktil operand just written (its 8 x 8 core matrices are the row-major fragments
+                // ldmatrix wants), hi + lo; B: Omega and q from shared memory into fragments, split into hi + lo in registers ----
+                const int mt = fw >> 2, nt = (fw & 3) - 1;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t btb = smem_u32(set + sm.set_bt);
                 const uint32_t a_row = btb + (uint32_t)(2 * mt + ((lane >> 3) & 1)) * LBO_M + (uint32_t)(lane >> 4) * SBO + (uint32_t)(lane & 7) * 16u;
                 const __nv_bfloat16* sq = reinterpret_cast<const __nv_bfloat16*>(sStg + sm.stg_q);
                 const int ncol = p.write_sketch ? R : 0;
                 const bool has_q = p.q != nullptr;
+                const int g = nt * 8 + (lane >> 2);
+                const int src = g < ncol ? 0 : (g == QA && has_q) ? 1 : 2;       // Omega column, query, padding
+#pragma unroll 4
                 for (int ks = 0; ks < K / 16; ++ks) {
                     uint32_t ahi[4], alo[4];
                     k_ldmatrix_x4(a_row + (uint32_t)(2 * ks) * SBO, ahi);
                     k_ldmatrix_x4(a_row + sm.set_bt_lo + (uint32_t)(2 * ks) * SBO, alo);
                     const int i0 = ks * 16 + (lane & 3) * 2;
-#pragma unroll
-                    for (int nt = 0; nt < 3; ++nt) {
-                        const int g = nt * 8 + (lane >> 2);
-                        float w[4] = {0.f, 0.f, 0.f, 0.f};
-                        if (g < ncol) {
-                            w[0] = sOm[i0 * 16 + g];
-                            w[1] = sOm[(i0 + 1) * 16 + g];
-                            w[2] = sOm[(i0 + 8) * 16 + g];
-                            w[3] = sOm[(i0 + 9) * 16 + g];
-                        } else if (g == QA && has_q) {
-                            w[0] = __bfloat162float(sq[i0]);
-                            w[1] = __bfloat162float(sq[i0 + 1]);
-                            w[2] = __bfloat162float(sq[i0 + 8]);
-                            w[3] = __bfloat162float(sq[i0 + 9]);
-                        }
-                        uint32_t bhi[2], blo[2];
-                        split_bf16x2(w[0], w[1], bhi[0], blo[0]);
-                        split_bf16x2(w[2], w[3], bhi[1], blo[1]);
-                        k_mma_16816(acc[nt], ahi, bhi);
-                        k_mma_16816(acc[nt], alo, bhi);
-                        k_mma_16816(acc[nt], ahi, blo);
+                    float w[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (src == 0) {
+                        w[0] = sOm[i0 * 16 + g];
+                        w[1] = sOm[(i0 + 1) * 16 + g];
+                        w[2] = sOm[(i0 + 8) * 16 + g];
+                        w[3] = sOm[(i0 + 9) * 16 + g];
+                    } else if (src == 1) {
+                        w[0] = __bfloat162float(sq[i0]);
+                        w[1] = __bfloat162float(sq[i0 + 1]);
+                        w[2] = __bfloat162float(sq[i0 + 8]);
+                        w[3] = __bfloat162float(sq[i0 + 9]);
                     }
+                    uint32_t bhi[2], blo[2];
+                    split_bf16x2(w[0], w[1], bhi[0], blo[0]);
+                    split_bf16x2(w[2], w[3], bhi[1], blo[1]);
+                    k_mma_16816(acc, ahi, bhi);
+                    k_mma_16816(acc, alo, bhi);
+                    k_mma_16816(acc, ahi, blo);
                 }
                 __nv_bfloat16* bchi = reinterpret_cast<__nv_bfloat16*>(set + sm.set_bc);
                 __nv_bfloat16* bclo = bchi + 1024;
-                auto put = [&](int s, int g, float x) {
+                auto put = [&](int s, int gc, float x) {
                     __nv_bfloat16 hi, lo;
                     split_bf16(x, hi, lo);
-                    const uint32_t o2 = ((uint32_t)(g & 7) * 16u + (uint32_t)(g >> 3) * SBO + (uint32_t)(s >> 3) * LBO_C + (uint32_t)(s & 7) * 2u) >> 1;
+                    const uint32_t o2 = ((uint32_t)(gc & 7) * 16u + (uint32_t)(gc >> 3) * SBO + (uint32_t)(s >> 3) * LBO_C + (uint32_t)(s & 7) * 2u) >> 1;
                     bchi[o2] = hi;
                     bclo[o2] = lo;
                 };
-#pragma unroll
-                for (int nt = 0; nt < 3; ++nt) {
-                    const int s0 = 16 * mt + (lane >> 2), g0 = nt * 8 + (lane & 3) * 2;
-                    put(s0, g0, acc[nt][0]);
-                    put(s0, g0 + 1, acc[nt][1]);
-                    put(s0 + 8, g0, acc[nt][2]);
-                    put(s0 + 8, g0 + 1, acc[nt][3]);
-                }
+                const int s0 = 16 * mt + (lane >> 2), g0 = nt * 8 + (lane & 3) * 2;
+                put(s0, g0, acc[0]);
+                put(s0, g0 + 1, acc[1]);
+                put(s0 + 8, g0, acc[2]);
+                put(s0 + 8, g0 + 1, acc[3]);
             }
             proxy_fence();         // operand sets and windows are read by MMAs (async proxy)
-            k_sync(2);
-            if (gt == 0) k_arrive(&bars[kPro + b]);
+            f_sync();
+            if (ft == 0) k_arrive(&bars[kPro + b]);
             next_tile(k + 1);      // the staging area has been read: the next tile's rows may come in
         }
-        if (gt == 0) {     // scheduler counters back to zero once every CTA is done claiming
+        if (ft == 0) {     // scheduler counters back to zero once every CTA is done claiming
             __threadfence();
             if (atomicAdd(&sched[0], 1) == (int)gridDim.x - 1) {
                 for (int hh = 0; hh < H; ++hh) cnt[hh] = 0;
