@@ -11,22 +11,25 @@
 //     [U | o] = S_0^T (G_n * [Omega | q]) + E^T (Ktil [Omega | q])         (Eq. 7 and the exact output of the flush step)
 // No quotient of cumulative decays is ever formed (they underflow within a window on real gates).
 //
-// Same schedule as the gated-delta-rule kernel: tile = one head (K = V = 128), TMEM lane = value column; the state is
-// read once by bulk copies into a ring of shared-memory stages; the pass-A group splits the S_0 chunks into bf16 hi + lo,
-// leaves G_n * S_0 in the accumulator of Ktil^T E (tcgen05.st); one thread issues every MMA; the pass-B
-// group forms E, writes the accumulator (S_new) back and stores the sketch rows; the front group builds the ring-only operands two
-// tiles ahead.  What differs: up to 32 tokens per pass (the MMAs over tokens take two k-steps), both key operands and the
-// basis operand are per tile and carry hi + lo halves, so the B operand of pass A is a double-buffered per-tile window
-// [Khat (32 rows) | G_n * [Omega | q] (32 rows)], and the kernel runs one CTA per SM.
+// Tile = one head (K = V = 128), TMEM lane = value column; the state is read once by bulk copies into a ring of
+// shared-memory stages; the pass-A group splits the S_0 chunks into bf16 hi + lo and leaves G_n * S_0 in the accumulator
+// of Ktil^T E (tcgen05.st); one thread issues every MMA; the pass-B group forms E, writes the accumulator (S_new) back
+// and stores the sketch rows; the front group builds the ring-only operands two tiles ahead.  Up to 32 tokens per pass
+// (the MMAs over tokens take two k-steps); both key operands and the basis operand are per tile and carry hi + lo
+// halves, so the B operand of pass A is a double-buffered per-tile window [Khat (32 rows) | G_n * [Omega | q] (32 rows)].
+// The kernel runs one CTA per SM (shared memory) and owns all 512 columns of tensor memory: two 64-column slots
+// [P | U0] and two 128-column accumulators for alternating tiles, so pass A of tile k + 1 (issued before the E step of
+// tile k) never waits for the write-back of tile k.
 //
-// Front group, thread = channel i: reads column i of the staged key and decay rows into registers, forms the running
-// products and writes Khat / Ktil / G_n * W in the operand layouts.  The 32 x 32 system is handled as two blocks of 16
-// tokens: the 2 x 120 pair sums inside the blocks are per-channel products reduced over the 128 channels by transposing
-// butterflies (per-warp partials summed in a fixed order: results are bitwise reproducible); the 16 x 16 block that
-// couples the two blocks is an mma.sync product of rescaled keys (the decay product splits at the block boundary without
-// a quotient); T_11 and T_22 by forward substitution (one column per thread, two warps) while two warps form
-// Ktil [Omega | q] with mma.sync.  The E step (E_1 = T_11 x_1, E_2 = T_22 (x_2 - A_21 E_1), 528 multiply-adds per lane) runs
-// on the pass-B group, between the write-back of one tile and the next, so that the pass-A group only streams.
+// Front group, 256 threads, thread = (token block, channel i): reads column i of its block's staged key and decay rows
+// into registers, forms the running products and writes its rows of Khat / Ktil / G_n * W in the operand layouts.  The
+// 32 x 32 system is handled as two blocks of 16 tokens: the 120 pair sums inside a block are per-channel products of
+// that block's threads reduced over the 128 channels by transposing butterflies (per-warp partials summed in a fixed
+// order: results are bitwise reproducible); the 16 x 16 block that couples the two blocks is an mma.sync product of
+// rescaled keys (the decay product splits at the block boundary without a quotient); T_11 and T_22 by forward
+// substitution (one column per thread, one warp each) while six warps form Ktil [Omega | q] with mma.sync.  The E step
+// (E_1 = T_11 x_1, E_2 = T_22 (x_2 - A_21 E_1), 528 multiply-adds per lane) runs on the pass-B group, between the
+// write-back of one tile and the next, so that the pass-A group only streams.
 //
 // Domain: KDA, bf16 I/O, K = V = 128, rank <= 16; 1..32 tokens per pass, up to 64 tokens per flush in blocks of 32.
 #include <type_traits>
@@ -48,6 +51,9 @@ constexpr int kAS = 36;              // (sizes the work area of A: 32 rows of 36
 constexpr int kAS2 = 20;             // row stride (floats) of the two 16 x 16 triangles of A
 constexpr uint32_t kZPitch = 272u;   // bytes between the rows of the rescaled keys Z[token][channel]: 256 + 16, so that the 8 rows of an ldmatrix fall in different banks
 constexpr uint32_t kZHalf = 32u * kZPitch;   // hi rows, then lo rows
+// Pass-A window [Khat 32 | G_n * W 32]: 64 rows of 16 bytes per group of 8 channels, the groups 16 bytes further apart than
+// they need to be, so that the per-channel threads of a warp (4 groups) store to different banks
+constexpr uint32_t kLboW = 64u * 16u + 16u;
 constexpr int kKA2 = 2;              // chunk buffers between the pass-A group and the MMA issue warp
 constexpr int kNPk = 32;             // columns of [Omega | q]: Omega in 0..R-1, q at column QA = round_up(R, 8) <= 16
 
@@ -62,7 +68,7 @@ __host__ __device__ inline KSmem make_ksmem(int stages) {
     s.a2 = off; off += (uint32_t)kKA2 * 2u * 128u * 16u * 2u;     // 16-row chunk buffers, hi + lo
     s.e = off; off += 2u * 128u * (uint32_t)kNT * 2u;             // E hi + lo: A operand of Ktil^T E (128 x 32 tokens each)
     // B operand of pass A, per tile and double-buffered: 64 rows [Khat (32) | G_n * [Omega | q] (32)] x 128 channels, hi then lo
-    s.w = off; s.w_lo = 64u * kK * 2u; s.w_stride = 2u * s.w_lo; off += 2u * s.w_stride;
+    s.w = off; s.w_lo = (uint32_t)(kK / 8) * kLboW; s.w_stride = 2u * s.w_lo; off += 2u * s.w_stride;
     // per-tile operand set, double-buffered: Ktil as B operand of Ktil^T E (MN-major, hi | lo), raw value rows, T,
     // Ktil [Omega | q] hi | lo (B operand of the sketch correction), G_n
     s.set = off;
@@ -91,19 +97,8 @@ enum { kPro = 0, kPfull = 2, kTfull = 4, kBdone = 6, kBufFree = 8, kA2free = 10,
 __device__ __forceinline__ void k_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool k_or(int id, bool flag) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 q, %2, 0;\n\t"
-        "bar.red.or.pred p, %1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r)
-        : "r"(id), "r"(flag ? 1u : 0u)
-        : "memory");
-    return r != 0;
-}
-// the same for the 256 threads of the front group (named barrier 2)
+// named barrier 2 over the 256 threads of the front group, and a group-wide bounded wait: one warp polls, the others
+// sleep in the barrier
 __device__ __forceinline__ void f_sync() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
 __device__ __forceinline__ bool f_wait(int ft, uint64_t* bar, uint32_t phase) {
     bool bad = false;
@@ -154,7 +149,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + sm.misc);
     unsigned char* sStg = smem + sm.stg;
 
-    constexpr uint32_t tmem_cols = 256u;
+    constexpr uint32_t tmem_cols = 512u;          // one CTA per SM (shared memory): two slots of 64 columns, two accumulators of 128
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(tmem_cols)
@@ -165,7 +160,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         *reinterpret_cast<volatile int*>(smem + sm.misc + 32) = 0;
         for (int i = 0; i < kNumBars; ++i) {
             // one arrival per warp of a stream group: chunk ready, E ready, stage empty, accumulator halves, pass-B done, slot free
-            const bool per_warp = (i >= kA2rdy && i <= kErdy) || i == kStDone || i >= kEmpty || (i >= kBdone && i < kBdone + 4);
+            const bool per_warp = (i >= kA2rdy && i <= kErdy) || i == kStDone || i == kStDone + 1 || i >= kEmpty || (i >= kBdone && i < kBdone + 4);
             mbar_init(&bars[i], per_warp ? 4 : 1);
         }
         mbar_fence_init();
@@ -186,7 +181,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
     //   K-major : elem(mn, k) at (mn%8)*16 + (mn/8)*128 + (k/8)*LBO + (k%8)*2,  LBO = 16*MN
     //   MN-major: elem(mn, k) at (k%8)*16 + (mn%8)*2 + (mn/8)*128 + (k/8)*2048
     constexpr uint32_t SBO = 128, LBO_M = 2048;
-    constexpr uint32_t LBO_W = 64u * 16u;                 // pass-A window: 64 rows
+    constexpr uint32_t LBO_W = kLboW;                     // pass-A window: 64 rows (+ 16 bytes of padding)
     constexpr uint32_t LBO_C = (uint32_t)NP * 16u;        // Ktil W: 32 rows
 
     const int tiles_per_h = B;
@@ -216,16 +211,15 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         bool bad = false;
 
         uint32_t phTf = 0;
-        // pass A of a tile with operand set b; `later`: not the CTA's first tile, so the Ktil^T E accumulator still holds
-        // the tile before until the pass-B group has read it (half by half)
-        auto pass_a = [&](int b, bool later) {
+        // pass A of the CTA's tile number kt with operand set b = kt & 1; the Ktil^T E accumulator b still holds tile kt - 2
+        // until the pass-B group has read it
+        auto pass_a = [&](int b, int kt) {
             const float* sGn = reinterpret_cast<const float*>(set_ptr(b) + sm.set_gn);
 #pragma unroll 2
             for (int c = 0; c < NCH; ++c) {
-                if (later && (c == 0 || c == NCH / 2)) {
-                    const int hf = c ? 1 : 0;
-                    bad |= !mbar_wait_bounded(&bars[kTfree + hf], (phTf >> hf) & 1u);
-                    phTf ^= 1u << hf;
+                if (c == 0 && kt >= 2) {
+                    bad |= !mbar_wait_bounded(&bars[kTfree + b], (phTf >> b) & 1u);
+                    phTf ^= 1u << b;
                     tc_fence_after();
                 }
                 bad |= !mbar_wait_bounded(&bars[kFull + stage], phF);
@@ -245,7 +239,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                         ds[i4 * 4 + 2] = g4.z * s0[i4 * 4 + 2];
                         ds[i4 * 4 + 3] = g4.w * s0[i4 * 4 + 3];
                     }
-                    if (!bad) tmem_st16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), ds);
+                    if (!bad) tmem_st16(tmem_base + 128u + (uint32_t)b * 128u + lane_sel + (uint32_t)(c * CH), ds);
                 }
                 const int ab = c & (kKA2 - 1);
                 if (gc >= kKA2) {     // the chunk buffer was read by the MMAs issued kKA2 chunks ago
@@ -272,7 +266,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             tmem_st_wait();            // this warp's G_n * S_0 columns are in tensor memory
             tc_fence_before();
             bad = __any_sync(0xffffffffu, bad);
-            if (lane == 0 && !bad) k_arrive(&bars[kStDone]);
+            if (lane == 0 && !bad) k_arrive(&bars[kStDone + b]);
         };
         auto wait_pro = [&](int b) {
             bad |= !mbar_wait_bounded(&bars[kPro + b], (phPro >> b) & 1u);
@@ -282,14 +276,14 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         int cur = seq_get(0);
         if (cur >= 0) {
             wait_pro(0);
-            pass_a(0, false);
+            pass_a(0, 0);
             for (int k = 0; !bad; ++k) {
                 const int b = k & 1;
                 const int raw = seq_get(k + 1);
                 if (raw < -1) { bad = true; break; }
                 if (raw < 0) break;
                 wait_pro(b ^ 1);
-                pass_a(b ^ 1, true);
+                pass_a(b ^ 1, k + 1);
             }
         } else if (cur < -1) {
             bad = true;
@@ -404,19 +398,17 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
             for (int c = 0; c < NCH; ++c) {
                 if (!bad) {
                     float t[CH];
-                    tmem_ld16(tmem_base + 128u + lane_sel + (uint32_t)(c * CH), t);
-                    if (c == NCH / 2 - 1 || c == NCH - 1) {      // this warp is done with a half of the accumulator
+                    tmem_ld16(tmem_base + 128u + (uint32_t)b * 128u + lane_sel + (uint32_t)(c * CH), t);
+                    if (c == NCH - 1) {      // this warp is done with the accumulator: pass A of tile k + 2 may overwrite it
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) k_arrive(&bars[kTfree + (c == NCH - 1 ? 1 : 0)]);
+                        if (lane == 0) k_arrive(&bars[kTfree + b]);
                     }
 #pragma unroll
                     for (int ii = 0; ii < CH; ++ii) So[(size_t)(c * CH + ii) * V] = t[ii];
                 }
             }
-            tc_fence_before();
             bad = __any_sync(0xffffffffu, bad);
-            if (lane == 0 && !bad) k_arrive(&bars[kBdone + b]);
             // [U | o] = S_0^T (G_n * W) + E^T (Ktil W) from the tile's slot of tensor memory: [correction 32 | U0 32]
             if (!bad) {
                 const uint32_t slot = tmem_base + (uint32_t)b * 64u + lane_sel;
@@ -463,48 +455,17 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
         if (lane == 0) {
             uint32_t phR = 0, phE = 0, phBuf = 0, phSt = 0;
             bool bad = false;
-            int where = 104;                // which wait gave up (status detail): 141 slot free, 142 chunk ready, 143 E ready, 144 accumulator read
+            int where = 104;                // which wait gave up (status detail): 141 slot free, 142 chunk ready, 143 E ready, 145 accumulator written
             const uint32_t a2base = smem_u32(smem + sm.a2);
-            // [P | U0](b) = S_0^T [Khat^T | G_n * W] chunk by chunk: one 64-row window per tile
-            auto pass_a = [&](int k) {
-                const int b = k & 1;
-                if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
-                    if (!mbar_wait_bounded(&bars[kBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 141; return; }
-                    phBuf ^= 1u << b;
-                    tc_fence_after();
-                }
-                const uint32_t slot = tmem_base + (uint32_t)b * 64u;
-                const uint32_t whi0 = smem_u32(w_ptr(b));
-                const uint32_t wlo0 = whi0 + sm.w_lo;
-#pragma unroll 2
-                for (int c = 0; c < NCH; ++c) {
-                    const int ab = c & (kKA2 - 1);
-                    if (!mbar_wait_bounded(&bars[kA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 142; return; }
-                    phR ^= 1u << ab;
-                    tc_fence_after();
-                    const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
-                    const uint64_t ahi = make_desc(a2, LBO_M, SBO);
-                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
-                    const uint64_t whi = make_desc(whi0 + (uint32_t)(c * (CH / 8)) * LBO_W, LBO_W, SBO);
-                    const uint64_t wlo = make_desc(wlo0 + (uint32_t)(c * (CH / 8)) * LBO_W, LBO_W, SBO);
-                    tc_mma_bf16(slot, ahi, whi, idescA, c ? 1u : 0u);
-                    tc_mma_bf16(slot, alo, whi, idescA, 1u);
-                    tc_mma_bf16(slot, ahi, wlo, idescA, 1u);
-                    tc_commit(&bars[kA2free + ab]);
-                    if (c == NCH - 1) tc_commit(&bars[kPfull + b]);
-                }
-            };
             auto step_e = [&](int k) {          // Ktil^T E onto G_n * S_0 (128 columns) and the sketch correction E^T (Ktil W) over the spent P
                 const int b = k & 1;
                 if (!mbar_wait_bounded(&bars[kErdy], phE)) { bad = true; where = 143; return; }
                 phE ^= 1u;
-                if (!mbar_wait_bounded(&bars[kStDone], phSt)) { bad = true; where = 145; return; }       // G_n * S_0 is in the accumulator
-                phSt ^= 1u;
-                if (k >= 1) {                   // the pass-B group must have read the accumulator of the tile before
-                    if (!mbar_wait_bounded(&bars[kBdone + (b ^ 1)], (uint32_t)((k - 1) >> 1) & 1u)) { bad = true; where = 144; return; }
-                }
+                // G_n * S_0 is in accumulator b (the pass-A group stored it after the pass-B group had read tile k - 2 from it)
+                if (!mbar_wait_bounded(&bars[kStDone + b], (phSt >> b) & 1u)) { bad = true; where = 145; return; }
+                phSt ^= 1u << b;
                 tc_fence_after();
-                const uint32_t tmem_t = tmem_base + 128u;
+                const uint32_t tmem_t = tmem_base + 128u + (uint32_t)b * 128u;
                 const uint32_t tmem_c = tmem_base + (uint32_t)b * 64u;
                 const uint32_t e = smem_u32(smem + sm.e);
                 const uint32_t bt = smem_u32(set_ptr(b) + sm.set_bt);
@@ -525,16 +486,63 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 }
                 tc_commit(&bars[kTfull + b]);
             };
+            // The E step of a tile is issued as soon as its E operand is ready, also in the middle of the next tile's pass A:
+            // every wait of pass A polls for it in turn (pend_e: the tile whose E step is still to be issued, or -1).
+            int pend_e = -1;
+            auto wait_or_e = [&](uint64_t* bar, uint32_t phase) -> bool {
+                for (uint32_t it = 0; it < (1u << 22); ++it) {
+                    if (mbar_test_wait(bar, phase)) return true;
+                    if (pend_e >= 0 && mbar_test_wait(&bars[kErdy], phE)) {
+                        const int ke = pend_e;
+                        pend_e = -1;
+                        step_e(ke);
+                        if (bad) return false;
+                    }
+                }
+                return false;
+            };
+            // [P | U0](b) = S_0^T [Khat^T | G_n * W] chunk by chunk: one 64-row window per tile
+            auto pass_a = [&](int k) {
+                const int b = k & 1;
+                if (k >= 2) {                   // the slot still holds the sketch data of tile k - 2 until they are stored
+                    if (!wait_or_e(&bars[kBufFree + b], (phBuf >> b) & 1u)) { bad = true; where = 141; return; }
+                    phBuf ^= 1u << b;
+                    tc_fence_after();
+                }
+                const uint32_t slot = tmem_base + (uint32_t)b * 64u;
+                const uint32_t whi0 = smem_u32(w_ptr(b));
+                const uint32_t wlo0 = whi0 + sm.w_lo;
+#pragma unroll 2
+                for (int c = 0; c < NCH; ++c) {
+                    const int ab = c & (kKA2 - 1);
+                    if (!wait_or_e(&bars[kA2rdy + ab], (phR >> ab) & 1u)) { bad = true; where = 142; return; }
+                    phR ^= 1u << ab;
+                    tc_fence_after();
+                    const uint32_t a2 = a2base + (uint32_t)ab * (2u * 128u * CH * 2u);
+                    const uint64_t ahi = make_desc(a2, LBO_M, SBO);
+                    const uint64_t alo = make_desc(a2 + 128u * CH * 2u, LBO_M, SBO);
+                    const uint64_t whi = make_desc(whi0 + (uint32_t)(c * (CH / 8)) * LBO_W, LBO_W, SBO);
+                    const uint64_t wlo = make_desc(wlo0 + (uint32_t)(c * (CH / 8)) * LBO_W, LBO_W, SBO);
+                    tc_mma_bf16(slot, ahi, whi, idescA, c ? 1u : 0u);
+                    tc_mma_bf16(slot, alo, whi, idescA, 1u);
+                    tc_mma_bf16(slot, ahi, wlo, idescA, 1u);
+                    tc_commit(&bars[kA2free + ab]);
+                    if (c == NCH - 1) tc_commit(&bars[kPfull + b]);
+                }
+            };
             int cur = seq_get(0);
             if (cur >= 0) {
+                // pass A of tile k + 1 starts before the E step of tile k: the stream of S_0 chunks does not wait for the
+                // pass-B group (two accumulators); the E step goes out as soon as that group has formed E
                 pass_a(0);
-                if (!bad) step_e(0);
                 for (int k = 0; !bad; ++k) {
+                    pend_e = k;
                     const int raw = seq_get(k + 1);
                     if (raw < -1) { bad = true; break; }
                     if (raw >= 0) pass_a(k + 1);
-                    if (raw < 0 || bad) break;
-                    step_e(k + 1);
+                    if (bad) break;
+                    if (pend_e >= 0) { pend_e = -1; step_e(k); }
+                    if (raw < 0) break;
                 }
             } else if (cur < -1) {
                 bad = true;
@@ -695,14 +703,6 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 cur_h = h;            // (visible to the group after the barrier below)
             }
             const float* og = sOm + i * 16;
-            // the operand set and window of tile k - 2 are free once its Ktil^T E has completed
-            if (k >= 2) {
-                if (!f_wait(ft, &bars[kTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
-                    if (ft == 0) record_fault(p.status, kFaultUpdateWait, 109);
-                    dead = true;
-                    break;
-                }
-            }
             // the staged rows, gates and query row of this tile must have landed
             if (!f_wait(ft, &bars[kStg], phS)) {
                 if (ft == 0) record_fault(p.status, kFaultUpdateWait, 106);
@@ -727,12 +727,12 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 const int t = 16 * (1 - fg) + s;
                 if (t < n_tot) gother *= bf16_at(sStg + sm.stg_g, (uint32_t)(t * K + i));
             }
+            uint4 vrow[2];            // 512 vectors of 16 bytes: 32 value rows, parked in registers until the set is free
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-                const int idx = ft + r * kKFront;          // 512 vectors of 16 bytes: 32 value rows
-                uint4 vv = make_uint4(0, 0, 0, 0);
-                if ((idx >> 4) < n_tot) vv = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)idx * 16);
-                *reinterpret_cast<uint4*>(set + sm.set_vv + (size_t)idx * 16) = vv;
+                const int idx = ft + r * kKFront;
+                vrow[r] = make_uint4(0, 0, 0, 0);
+                if ((idx >> 4) < n_tot) vrow[r] = *reinterpret_cast<const uint4*>(sStg + sm.stg_v + (size_t)idx * 16);
             }
             const float q_i = p.q != nullptr ? bf16_at(sStg + sm.stg_q, (uint32_t)i) : 0.f;
             if (ft < kNT) {
@@ -776,6 +776,19 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     part[bi * 32 + lane] = vals[0];
                 }
             }
+
+            // Up to here nothing of the operand set and window b was touched: they are free once Ktil^T E of tile k - 2 has
+            // completed, so the loads and pair sums above overlap the tail of that tile.
+            if (k >= 2) {
+                if (!f_wait(ft, &bars[kTfull + b], (uint32_t)((k - 2) >> 1) & 1u)) {
+                    if (ft == 0) record_fault(p.status, kFaultUpdateWait, 109);
+                    dead = true;
+                    break;
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 2; ++r)
+                *reinterpret_cast<uint4*>(set + sm.set_vv + (size_t)(ft + r * kKFront) * 16) = vrow[r];
 
             // ---- running products of this block.  Khat -> window rows 0..31; Ktil -> set (MN-major); G_n * W -> window
             // rows 32..; and for the 16 x 16 block of A that couples the two token blocks, whose decay product splits at
