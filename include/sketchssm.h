@@ -102,6 +102,14 @@ typedef struct sketchssm_config {
                                non-flush read, Appendix D).  U is rounded to bfloat16 once, when the flush stores it; all
                                arithmetic stays fp32.  With bfloat16 storage C is the fixed offline map (coef_per_seq = 0),
                                handed over as bfloat16 [H][r][K], and only the default one-kernel decode is available. */
+    int32_t erase_factors;  /* GDN / KDA only.  0 (default): the decode step forms the effective query q~_t by the backward
+                               sweep over the ring and then c_t = C q~_t.  1: it forms c_t from projected erase vectors
+                               (Appendix C.2, Eq. 44-45): every appended token leaves f_s = beta_s [C (d_[s] * k_s) -
+                               sum_{j<s} f_j <l_j(s), k_s>] in R^r in the `erase` buffer, and c_t = C (d_[t] * q_t) -
+                               sum_{s<=t} f_s <l_s(t), q_t> with <l_s(t), y> taken from the stored ring keys and the
+                               cumulative decays (Eq. 46).  Exact for the map in force during the window (the same c_t up
+                               to rounding order); costs 4 r bytes per buffered token and step.  Needs rank % 4 == 0 and
+                               buf_len <= 32; only the default one-kernel decode supports it. */
 } sketchssm_config;
 
 typedef struct sketchssm_sizes {
@@ -112,6 +120,7 @@ typedef struct sketchssm_sizes {
     size_t ring_head_bytes;  /* stride of one (b, h) ring block */
     size_t ring_v_offset, ring_beta_offset, ring_decay_offset; /* byte offsets inside a ring block (k is at 0) */
     size_t alignment;        /* required alignment of every pointer (16) */
+    size_t erase_bytes;      /* erase_factors = 1: B*H*L*rank floats (else 0) */
 } sketchssm_sizes;
 
 typedef struct sketchssm_buffers {
@@ -136,6 +145,10 @@ typedef struct sketchssm_buffers {
                       fetches only that many); 0 = a dense-fallback head whose decode step reads the full state
                       exactly, inside the same launch.  Layouts keep the configured `rank` as their row stride.
                       Only the default one-kernel decode supports the table. */
+    void* erase;   /* erase_factors = 1: erase_bytes, [B][H][L][rank] fp32: slot s of a (b, h) block holds f_s of the token
+                      in ring slot s (written by the decode step that appends the token, read by the later steps of the
+                      window; a state update empties the ring and with it these slots).  Contents need no
+                      initialisation.  Ignored (may be NULL) when erase_factors = 0. */
 } sketchssm_buffers;
 
 typedef struct sketchssm_ctx sketchssm_ctx; /* host-only metadata; owns no device memory */

@@ -25,7 +25,8 @@ the scalar alpha_t (GDN) or the vector g_t in (0,1)^K (KDA).
 Pinned by tests/test_oracle_pins.py against: the exact decomposition of the
 read (Eq. 4), explicit dense transition matrices built with Python loops, the
 identity-basis special case, replay == repeated single updates, the empty-buffer
-case, the WY identities (Eq. 41-45), the PCA closed forms of Appendix A.1, the
+case, the WY identities (Eq. 41-45; the projected erase vectors against C times
+the erase factors), the PCA closed forms of Appendix A.1, the
 traffic-reduction values printed in Tables 4-7, and for the state-dependent
 coefficient maps of Appendix A.2: a library least-squares solve of the ridge
 problem, the range projection in the limit of no ridge, independence of the
@@ -239,12 +240,13 @@ def wy_effective_query(kind, tokens, q):
     return out
 
 
-def wy_coefficients(kind, tokens, q, C):
-    """c_t = C (d_[t] * q_t) - sum_s f_s <l_s(t), q_t> with the projected erase
-    factors f_s = beta_s [C (d_[s] * k_s) - sum_{j<s} f_j <l_j(s), k_s>] (Eq. 44-45)."""
+def projected_erase_vectors(kind, tokens, C):
+    """f_s = beta_s [C (d_[s] * k_s) - sum_{j<s} f_j <l_j(s), k_s>] for every buffered token (Eq. 45),
+    with the left factors l_j(s) = (D_s ... D_{j+1}) k_j kept as running products.
+    Returns (f list, l list, d) where l[j] = l_j(t) and d = d_[t] for t = len(tokens)."""
     assert kind != MAMBA2
-    q, C = _f64(q), _f64(C)
-    K = q.shape[-1]
+    C = _f64(C)
+    K = C.shape[-1]
     fs, ls = [], []
     d_run = None
     for (k, _v, beta, decay) in tokens:
@@ -257,6 +259,14 @@ def wy_coefficients(kind, tokens, q, C):
             acc = acc - f_j * np.einsum("...k,...k->...", l_j, k)[..., None]
         fs.append(beta[..., None] * acc)
         ls.append(k.copy())
+    return fs, ls, d_run
+
+
+def wy_coefficients(kind, tokens, q, C):
+    """c_t = C (d_[t] * q_t) - sum_s f_s <l_s(t), q_t> with the projected erase
+    factors f_s of Eq. 45 (Eq. 44)."""
+    q, C = _f64(q), _f64(C)
+    fs, ls, d_run = projected_erase_vectors(kind, tokens, C)
     c = np.einsum("...gk,...k->...g", C, d_run * q)
     for l_s, f_s in zip(ls, fs):
         c = c - f_s * np.einsum("...k,...k->...", l_s, q)[..., None]

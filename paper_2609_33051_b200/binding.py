@@ -34,17 +34,20 @@ OP_DECODE, OP_FULL_READ, OP_UPDATE = 0, 1, 2
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("kind", "batch", "heads", "dk", "dv", "rank", "buf_len", "io_dtype", "out_dtype", "device",
-                 "coef_per_seq", "coef_pivots")] + [("ridge_lambda", ctypes.c_float), ("sketch_dtype", ctypes.c_int32)]
+                 "coef_per_seq", "coef_pivots")] + [("ridge_lambda", ctypes.c_float), ("sketch_dtype", ctypes.c_int32),
+                                                            ("erase_factors", ctypes.c_int32)]
 
 
 class Sizes(ctypes.Structure):
     _fields_ = [(n, ctypes.c_size_t) for n in
                 ("state_bytes", "sketch_bytes", "ring_bytes", "omega_bytes", "coef_bytes", "status_bytes",
-                 "work_bytes", "ring_head_bytes", "ring_v_offset", "ring_beta_offset", "ring_decay_offset", "alignment")]
+                 "work_bytes", "ring_head_bytes", "ring_v_offset", "ring_beta_offset", "ring_decay_offset", "alignment",
+                 "erase_bytes")]
 
 
 class Buffers(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status", "work", "head_rank")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("state", "sketch", "ring", "omega", "coef", "status", "work", "head_rank",
+                                                "erase")]
 
 
 class Staging(ctypes.Structure):
@@ -108,24 +111,27 @@ class SketchSSM:
     omega [H,K,r] f32, coef [H,r,K] f32 (or [B,H,r,K] with coef_per_seq: the state-dependent map that every
     state update rebuilds).  Token arguments follow the C header:
     q,k [B,H,K] io; v [B,H,V] io; beta [B,H] f32; decay [B,H] f32 or [B,H,K] io (KDA).
+    With erase_factors (GDN / KDA) the decode step forms c_t from projected erase vectors kept in `erase` [B,H,L,r] f32.
     """
 
     def __init__(self, kind: str, batch: int, heads: int, dk: int, dv: int, rank: int, buf_len: int,
                  io: str = "bf16", out: str = "f32", device: int = 0, allocate: bool = True,
-                 coef_per_seq: bool = False, coef_pivots: int = 4, ridge_lambda: float = 0.1, sketch: str = "f32"):
+                 coef_per_seq: bool = False, coef_pivots: int = 4, ridge_lambda: float = 0.1, sketch: str = "f32",
+                 erase_factors: bool = False):
         self.lib = load_library()
         self.kind, self.io, self.out = kind, io, out
         self.B, self.H, self.K, self.V, self.R, self.L = batch, heads, dk, dv, rank, buf_len
         self.device = torch.device("cuda", device)
         self.coef_per_seq = bool(coef_per_seq)
         self.cfg = Config(KIND[kind], batch, heads, dk, dv, rank, buf_len, DTYPE[io], DTYPE[out], device,
-                          int(self.coef_per_seq), coef_pivots, ridge_lambda, DTYPE[sketch])
+                          int(self.coef_per_seq), coef_pivots, ridge_lambda, DTYPE[sketch], int(bool(erase_factors)))
+        self.erase_factors = bool(erase_factors)
         self.sketch_dtype = sketch
         self._ctx = ctypes.c_void_p()
         self._check("sketchssm_create", self.lib.sketchssm_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.sizes = Sizes()
         self._check("sketchssm_query_sizes", self.lib.sketchssm_query_sizes(self._ctx, ctypes.byref(self.sizes)))
-        self.state = self.sketch = self.ring = self.omega = self.coef = self.status = self.work = None
+        self.state = self.sketch = self.ring = self.omega = self.coef = self.status = self.work = self.erase = None
         self.head_rank = None        # optional int32 [H] device tensor: per-head sketch rank (0 = full-state read); set, then bind()
         if allocate:
             self.allocate()
@@ -141,6 +147,8 @@ class SketchSSM:
                                 dtype=TORCH_DTYPE[self.sketch_dtype], device=d)
         self.status = torch.zeros(self.sizes.status_bytes // 4, dtype=torch.int32, device=d)
         self.work = torch.zeros(self.sizes.work_bytes // 4, dtype=torch.float32, device=d)
+        if self.erase_factors:
+            self.erase = torch.zeros(self.B, self.H, self.L, self.R, dtype=torch.float32, device=d)
         self.bind()
 
     def bind(self):
@@ -149,7 +157,8 @@ class SketchSSM:
         assert self.ring.numel() == self.sizes.ring_bytes
         b = Buffers(self.state.data_ptr(), self.sketch.data_ptr(), self.ring.data_ptr(),
                     self.omega.data_ptr(), self.coef.data_ptr(), self.status.data_ptr(), self.work.data_ptr(),
-                    self.head_rank.data_ptr() if self.head_rank is not None else None)
+                    self.head_rank.data_ptr() if self.head_rank is not None else None,
+                    self.erase.data_ptr() if self.erase is not None else None)
         self._check("sketchssm_bind", self.lib.sketchssm_bind(self._ctx, ctypes.byref(b)))
 
     def close(self):

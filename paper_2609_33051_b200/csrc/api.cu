@@ -64,6 +64,7 @@ Params base_params(const sketchssm_ctx* ctx) {
     p.pivots = ctx->cfg.coef_pivots;
     p.ridge_lambda = ctx->cfg.ridge_lambda;
     p.sketch_bf16 = ctx->cfg.sketch_dtype == SKETCHSSM_BF16;
+    p.erase = ctx->cfg.erase_factors ? static_cast<float*>(ctx->bufs.erase) : nullptr;
     return p;
 }
 
@@ -126,7 +127,8 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     if (rc != SKETCHSSM_OK) return rc;
     // Only a state update writes the sketch.  Unless that was the previous call on this context (it may still be running:
     // programmatic dependent launch), a decode step may read U before it waits for its predecessor in the stream.
-    p.early_sketch = (!full_read && !ctx->sketch_fresh) ? 1 : 0;
+    // (The projected erase vectors travel with the sketch rows and are written by the previous decode step: no early read.)
+    p.early_sketch = (!full_read && !ctx->sketch_fresh && p.erase == nullptr) ? 1 : 0;
     ctx->sketch_fresh = false;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (p.early_sketch) {
@@ -138,7 +140,8 @@ int decode_common(sketchssm_ctx* ctx, int full_read, int n_before, const void* q
     const bool bf = ctx->cfg.io_dtype == SKETCHSSM_BF16;
     if (ctx->tune_decode_impl == 1) return launch_decode(ctx, p, cs);
     // the two-kernel decode stages one map per head index, knows one rank and the value widths 64 and 128
-    if ((p.coef_per_seq && !full_read) || p.head_rank != nullptr || ctx->cfg.dv == 80 || (p.sketch_bf16 && !full_read))
+    if ((p.coef_per_seq && !full_read) || p.head_rank != nullptr || ctx->cfg.dv == 80 || (p.sketch_bf16 && !full_read) ||
+        (p.erase != nullptr && !full_read))
         return SKETCHSSM_UNSUPPORTED_SHAPE;
     switch (ctx->cfg.kind) {
         case SKETCHSSM_MAMBA2:
@@ -170,6 +173,13 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     if (cfg->coef_per_seq != 0 && cfg->coef_per_seq != 1) return SKETCHSSM_INVALID_ARG;
     if (cfg->sketch_dtype != SKETCHSSM_F32 && cfg->sketch_dtype != SKETCHSSM_BF16) return SKETCHSSM_INVALID_ARG;
     if (cfg->sketch_dtype == SKETCHSSM_BF16 && cfg->coef_per_seq) return SKETCHSSM_UNSUPPORTED_SHAPE;   // bfloat16 storage: fixed offline map
+    if (cfg->erase_factors != 0 && cfg->erase_factors != 1) return SKETCHSSM_INVALID_ARG;
+    if (cfg->erase_factors) {
+        if (cfg->kind == SKETCHSSM_MAMBA2) return SKETCHSSM_INVALID_ARG;            // no erase term: nothing to project
+        // rows of r floats travel as bulk copies (16-byte units); the per-slot dot products and the two coefficient
+        // vectors share the decode kernel's per-warp scratch
+        if ((cfg->rank & 3) || cfg->buf_len > 32 || 2 * ((cfg->rank + 7) & ~7) > cfg->dk) return SKETCHSSM_UNSUPPORTED_SHAPE;
+    }
     if (cfg->coef_per_seq) {
         if (!(cfg->ridge_lambda > 0.f) || cfg->coef_pivots < 0) return SKETCHSSM_INVALID_ARG;
         if (cfg->coef_pivots > 8) return SKETCHSSM_UNSUPPORTED_SHAPE;
@@ -218,6 +228,7 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
     out->ring_beta_offset = ctx->ring.beta_off;
     out->ring_decay_offset = ctx->ring.decay_off;
     out->alignment = 16;
+    out->erase_bytes = c.erase_factors ? bh * (size_t)c.buf_len * c.rank * 4 : 0;
     return SKETCHSSM_OK;
 }
 
@@ -228,6 +239,7 @@ int sketchssm_bind(sketchssm_ctx* ctx, const sketchssm_buffers* b) {
         if (p == nullptr || !aligned16(p)) return SKETCHSSM_INVALID_ARG;
     }
     if (b->head_rank != nullptr && (reinterpret_cast<uintptr_t>(b->head_rank) & 3u)) return SKETCHSSM_INVALID_ARG;
+    if (ctx->cfg.erase_factors && (b->erase == nullptr || !aligned16(b->erase))) return SKETCHSSM_INVALID_ARG;
     ctx->bufs = *b;
     ctx->bound = true;
     ctx->sketch_fresh = true;       // whatever filled the buffers may still be running
@@ -329,7 +341,8 @@ int sketchssm_decode_step_static(sketchssm_ctx* ctx, int n_before, const void* q
     int rc = decode_params(ctx, 0, n_before, q, k, v, beta, decay, out, flags, &p);
     if (rc != SKETCHSSM_OK) return rc;
     // runs the two-kernel decode (one map per head index, one rank, value widths 64 and 128)
-    if (ctx->cfg.coef_per_seq || ctx->bufs.head_rank != nullptr || ctx->cfg.dv == 80 || ctx->cfg.sketch_dtype == SKETCHSSM_BF16)
+    if (ctx->cfg.coef_per_seq || ctx->bufs.head_rank != nullptr || ctx->cfg.dv == 80 || ctx->cfg.sketch_dtype == SKETCHSSM_BF16 ||
+        ctx->cfg.erase_factors)
         return SKETCHSSM_UNSUPPORTED_SHAPE;
     // the size limit of the library's static array is checked (on the host, before any CUDA call) by the launcher
     const sketchssm_config& c = ctx->cfg;

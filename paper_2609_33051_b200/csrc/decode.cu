@@ -33,6 +33,7 @@ namespace {
 struct StageLayout {
     uint32_t u_off, u_bytes;        // sketch U (sketch mode only)
     uint32_t c_off, c_bytes;        // the head's own coefficient map (sketch mode with a per-sequence map only)
+    uint32_t f_off, f_bytes;        // projected erase vectors of the n buffered tokens (n rows of R floats; erase mode only)
     uint32_t k_off, k_bytes;        // n buffered keys
     uint32_t v_off, v_bytes;        // n buffered values
     uint32_t gate_off, gate_bytes;  // beta[L] (+ decay[L] for scalar kinds)
@@ -42,13 +43,15 @@ struct StageLayout {
 };
 
 __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K, int V, int R, int L, int n,
-                                                         int full_read, int coef_per_seq, int sketch_bytes = 4) {
+                                                         int full_read, int coef_per_seq, int sketch_bytes = 4,
+                                                         int erase = 0) {
     StageLayout s;
     uint32_t off = 0;
     s.u_off = off; s.u_bytes = full_read ? 0u : (uint32_t)(R * V * sketch_bytes); off += (s.u_bytes + 15u) & ~15u;
     // rows padded to the reduction width are read (their sums are never used), so they get room but are not copied
     s.c_off = off; s.c_bytes = (!full_read && coef_per_seq) ? (uint32_t)(R * K * 4) : 0u;
     off += (!full_read && coef_per_seq) ? (uint32_t)(((R + 7) & ~7) * K * 4) : 0u;
+    s.f_off = off; s.f_bytes = (!full_read && erase) ? (uint32_t)(n * R * 4) : 0u; off += s.f_bytes;
     s.k_off = off; s.k_bytes = (uint32_t)(n * K * io); off += s.k_bytes;
     s.v_off = off; s.v_bytes = (uint32_t)(n * V * io); off += s.v_bytes;
     s.gate_off = off;
@@ -87,7 +90,8 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
 
 // RT: the sketch rank as a compile-time constant (loops over ranks unroll fully), or 0 for any rank.
 // GEN: 0 = one ring fill and one rank for every head of the launch (copy sizes are per-lane constants);
-//      1 = per-sequence phases and / or a per-head rank table (sizes follow the head).
+//      1 = per-sequence phases and / or a per-head rank table (sizes follow the head);
+//      2 = 1 with the coefficient vector formed from projected erase vectors (delta-rule kinds).
 template <int KIND, typename IO, int K, int V, int RT, int GEN>
 __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
@@ -107,8 +111,11 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     const bool u_bf16 = GEN && p.sketch_bf16;           // sketch rows (and the fixed coefficient map) stored as bfloat16
     const int su = u_bf16 ? 2 : 4;
     const int RP = (R + 7) & ~7;
+    // c_t from the projected erase vectors of the buffered tokens instead of the swept query (delta-rule kinds)
+    constexpr bool ER = GEN == 2;
+    const bool er = ER && !p.full_read;
 
-    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, per_seq, su);
+    const StageLayout sl = make_stage_layout(KIND, (int)sizeof(IO), K, V, R, L, n_cap, p.full_read, per_seq, su, er);
     const DecodeSmem ds = make_decode_smem(K, R, nwarps, p.full_read, per_seq, sl.total);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ds.bar_off) + warp * 2;
     float* sX = reinterpret_cast<float*>(smem + ds.scratch_off + (size_t)warp * ds.scratch_stride);   // c or q~
@@ -175,6 +182,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_unit = KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u; cp_mode = 1; break;
         case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * su; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * su); cp_mode = 3; break;
         case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_unit = per_seq ? (uint32_t)(K * 4) : 0u; cp_mode = 3; break;
+        case 10: cp_base = reinterpret_cast<const unsigned char*>(p.erase); cp_stride = (size_t)L * R * 4; cp_dst = sl.f_off; cp_unit = er ? (uint32_t)(R * 4) : 0u; cp_mode = 1; break;
         default: break;
     }
     const uint32_t tokA = 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
@@ -201,12 +209,15 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
             if (lane < 8 && cp_fixed) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_fixed, barA);
         }
     };
-    auto issue_b = [&](size_t bh, int r_it) {      // whole warp; r_it: sketch rank of the head (0: nothing to fetch)
+    // whole warp; r_it: sketch rank of the head (0: nothing to fetch), n_it: its ring fill (rows of erase vectors)
+    auto issue_b = [&](size_t bh, int r_it, int n_it) {
         if constexpr (GEN) {
-            if (lane == 8 && r_it > 0) mbar_expect_tx(barB, (uint32_t)r_it * rowB);
+            const uint32_t fbytes = er ? (uint32_t)n_it * (uint32_t)(R * 4) : 0u;
+            if (lane == 8 && r_it > 0) mbar_expect_tx(barB, (uint32_t)r_it * rowB + fbytes);
             __syncwarp();
             if ((lane == 8 || lane == 9) && cp_unit && r_it > 0)
                 bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, cp_unit * (uint32_t)r_it, barB);
+            if (lane == 10 && fbytes && r_it > 0) bulk_g2s(my_stage + cp_dst, cp_base + bh * cp_stride, fbytes, barB);
         } else {
             if (lane == 8 && txB_fixed) mbar_expect_tx(barB, txB_fixed);
             __syncwarp();
@@ -263,7 +274,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
     // head's sketch rows are requested before the predecessor in the stream is waited for, so they travel during its tail.
     // (Not with per-sequence phases: whether the head takes part at all is only known after the wait.)
     const bool early_u = p.early_sketch != 0 && p.n_dev == nullptr;
-    if (item < item1 && early_u) issue_b((size_t)b * H + h, rk);
+    if (item < item1 && early_u) issue_b((size_t)b * H + h, rk, 0);
     grid_dep_wait();                 // from here on the ring and the token tensors (and otherwise the sketch) are read
     // Dependents are released only now: a successor that reads its sketch early must not start before this kernel has
     // seen its own predecessor (possibly a state update) complete.
@@ -273,7 +284,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
         n = fill_of(b);
         if (!GEN || n >= 0) {
             issue_a(bh0, n);
-            if (!early_u) issue_b(bh0, rk);
+            if (!early_u) issue_b(bh0, rk, n);
             scalar_gates(bh0, bt_next, dsc_next);
         }
     }
@@ -299,12 +310,13 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 
         if constexpr (GEN) {
             if (n < 0) {             // this sequence takes the flush step in this call: nothing to do here
-                if (go_next) { issue_a(bh_next, n_next); issue_b(bh_next, rk_next); }
+                if (go_next) { issue_a(bh_next, n_next); issue_b(bh_next, rk_next, n_next); }
                 item = item_next; h = hn; b = bn; n = n_next; rk = rk_next;
                 continue;
             }
         }
         const bool full = rk == 0;   // exact read of the whole state for this head
+        const bool er_h = er && !full;       // this head forms c_t from projected erase vectors
 
         if (__any_sync(0xffffffffu, !DEC_WAIT(barA, parA))) {
             if (lane == 0) record_fault(p.status, p.full_read ? kFaultFullReadWait : kFaultDecodeWait, (int)blockIdx.x);
@@ -343,11 +355,13 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 
         // ---- current token, s = t ----
         float dsuf = 1.f;
+        float kq_t;                  // <k_t, q_t>
         {
             float part = 0.f;
 #pragma unroll
             for (int e = 0; e < EK; ++e) part = fmaf(kk[e], q0[e], part);
-            const float a = bt * warp_sum(part);
+            kq_t = warp_sum(part);
+            const float a = bt * kq_t;
 #pragma unroll
             for (int e = 0; e < EV; ++e) o[e] = a * vv[e];
             if constexpr (KIND == SKETCHSSM_MAMBA2) {
@@ -408,29 +422,68 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 #pragma unroll
             for (int e = 0; e < EK; ++e) x[e] = dsuf * q0[e];
         } else {
+            // Erase mode: next to the sweep (which the exact output of the buffered tokens needs anyway), the left factors
+            // l_s(t) = (D_t ... D_{s+1}) k_s give <l_s(t), q_t> and <l_s(t), k_t> for every slot (Eq. 46: from the stored keys
+            // and the running product of the decays); dl / dlv end up as the cumulative decay d_[t].
+            float dl = dsc;
+            float dlv[EK];
+#pragma unroll
+            for (int e = 0; e < EK; ++e) dlv[e] = KIND == SKETCHSSM_KDA ? gg[e] : 1.f;
 #pragma unroll 2
             for (int s = n - 1; s >= 0; --s) {
-                float kr[EK], vr[EV];
+                float kr[EK], vr[EV], gr[EK];
                 load_io<EK>(sK, s * K + lane * EK, kr);
 #pragma unroll
                 for (int e = 0; e < EV; ++e) vr[e] = 0.f;
                 if (vlane) load_io<EV>(sV, s * V + lane * EV, vr);
+                if constexpr (KIND == SKETCHSSM_KDA && ER) load_io<EK>(sG, s * K + lane * EK, gr);
                 float part = 0.f;
 #pragma unroll
                 for (int e = 0; e < EK; ++e) part = fmaf(kr[e], x[e], part);
                 const float a = sBeta[s] * warp_sum(part);
+                if constexpr (ER) {
+                    if (er_h) {
+                        float pq = 0.f, pk = 0.f;
+#pragma unroll
+                        for (int e = 0; e < EK; ++e) {
+                            const float le = KIND == SKETCHSSM_KDA ? dlv[e] * kr[e] : kr[e];
+                            pq = fmaf(le, q0[e], pq);
+                            pk = fmaf(le, kk[e], pk);
+                        }
+                        pq = warp_sum(pq);
+                        pk = warp_sum(pk);
+                        if constexpr (KIND == SKETCHSSM_GDN) {
+                            pq *= dl;
+                            pk *= dl;
+                            dl *= sDec[s];
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < EK; ++e) dlv[e] *= gr[e];
+                        }
+                        if (lane == 0) { sP[s] = pq; sP[32 + s] = pk; }
+                    }
+                }
                 if constexpr (KIND == SKETCHSSM_GDN) {
                     const float d = sDec[s];
 #pragma unroll
                     for (int e = 0; e < EK; ++e) x[e] = d * fmaf(-a, kr[e], x[e]);
                 } else {
-                    float gr[EK];
-                    load_io<EK>(sG, s * K + lane * EK, gr);
+                    if constexpr (!ER) load_io<EK>(sG, s * K + lane * EK, gr);
 #pragma unroll
                     for (int e = 0; e < EK; ++e) x[e] = gr[e] * fmaf(-a, kr[e], x[e]);
                 }
 #pragma unroll
                 for (int e = 0; e < EV; ++e) o[e] = fmaf(a, vr[e], o[e]);
+            }
+            if constexpr (ER) {
+                if (er_h) {      // x <- d_[t] * q_t; kk <- d_[t] * k_t (the token's key has been stored and swept by now)
+#pragma unroll
+                    for (int e = 0; e < EK; ++e) {
+                        const float d = KIND == SKETCHSSM_KDA ? dlv[e] : dl;
+                        x[e] = d * q0[e];
+                        kk[e] *= d;
+                    }
+                }
             }
         }
 
@@ -466,6 +519,24 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 group_reduce_transpose<32, NB>(part, lane);
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
+            if constexpr (ER) {
+                if (er_h) {      // C (d_[t] * k_t) behind C (d_[t] * q_t) in the scratch
+                    for (int g0 = 0; g0 < rp_it; g0 += NB) {
+                        float part[NB];
+#pragma unroll
+                        for (int i = 0; i < NB; ++i) {
+                            float cw[EK];
+                            load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
+                            float acc = 0.f;
+#pragma unroll
+                            for (int e = 0; e < EK; ++e) acc = fmaf(cw[e], kk[e], acc);
+                            part[i] = acc;
+                        }
+                        group_reduce_transpose<32, NB>(part, lane);
+                        if ((lane & 3) == 0) sX[rp_it + g0 + (lane >> 2)] = part[0];
+                    }
+                }
+            }
             __syncwarp();
             if (!per_seq) {
                 if (__any_sync(0xffffffffu, !DEC_WAIT(barB, PARB))) {
@@ -476,6 +547,25 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 }
             }
             if constexpr (GEN) parB ^= 1u;
+            if constexpr (ER) {
+                if (er_h) {
+                    // f_t = beta_t [C (d_[t] * k_t) - sum_{s<t} f_s <l_s(t), k_t>]  (Eq. 45), stored for the later steps;
+                    // c_t = C (d_[t] * q_t) - sum_{s<t} f_s <l_s(t), q_t> - f_t <k_t, q_t>  (Eq. 44).  One coefficient per lane.
+                    const float* sF = reinterpret_cast<const float*>(sb + sl.f_off);
+                    for (int g = lane; g < rk; g += 32) {
+                        float fq = sX[g], fk = sX[rp_it + g];
+                        for (int s = 0; s < n; ++s) {
+                            const float f = sF[s * R + g];
+                            fq = fmaf(-f, sP[s], fq);
+                            fk = fmaf(-f, sP[32 + s], fk);
+                        }
+                        const float f_t = bt * fk;
+                        sX[g] = fmaf(-f_t, kq_t, fq);
+                        if (p.append) p.erase[(bh * L + n) * (size_t)R + g] = f_t;
+                    }
+                    __syncwarp();
+                }
+            }
             const float* sU = reinterpret_cast<const float*>(sb + sl.u_off);
             if (vlane) {
 #pragma unroll (RT ? RT : 4)
@@ -489,7 +579,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 }
             }
             __syncwarp();
-            if (go_next) issue_b(bh_next, rk_next);
+            if (go_next) issue_b(bh_next, rk_next, n_next);
         } else {
             __syncwarp();
             store_io<EK>(sX, lane * EK, x);
@@ -510,7 +600,7 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
                 }
             }
             // a head that reads the full state fetched no sketch rows; the next head's are requested here
-            if (go_next) issue_b(bh_next, rk_next);
+            if (go_next) issue_b(bh_next, rk_next, n_next);
         }
 
         if (vlane) {
@@ -537,7 +627,8 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 template <int KIND, typename IO, int K, int V>
 static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     const int io = (int)sizeof(IO);
-    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq, p.sketch_bf16 ? 2 : 4);   // (the general instantiation runs whenever coef_per_seq or sketch_bf16 is set)
+    const int erase = (KIND != SKETCHSSM_MAMBA2 && p.erase != nullptr && !p.full_read) ? 1 : 0;
+    const StageLayout sl = make_stage_layout(KIND, io, K, V, p.R, p.L, p.n_before, p.full_read, p.coef_per_seq, p.sketch_bf16 ? 2 : 4, erase);   // (the general instantiation runs whenever coef_per_seq or sketch_bf16 is set)
     const uint32_t smem_budget = 227u * 1024u;
     if (ctx->sm_count == 0) {
         int dev = 0, sms = 0;
@@ -549,12 +640,15 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
     // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
-    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq || p.sketch_bf16;
+    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq || p.sketch_bf16 || erase;
     const bool fixed16 = p.R == 16 && !gen;     // the unrolled rank-16 instantiation needs one rank for all heads
     auto kern = gen ? decode_kernel<KIND, IO, K, V, 0, 1> : fixed16 ? decode_kernel<KIND, IO, K, V, 16, 0> : decode_kernel<KIND, IO, K, V, 0, 0>;
+    if constexpr (KIND != SKETCHSSM_MAMBA2) {
+        if (erase) kern = decode_kernel<KIND, IO, K, V, 0, 2>;
+    }
     // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does
-    static int regs_per_thread[3] = {0, 0, 0};
-    int& regs = regs_per_thread[gen ? 2 : fixed16 ? 1 : 0];
+    static int regs_per_thread[4] = {0, 0, 0, 0};
+    int& regs = regs_per_thread[erase ? 3 : gen ? 2 : fixed16 ? 1 : 0];
     if (regs == 0) {
         cudaFuncAttributes fa;
         if ((ctx->last_cuda_error = cudaFuncGetAttributes(&fa, kern)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;

@@ -80,6 +80,7 @@ struct Params {
                           // -v - 1 buffered tokens); nullptr: n_before for every sequence
     int n_cap;            // update (CUDA cores) with per-sequence phases: ring rows the shared-memory layout has room for
     int sketch_bf16;      // U (and the fixed C) are stored as bfloat16
+    float* erase;         // projected erase vectors f_s [B][H][L][R] (Eq. 44-45), or nullptr: c_t = C q~_t from the swept query
     int tok_base;         // update (GDN tensor-core kernel): first ring row of this pass when a flush is replayed in blocks of 16 tokens
 };
 

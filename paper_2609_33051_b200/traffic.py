@@ -22,9 +22,10 @@ def token_bytes(kind: str, K: int, V: int, io: str) -> int:
 
 
 def decode_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, full_read=False, append=True,
-                 sketch_bytes=4, coef_per_seq=False) -> int:
+                 sketch_bytes=4, coef_per_seq=False, erase_factors=False) -> int:
     """decode_step / full_read_decode launch at ring fill n_before.  sketch_bytes: storage of U and C (4 or 2);
-    coef_per_seq: every head reads its own coefficient map instead of the one shared by the batch."""
+    coef_per_seq: every head reads its own coefficient map instead of the one shared by the batch;
+    erase_factors: the projected erase vectors f_s (r floats per buffered token) are read, and the token's is written."""
     per_head = (K * V * 4 if full_read else r * V * sketch_bytes)   # S or U
     per_head += n_before * slot_bytes(kind, K, V, io)               # ring read
     per_head += token_bytes(kind, K, V, io)                         # q, k, v, gates of the token
@@ -36,6 +37,8 @@ def decode_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, full_rea
             per_head += r * K * 4                                   # the head's own C (fp32)
         else:
             shared = H * r * K * sketch_bytes                       # C, once per launch
+        if erase_factors and kind != "mamba2":
+            per_head += (n_before + (1 if append else 0)) * r * 4   # f_s of the buffered tokens in, f_t out
     return B * H * per_head + shared
 
 

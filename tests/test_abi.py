@@ -68,6 +68,23 @@ def test_create_validates_configuration(lib):
     s = binding.Sizes()
     assert rc == 0 and lib.sketchssm_query_sizes(ctx, ctypes.byref(s)) == 0
     assert s.coef_bytes == 3 * 5 * 8 * 128 * 4                  # one map per (batch, head)
+    assert s.erase_bytes == 0
+    lib.sketchssm_destroy(ctx)
+    # projected erase vectors: delta-rule kinds only, rank a multiple of 4, windows of at most 32 tokens, and room for two
+    # coefficient vectors in the scratch (2 * round_up(rank, 8) <= dk)
+    assert make(lib, erase_factors=1)[0] == 0
+    assert make(lib, erase_factors=2)[0] == -1
+    assert make(lib, kind=0, dv=64, erase_factors=1)[0] == -1
+    assert make(lib, rank=6, erase_factors=1)[0] == -2
+    assert make(lib, buf_len=64, erase_factors=1)[0] == -2
+    assert make(lib, dk=64, dv=64, rank=36, erase_factors=1)[0] == -2
+    rc, ctx = make(lib, erase_factors=1, batch=3, heads=5, rank=8, buf_len=8)
+    assert rc == 0 and lib.sketchssm_query_sizes(ctx, ctypes.byref(s)) == 0
+    assert s.erase_bytes == 3 * 5 * 8 * 8 * 4
+    b = binding.Buffers(*([1 << 20] * 7), None, None)             # (addresses are only checked, never dereferenced, by bind)
+    assert lib.sketchssm_bind(ctx, ctypes.byref(b)) == -1         # the erase buffer is required
+    b.erase = 1 << 20
+    assert lib.sketchssm_bind(ctx, ctypes.byref(b)) == 0
     lib.sketchssm_destroy(ctx)
 
 

@@ -25,14 +25,16 @@ def _device():
     return torch.device("cuda", 0)
 
 
-def make_layer(w, layer=0, out="f32", coef=None, lam=0.1, pivots=4, sketch="f32"):
+def make_layer(w, layer=0, out="f32", coef=None, lam=0.1, pivots=4, sketch="f32", erase=False):
     """coef: None (fixed offline map, an input), "pivot" or "ridge" (state-dependent map, rebuilt by every flush).
-    sketch: storage type of U and C ("bf16": the fixed map is rounded to bfloat16 before either side sees it)."""
+    sketch: storage type of U and C ("bf16": the fixed map is rounded to bfloat16 before either side sees it).
+    erase: the decode step forms c_t from projected erase vectors (Eq. 44-45) instead of the swept query."""
     from paper_2609_33051_b200.binding import SketchSSM
     dev = _device()
     Om, C = harness.basis_for(w, layer)
     m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out=out, device=0,
-                  coef_per_seq=coef is not None, coef_pivots=pivots if coef == "pivot" else 0, ridge_lambda=lam, sketch=sketch)
+                  coef_per_seq=coef is not None, coef_pivots=pivots if coef == "pivot" else 0, ridge_lambda=lam, sketch=sketch,
+                  erase_factors=erase)
     if sketch == "bf16":
         C = synth.round_io(C, "bf16")
     S0 = synth.initial_state(w, layer)
@@ -44,7 +46,7 @@ def make_layer(w, layer=0, out="f32", coef=None, lam=0.1, pivots=4, sketch="f32"
 
 
 def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", input_batch=None, per_element=None,
-                 coef=None, lam=0.1, pivots=4, sketch="f32"):
+                 coef=None, lam=0.1, pivots=4, sketch="f32", erase=False):
     """Algorithm 1 on GPU and oracle; returns the worst per-step relative error and the final-state errors.
 
     input_batch: generate the token inputs for this many batch entries and repeat them over the batch (the initial
@@ -52,8 +54,13 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
     generation of the largest batches short.  per_element: optional callable(got, ref) run on every step's outputs.
     errs["windows"] lists the worst output error of each window, so drift across flushes is visible.
     coef: None, or "pivot" / "ridge": the state-dependent coefficient map, which both sides rebuild from the state at
-    the initial sketch construction and at every flush (errs["C"]: the final maps)."""
-    m, S0, Om, C, dev = make_layer(w, out=out, coef=coef, lam=lam, pivots=pivots, sketch=sketch)
+    the initial sketch construction and at every flush (errs["C"]: the final maps).
+    erase: decode through the projected erase vectors; errs["f"] compares the vector every decode step stores with the
+    oracle's f_s of that token (Eq. 45)."""
+    m, S0, Om, C, dev = make_layer(w, out=out, coef=coef, lam=lam, pivots=pivots, sketch=sketch, erase=erase)
+    if erase:
+        m.erase.fill_(float("nan"))                     # the buffer needs no initialisation: stale contents must not matter
+        errs_f = 0.0
     stored = (lambda u: orc.round_bf16(u)) if sketch == "bf16" else (lambda u: u)      # the oracle rounds U where the flush stores it
     for key, val in (tune or {}).items():
         m.tune(key, val)
@@ -88,6 +95,9 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
             if mode == "sketch":
                 m.decode_step(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
                 ref = orc.decode_step(w.kind, U, C_s, ring, q)
+                if erase:
+                    f_ref = orc.projected_erase_vectors(w.kind, ring, C_s)[0][-1]
+                    errs_f = max(errs_f, harness.rel_err(m.erase[bs_t, hs_t, n].cpu().numpy(), f_ref))
             else:
                 m.full_read_decode(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
                 ref = orc.full_read_decode(w.kind, S, ring, q)
@@ -118,6 +128,8 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
         errs["u_mismatch"] = float(np.mean(got_u != U))
     if coef is not None:
         errs["C"] = harness.rel_err(m.coef[bs_t, hs_t].cpu().numpy(), C_s)
+    if erase:
+        errs["f"] = errs_f
     errs["windows"] = windows
     return errs
 

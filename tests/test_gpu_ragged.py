@@ -26,15 +26,16 @@ def _dev():
     return torch.device("cuda", 0)
 
 
-@pytest.mark.parametrize("kind,dv", [("mamba2", 64), ("gdn", 128), ("kda", 128), ("mamba2", 80)])
+@pytest.mark.parametrize("kind,dv,erase", [("mamba2", 64, False), ("gdn", 128, False), ("kda", 128, False), ("mamba2", 80, False),
+                                            ("gdn", 128, True), ("kda", 128, True)])
 @pytest.mark.parametrize("coef", [None, "pivot"])
-def test_per_head_ranks_and_dense_fallback_heads(kind, dv, coef):
+def test_per_head_ranks_and_dense_fallback_heads(kind, dv, coef, erase):
     """Heads of one layer with ranks (8, 3, 0, 5, 1, 8): rank-g heads use the first g columns of Omega (and the first g rows
     of C, or their own state-dependent map of that rank); rank 0 reads the full state exactly.  Two windows."""
     dev = _dev()
     ranks = np.array([8, 3, 0, 5, 1, 8], dtype=np.int32)
     w = synth.Workload("t", kind, 5, len(ranks), 128, dv, 8, 8, 0, "bf16", 131, basis="qr")
-    m, S0, Om, C, _ = make_layer(w, coef=coef)
+    m, S0, Om, C, _ = make_layer(w, coef=coef, erase=erase)
     m.head_rank = torch.from_numpy(ranks).to(dev)
     m.bind()
     m.state_update(0)
@@ -84,15 +85,17 @@ def test_per_head_ranks_and_dense_fallback_heads(kind, dv, coef):
     assert harness.rel_err(m.state.cpu().numpy(), S) <= FP32_GUARD
 
 
-@pytest.mark.parametrize("kind,dv,coef", [("mamba2", 64, None), ("gdn", 128, None), ("kda", 128, None), ("mamba2", 80, None),
-                                           ("gdn", 128, "pivot"), ("mamba2", 64, "ridge")])
-def test_sequences_at_different_window_phases_in_one_call(kind, dv, coef):
+@pytest.mark.parametrize("kind,dv,coef,erase", [("mamba2", 64, None, False), ("gdn", 128, None, False), ("kda", 128, None, False),
+                                                 ("mamba2", 80, None, False), ("gdn", 128, "pivot", False),
+                                                 ("mamba2", 64, "ridge", False), ("gdn", 128, None, True),
+                                                 ("kda", 128, "pivot", True)])
+def test_sequences_at_different_window_phases_in_one_call(kind, dv, coef, erase):
     """Sequence b takes its first flush when b mod L tokens are buffered and then one every L tokens, so every call mixes
     decode steps at different ring fills with flush steps.  The oracle follows every sequence with its own ring."""
     dev = _dev()
     L = 8
     w = synth.Workload("t", kind, 11, 3, 128, dv, 8, L, 0, "bf16", 137, basis="qr")
-    m, S0, Om, C, _ = make_layer(w, coef=coef)
+    m, S0, Om, C, _ = make_layer(w, coef=coef, erase=erase)
     m.state_update(0)
     Om64 = Om.astype(np.float64)
     S = [S0[b].astype(np.float64) for b in range(w.batch)]                       # per sequence: [H, K, V]

@@ -267,6 +267,28 @@ def test_projected_factors_give_C_qtilde_exactly(kind):
     np.testing.assert_allclose(orc.wy_coefficients(kind, toks, q, C), C @ x, atol=1e-13)
 
 
+@pytest.mark.parametrize("kind", ("gdn", "kda"))
+def test_projected_erase_vectors_are_C_times_the_erase_factors(kind):
+    # f_s := C pi_s (the definition above Eq. 44), with pi_s from the recurrence of Eq. 42 that the dense transition
+    # product pins; and the returned left factors / cumulative decay are those of the WY form
+    K, V, n, G = 10, 3, 7, 4
+    rng = np.random.default_rng(15)
+    toks = rand_tokens(rng, kind, n, K, V, (2,))
+    C = rng.standard_normal((2, G, K))
+    d_cum, pis, ls = orc.wy_factors(kind, toks)
+    fs, ls_f, d = orc.projected_erase_vectors(kind, toks, C)
+    assert len(fs) == n
+    for f_s, pi_s in zip(fs, pis):
+        np.testing.assert_allclose(f_s, np.einsum("bgk,bk->bg", C, pi_s), atol=1e-13)
+    for a, b in zip(ls_f, ls):
+        np.testing.assert_allclose(a, b, atol=1e-15)
+    np.testing.assert_allclose(d, d_cum[-1], atol=1e-15)
+    # a prefix of the window gives the same vectors: f_s does not depend on later tokens
+    fs5, _, _ = orc.projected_erase_vectors(kind, toks[:5], C)
+    for a, b in zip(fs5, fs[:5]):
+        np.testing.assert_allclose(a, b, atol=1e-15)
+
+
 # ---------------------------------------------------------------------------
 # Eq. 5-6: output error identity
 # ---------------------------------------------------------------------------
