@@ -226,12 +226,12 @@ class Stack:
     """`logical` layers of one workload on one GPU, mapped round-robin onto `n_phys` physical layer slots, with one
     window of device-resident inputs per slot."""
 
-    def __init__(self, w: synth.Workload, n_phys: int, logical: int, device: int, coef=None, sketch="f32"):
+    def __init__(self, w: synth.Workload, n_phys: int, logical: int, device: int, coef=None, sketch="f32", erase=False):
         """coef: None (fixed offline map) or "pivot" / "ridge" (state-dependent map rebuilt by every flush);
-        sketch: storage type of U and C."""
+        sketch: storage type of U and C; erase: decode through projected erase vectors (GDN / KDA)."""
         from paper_2609_33051_b200.binding import SketchSSM
         self.w, self.n_phys, self.logical, self.device = w, n_phys, logical, device
-        self.coef, self.sketch = coef, sketch
+        self.coef, self.sketch, self.erase = coef, sketch, erase
         dev = torch.device("cuda", device)
         Om, C = fitted_basis(w)
         wi = input_workload(w)
@@ -252,7 +252,8 @@ class Stack:
         Om_t, C_t = torch.from_numpy(Om), torch.from_numpy(C)
         for li in range(n_phys):
             m = SketchSSM(w.kind, w.batch, w.heads, w.dk, w.dv, w.rank, w.buf_len, io=w.io, out="f32", device=device,
-                          coef_per_seq=coef is not None, coef_pivots=4 if coef == "pivot" else 0, sketch=sketch)
+                          coef_per_seq=coef is not None, coef_pivots=4 if coef == "pivot" else 0, sketch=sketch,
+                          erase_factors=erase)
             gen.manual_seed(w.seed * 1000 + li)
             m.state.normal_(0.0, w.state_std, generator=gen)          # S_init ~ N(0, 0.02^2), drawn on the device
             m.omega.copy_(Om_t)
@@ -373,10 +374,11 @@ class Stack:
         return h2d, d2h
 
 
-def make_stack(w: synth.Workload, budget_gb: float, logical: int, device: int, coef=None, sketch="f32") -> Stack:
+def make_stack(w: synth.Workload, budget_gb: float, logical: int, device: int, coef=None, sketch="f32", erase=False) -> Stack:
     per = layer_bytes(w) + (w.batch * w.heads * w.rank * w.dk * 4 if coef else 0)
+    per += w.batch * w.heads * w.buf_len * w.rank * 4 if erase else 0
     n_phys = physical_layers(per, int(budget_gb * 1e9), logical)
-    return Stack(w, n_phys, logical, device, coef=coef, sketch=sketch)
+    return Stack(w, n_phys, logical, device, coef=coef, sketch=sketch, erase=erase)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -450,12 +452,13 @@ def kernel_figures(w, stack, timer, ms_window, reps, peak):
     L, B, H = w.buf_len, w.batch, w.heads
     n_log = stack.logical
     tkw = dict(sketch_bytes=2 if stack.sketch == "bf16" else 4, coef_per_seq=stack.coef is not None)
+    dkw = dict(tkw, erase_factors=stack.erase)
     ms_d, _, _ = timer.region(stack.run_decode_only, reps, 1)
     us_dec_b2b = 1e3 * ms_d / ((L - 1) * n_log)
     ms_u, _, _ = timer.region(stack.run_update_only, reps, 1)
     us_upd = 1e3 * ms_u / n_log
     stack.run_window("sketch", None)     # leave every layer at the start of a window again
-    by_d = sum(traffic.decode_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io, **tkw) for t in range(L - 1)) / (L - 1)
+    by_d = sum(traffic.decode_bytes(w.kind, B, H, w.dk, w.dv, w.rank, t, w.io, **dkw) for t in range(L - 1)) / (L - 1)
     by_u = traffic.update_bytes(w.kind, B, H, w.dk, w.dv, w.rank, L - 1, w.io, **tkw)
     # what a decode launch costs inside the window: the window minus the flush, over its L-1 decode launches
     us_dec_win = max((1e3 * ms_window / n_log - us_upd) / (L - 1), 1e-3)
@@ -473,9 +476,9 @@ def kernel_figures(w, stack, timer, ms_window, reps, peak):
     }
 
 
-def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25, coef=None, sketch="f32"):
+def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25, coef=None, sketch="f32", erase=False):
     """One sweep record: the sketch window, the full-read window, per-kernel figures, byte accounting, clocks."""
-    stack = make_stack(w, budget_gb, logical, device, coef=coef, sketch=sketch)
+    stack = make_stack(w, budget_gb, logical, device, coef=coef, sketch=sketch, erase=erase)
     try:
         L, B, H = w.buf_len, w.batch, w.heads
         tokens = B * L * logical
@@ -494,7 +497,7 @@ def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25, 
             m.check_status()
         mean_n = (L - 2) / 2.0
         tkw = dict(sketch_bytes=2 if sketch == "bf16" else 4, coef_per_seq=coef is not None)
-        dec_b = traffic.decode_bytes(w.kind, 1, 1, w.dk, w.dv, w.rank, 0, w.io, **tkw)
+        dec_b = traffic.decode_bytes(w.kind, 1, 1, w.dk, w.dv, w.rank, 0, w.io, erase_factors=erase, **tkw)
         if coef is None:
             dec_b -= w.rank * w.dk * tkw["sketch_bytes"]          # the shared map is read once per launch, not per head
         from paper_2609_33051_b200.binding import NO_SKETCH
@@ -507,6 +510,7 @@ def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25, 
             "coefficient_map": {None: "fixed offline map [H][r][K]", "pivot": "state-dependent, P = 4 approximation, lambda 0.1, "
                                 "rebuilt by every flush [B][H][r][K]", "ridge": "state-dependent, exact ridge solve, lambda 0.1"}[coef],
             "sketch_storage": sketch,
+            "erase_factors": bool(erase),
             "flush_without_sketch_us": 1e3 * ms_u0 / logical,
             "sketch_and_map_overhead_on_flush": figs["update"]["back_to_back_us"] / (1e3 * ms_u0 / logical) - 1.0,
             "n_phys": stack.n_phys, "device_bytes": stack.device_bytes(), "steps": steps,
@@ -520,7 +524,7 @@ def measure_point(w, budget_gb, logical, device, timer, peak, min_seconds=0.25, 
             "update_frac_of_measured": figs["update"]["frac_of_measured"],
             "update_frac_of_8TBs_nominal": figs["update"]["frac_of_8TBs_nominal"],
             "full_read": {"value": tokens / (ms_full * 1e-3), "unit": UNIT, "sketch_speedup": ms_full / ms},
-            "decode_bytes_per_token_head": dec_b + mean_n * slot, "full_read_bytes_per_token_head": full_b + mean_n * slot,
+            "decode_bytes_per_token_head": dec_b + mean_n * (slot + (w.rank * 4 if erase else 0)), "full_read_bytes_per_token_head": full_b + mean_n * slot,
             "state_read_ratio_dk_over_r": w.dk / w.rank,
             "clocks": clocks,
         }
@@ -589,6 +593,7 @@ def main():
     ap.add_argument("--tune", default="", help="comma list key=value passed to sketchssm_tune")
     ap.add_argument("--coef", default="fixed", choices=["fixed", "pivot", "ridge"], help="coefficient map of the headline stack")
     ap.add_argument("--sketch", default="f32", choices=["f32", "bf16"], help="storage type of U and C of the headline stack")
+    ap.add_argument("--erase-factors", action="store_true", help="GDN / KDA workloads: decode through projected erase vectors (Eq. 44-45)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -651,7 +656,8 @@ def main():
     timer = Timer(dist, local_rank)
     peak, peak_kind = measured_peaks()
 
-    stack = make_stack(w, args.budget_gb, logical, local_rank, coef=None if args.coef == "fixed" else args.coef, sketch=args.sketch)
+    stack = make_stack(w, args.budget_gb, logical, local_rank, coef=None if args.coef == "fixed" else args.coef, sketch=args.sketch,
+                       erase=args.erase_factors)
     for kv in filter(None, args.tune.split(",")):
         k, v = kv.split("=")
         for m in stack.layers:
@@ -793,7 +799,9 @@ def main():
     if not args.no_sweep and world == 1:
         variants = [measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, coef="pivot"),
                     measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, sketch="bf16"),
-                    measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, coef="pivot")]
+                    measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, coef="pivot"),
+                    measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True),
+                    measure_point(synth.CONFIGS["c4_kda"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True)]
 
     # ---- CPU oracle on a bounded sample (rank 0, N = 1) ----
     cpu = None

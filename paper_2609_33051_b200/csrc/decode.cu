@@ -93,7 +93,7 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
 //      1 = per-sequence phases and / or a per-head rank table (sizes follow the head);
 //      2 = 1 with the coefficient vector formed from projected erase vectors (delta-rule kinds).
 template <int KIND, typename IO, int K, int V, int RT, int GEN>
-__global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
+__global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
     constexpr int EV = V % 32 == 0 ? V / 32 : 4;        // value elements per lane ...
     constexpr int VL = V / EV;                          // ... on the first VL lanes (all 32, or 20 for V = 80)
@@ -422,53 +422,75 @@ __global__ void __launch_bounds__(256, 4) decode_kernel(const Params p) {
 #pragma unroll
             for (int e = 0; e < EK; ++e) x[e] = dsuf * q0[e];
         } else {
-            // Erase mode: next to the sweep (which the exact output of the buffered tokens needs anyway), the left factors
+            // Erase mode: before the sweep (which the exact output of the buffered tokens needs anyway), the left factors
             // l_s(t) = (D_t ... D_{s+1}) k_s give <l_s(t), q_t> and <l_s(t), k_t> for every slot (Eq. 46: from the stored keys
-            // and the running product of the decays); dl / dlv end up as the cumulative decay d_[t].
+            // and the running product of the decays), eight slots per transposing reduction, from the newest slot down.
+            // KDA: dlv ends up as the cumulative decay d_[t].  GDN: the dot products are those of the raw keys, scaled by
+            // the running scalar product inside the sweep below, where dl ends up as d_[t].
             float dl = dsc;
             float dlv[EK];
 #pragma unroll
             for (int e = 0; e < EK; ++e) dlv[e] = KIND == SKETCHSSM_KDA ? gg[e] : 1.f;
+            if constexpr (ER) {
+                if (er_h) {
+                    for (int sb = n - 1; sb >= 0; sb -= NB) {
+                        float pq[NB], pk[NB];
+#pragma unroll
+                        for (int i = 0; i < NB; ++i) {
+                            const int s = sb - i;
+                            const int sc = s < 0 ? 0 : s;              // (rows below slot 0: computed, never stored)
+                            float kr[EK];
+                            load_io<EK>(sK, sc * K + lane * EK, kr);
+                            float aq = 0.f, ak = 0.f;
+#pragma unroll
+                            for (int e = 0; e < EK; ++e) {
+                                const float le = KIND == SKETCHSSM_KDA ? dlv[e] * kr[e] : kr[e];
+                                aq = fmaf(le, q0[e], aq);
+                                ak = fmaf(le, kk[e], ak);
+                            }
+                            pq[i] = aq;
+                            pk[i] = ak;
+                            if constexpr (KIND == SKETCHSSM_KDA) {
+                                if (s >= 0) {
+                                    float gr[EK];
+                                    load_io<EK>(sG, s * K + lane * EK, gr);
+#pragma unroll
+                                    for (int e = 0; e < EK; ++e) dlv[e] *= gr[e];
+                                }
+                            }
+                        }
+                        group_reduce_transpose<32, NB>(pq, lane);       // lane l holds entry l / 4: slot sb - l / 4
+                        group_reduce_transpose<32, NB>(pk, lane);
+                        const int s = sb - (lane >> 2);
+                        if ((lane & 3) == 0 && s >= 0) { sP[s] = pq[0]; sP[32 + s] = pk[0]; }
+                    }
+                    __syncwarp();
+                }
+            }
 #pragma unroll 2
             for (int s = n - 1; s >= 0; --s) {
-                float kr[EK], vr[EV], gr[EK];
+                float kr[EK], vr[EV];
                 load_io<EK>(sK, s * K + lane * EK, kr);
 #pragma unroll
                 for (int e = 0; e < EV; ++e) vr[e] = 0.f;
                 if (vlane) load_io<EV>(sV, s * V + lane * EV, vr);
-                if constexpr (KIND == SKETCHSSM_KDA && ER) load_io<EK>(sG, s * K + lane * EK, gr);
                 float part = 0.f;
 #pragma unroll
                 for (int e = 0; e < EK; ++e) part = fmaf(kr[e], x[e], part);
                 const float a = sBeta[s] * warp_sum(part);
-                if constexpr (ER) {
-                    if (er_h) {
-                        float pq = 0.f, pk = 0.f;
-#pragma unroll
-                        for (int e = 0; e < EK; ++e) {
-                            const float le = KIND == SKETCHSSM_KDA ? dlv[e] * kr[e] : kr[e];
-                            pq = fmaf(le, q0[e], pq);
-                            pk = fmaf(le, kk[e], pk);
-                        }
-                        pq = warp_sum(pq);
-                        pk = warp_sum(pk);
-                        if constexpr (KIND == SKETCHSSM_GDN) {
-                            pq *= dl;
-                            pk *= dl;
-                            dl *= sDec[s];
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < EK; ++e) dlv[e] *= gr[e];
-                        }
-                        if (lane == 0) { sP[s] = pq; sP[32 + s] = pk; }
-                    }
-                }
                 if constexpr (KIND == SKETCHSSM_GDN) {
                     const float d = sDec[s];
+                    if constexpr (ER) {
+                        if (er_h) {
+                            if (lane == 0) { sP[s] *= dl; sP[32 + s] *= dl; }
+                            dl *= d;
+                        }
+                    }
 #pragma unroll
                     for (int e = 0; e < EK; ++e) x[e] = d * fmaf(-a, kr[e], x[e]);
                 } else {
-                    if constexpr (!ER) load_io<EK>(sG, s * K + lane * EK, gr);
+                    float gr[EK];
+                    load_io<EK>(sG, s * K + lane * EK, gr);
 #pragma unroll
                     for (int e = 0; e < EK; ++e) x[e] = gr[e] * fmaf(-a, kr[e], x[e]);
                 }

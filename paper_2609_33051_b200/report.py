@@ -61,7 +61,7 @@ def table(rows) -> str:
         name = s["workload"].split(":")[0]
         shape = s["workload"].split(":")[1].strip()
         var = ("fixed" if s["coefficient_map"].startswith("fixed") else "state-dep. P=4" if "P = 4" in s["coefficient_map"] else "state-dep. exact") \
-            + " / " + s["sketch_storage"]
+            + " / " + s["sketch_storage"] + (" / erase vectors" if s.get("erase_factors") else "")
         out.append(f"| {name} ({shape}) | {var} | {s['n_phys']} | {s['value'] / 1e6:.2f} | {s['decode_in_window_us']:.1f} | "
                    f"{s['decode_frac_of_measured']:.2f} | {s['decode_frac_of_8TBs_nominal']:.2f} | {s['update_kernel']} | {s['update_us']:.0f} | "
                    f"{s['update_frac_of_measured']:.2f} | {100 * s['sketch_and_map_overhead_on_flush']:.0f} % | "
