@@ -92,7 +92,9 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
 // GEN: 0 = one ring fill and one rank for every head of the launch (copy sizes are per-lane constants);
 //      1 = per-sequence phases and / or a per-head rank table (sizes follow the head);
 //      2 = 1 with the coefficient vector formed from projected erase vectors (delta-rule kinds).
-template <int KIND, typename IO, int K, int V, int RT, int GEN>
+// UB: the sketch rows and the fixed coefficient map are stored as bfloat16 (a compile-time fact for the lean
+//     instantiation; the general ones read the flag of the launch).
+template <int KIND, typename IO, int K, int V, int RT, int GEN, bool UB = false>
 __global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
     constexpr int EV = V % 32 == 0 ? V / 32 : 4;        // value elements per lane ...
@@ -108,7 +110,7 @@ __global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Par
     const int n_cap = p.n_before;                       // ring rows the stage has room for (per-sequence phases: the largest fill)
     const bool vlane = VL == 32 || lane < VL;           // this lane holds value elements
     const bool per_seq = GEN && p.coef_per_seq;         // the head's own coefficient map travels with its sketch rows
-    const bool u_bf16 = GEN && p.sketch_bf16;           // sketch rows (and the fixed coefficient map) stored as bfloat16
+    const bool u_bf16 = UB || (GEN && p.sketch_bf16);   // sketch rows (and the fixed coefficient map) stored as bfloat16
     const int su = u_bf16 ? 2 : 4;
     const int RP = (R + 7) & ~7;
     // c_t from the projected erase vectors of the buffered tokens instead of the swept query (delta-rule kinds)
@@ -662,15 +664,19 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     // warps per CTA / CTAs per SM: as many resident warps per SM as shared memory allows (capped), preferring
     // fewer, larger CTAs
     const int cap = p.max_warps_per_sm > 0 ? p.max_warps_per_sm : 32;
-    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq || p.sketch_bf16 || erase;
+    // bfloat16 storage with nothing else that needs the general kernel: the lean rank-16 instantiation reads it too
+    const bool lean_bf16 = p.sketch_bf16 && p.R == 16 && !p.full_read && p.head_rank == nullptr && p.n_dev == nullptr &&
+                           !p.coef_per_seq && !erase;
+    const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq || (p.sketch_bf16 && !lean_bf16) || erase;
     const bool fixed16 = p.R == 16 && !gen;     // the unrolled rank-16 instantiation needs one rank for all heads
     auto kern = gen ? decode_kernel<KIND, IO, K, V, 0, 1> : fixed16 ? decode_kernel<KIND, IO, K, V, 16, 0> : decode_kernel<KIND, IO, K, V, 0, 0>;
+    if (lean_bf16) kern = decode_kernel<KIND, IO, K, V, 16, 0, true>;
     if constexpr (KIND != SKETCHSSM_MAMBA2) {
         if (erase) kern = decode_kernel<KIND, IO, K, V, 0, 2>;
     }
     // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does
-    static int regs_per_thread[4] = {0, 0, 0, 0};
-    int& regs = regs_per_thread[erase ? 3 : gen ? 2 : fixed16 ? 1 : 0];
+    static int regs_per_thread[5] = {0, 0, 0, 0, 0};
+    int& regs = regs_per_thread[lean_bf16 ? 4 : erase ? 3 : gen ? 2 : fixed16 ? 1 : 0];
     if (regs == 0) {
         cudaFuncAttributes fa;
         if ((ctx->last_cuda_error = cudaFuncGetAttributes(&fa, kern)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
