@@ -37,6 +37,15 @@ def test_erase_factors_with_the_state_dependent_map(kind, coef):
     assert errs["S"] <= FP32_GUARD and errs["U"] <= FP32_GUARD, errs
 
 
+@pytest.mark.parametrize("kind", ("gdn", "kda"))
+def test_erase_factors_with_bfloat16_sketch_storage(kind):
+    # U and the fixed map stored as bfloat16 (the oracle rounds U where the flush stores it, and both sides get the map
+    # already rounded); the erase vectors themselves stay fp32
+    w = synth.Workload("t", kind, 6, 4, 128, 128, 16, 16, 0, "bf16", 229, basis="qr")
+    errs = run_schedule(w, 2 * w.buf_len + 2, max_heads=10**9, sketch="bf16", erase=True)
+    assert errs["out"] <= 2e-3 + 2.0 ** -9 and errs["f"] <= FP32_GUARD and errs["S"] <= FP32_GUARD, errs
+
+
 def test_erase_factors_give_the_same_outputs_as_the_swept_query():
     # same layer, same tokens, with and without the projected vectors: equal up to rounding order
     dev = torch.device("cuda", 0)
