@@ -31,7 +31,8 @@ traffic-reduction values printed in Tables 4-7, and for the state-dependent
 coefficient maps of Appendix A.2: a library least-squares solve of the ridge
 problem, the range projection in the limit of no ridge, independence of the
 orthogonal completion, the Woodbury step against a dense inverse, exactness of
-the pivot approximation when P >= G, and a hand-rolled brute force on tiny heads.  Absolute output values on
+the pivot approximation when P >= G, a hand-rolled brute force on tiny heads, and the sketch-form restatements
+(*_from_sketch) against the appendix forms at the exact sketch.  Absolute output values on
 the benchmark workloads have no printed counterpart in the paper: for those,
 parity is pinned only through the identities above ("parity unpinned" by a
 worked numeric example).
@@ -404,10 +405,59 @@ def pivot_coefficient_map(S0, Omega, lam=0.1, P=4):
     return A_inv_rhs @ R
 
 
-def coefficient_maps(S, Omega, mode, lam=0.1, P=4):
+def ridge_coefficient_map_from_sketch(S0, U, lam=0.1):
+    """The ridge map of Eq. 28-29 carried back from the rotated coordinates to the quantities a kernel holds
+    (J^T H J = U^T U / mu, J^T H R = U^T S_0^T / mu for U = S_0^T Omega):  C = (U^T U + lam mu I)^{-1} U^T S_0^T,
+    mu = ||S_0||_F^2 / K (1 for a zero state).  Equal to ridge_coefficient_map when U is the exact sketch; stated in
+    terms of U so that it also defines the map built from a sketch that was rounded when it was stored.
+    S0 [K, V], U [V, G]."""
+    S0, U = _f64(S0), _f64(U)
+    K, G = S0.shape[0], U.shape[1]
+    mu = float(np.sum(S0 * S0)) / K
+    if mu == 0.0:
+        mu = 1.0
+    return np.linalg.solve(U.T @ U + lam * mu * np.eye(G), U.T @ S0.T)
+
+
+def pivot_coefficient_map_from_sketch(S0, U, Omega, lam=0.1, P=4):
+    """The approximated map of Eq. 30-37 in the same carried-back form: with Q the Gram-Schmidt basis of the first p
+    sketch columns, L_G = U^T Q / sqrt(mu), d_g = max((||U_g||^2 - ||Q^T U_g||^2) / mu, 0), D_G = Diag(d) + lam I,
+    C = (D_G + L_G L_G^T)^{-1} [L_G Q^T S_0^T / sqrt(mu) + Diag(d) Omega^T], the inverse through the p x p Woodbury
+    system.  Equal to pivot_coefficient_map when U is the exact sketch.  S0 [K, V], U [V, G], Omega [K, G]."""
+    S0, U, Omega = _f64(S0), _f64(U), _f64(Omega)
+    K, G = Omega.shape
+    mu = float(np.sum(S0 * S0)) / K
+    if mu == 0.0:
+        mu = 1.0
+    p = min(G, P)
+    Q = np.zeros((U.shape[0], p))
+    for j in range(p):
+        u = U[:, j].copy()
+        for i in range(j):
+            u -= Q[:, i] * (Q[:, i] @ U[:, j])
+        for i in range(j):
+            u -= Q[:, i] * (Q[:, i] @ u)
+        nrm, ref = np.linalg.norm(u), np.linalg.norm(U[:, j])
+        Q[:, j] = u / nrm if nrm > 1e-10 * max(ref, 1e-300) and ref > 0 else 0.0
+    LG = U.T @ Q / np.sqrt(mu)                                     # G x p
+    d = np.maximum((np.sum(U * U, axis=0) - np.sum((Q.T @ U) ** 2, axis=0)) / mu, 0.0)
+    DG = d + lam
+    rhs = LG @ (Q.T @ S0.T) / np.sqrt(mu) + d[:, None] * Omega.T   # G x K
+    TP = np.eye(p) + LG.T @ (LG / DG[:, None])
+    Dinv_rhs = rhs / DG[:, None]
+    return Dinv_rhs - (LG / DG[:, None]) @ np.linalg.solve(TP, LG.T @ Dinv_rhs)
+
+
+def coefficient_maps(S, Omega, mode, lam=0.1, P=4, U=None):
     """Per-head state-dependent maps for a batch of heads: S [N, K, V], Omega [N, K, G] -> C [N, G, K].
-    mode "ridge": ridge_coefficient_map; mode "pivot": pivot_coefficient_map."""
+    mode "ridge": ridge_coefficient_map; mode "pivot": pivot_coefficient_map.  With U [N, V, G] given (the sketch as it
+    was stored, e.g. rounded to bfloat16) the maps are built from that sketch by the *_from_sketch forms."""
     S, Omega = _f64(S), _f64(Omega)
+    if U is not None:
+        U = _f64(U)
+        fn = {"ridge": lambda i: ridge_coefficient_map_from_sketch(S[i], U[i], lam),
+              "pivot": lambda i: pivot_coefficient_map_from_sketch(S[i], U[i], Omega[i], lam, P)}[mode]
+        return np.stack([fn(i) for i in range(S.shape[0])])
     fn = {"ridge": lambda s, o: ridge_coefficient_map(s, o, lam), "pivot": lambda s, o: pivot_coefficient_map(s, o, lam, P)}[mode]
     return np.stack([fn(S[i], Omega[i]) for i in range(S.shape[0])])
 

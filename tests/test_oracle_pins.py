@@ -572,6 +572,38 @@ def test_pivot_map_handles_dependent_pivot_columns_and_the_zero_state():
     assert np.allclose(orc.pivot_coefficient_map(Z, Om), 0.0) and np.allclose(orc.ridge_coefficient_map(Z, Om), 0.0)
 
 
+def test_sketch_form_maps_equal_the_appendix_forms_at_the_exact_sketch():
+    """The restatements in terms of (S_0, U, Omega) that define the map built from a stored sketch: at U = S_0^T Omega
+    they are the appendix's maps (which are pinned above); with a dependent pivot column and the zero state too; and
+    the ridge form at a perturbed U is still the regularised least-squares solution for that U."""
+    rng = np.random.default_rng(18)
+    for (K, V, G, P, lam) in [(16, 12, 5, 4, 0.1), (24, 8, 8, 4, 0.1), (12, 10, 3, 4, 0.7), (20, 16, 6, 2, 0.1)]:
+        S, Om = _head(rng, K, V, G)
+        U = S.T @ Om
+        np.testing.assert_allclose(orc.ridge_coefficient_map_from_sketch(S, U, lam), orc.ridge_coefficient_map(S, Om, lam),
+                                   rtol=0, atol=1e-10)
+        np.testing.assert_allclose(orc.pivot_coefficient_map_from_sketch(S, U, Om, lam, P),
+                                   orc.pivot_coefficient_map(S, Om, lam, P), rtol=0, atol=1e-10)
+        Cb = orc.coefficient_maps(S[None], Om[None], "pivot", lam, P, U=U[None])
+        np.testing.assert_allclose(Cb[0], orc.pivot_coefficient_map(S, Om, lam, P), atol=1e-10)
+        # a sketch that is not exactly S^T Omega (as after rounding): the ridge form solves the least-squares problem of that U
+        Up = U * (1.0 + 2.0 ** -8 * (rng.random(U.shape) < 0.3))
+        C = orc.ridge_coefficient_map_from_sketch(S, Up, lam)
+        mu = float((S * S).sum()) / K
+        q = rng.standard_normal(K)
+        A = np.concatenate([Up / np.sqrt(mu), np.sqrt(lam) * np.eye(G)])
+        b = np.concatenate([S.T @ q / np.sqrt(mu), np.zeros(G)])
+        np.testing.assert_allclose(C @ q, np.linalg.lstsq(A, b, rcond=None)[0], atol=1e-10)
+    K, V, G = 10, 8, 4
+    S, Om = _head(rng, K, V, G)
+    w = Om[:, 1] - 3.0 * Om[:, 0]
+    S = S - np.outer(w, w @ S) / (w @ w)
+    np.testing.assert_allclose(orc.pivot_coefficient_map_from_sketch(S, S.T @ Om, Om), orc.pivot_coefficient_map(S, Om), atol=1e-9)
+    Z = np.zeros((K, V))
+    assert np.allclose(orc.pivot_coefficient_map_from_sketch(Z, Z.T @ Om, Om), 0.0)
+    assert np.allclose(orc.ridge_coefficient_map_from_sketch(Z, Z.T @ Om), 0.0)
+
+
 def test_pivot_map_brute_force_on_tiny_heads():
     """K, V <= 4 with Python loops only: rotate the state, build mu, H, the Gram-Schmidt basis of the first p sketch
     columns, L, d and H^ entry by entry, and solve the G x G normal equations by hand-written elimination."""
