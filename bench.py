@@ -375,7 +375,7 @@ class Stack:
 
 
 def make_stack(w: synth.Workload, budget_gb: float, logical: int, device: int, coef=None, sketch="f32", erase=False) -> Stack:
-    per = layer_bytes(w) + (w.batch * w.heads * w.rank * w.dk * 4 if coef else 0)
+    per = layer_bytes(w) + (w.batch * w.heads * w.rank * w.dk * (2 if sketch == "bf16" else 4) if coef else 0)
     per += w.batch * w.heads * w.buf_len * w.rank * 4 if erase else 0
     n_phys = physical_layers(per, int(budget_gb * 1e9), logical)
     return Stack(w, n_phys, logical, device, coef=coef, sketch=sketch, erase=erase)
@@ -799,6 +799,7 @@ def main():
     if not args.no_sweep and world == 1:
         variants = [measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, coef="pivot"),
                     measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, sketch="bf16"),
+                    measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, coef="pivot", sketch="bf16"),
                     measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, coef="pivot"),
                     measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True),
                     measure_point(synth.CONFIGS["c4_kda"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True)]

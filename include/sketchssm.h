@@ -100,8 +100,10 @@ typedef struct sketchssm_config {
     int32_t sketch_dtype;   /* sketchssm_dtype of the stored sketch U and coefficient map C: SKETCHSSM_F32 (default) or
                                SKETCHSSM_BF16, the storage the paper's traffic model assumes (T_G = 2 G (V + K) bytes per
                                non-flush read, Appendix D).  U is rounded to bfloat16 once, when the flush stores it; all
-                               arithmetic stays fp32.  With bfloat16 storage C is the fixed offline map (coef_per_seq = 0),
-                               handed over as bfloat16 [H][r][K], and only the default one-kernel decode is available. */
+                               arithmetic stays fp32.  The fixed offline map (coef_per_seq = 0) is then handed over as
+                               bfloat16 [H][r][K]; the state-dependent map (coef_per_seq = 1) is built from the sketch as
+                               stored (the rounded rows) and rounded to bfloat16 once, when it is stored [B][H][r][K].
+                               Only the default one-kernel decode is available with bfloat16 storage. */
     int32_t erase_factors;  /* GDN / KDA only.  0 (default): the decode step forms the effective query q~_t by the backward
                                sweep over the ring and then c_t = C q~_t.  1: it forms c_t from projected erase vectors
                                (Appendix C.2, Eq. 44-45): every appended token leaves f_s = beta_s [C (d_[s] * k_s) -

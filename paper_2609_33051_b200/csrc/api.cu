@@ -172,7 +172,6 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
     if ((size_t)cfg->batch * cfg->heads > (size_t)1 << 24) return SKETCHSSM_UNSUPPORTED_SHAPE;
     if (cfg->coef_per_seq != 0 && cfg->coef_per_seq != 1) return SKETCHSSM_INVALID_ARG;
     if (cfg->sketch_dtype != SKETCHSSM_F32 && cfg->sketch_dtype != SKETCHSSM_BF16) return SKETCHSSM_INVALID_ARG;
-    if (cfg->sketch_dtype == SKETCHSSM_BF16 && cfg->coef_per_seq) return SKETCHSSM_UNSUPPORTED_SHAPE;   // bfloat16 storage: fixed offline map
     if (cfg->erase_factors != 0 && cfg->erase_factors != 1) return SKETCHSSM_INVALID_ARG;
     if (cfg->erase_factors) {
         if (cfg->kind == SKETCHSSM_MAMBA2) return SKETCHSSM_INVALID_ARG;            // no erase term: nothing to project

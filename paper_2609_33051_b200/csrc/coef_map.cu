@@ -93,15 +93,34 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
     constexpr int RUP = PM;                // pitch of RU in the pivot form (16- or 32-byte rows, zero beyond m)
 
     const int RS = p.R;                // row strides of U, C and Omega follow the configured rank
-    const float* Ug = p.sketch + bh * (size_t)RS * V;
+    const float* Ug = p.sketch + bh * (size_t)RS * V;                  // (fp32 storage)
     const float* Sg = p.state + bh * (size_t)K * V;
+    // the map is stored like the sketch: fp32, or rounded to bfloat16 once, here
     float* Cg = const_cast<float*>(p.coef) + bh * (size_t)RS * K;
+    __nv_bfloat16* Cg16 = reinterpret_cast<__nv_bfloat16*>(const_cast<float*>(p.coef)) + bh * (size_t)RS * K;
+    const bool bf = p.sketch_bf16 != 0;
+    auto store_c = [&](size_t idx, float x) {
+        if (bf) Cg16[idx] = __float2bfloat16_rn(x);
+        else Cg[idx] = x;
+    };
     const float* Om = p.omega + (size_t)h * K * RS;
 
     // ---- sketch rows into shared memory ----
-    for (int i = tid; i < G * V / 4; i += kCoefThreads) {
-        const int g = i / (V / 4), c = i - g * (V / 4);
-        *reinterpret_cast<float4*>(sU + g * PT + 4 * c) = *reinterpret_cast<const float4*>(Ug + (size_t)g * V + 4 * c);
+    // (with bfloat16 storage the map is built from the sketch as stored, i.e. from the rounded rows)
+    if (bf) {
+        const uint2* Ug16 = reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(p.sketch) + bh * (size_t)RS * V);
+        for (int i = tid; i < G * V / 4; i += kCoefThreads) {
+            const int g = i / (V / 4), c = i - g * (V / 4);
+            const uint2 t = Ug16[(size_t)g * (V / 4) + c];
+            *reinterpret_cast<float4*>(sU + g * PT + 4 * c) =
+                make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
+                            __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+        }
+    } else {
+        for (int i = tid; i < G * V / 4; i += kCoefThreads) {
+            const int g = i / (V / 4), c = i - g * (V / 4);
+            *reinterpret_cast<float4*>(sU + g * PT + 4 * c) = *reinterpret_cast<const float4*>(Ug + (size_t)g * V + 4 * c);
+        }
     }
     __syncthreads();
     // ||U_g||^2, one row per thread
@@ -325,7 +344,7 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
 #pragma unroll
                 for (int j = 0; j < PM; ++j) { Mg = fmaf(ru[j], y[j], Mg); corr = fmaf(ru[j], wv[j], corr); }
                 Mg = fmaf(Mg, inv_mu, sUU[g] * omk[g]);
-                Cg[(size_t)g * K + k] = (Mg - corr) * sD[g];
+                store_c((size_t)g * K + k, (Mg - corr) * sD[g]);
             }
         }
     } else {
@@ -358,7 +377,7 @@ __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) 
                 float t = y[g];
                 for (int j = g + 1; j < G; ++j) t = fmaf(-sRU[j * MP + g], y[j], t);
                 y[g] = t / sRU[g * MP + g];
-                Cg[(size_t)g * K + k] = y[g];
+                store_c((size_t)g * K + k, y[g]);
             }
         }
     }

@@ -49,8 +49,8 @@ __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K
     uint32_t off = 0;
     s.u_off = off; s.u_bytes = full_read ? 0u : (uint32_t)(R * V * sketch_bytes); off += (s.u_bytes + 15u) & ~15u;
     // rows padded to the reduction width are read (their sums are never used), so they get room but are not copied
-    s.c_off = off; s.c_bytes = (!full_read && coef_per_seq) ? (uint32_t)(R * K * 4) : 0u;
-    off += (!full_read && coef_per_seq) ? (uint32_t)(((R + 7) & ~7) * K * 4) : 0u;
+    s.c_off = off; s.c_bytes = (!full_read && coef_per_seq) ? (uint32_t)(R * K * sketch_bytes) : 0u;
+    off += (!full_read && coef_per_seq) ? (uint32_t)(((R + 7) & ~7) * K * sketch_bytes) : 0u;
     s.f_off = off; s.f_bytes = (!full_read && erase) ? (uint32_t)(n * R * 4) : 0u; off += s.f_bytes;
     s.k_off = off; s.k_bytes = (uint32_t)(n * K * io); off += s.k_bytes;
     s.v_off = off; s.v_bytes = (uint32_t)(n * V * io); off += s.v_bytes;
@@ -183,14 +183,14 @@ __global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Par
         case 6: cp_base = p.ring + p.rl.v_off; cp_stride = p.rl.head_bytes; cp_dst = sl.v_off; cp_unit = (uint32_t)(V * sizeof(IO)); cp_mode = 1; break;
         case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_unit = KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u; cp_mode = 1; break;
         case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * su; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * su); cp_mode = 3; break;
-        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * 4; cp_dst = sl.c_off; cp_unit = per_seq ? (uint32_t)(K * 4) : 0u; cp_mode = 3; break;
+        case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * su; cp_dst = sl.c_off; cp_unit = per_seq ? (uint32_t)(K * su) : 0u; cp_mode = 3; break;
         case 10: cp_base = reinterpret_cast<const unsigned char*>(p.erase); cp_stride = (size_t)L * R * 4; cp_dst = sl.f_off; cp_unit = er ? (uint32_t)(R * 4) : 0u; cp_mode = 1; break;
         default: break;
     }
     const uint32_t tokA = 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
     const uint32_t rowA = (uint32_t)((K + V) * sizeof(IO)) + (KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u);
     const uint32_t gateA = (uint32_t)((KIND == SKETCHSSM_KDA ? 1 : 2) * L * 4);
-    const uint32_t rowB = (uint32_t)(V * su) + (per_seq ? (uint32_t)(K * 4) : 0u);
+    const uint32_t rowB = (uint32_t)(V * su) + (per_seq ? (uint32_t)(K * su) : 0u);
     const int r_uni = p.full_read ? 0 : R;          // GEN = 0: the rank of every head
     // GEN = 0: the size of this lane's copy and the two transaction totals are constants of the launch
     const uint32_t cp_fixed = cp_mode == 0 ? cp_unit : cp_mode == 1 ? cp_unit * (uint32_t)n_cap
@@ -527,6 +527,7 @@ __global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Par
                     break;
                 }
             }
+            const bool c16 = GEN && per_seq && u_bf16;       // the head's own map travels as bfloat16 (the shared map was widened when staged)
             const int rp_it = RT ? ((RT + 7) & ~7) : ((rk + 7) & ~7);
 #pragma unroll
             for (int g0 = 0; g0 < (RT ? ((RT + 7) & ~7) : rp_it); g0 += NB) {
@@ -534,7 +535,8 @@ __global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Par
 #pragma unroll
                 for (int i = 0; i < NB; ++i) {
                     float cw[EK];
-                    load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
+                    if (c16) load_io<EK>(reinterpret_cast<const __nv_bfloat16*>(sC), (g0 + i) * K + lane * EK, cw);
+                    else load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
                     float acc = 0.f;
 #pragma unroll
                     for (int e = 0; e < EK; ++e) acc = fmaf(cw[e], x[e], acc);
@@ -550,7 +552,8 @@ __global__ void __launch_bounds__(256, GEN == 2 ? 3 : 4) decode_kernel(const Par
 #pragma unroll
                         for (int i = 0; i < NB; ++i) {
                             float cw[EK];
-                            load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
+                            if (c16) load_io<EK>(reinterpret_cast<const __nv_bfloat16*>(sC), (g0 + i) * K + lane * EK, cw);
+                            else load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
                             float acc = 0.f;
 #pragma unroll
                             for (int e = 0; e < EK; ++e) acc = fmaf(cw[e], kk[e], acc);

@@ -34,7 +34,7 @@ def decode_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, full_rea
     shared = 0
     if not full_read:
         if coef_per_seq:
-            per_head += r * K * 4                                   # the head's own C (fp32)
+            per_head += r * K * sketch_bytes                        # the head's own C
         else:
             shared = H * r * K * sketch_bytes                       # C, once per launch
         if erase_factors and kind != "mamba2":
@@ -53,6 +53,6 @@ def update_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, has_toke
     per_head += slot_bytes(kind, K, V, io) if has_token else 0
     per_head += (K * _io(io) + V * out_bytes) if with_output else 0  # q in, o out
     per_head += r * V * sketch_bytes if sketch else 0               # U write
-    per_head += r * K * 4 if (sketch and coef_per_seq) else 0       # C write
+    per_head += r * K * sketch_bytes if (sketch and coef_per_seq) else 0   # C write
     shared = H * K * r * 4 if sketch else 0                         # Omega
     return B * H * per_head + shared

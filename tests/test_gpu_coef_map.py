@@ -35,6 +35,21 @@ def test_state_dependent_map_ranks_and_shapes(rank, dk, dv, coef):
     check_coef(run_schedule(w, w.buf_len + 3, max_heads=10**9, coef=coef))
 
 
+@pytest.mark.parametrize("kind,dv", [("mamba2", 64), ("gdn", 128), ("kda", 128)])
+@pytest.mark.parametrize("coef", ["pivot", "ridge"])
+def test_state_dependent_map_with_bfloat16_storage(kind, dv, coef):
+    """The paper's storage of the paper's method: U and the per-head maps as bfloat16.  The map is built from the sketch
+    as stored (the oracle's sketch-form restatement, from its own rounded U) and rounded once where it is stored.  A
+    stored element next to a rounding boundary may fall on the other side of it on the two sides (one bfloat16 spacing,
+    2^-8 relative): U and C are held to 2^-7 of their largest element; such an element of U also moves the map a little
+    (measured: a few 1e-4 of max |C|), so the outputs get the bar of the bfloat16 sketch test."""
+    w = synth.Workload("t", kind, 5, 3, 128, dv, 16, 8, 0, "bf16", 113, basis="qr")
+    errs = run_schedule(w, 2 * w.buf_len + 3, max_heads=10**9, coef=coef, sketch="bf16")
+    assert errs["out"] <= 2e-3 + 2.0 ** -9, errs
+    assert errs["S"] <= FP32_GUARD, errs
+    assert max(errs["U"], errs["u0"], errs["C"], errs["c0"]) <= 2.0 ** -7, errs
+
+
 @pytest.mark.parametrize("name", ["c2_mamba2", "c3_gdn"])
 def test_state_dependent_map_full_batch_sampled_heads(name):
     w = synth.CONFIGS[name]
