@@ -110,6 +110,77 @@ def test_no_kernel_writes_outside_a_caller_buffer(kind, batch, heads, dv, rank, 
     assert int(m.status.abs().sum().item()) == 0
 
 
+@pytest.mark.parametrize("kind,coef,sketch,erase,ranks", [
+    ("mamba2", "pivot", "bf16", False, False), ("gdn", "pivot", "f32", True, True), ("kda", None, "bf16", True, False),
+    ("gdn", "ridge", "bf16", False, True), ("kda", "pivot", "f32", False, False)])
+def test_no_kernel_writes_outside_a_caller_buffer_in_the_optional_modes(kind, coef, sketch, erase, ranks):
+    """The same check for the buffers and kernels of the optional modes: per-head coefficient maps (written by the map
+    kernel, fp32 or bfloat16), bfloat16 sketch storage, the erase vectors, a per-head rank table, and calls with
+    per-sequence phases (decode kernel of the general kind, CUDA-core flush, map kernel in one call)."""
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    dev = torch.device("cuda", 0)
+    dv = 64 if kind == "mamba2" else 128
+    L = 8
+    w = synth.Workload("t", kind, 7, 3, 128, dv, 8, L, 0, "bf16", 67, basis="qr")
+    m = binding.SketchSSM(kind, w.batch, w.heads, w.dk, w.dv, w.rank, L, io="bf16", device=0, allocate=False,
+                          coef_per_seq=coef is not None, coef_pivots=4 if coef == "pivot" else 0, sketch=sketch,
+                          erase_factors=erase)
+    sz = m.sizes
+    names = ["state", "sketch", "ring", "omega", "coef", "status", "work"] + (["erase"] if erase else [])
+    g = {n: Guarded(getattr(sz, n + "_bytes"), dev) for n in names}
+    f32, st = torch.float32, binding.TORCH_DTYPE[sketch]
+    m.state = g["state"].view(f32, w.batch, w.heads, w.dk, w.dv)
+    m.sketch = g["sketch"].view(st, w.batch, w.heads, w.rank, w.dv)
+    m.ring = g["ring"].inner
+    m.omega = g["omega"].view(f32, w.heads, w.dk, w.rank)
+    m.coef = g["coef"].view(st, *((w.batch,) if coef else ()), w.heads, w.rank, w.dk)
+    m.status = g["status"].view(torch.int32, sz.status_bytes // 4)
+    m.work = g["work"].view(f32, sz.work_bytes // 4)
+    if erase:
+        m.erase = g["erase"].view(f32, w.batch, w.heads, L, w.rank)
+    if ranks:
+        g["head_rank"] = Guarded(w.heads * 4, dev)
+        m.head_rank = g["head_rank"].view(torch.int32, w.heads)
+        m.head_rank.copy_(torch.tensor([8, 0, 4], dtype=torch.int32))
+    m.bind()
+    Om, C = harness.basis_for(w)
+    m.state.copy_(torch.from_numpy(synth.initial_state(w)))
+    m.omega.copy_(torch.from_numpy(Om))
+    if coef is None:
+        m.coef.copy_(torch.from_numpy(C))
+    m.state_update(0)
+    token_guards = []
+    for t in range(L + 2):                            # a lock-step window, then the start of the next
+        tt, tg = guarded_tokens(w, synth.step_inputs(w, 0, t), dev)
+        token_guards += tg
+        n = t % L
+        if n < L - 1:
+            m.decode_step(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], tt["out"])
+        else:
+            m.state_update(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], tt["out"])
+    # calls with per-sequence phases: every sequence flushes once at its own ring fill (the lock-step steps left 2 tokens)
+    fill = [2] * w.batch
+    for t in range(L + 2, 2 * L + 2):
+        tt, tg = guarded_tokens(w, synth.step_inputs(w, 0, t), dev)
+        token_guards += tg
+        phase = []
+        for b in range(w.batch):
+            if fill[b] == L - 1 or fill[b] == 2 + b % 4 + 1:
+                phase.append(-(fill[b] + 1)); fill[b] = 0
+            else:
+                phase.append(fill[b]); fill[b] += 1
+        gp = Guarded(w.batch * 4, dev)
+        ph = gp.view(torch.int32, w.batch)
+        ph.copy_(torch.tensor(phase, dtype=torch.int32))
+        token_guards.append(("phase", gp))
+        m.step_mixed(ph, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], tt["out"])
+    torch.cuda.synchronize()
+    m.check_status()
+    for name, gb in list(g.items()) + token_guards:
+        assert gb.intact(), f"guard region around `{name}` was overwritten"
+    assert bool(torch.isfinite(m.state).all().item()) and bool(torch.isfinite(m.sketch.float()).all().item())
+
+
 def _window(w, dev, poison_at=None, poison_bh=(1, 1), tune=None):
     """Two windows on a fresh layer; optionally one step's q, k, v of one (batch, head) are NaN.  Returns the outputs of
     every step, the final state and the final sketch (device tensors)."""
