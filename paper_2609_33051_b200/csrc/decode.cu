@@ -95,7 +95,7 @@ __host__ __device__ inline DecodeSmem make_decode_smem(int K, int R, int nwarps,
 // UB: the sketch rows and the fixed coefficient map are stored as bfloat16 (a compile-time fact for the lean
 //     instantiation; the general ones read the flag of the launch).
 template <int KIND, typename IO, int K, int V, int RT, int GEN, bool UB = false>
-__global__ void __launch_bounds__(256, (GEN == 2 || KIND != SKETCHSSM_MAMBA2) ? 3 : 4) decode_kernel(const Params p) {
+__global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 3 : 4) decode_kernel(const Params p) {
     constexpr int EK = K / 32;
     constexpr int EV = V % 32 == 0 ? V / 32 : 4;        // value elements per lane ...
     constexpr int VL = V / EV;                          // ... on the first VL lanes (all 32, or 20 for V = 80)
