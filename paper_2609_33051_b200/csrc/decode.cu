@@ -433,8 +433,21 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
             float dlv[EK];
 #pragma unroll
             for (int e = 0; e < EK; ++e) dlv[e] = KIND == SKETCHSSM_KDA ? gg[e] : 1.f;
+            float dl_lane = 1.f;          // GDN, erase mode: lane l holds the product of the decays after slot l (the token's included)
             if constexpr (ER) {
                 if (er_h) {
+                    if constexpr (KIND == SKETCHSSM_GDN) {
+                        float incl = lane < n ? sDec[lane] : 1.f;       // inclusive suffix product over the slots
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const float other = __shfl_down_sync(0xffffffffu, incl, o);
+                            if (lane + o < 32) incl *= other;
+                        }
+                        float excl = __shfl_down_sync(0xffffffffu, incl, 1);
+                        if (lane == 31) excl = 1.f;
+                        dl_lane = dsc * excl;
+                        dl = dsc * __shfl_sync(0xffffffffu, incl, 0);     // the cumulative decay d_[t]
+                    }
                     for (int sb = n - 1; sb >= 0; sb -= NB) {
                         float pq[NB], pk[NB];
 #pragma unroll
@@ -464,7 +477,9 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
                         group_reduce_transpose<32, NB>(pq, lane);       // lane l holds entry l / 4: slot sb - l / 4
                         group_reduce_transpose<32, NB>(pk, lane);
                         const int s = sb - (lane >> 2);
-                        if ((lane & 3) == 0 && s >= 0) { sP[s] = pq[0]; sP[32 + s] = pk[0]; }
+                        float sc = 1.f;
+                        if constexpr (KIND == SKETCHSSM_GDN) sc = __shfl_sync(0xffffffffu, dl_lane, s < 0 ? 0 : s);
+                        if ((lane & 3) == 0 && s >= 0) { sP[s] = pq[0] * sc; sP[32 + s] = pk[0] * sc; }
                     }
                     __syncwarp();
                 }
@@ -482,12 +497,6 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
                 const float a = sBeta[s] * warp_sum(part);
                 if constexpr (KIND == SKETCHSSM_GDN) {
                     const float d = sDec[s];
-                    if constexpr (ER) {
-                        if (er_h) {
-                            if (lane == 0) { sP[s] *= dl; sP[32 + s] *= dl; }
-                            dl *= d;
-                        }
-                    }
 #pragma unroll
                     for (int e = 0; e < EK; ++e) x[e] = d * fmaf(-a, kr[e], x[e]);
                 } else {
@@ -529,6 +538,9 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
             }
             const bool c16 = GEN && per_seq && u_bf16;       // the head's own map travels as bfloat16 (the shared map was widened when staged)
             const int rp_it = RT ? ((RT + 7) & ~7) : ((rk + 7) & ~7);
+            bool both = false;       // erase mode: C (d_[t] * q_t) and C (d_[t] * k_t) in one pass over the rows of C
+            if constexpr (ER) both = er_h;
+            if (!both) {
 #pragma unroll
             for (int g0 = 0; g0 < (RT ? ((RT + 7) & ~7) : rp_it); g0 += NB) {
                 float part[NB];
@@ -545,22 +557,24 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
                 group_reduce_transpose<32, NB>(part, lane);
                 if ((lane & 3) == 0) sX[g0 + (lane >> 2)] = part[0];
             }
-            if constexpr (ER) {
-                if (er_h) {      // C (d_[t] * k_t) behind C (d_[t] * q_t) in the scratch
+            } else {
+                if constexpr (ER) {
                     for (int g0 = 0; g0 < rp_it; g0 += NB) {
-                        float part[NB];
+                        float part[2 * NB];
 #pragma unroll
                         for (int i = 0; i < NB; ++i) {
                             float cw[EK];
                             if (c16) load_io<EK>(reinterpret_cast<const __nv_bfloat16*>(sC), (g0 + i) * K + lane * EK, cw);
                             else load_io<EK>(sC, (g0 + i) * K + lane * EK, cw);
-                            float acc = 0.f;
+                            float aq = 0.f, ak = 0.f;
 #pragma unroll
-                            for (int e = 0; e < EK; ++e) acc = fmaf(cw[e], kk[e], acc);
-                            part[i] = acc;
+                            for (int e = 0; e < EK; ++e) { aq = fmaf(cw[e], x[e], aq); ak = fmaf(cw[e], kk[e], ak); }
+                            part[i] = aq;
+                            part[NB + i] = ak;
                         }
-                        group_reduce_transpose<32, NB>(part, lane);
-                        if ((lane & 3) == 0) sX[rp_it + g0 + (lane >> 2)] = part[0];
+                        group_reduce_transpose<32, 2 * NB>(part, lane);      // lane l holds entry l / 2
+                        const int en = lane >> 1;
+                        if ((lane & 1) == 0) sX[(en < NB ? g0 + en : rp_it + g0 + en - NB)] = part[0];
                     }
                 }
             }
