@@ -148,15 +148,21 @@ def full_read_decode(kind, S0, tokens, q):
     return exact_read(S0, x) + ob
 
 
-def decode_step(kind, U, C, tokens, q):
+def decode_step(kind, U, C, tokens, q, erase_store=None):
     """Non-flush decode step of Algorithm 1: o_t = U C q~_t + o_t^buffer.
 
     U [..., V, G] is the sketch of the window-start state, C [..., G, K] the
     coefficient map; c_t = C q~_t (Section 4.1, "Per-step: coefficient vector").
     `tokens` already contains the current token (Algorithm 1 appends first).
+    erase_store: if given (GDN / KDA), c_t is formed from projected erase vectors (Eq. 44-45) each of which is passed
+    through this function when it is stored (e.g. round_bf16: the paper keeps the vectors in BF16); with the identity
+    this is the same c_t.
     """
     x, a = effective_query(kind, tokens, q)
-    c = np.einsum("...gk,...k->...g", _f64(C), x)
+    if erase_store is None:
+        c = np.einsum("...gk,...k->...g", _f64(C), x)
+    else:
+        c = wy_coefficients(kind, tokens, q, C, store=erase_store)
     o_state = np.einsum("...vg,...g->...v", _f64(U), c)
     ob = buffer_output(tokens, a) if tokens else 0.0
     return o_state + ob
@@ -241,9 +247,10 @@ def wy_effective_query(kind, tokens, q):
     return out
 
 
-def projected_erase_vectors(kind, tokens, C):
+def projected_erase_vectors(kind, tokens, C, store=None):
     """f_s = beta_s [C (d_[s] * k_s) - sum_{j<s} f_j <l_j(s), k_s>] for every buffered token (Eq. 45),
     with the left factors l_j(s) = (D_s ... D_{j+1}) k_j kept as running products.
+    store: applied to every f_s when it is stored (default: nothing); later vectors are formed from the stored ones.
     Returns (f list, l list, d) where l[j] = l_j(t) and d = d_[t] for t = len(tokens)."""
     assert kind != MAMBA2
     C = _f64(C)
@@ -258,16 +265,17 @@ def projected_erase_vectors(kind, tokens, C):
         acc = np.einsum("...gk,...k->...g", C, d_run * k)
         for l_j, f_j in zip(ls, fs):
             acc = acc - f_j * np.einsum("...k,...k->...", l_j, k)[..., None]
-        fs.append(beta[..., None] * acc)
+        f_s = beta[..., None] * acc
+        fs.append(f_s if store is None else _f64(store(f_s)))
         ls.append(k.copy())
     return fs, ls, d_run
 
 
-def wy_coefficients(kind, tokens, q, C):
+def wy_coefficients(kind, tokens, q, C, store=None):
     """c_t = C (d_[t] * q_t) - sum_s f_s <l_s(t), q_t> with the projected erase
-    factors f_s of Eq. 45 (Eq. 44)."""
+    factors f_s of Eq. 45 (Eq. 44), each passed through `store` when it is stored."""
     q, C = _f64(q), _f64(C)
-    fs, ls, d_run = projected_erase_vectors(kind, tokens, C)
+    fs, ls, d_run = projected_erase_vectors(kind, tokens, C, store)
     c = np.einsum("...gk,...k->...g", C, d_run * q)
     for l_s, f_s in zip(ls, fs):
         c = c - f_s * np.einsum("...k,...k->...", l_s, q)[..., None]

@@ -289,6 +289,32 @@ def test_projected_erase_vectors_are_C_times_the_erase_factors(kind):
         np.testing.assert_allclose(a, b, atol=1e-15)
 
 
+@pytest.mark.parametrize("kind", ("gdn", "kda"))
+def test_stored_erase_vectors_with_rounding_stay_within_their_rounding_budget(kind):
+    # With the vectors rounded to bfloat16 where they are stored, c_t moves by at most the sum over slots of the rounding
+    # of each vector times |<l_s(t), q_t>|, plus what the rounded vectors pass on to later ones (second order); with the
+    # identity as the store function nothing changes; and the decode step with such a store is U c_t + o^buffer.
+    K, V, n, G = 12, 5, 7, 4
+    rng = np.random.default_rng(19)
+    toks = rand_tokens(rng, kind, n, K, V)
+    q = rng.standard_normal(K)
+    C = rng.standard_normal((G, K))
+    U = rng.standard_normal((V, G))
+    c0 = orc.wy_coefficients(kind, toks, q, C)
+    np.testing.assert_allclose(orc.wy_coefficients(kind, toks, q, C, store=lambda f: f), c0, atol=0)
+    cr = orc.wy_coefficients(kind, toks, q, C, store=orc.round_bf16)
+    fs, ls, _ = orc.projected_erase_vectors(kind, toks, C)
+    fr, _, _ = orc.projected_erase_vectors(kind, toks, C, store=orc.round_bf16)
+    for f in fr:
+        np.testing.assert_array_equal(f, orc.round_bf16(f))                    # stored values are bfloat16 values
+    budget = sum(np.abs(fr_s - f_s) * abs(l_s @ q) for fr_s, f_s, l_s in zip(fr, fs, ls))
+    assert np.all(np.abs(cr - c0) <= budget + 1e-12) and np.all(budget <= 2.0 ** -7 * sum(np.abs(f) * abs(l @ q) for f, l in zip(fs, ls)) + 1e-12)
+    x, a = orc.effective_query(kind, toks, q)
+    np.testing.assert_allclose(orc.decode_step(kind, U, C, toks, q, erase_store=orc.round_bf16),
+                               U @ cr + orc.buffer_output(toks, a), atol=1e-13)
+    np.testing.assert_allclose(orc.decode_step(kind, U, C, toks, q, erase_store=lambda f: f), orc.decode_step(kind, U, C, toks, q), atol=1e-12)
+
+
 # ---------------------------------------------------------------------------
 # Eq. 5-6: output error identity
 # ---------------------------------------------------------------------------
