@@ -122,7 +122,7 @@ typedef struct sketchssm_sizes {
     size_t ring_head_bytes;  /* stride of one (b, h) ring block */
     size_t ring_v_offset, ring_beta_offset, ring_decay_offset; /* byte offsets inside a ring block (k is at 0) */
     size_t alignment;        /* required alignment of every pointer (16) */
-    size_t erase_bytes;      /* erase_factors = 1: B*H*L*rank floats (else 0) */
+    size_t erase_bytes;      /* erase_factors = 1: B*H*L*rank elements of the sketch's storage type (else 0) */
 } sketchssm_sizes;
 
 typedef struct sketchssm_buffers {
@@ -147,7 +147,8 @@ typedef struct sketchssm_buffers {
                       fetches only that many); 0 = a dense-fallback head whose decode step reads the full state
                       exactly, inside the same launch.  Layouts keep the configured `rank` as their row stride.
                       Only the default one-kernel decode supports the table. */
-    void* erase;   /* erase_factors = 1: erase_bytes, [B][H][L][rank] fp32: slot s of a (b, h) block holds f_s of the token
+    void* erase;   /* erase_factors = 1: erase_bytes, [B][H][L][rank] in the sketch's storage type (fp32, or bfloat16: then
+                      every vector is rounded once, where it is stored, and rank % 8 = 0): slot s of a (b, h) block holds f_s of the token
                       in ring slot s (written by the decode step that appends the token, read by the later steps of the
                       window; a state update empties the ring and with it these slots).  Contents need no
                       initialisation.  Ignored (may be NULL) when erase_factors = 0. */

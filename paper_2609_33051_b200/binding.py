@@ -148,7 +148,7 @@ class SketchSSM:
         self.status = torch.zeros(self.sizes.status_bytes // 4, dtype=torch.int32, device=d)
         self.work = torch.zeros(self.sizes.work_bytes // 4, dtype=torch.float32, device=d)
         if self.erase_factors:
-            self.erase = torch.zeros(self.B, self.H, self.L, self.R, dtype=torch.float32, device=d)
+            self.erase = torch.zeros(self.B, self.H, self.L, self.R, dtype=TORCH_DTYPE[self.sketch_dtype], device=d)
         self.bind()
 
     def bind(self):

@@ -178,6 +178,7 @@ int sketchssm_create(const sketchssm_config* cfg, sketchssm_ctx** out) {
         // rows of r floats travel as bulk copies (16-byte units); the per-slot dot products and the two coefficient
         // vectors share the decode kernel's per-warp scratch
         if ((cfg->rank & 3) || cfg->buf_len > 32 || 2 * ((cfg->rank + 7) & ~7) > cfg->dk) return SKETCHSSM_UNSUPPORTED_SHAPE;
+        if (cfg->sketch_dtype == SKETCHSSM_BF16 && (cfg->rank & 7)) return SKETCHSSM_UNSUPPORTED_SHAPE;      // bfloat16 rows of 16-byte units
     }
     if (cfg->coef_per_seq) {
         if (!(cfg->ridge_lambda > 0.f) || cfg->coef_pivots < 0) return SKETCHSSM_INVALID_ARG;
@@ -227,7 +228,7 @@ int sketchssm_query_sizes(const sketchssm_ctx* ctx, sketchssm_sizes* out) {
     out->ring_beta_offset = ctx->ring.beta_off;
     out->ring_decay_offset = ctx->ring.decay_off;
     out->alignment = 16;
-    out->erase_bytes = c.erase_factors ? bh * (size_t)c.buf_len * c.rank * 4 : 0;
+    out->erase_bytes = c.erase_factors ? bh * (size_t)c.buf_len * c.rank * su : 0;
     return SKETCHSSM_OK;
 }
 

@@ -51,7 +51,7 @@ __host__ __device__ inline StageLayout make_stage_layout(int kind, int io, int K
     // rows padded to the reduction width are read (their sums are never used), so they get room but are not copied
     s.c_off = off; s.c_bytes = (!full_read && coef_per_seq) ? (uint32_t)(R * K * sketch_bytes) : 0u;
     off += (!full_read && coef_per_seq) ? (uint32_t)(((R + 7) & ~7) * K * sketch_bytes) : 0u;
-    s.f_off = off; s.f_bytes = (!full_read && erase) ? (uint32_t)(n * R * 4) : 0u; off += s.f_bytes;
+    s.f_off = off; s.f_bytes = (!full_read && erase) ? (uint32_t)(n * R * sketch_bytes) : 0u; off += (s.f_bytes + 15u) & ~15u;
     s.k_off = off; s.k_bytes = (uint32_t)(n * K * io); off += s.k_bytes;
     s.v_off = off; s.v_bytes = (uint32_t)(n * V * io); off += s.v_bytes;
     s.gate_off = off;
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
         case 7: cp_base = p.ring + p.rl.decay_off; cp_stride = p.rl.head_bytes; cp_dst = sl.g_off; cp_unit = KIND == SKETCHSSM_KDA ? (uint32_t)(K * sizeof(IO)) : 0u; cp_mode = 1; break;
         case 8: cp_base = reinterpret_cast<const unsigned char*>(p.sketch); cp_stride = (size_t)R * V * su; cp_dst = sl.u_off; cp_unit = (uint32_t)(V * su); cp_mode = 3; break;
         case 9: cp_base = reinterpret_cast<const unsigned char*>(p.coef); cp_stride = (size_t)R * K * su; cp_dst = sl.c_off; cp_unit = per_seq ? (uint32_t)(K * su) : 0u; cp_mode = 3; break;
-        case 10: cp_base = reinterpret_cast<const unsigned char*>(p.erase); cp_stride = (size_t)L * R * 4; cp_dst = sl.f_off; cp_unit = er ? (uint32_t)(R * 4) : 0u; cp_mode = 1; break;
+        case 10: cp_base = reinterpret_cast<const unsigned char*>(p.erase); cp_stride = (size_t)L * R * su; cp_dst = sl.f_off; cp_unit = er ? (uint32_t)(R * su) : 0u; cp_mode = 1; break;
         default: break;
     }
     const uint32_t tokA = 2u * sl.tqk_bytes + sl.tv_bytes + sl.tg_bytes;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
     // whole warp; r_it: sketch rank of the head (0: nothing to fetch), n_it: its ring fill (rows of erase vectors)
     auto issue_b = [&](size_t bh, int r_it, int n_it) {
         if constexpr (GEN) {
-            const uint32_t fbytes = er ? (uint32_t)n_it * (uint32_t)(R * 4) : 0u;
+            const uint32_t fbytes = er ? (uint32_t)n_it * (uint32_t)(R * su) : 0u;
             if (lane == 8 && r_it > 0) mbar_expect_tx(barB, (uint32_t)r_it * rowB + fbytes);
             __syncwarp();
             if ((lane == 8 || lane == 9) && cp_unit && r_it > 0)
@@ -592,17 +592,24 @@ __global__ void __launch_bounds__(256, (GEN >= 1 || KIND != SKETCHSSM_MAMBA2) ? 
                 if (er_h) {
                     // f_t = beta_t [C (d_[t] * k_t) - sum_{s<t} f_s <l_s(t), k_t>]  (Eq. 45), stored for the later steps;
                     // c_t = C (d_[t] * q_t) - sum_{s<t} f_s <l_s(t), q_t> - f_t <k_t, q_t>  (Eq. 44).  One coefficient per lane.
+                    // (with bfloat16 storage the vectors are rounded once, where they are stored; this step uses the rounded f_t too)
                     const float* sF = reinterpret_cast<const float*>(sb + sl.f_off);
+                    const __nv_bfloat16* sF16 = reinterpret_cast<const __nv_bfloat16*>(sb + sl.f_off);
                     for (int g = lane; g < rk; g += 32) {
                         float fq = sX[g], fk = sX[rp_it + g];
                         for (int s = 0; s < n; ++s) {
-                            const float f = sF[s * R + g];
+                            const float f = u_bf16 ? __bfloat162float(sF16[s * R + g]) : sF[s * R + g];
                             fq = fmaf(-f, sP[s], fq);
                             fk = fmaf(-f, sP[32 + s], fk);
                         }
-                        const float f_t = bt * fk;
+                        float f_t = bt * fk;
+                        if (u_bf16) f_t = __bfloat162float(__float2bfloat16_rn(f_t));
                         sX[g] = fmaf(-f_t, kq_t, fq);
-                        if (p.append) p.erase[(bh * L + n) * (size_t)R + g] = f_t;
+                        if (p.append) {
+                            const size_t idx = (bh * L + n) * (size_t)R + g;
+                            if (u_bf16) reinterpret_cast<__nv_bfloat16*>(p.erase)[idx] = __float2bfloat16_rn(f_t);
+                            else p.erase[idx] = f_t;
+                        }
                     }
                     __syncwarp();
                 }

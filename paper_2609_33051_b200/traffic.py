@@ -38,7 +38,7 @@ def decode_bytes(kind, B, H, K, V, r, n_before, io="bf16", out_bytes=4, full_rea
         else:
             shared = H * r * K * sketch_bytes                       # C, once per launch
         if erase_factors and kind != "mamba2":
-            per_head += (n_before + (1 if append else 0)) * r * 4   # f_s of the buffered tokens in, f_t out
+            per_head += (n_before + (1 if append else 0)) * r * sketch_bytes   # f_s of the buffered tokens in, f_t out
     return B * H * per_head + shared
 
 

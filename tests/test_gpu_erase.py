@@ -39,11 +39,17 @@ def test_erase_factors_with_the_state_dependent_map(kind, coef):
 
 @pytest.mark.parametrize("kind", ("gdn", "kda"))
 def test_erase_factors_with_bfloat16_sketch_storage(kind):
-    # U and the fixed map stored as bfloat16 (the oracle rounds U where the flush stores it, and both sides get the map
-    # already rounded); the erase vectors themselves stay fp32
+    # U, the fixed map and the erase vectors stored as bfloat16, the paper's storage (the oracle rounds U where the flush
+    # stores it and every erase vector where the decode step stores it; both sides get the map already rounded).  A stored
+    # value next to a rounding boundary may fall on the other side of it: the vectors are held to 2^-7 of their largest
+    # element, the outputs to the bar of the bfloat16 sketch test
     w = synth.Workload("t", kind, 6, 4, 128, 128, 16, 16, 0, "bf16", 229, basis="qr")
     errs = run_schedule(w, 2 * w.buf_len + 2, max_heads=10**9, sketch="bf16", erase=True)
-    assert errs["out"] <= 2e-3 + 2.0 ** -9 and errs["f"] <= FP32_GUARD and errs["S"] <= FP32_GUARD, errs
+    assert errs["out"] <= 2e-3 + 2.0 ** -9 and errs["f"] <= 2.0 ** -7 and errs["S"] <= FP32_GUARD, errs
+    m = binding.SketchSSM(kind, 2, 2, 128, 128, 16, 16, sketch="bf16", erase_factors=True, allocate=False)
+    assert m.sizes.erase_bytes == 2 * 2 * 16 * 16 * 2
+    with pytest.raises(binding.SketchSSMError):          # bfloat16 rows travel in 16-byte units: rank % 8 = 0
+        binding.SketchSSM(kind, 2, 2, 128, 128, 12, 16, sketch="bf16", erase_factors=True, allocate=False)
 
 
 def test_erase_factors_give_the_same_outputs_as_the_swept_query():

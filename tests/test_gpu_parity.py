@@ -100,10 +100,12 @@ def run_schedule(w, steps, max_heads=64, mode="sketch", tune=None, out="f32", in
         if n < L - 1:
             if mode == "sketch":
                 m.decode_step(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
-                ref = orc.decode_step(w.kind, U, C_s, ring, q)
+                # (erase vectors stored as bfloat16 are rounded where they are stored, on both sides)
+                f_store = orc.round_bf16 if (erase and sketch == "bf16") else None
+                ref = orc.decode_step(w.kind, U, C_s, ring, q, erase_store=f_store)
                 if erase:
-                    f_ref = orc.projected_erase_vectors(w.kind, ring, C_s)[0][-1]
-                    errs_f = max(errs_f, harness.rel_err(m.erase[bs_t, hs_t, n].cpu().numpy(), f_ref))
+                    f_ref = orc.projected_erase_vectors(w.kind, ring, C_s, store=f_store)[0][-1]
+                    errs_f = max(errs_f, harness.rel_err(m.erase[bs_t, hs_t, n].float().cpu().numpy(), f_ref))
             else:
                 m.full_read_decode(n, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o_dev)
                 ref = orc.full_read_decode(w.kind, S, ring, q)

@@ -137,7 +137,7 @@ def test_no_kernel_writes_outside_a_caller_buffer_in_the_optional_modes(kind, co
     m.status = g["status"].view(torch.int32, sz.status_bytes // 4)
     m.work = g["work"].view(f32, sz.work_bytes // 4)
     if erase:
-        m.erase = g["erase"].view(f32, w.batch, w.heads, L, w.rank)
+        m.erase = g["erase"].view(st, w.batch, w.heads, L, w.rank)
     if ranks:
         g["head_rank"] = Guarded(w.heads * 4, dev)
         m.head_rank = g["head_rank"].view(torch.int32, w.heads)
