@@ -802,7 +802,9 @@ def main():
                     measure_point(w, args.sweep_budget_gb, logical, local_rank, timer, peak, coef="pivot", sketch="bf16"),
                     measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, coef="pivot"),
                     measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True),
-                    measure_point(synth.CONFIGS["c4_kda"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True)]
+                    measure_point(synth.CONFIGS["c4_kda"], args.sweep_budget_gb, 8, local_rank, timer, peak, erase=True),
+                    measure_point(synth.CONFIGS["c3_gdn"], args.sweep_budget_gb, 8, local_rank, timer, peak, coef="pivot",
+                                  sketch="bf16", erase=True)]
 
     # ---- CPU oracle on a bounded sample (rank 0, N = 1) ----
     cpu = None

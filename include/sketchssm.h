@@ -110,7 +110,8 @@ typedef struct sketchssm_config {
                                sum_{j<s} f_j <l_j(s), k_s>] in R^r in the `erase` buffer, and c_t = C (d_[t] * q_t) -
                                sum_{s<=t} f_s <l_s(t), q_t> with <l_s(t), y> taken from the stored ring keys and the
                                cumulative decays (Eq. 46).  Exact for the map in force during the window (the same c_t up
-                               to rounding order); costs 4 r bytes per buffered token and step.  Needs rank % 4 == 0 and
+                               to rounding order); costs r stored elements (fp32 or bfloat16, like the sketch) per buffered token and step.
+                               Needs rank % 4 == 0 (% 8 with bfloat16 storage) and
                                buf_len <= 32; only the default one-kernel decode supports it. */
 } sketchssm_config;
 

@@ -52,6 +52,15 @@ def test_erase_factors_with_bfloat16_sketch_storage(kind):
         binding.SketchSSM(kind, 2, 2, 128, 128, 12, 16, sketch="bf16", erase_factors=True, allocate=False)
 
 
+@pytest.mark.parametrize("kind", ("gdn", "kda"))
+def test_the_papers_storage_and_map_together_with_erase_vectors(kind):
+    # state-dependent map (P = 4), bfloat16 U / C / f_s: every piece of the paper's decode configuration at once
+    w = synth.Workload("t", kind, 5, 3, 128, 128, 16, 8, 0, "bf16", 233, basis="qr")
+    errs = run_schedule(w, 3 * w.buf_len, max_heads=10**9, coef="pivot", sketch="bf16", erase=True)
+    assert errs["out"] <= 2e-3 + 2.0 ** -9 and errs["S"] <= FP32_GUARD, errs
+    assert max(errs["U"], errs["C"], errs["c0"], errs["f"]) <= 2.0 ** -7, errs
+
+
 def test_erase_factors_give_the_same_outputs_as_the_swept_query():
     # same layer, same tokens, with and without the projected vectors: equal up to rounding order
     dev = torch.device("cuda", 0)
