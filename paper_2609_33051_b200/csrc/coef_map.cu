@@ -78,7 +78,9 @@ template <int K, int V, int EXACT, int PM>
 __global__ void __launch_bounds__(kCoefThreads) coef_map_kernel(const Params p) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const size_t bh = blockIdx.x;
+    // Heads in descending order: the flush kernel before this one works through every head index from batch 0 upwards,
+    // so what it wrote last -- the part of the new state that is still in L2 -- belongs to the highest batch indices.
+    const size_t bh = (size_t)gridDim.x - 1 - blockIdx.x;
     // the single-warp stages (Gram-Schmidt, the p x p system) rotate over the warps from CTA to CTA: the warps of equal
     // index of all resident CTAs share one scheduler of the SM
     const int w0 = (int)(blockIdx.x & 3u);
