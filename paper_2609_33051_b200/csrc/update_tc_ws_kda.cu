@@ -54,6 +54,10 @@ constexpr uint32_t kZHalf = 32u * kZPitch;   // hi rows, then lo rows
 // Pass-A window [Khat 32 | G_n * W 32]: 64 rows of 16 bytes per group of 8 channels, the groups 16 bytes further apart than
 // they need to be, so that the per-channel threads of a warp (4 groups) store to different banks
 constexpr uint32_t kLboW = 64u * 16u + 16u;
+// Ktil operand (MN-major: 8 channels x 8 tokens per core matrix): the four token groups of a channel group lie side by
+// side and the channel groups 16 bytes further apart than that, so the four channel groups a warp stores to for one
+// token fall into different banks
+constexpr uint32_t kLboT = 128u, kSboT = 4u * 128u + 16u, kKtHalf = (uint32_t)(kK / 8) * kSboT;
 constexpr int kKA2 = 2;              // chunk buffers between the pass-A group and the MMA issue warp
 constexpr int kNPk = 32;             // columns of [Omega | q]: Omega in 0..R-1, q at column QA = round_up(R, 8) <= 16
 
@@ -72,8 +76,9 @@ __host__ __device__ inline KSmem make_ksmem(int stages) {
     // per-tile operand set, double-buffered: Ktil as B operand of Ktil^T E (MN-major, hi | lo), raw value rows, T,
     // Ktil [Omega | q] hi | lo (B operand of the sketch correction), G_n
     s.set = off;
-    s.set_bt = 0u; s.set_bt_lo = 8192u; s.set_vv = 16384u; s.set_t1 = 24576u; s.set_bc = 28672u; s.set_gn = 32768u;
-    s.set_stride = 33280u;
+    s.set_bt = 0u; s.set_bt_lo = kKtHalf; s.set_vv = 2u * kKtHalf; s.set_t1 = s.set_vv + 8192u; s.set_bc = s.set_t1 + 4096u;
+    s.set_gn = s.set_bc + 4096u;
+    s.set_stride = s.set_gn + 512u;
     off += 2u * s.set_stride;
     // staging of the next tile's raw rows: keys [32][256 B], decays [32][256 B], values [32][256 B], beta [L] floats, query row.
     // Once a tile's rows are in registers the key / decay area is re-used (A partials, then Ktil in fp32).
@@ -473,8 +478,8 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 for (int kk = 0; kk < ksteps; ++kk) {
                     const uint64_t ehi = make_desc(e + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
                     const uint64_t elo = make_desc(e + 128u * (uint32_t)kNT * 2u + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
-                    const uint64_t bthi = make_desc(bt + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
-                    const uint64_t btlo = make_desc(bt + sm.set_bt_lo + (uint32_t)kk * 2u * LBO_M, LBO_M, SBO);
+                    const uint64_t bthi = make_desc(bt + (uint32_t)kk * 2u * kLboT, kLboT, kSboT);
+                    const uint64_t btlo = make_desc(bt + sm.set_bt_lo + (uint32_t)kk * 2u * kLboT, kLboT, kSboT);
                     const uint64_t bchi = make_desc(bc + (uint32_t)kk * 2u * LBO_C, LBO_C, SBO);
                     const uint64_t bclo = make_desc(bc + 2048u + (uint32_t)kk * 2u * LBO_C, LBO_C, SBO);
                     tc_mma_bf16(tmem_t, ehi, bthi, idescT, 1u);
@@ -803,7 +808,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 __nv_bfloat16* zhi = reinterpret_cast<__nv_bfloat16*>(sStg);
                 __nv_bfloat16* zlo = reinterpret_cast<__nv_bfloat16*>(sStg + kZHalf);
                 const uint32_t wcol = ((uint32_t)(i >> 3) * LBO_W + (uint32_t)(i & 7) * 2u) >> 1;        // K-major: k = channel
-                const uint32_t bcol = ((uint32_t)(i & 7) * 2u + (uint32_t)(i >> 3) * SBO) >> 1;          // MN-major: mn = channel
+                const uint32_t bcol = ((uint32_t)(i & 7) * 2u + (uint32_t)(i >> 3) * kSboT) >> 1;        // MN-major: mn = channel
                 float G = fg ? gother : 1.f, X = 1.f;
 #pragma unroll
                 for (int s = 0; s < 16; ++s) {
@@ -828,7 +833,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                     Dn *= gg[s];
                     __nv_bfloat16 hi, lo;
                     split_bf16(kt, hi, lo);
-                    const uint32_t o = bcol + (((uint32_t)(s & 7) * 16u + (uint32_t)((s >> 3) + 2 * fg) * LBO_M) >> 1);
+                    const uint32_t o = bcol + (((uint32_t)(s & 7) * 16u + (uint32_t)((s >> 3) + 2 * fg) * kLboT) >> 1);
                     bthi[o] = hi;
                     btlo[o] = lo;
                     if (!fg) {
@@ -941,7 +946,7 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
                 const int mt = fw >> 2, nt = (fw & 3) - 1;
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 const uint32_t btb = smem_u32(set + sm.set_bt);
-                const uint32_t a_row = btb + (uint32_t)(2 * mt + ((lane >> 3) & 1)) * LBO_M + (uint32_t)(lane >> 4) * SBO + (uint32_t)(lane & 7) * 16u;
+                const uint32_t a_row = btb + (uint32_t)(2 * mt + ((lane >> 3) & 1)) * kLboT + (uint32_t)(lane >> 4) * kSboT + (uint32_t)(lane & 7) * 16u;
                 const __nv_bfloat16* sq = reinterpret_cast<const __nv_bfloat16*>(sStg + sm.stg_q);
                 const int ncol = p.write_sketch ? R : 0;
                 const bool has_q = p.q != nullptr;
@@ -950,8 +955,8 @@ __global__ void __launch_bounds__(kKThreads, 1) update_tc_ws_kda_kernel(const Pa
 #pragma unroll 4
                 for (int ks = 0; ks < K / 16; ++ks) {
                     uint32_t ahi[4], alo[4];
-                    k_ldmatrix_x4(a_row + (uint32_t)(2 * ks) * SBO, ahi);
-                    k_ldmatrix_x4(a_row + sm.set_bt_lo + (uint32_t)(2 * ks) * SBO, alo);
+                    k_ldmatrix_x4(a_row + (uint32_t)(2 * ks) * kSboT, ahi);
+                    k_ldmatrix_x4(a_row + sm.set_bt_lo + (uint32_t)(2 * ks) * kSboT, alo);
                     const int i0 = ks * 16 + (lane & 3) * 2;
                     float w[4] = {0.f, 0.f, 0.f, 0.f};
                     if (src == 0) {
