@@ -694,13 +694,18 @@ static int launch_decode_t(Ctx* ctx, Params p, cudaStream_t stream) {
     const bool gen = p.head_rank != nullptr || p.n_dev != nullptr || p.coef_per_seq || (p.sketch_bf16 && !lean_bf16) || erase;
     const bool fixed16 = p.R == 16 && !gen;     // the unrolled rank-16 instantiation needs one rank for all heads
     auto kern = gen ? decode_kernel<KIND, IO, K, V, 0, 1> : fixed16 ? decode_kernel<KIND, IO, K, V, 16, 0> : decode_kernel<KIND, IO, K, V, 0, 0>;
+    // rank 32 unrolled as well (state rows of 128 only: every instantiation costs build time; rank 8 measured no gain)
+    bool fixed32 = false;
+    if constexpr (K == 128) {
+        if (!gen && p.R == 32) { kern = decode_kernel<KIND, IO, K, V, 32, 0>; fixed32 = true; }
+    }
     if (lean_bf16) kern = decode_kernel<KIND, IO, K, V, 16, 0, true>;
     if constexpr (KIND != SKETCHSSM_MAMBA2) {
         if (erase) kern = decode_kernel<KIND, IO, K, V, 0, 2>;
     }
     // registers per thread of the two instantiations (queried once): they bound the resident warps like shared memory does
-    static int regs_per_thread[5] = {0, 0, 0, 0, 0};
-    int& regs = regs_per_thread[lean_bf16 ? 4 : erase ? 3 : gen ? 2 : fixed16 ? 1 : 0];
+    static int regs_per_thread[6] = {0, 0, 0, 0, 0, 0};
+    int& regs = regs_per_thread[fixed32 ? 5 : lean_bf16 ? 4 : erase ? 3 : gen ? 2 : fixed16 ? 1 : 0];
     if (regs == 0) {
         cudaFuncAttributes fa;
         if ((ctx->last_cuda_error = cudaFuncGetAttributes(&fa, kern)) != cudaSuccess) return SKETCHSSM_CUDA_ERROR;
