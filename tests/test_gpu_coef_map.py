@@ -87,3 +87,30 @@ def test_zero_state_gives_a_zero_map_and_unsupported_paths_say_so():
         m.decode_step_static(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)
     m.full_read_decode(0, tt["q"], tt["k"], tt["v"], tt["beta"], tt["decay"], o)      # unaffected by the map
     m.check_status()
+
+
+@pytest.mark.parametrize("kind,dv", [("mamba2", 64), ("gdn", 128)])
+@pytest.mark.parametrize("state_rank", [1, 2, 3])
+def test_state_of_lower_rank_than_the_pivot_count(kind, dv, state_rank):
+    """A state of rank < P: the later pivot rows of the sketch lie in the span of the earlier ones, Gram-Schmidt drops
+    them on both sides (zero probe rows), and the map is still the oracle's.  Every sketch row then lies in the span of
+    the kept probes, so the residual diagonal d is rounding noise relative to the ridge and the comparison is as well
+    conditioned as for a full-rank state."""
+    from oracle import sketchssm_oracle as orc
+    w = synth.Workload("t", kind, 3, 2, 128, dv, 16, 8, 0, "bf16", 113, basis="qr")
+    m, S0, Om, C, dev = make_layer(w, coef="pivot", pivots=4)
+    rng = np.random.default_rng(17 + state_rank)
+    A = rng.standard_normal((w.batch, w.heads, w.dk, state_rank))
+    Bm = rng.standard_normal((w.batch, w.heads, state_rank, w.dv))
+    S = (A @ Bm / np.sqrt(state_rank)).astype(np.float32)
+    m.state.copy_(torch.from_numpy(S))
+    m.coef.fill_(float("nan"))
+    m.state_update(0)
+    m.check_status()
+    got = m.coef.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    worst = 0.0
+    for b in range(w.batch):
+        ref = orc.coefficient_maps(S[b].astype(np.float64), Om.astype(np.float64), "pivot", 0.1, 4)
+        worst = max(worst, float(np.abs(got[b] - ref).max() / np.abs(ref).max()))
+    assert worst <= COEF_GUARD, worst
